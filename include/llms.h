@@ -1,0 +1,207 @@
+/*
+ * llms.h - C ABI of the B200 chunk-wise KV-cache codec and tolerance score.
+ *
+ * The library implements the data-parallel part of context switching in LLMS
+ * ("LLM as a System Service on Mobile Devices", arXiv 2403.11805): per-chunk
+ * quantize + bit-pack on swap-out, unpack + dequantize on swap-in, the per-chunk
+ * information density that ranks chunks, the rank -> bit-width rule, the LCTRU
+ * eviction order and the copy of packed records to and from pinned host memory.
+ *
+ * Conventions
+ *  - Every function returns LLMS_OK (0) or a negative llms_status.  Arguments are
+ *    checked on the host before anything is enqueued; after an argument error
+ *    nothing has been launched or written.
+ *  - "device" pointers are CUDA device addresses of the current device, "host"
+ *    pointers are ordinary host addresses, "pinned" means page-locked host memory.
+ *  - The library never allocates or frees device or pinned memory.  Scratch
+ *    ("workspace") is passed in by the caller.
+ *  - Device work is enqueued on the given stream (a cudaStream_t passed as void*;
+ *    NULL is the legacy default stream) and the call returns without synchronising.
+ *    Host arrays passed in are consumed before the call returns unless stated.
+ *  - fp16 values are IEEE binary16; multi-byte fields in records are little-endian.
+ *
+ * KV layout.  Element (l, s, h, t, c) - layer, 0 = K / 1 = V, KV head, token,
+ * channel - lives at  l*stride_l + s*stride_s + h*stride_h + t*head_dim + c
+ * (strides in elements).  A *chunk* i is tokens [i*chunk_len, (i+1)*chunk_len) of
+ * every layer, of K and V, of every head (Sec. 3.1: chunks hold the same number of
+ * tokens and carry one compression ratio each); floor(n_tokens / chunk_len)
+ * chunks exist and a shorter tail is not a chunk.  A *slab* is the chunk's
+ * chunk_len*head_dim contiguous elements of one (l, s, h); slabs are numbered
+ * s_idx = (l*2 + s)*n_kv_heads + h.  A descriptor may equally describe a pool of
+ * chunk slots: chunk ids are then slot numbers.
+ *
+ * Record of one chunk at bit-width b (Sec. 3.2 "Compressing chunks": linear
+ * quantization to a lower bit-width; Sec. 4: sub-byte codes packed with bit shifts):
+ *     [ n_groups x { u16 scale (fp16 bits), u16 zero-point (fp16 bits) } ]
+ *     zero bytes up to a multiple of 16
+ *     [ codes: element e of the chunk, in memory order (slab, token, channel),
+ *       occupies bits [e*b, (e+1)*b) of a little-endian bit stream ]
+ *     zero bytes up to a multiple of 256
+ * quant_mode 0: a group is group_size consecutive channels of one token of one
+ * slab (group index = (s_idx*chunk_len + t)*(head_dim/group_size) + j).
+ * quant_mode 1: a group is one channel of one slab across the chunk's tokens
+ * (group index = s_idx*head_dim + c), the paper's "channel-wise" wording.
+ * Per group, in binary32 with IEEE round-to-nearest and no fused operations:
+ *     zero = min x (stored as +0 when it is a zero);  scale = fp16((max x - min x) / (2^b - 1));
+ *     code = min(2^b - 1, rint((x - zero) * (1 / scale)))  (ties to even; all codes 0 when scale == 0);
+ *     decoded value = fp16(clamp(zero + code*scale, -65504, 65504)).
+ * Inputs must be finite.
+ */
+#ifndef LLMS_H
+#define LLMS_H
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum llms_status {
+    LLMS_OK = 0,
+    LLMS_ERR_INVALID_ARG = -1,   /* null pointer, non-positive size, id out of range, duplicate chunk id */
+    LLMS_ERR_BAD_BITS = -2,      /* a bit-width other than 2, 4, 8 */
+    LLMS_ERR_MISALIGNED = -3,    /* pointer, stride or offset not aligned as required */
+    LLMS_ERR_BUF_TOO_SMALL = -4, /* output buffer or workspace smaller than needed */
+    LLMS_ERR_CUDA = -5,          /* a CUDA runtime call failed (see llms_last_cuda_error) */
+    LLMS_ERR_TIMEOUT = -6,       /* llms_wait ran out of time */
+    LLMS_ERR_CORRUPT = -7,       /* a record's checksum does not match */
+    LLMS_ERR_UNSUPPORTED = -8    /* valid in the format but not implemented by the kernels */
+} llms_status;
+
+/* Shape of a KV tensor (or slot pool) and of the codec applied to it.
+ * Requirements of the codec kernels: head_dim a multiple of 16; for quant_mode 0,
+ * group_size a power of two in [16, 512] dividing head_dim; strides multiples of 8
+ * elements; n_q_heads a multiple of n_kv_heads. */
+typedef struct llms_kv_desc {
+    int32_t n_layers, n_kv_heads, n_q_heads, head_dim;
+    int32_t n_tokens, chunk_len, group_size, quant_mode;
+    int64_t stride_l, stride_s, stride_h;
+} llms_kv_desc;
+
+/* One record of a swap buffer: where it is and what is in it (32 bytes). */
+typedef struct llms_chunk_meta {
+    uint32_t chunk_id;  /* chunk (slot) the record was made from */
+    uint32_t bits;      /* 2, 4 or 8 */
+    uint64_t offset;    /* byte offset of the record in its swap buffer, multiple of 256 */
+    uint64_t nbytes;    /* record size, multiple of 256 */
+    uint32_t n_groups;
+    uint32_t checksum;  /* sum of the record's little-endian u32 words, mod 2^32 */
+} llms_chunk_meta;
+
+/* One row of the host-side chunk table that the LCTRU order is taken over. */
+typedef struct llms_chunk_state {
+    uint32_t ctx_id, chunk_id, bits;
+    uint32_t resident;  /* non-zero: in device memory */
+    uint32_t locked;    /* non-zero: its context is being served (working-set lock) */
+    uint32_t pad_;
+    uint64_t last_access_step;
+} llms_chunk_state;
+
+const char *llms_strerror(int status);
+/* Text of the last CUDA error a call of this thread ran into ("" if none). */
+const char *llms_last_cuda_error(void);
+
+/* ------------------------------------------------------------------ sizes (host only) */
+
+/* Record layout at `bits`: byte offset of the code stream inside the record and the
+ * padded record size (see the layout above).  Either output may be NULL. */
+int llms_record_layout(const llms_kv_desc *desc, int bits, uint64_t *codes_offset, uint64_t *nbytes);
+int llms_record_bytes(const llms_kv_desc *desc, int bits, uint64_t *nbytes);
+/* Sum of the record sizes of n chunks with the given bit-widths (host array). */
+int llms_compressed_size(const llms_kv_desc *desc, const uint8_t *bits, int n, uint64_t *nbytes);
+/* Device scratch needed by llms_compress_chunks / llms_decompress_chunks for n chunks. */
+int llms_codec_workspace_bytes(int n, uint64_t *nbytes);
+
+/* ------------------------------------------------------------------ swap-out: quantize + pack */
+
+/* Reclaim's compression half (Sec. 3.1 primitives; Sec. 3.2; Sec. 4).
+ * For i < n: chunk chunk_ids[i] of `kv` is quantized at bits[i] bits and its record is laid
+ * down in out_buf at the running offset (records in list order, each 256-byte aligned).
+ *   kv         device, fp16, 16-byte aligned, read only
+ *   chunk_ids  host, n distinct ids < floor(n_tokens/chunk_len)
+ *   bits       host, n values from {2, 4, 8}
+ *   out_buf    device, 256-byte aligned, out_bytes >= llms_compressed_size(...); every byte of
+ *              every record, padding included, is written
+ *   meta       host, n entries, filled before return except `checksum`, which the device
+ *              computes: it is copied back into meta[] in stream order, so it is valid once the
+ *              stream has been synchronised (pass pinned memory to keep that copy asynchronous;
+ *              with pageable memory the call may block until the kernel is done)
+ *   workspace  device, 16-byte aligned, llms_codec_workspace_bytes(n); may be reused by the
+ *              next call on the same stream
+ * n == 0 is valid and does nothing. */
+int llms_compress_chunks(const llms_kv_desc *desc, const void *kv, const uint32_t *chunk_ids,
+                         const uint8_t *bits, int n, void *out_buf, uint64_t out_bytes,
+                         llms_chunk_meta *meta, void *workspace, uint64_t workspace_bytes, void *stream);
+
+/* ------------------------------------------------------------------ swap-in: unpack + dequantize */
+
+/* Load's decompression half.  Record i (meta[i], inside `buf`) is decoded into chunk slot
+ * dst_chunk_ids[i] of kv_out (dst_chunk_ids == NULL: meta[i].chunk_id).  Other chunks of kv_out
+ * are not touched.  While decoding, each record's checksum is recomputed; the number of
+ * records whose sum differs from meta[i].checksum is left in the workspace and can be read
+ * with llms_codec_corrupt_count (decoded values of such a record are still written).
+ *   buf        device, 256-byte aligned;  meta, dst_chunk_ids  host;  kv_out  device fp16 */
+int llms_decompress_chunks(const llms_kv_desc *desc, const void *buf, const llms_chunk_meta *meta,
+                           const uint32_t *dst_chunk_ids, int n, void *kv_out,
+                           void *workspace, uint64_t workspace_bytes, void *stream);
+
+/* Synchronises `stream`, then returns LLMS_OK if the last llms_decompress_chunks that used this
+ * workspace saw no checksum mismatch, LLMS_ERR_CORRUPT otherwise; *n_corrupt (host, may be NULL)
+ * receives the count. */
+int llms_codec_corrupt_count(const void *workspace, uint32_t *n_corrupt, void *stream);
+
+/* ------------------------------------------------------------------ tolerance score (Eq. 1) */
+
+/* Information density D_i of every chunk (Sec. 3.2 Eq. 1): the attention matrix
+ * A = softmax(mask(Q K^T / sqrt(head_dim))) of the last W query positions (row r sits at token
+ * position n_tokens - W + r and sees columns 0..that position) is averaged down each column over
+ * the rows that see it, then over heads, layers and the chunk's tokens.  W = n_tokens gives the
+ * paper's full lower-triangular matrix.  Query head h reads KV head h / (n_q_heads/n_kv_heads).
+ *   kv      device fp16 (only K, the s = 0 half, is read)
+ *   q_win   device fp16 [n_layers][n_q_heads][W][head_dim], contiguous, 16-byte aligned
+ *   scores  device fp32 [floor(n_tokens/chunk_len)]
+ *   workspace device, llms_tolerance_workspace_bytes(desc, W) */
+int llms_tolerance_workspace_bytes(const llms_kv_desc *desc, int W, uint64_t *nbytes);
+int llms_chunk_tolerance(const llms_kv_desc *desc, const void *kv, const void *q_win, int W,
+                         float *scores, void *workspace, uint64_t workspace_bytes, void *stream);
+/* The same reduction from attention probabilities that inference already produced:
+ *   probs   device fp32 [n_layers][n_q_heads][W][n_tokens]; entries above the causal boundary
+ *           (col > n_tokens - W + r) are ignored. */
+int llms_chunk_tolerance_from_probs(const llms_kv_desc *desc, const float *probs, int W,
+                                    float *scores, void *workspace, uint64_t workspace_bytes, void *stream);
+
+/* ------------------------------------------------------------------ policy (host only) */
+
+/* Eq. 2: rank chunks by density and map rank to a bit-width.  order_out (may be NULL) receives
+ * chunk indices, densest first, ties to the lower index.  With frac = {f8, f4, f2} (sum 1):
+ * the first n8 = floor(f8*n + 1/2) chunks of that order keep 8 bits, up to
+ * floor((f8+f4)*n + 1/2) get 4, the rest 2 - low density means high tolerance means fewer bits. */
+int llms_assign_bits(const float *scores, int n, const float frac[3], uint8_t *bits_out, uint32_t *order_out);
+
+/* Sec. 3.4 (ii): eviction order over the rows that are resident and not locked - the 8-bit
+ * sub-queue first, then 4, then 2 ("heavy chunks first"), least recently used first inside a
+ * sub-queue, ties by (ctx_id, chunk_id).  order_out (n entries) receives row indices; the return
+ * value is their count, or a negative status. */
+int llms_lctru_order(const llms_chunk_state *table, int n, uint32_t *order_out);
+
+/* ------------------------------------------------------------------ swap copies */
+
+/* Copy n records between a device swap buffer and a pinned host arena on `side_stream`
+ * (Sec. 3.1 Reclaim / Load, with pinned host memory in the place of the paper's disk; Sec. 4:
+ * an I/O thread of its own).  Record i sits at meta[i].offset in the device buffer and at
+ * host_offsets[i] in the arena (host_offsets == NULL: the same offsets).  Runs of records
+ * adjacent on both sides travel as one copy.  If `after` (a cudaEvent_t) is not NULL the side
+ * stream first waits for it - record it on the stream that produced (swap-out) or last used
+ * (swap-in) the device buffer.  If `done` is not NULL it is recorded on the side stream after
+ * the last copy. */
+int llms_swap_out(const void *dev_buf, const llms_chunk_meta *meta, int n, void *pinned_dst,
+                  const uint64_t *host_offsets, void *side_stream, void *after, void *done);
+int llms_swap_in(const void *pinned_src, const uint64_t *host_offsets, const llms_chunk_meta *meta, int n,
+                 void *dev_buf, void *side_stream, void *after, void *done);
+/* Poll a cudaEvent_t until it has completed or timeout_ms has passed (LLMS_ERR_TIMEOUT). */
+int llms_wait(void *event, uint32_t timeout_ms);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* LLMS_H */

@@ -1,0 +1,58 @@
+// Shared host-side helpers of the library: argument checks, record layout arithmetic, CUDA error capture.
+#pragma once
+
+#include <cuda_runtime.h>
+#include <cuda_fp16.h>
+#include <stdint.h>
+
+#include "llms.h"
+
+namespace llms {
+
+void set_cuda_error(cudaError_t e, const char *where);
+
+#define LLMS_CUDA_TRY(expr)                                   \
+    do {                                                      \
+        cudaError_t e__ = (expr);                             \
+        if (e__ != cudaSuccess) {                             \
+            ::llms::set_cuda_error(e__, #expr);               \
+            return LLMS_ERR_CUDA;                             \
+        }                                                     \
+    } while (0)
+
+inline uint64_t round_up(uint64_t x, uint64_t a) { return (x + a - 1) / a * a; }
+inline bool aligned(const void *p, uintptr_t a) { return (reinterpret_cast<uintptr_t>(p) & (a - 1)) == 0; }
+inline bool is_pow2(int x) { return x > 0 && (x & (x - 1)) == 0; }
+
+inline int64_t slabs_per_chunk(const llms_kv_desc &d) { return (int64_t)d.n_layers * 2 * d.n_kv_heads; }
+inline int64_t slab_elems(const llms_kv_desc &d) { return (int64_t)d.chunk_len * d.head_dim; }
+inline int n_chunks(const llms_kv_desc &d) { return d.n_tokens / d.chunk_len; }
+inline uint64_t groups_per_slab(const llms_kv_desc &d)
+{
+    return d.quant_mode == 0 ? (uint64_t)d.chunk_len * (d.head_dim / d.group_size) : (uint64_t)d.head_dim;
+}
+inline uint64_t groups_per_chunk(const llms_kv_desc &d) { return (uint64_t)slabs_per_chunk(d) * groups_per_slab(d); }
+
+// Shape checks common to every entry point.
+int check_desc(const llms_kv_desc *d);
+// Shape + alignment checks for the codec kernels (vector loads need 16-byte aligned slabs).
+int check_desc_codec(const llms_kv_desc *d);
+inline int check_bits(int b) { return (b == 2 || b == 4 || b == 8) ? LLMS_OK : LLMS_ERR_BAD_BITS; }
+
+// Number of SMs of the current device (cached per device).
+int sm_count();
+
+// Device-side copy of the per-chunk table, kept in the workspace.
+struct ChunkEntry {          // same bytes as llms_chunk_meta
+    uint32_t chunk_id, bits;
+    uint64_t offset, nbytes;
+    uint32_t n_groups, checksum;
+};
+static_assert(sizeof(ChunkEntry) == sizeof(llms_chunk_meta) && sizeof(ChunkEntry) == 32, "meta layout");
+
+// Workspace of the codec calls: [status word, padded to 16 bytes][n entries][n recomputed sums].
+constexpr uint64_t kWsEntriesOffset = 16;
+inline uint64_t ws_sums_offset(int n) { return kWsEntriesOffset + (uint64_t)n * sizeof(ChunkEntry); }
+inline uint64_t ws_total(int n) { return round_up(ws_sums_offset(n) + (uint64_t)n * 4, 16); }
+
+}  // namespace llms

@@ -1,0 +1,49 @@
+// Host-side policies: rank -> bit-width (Eq. 2) and the LCTRU eviction order (Sec. 3.4 ii).
+#include <algorithm>
+#include <cmath>
+#include <numeric>
+#include <vector>
+
+#include "llms_internal.cuh"
+
+extern "C" int llms_assign_bits(const float *scores, int n, const float frac[3], uint8_t *bits_out, uint32_t *order_out)
+{
+    if (n < 0 || !frac || (n > 0 && (!scores || !bits_out))) return LLMS_ERR_INVALID_ARG;
+    const double f8 = frac[0], f4 = frac[1], f2 = frac[2];
+    if (!(f8 >= 0) || !(f4 >= 0) || !(f2 >= 0) || std::fabs(f8 + f4 + f2 - 1.0) > 1e-3) return LLMS_ERR_INVALID_ARG;
+    std::vector<uint32_t> order(n);
+    std::iota(order.begin(), order.end(), 0u);
+    // densest first; equal densities keep index order
+    std::stable_sort(order.begin(), order.end(), [&](uint32_t a, uint32_t b) { return scores[a] > scores[b]; });
+    long n8 = (long)std::floor(f8 * n + 0.5);
+    long n84 = (long)std::floor((f8 + f4) * n + 0.5);
+    n8 = std::min<long>(n8, n);
+    n84 = std::max(std::min<long>(n84, n), n8);
+    for (long r = 0; r < n; ++r) {
+        bits_out[order[r]] = r < n8 ? 8 : (r < n84 ? 4 : 2);
+        if (order_out) order_out[r] = order[r];
+    }
+    return LLMS_OK;
+}
+
+extern "C" int llms_lctru_order(const llms_chunk_state *table, int n, uint32_t *order_out)
+{
+    if (n < 0 || (n > 0 && (!table || !order_out))) return LLMS_ERR_INVALID_ARG;
+    int m = 0;
+    for (int i = 0; i < n; ++i) {
+        if (table[i].resident && !table[i].locked) {
+            if (llms::check_bits((int)table[i].bits)) return LLMS_ERR_BAD_BITS;
+            order_out[m++] = (uint32_t)i;
+        }
+    }
+    // concatenated sub-queues: 8-bit chunks first, then 4, then 2; least recently used first inside each
+    std::sort(order_out, order_out + m, [&](uint32_t x, uint32_t y) {
+        const llms_chunk_state &a = table[x], &b = table[y];
+        if (a.bits != b.bits) return a.bits > b.bits;
+        if (a.last_access_step != b.last_access_step) return a.last_access_step < b.last_access_step;
+        if (a.ctx_id != b.ctx_id) return a.ctx_id < b.ctx_id;
+        if (a.chunk_id != b.chunk_id) return a.chunk_id < b.chunk_id;
+        return x < y;
+    });
+    return m;
+}
