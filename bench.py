@@ -1,0 +1,382 @@
+"""Throughput of the context-switching hot path on synthetic KV caches.
+
+One step = one pass of the whole path over one context that is resident in HBM:
+tolerance score (Eq. 1) -> rank -> bits on the host (Eq. 2) -> quantize + pack every chunk -> unpack + dequantize
+every chunk.  `value` counts the fp16 bytes the codec processed (compress + decompress: 2 x the KV size) per
+second of step time.  `e2e` runs compress -> swap-out to pinned host memory -> swap-in -> decompress through
+the same C-ABI calls, with the host copies inside the timed region.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload llama7b] [--impl ours|reference]
+"""
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import tempfile
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "KV compress+decompress GB/s (fp16 bytes)"
+UNIT = "GB/s"
+
+
+def parse_args():
+    p = argparse.ArgumentParser()
+    p.add_argument("--gpus", type=int, default=1)
+    p.add_argument("--steps", type=int, default=200)
+    p.add_argument("--warmup", type=int, default=10)
+    p.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    p.add_argument("--workload", default="llama7b", help="a key of synth.CONFIGS (single-context workloads)")
+    p.add_argument("--layers", type=int, default=0, help="use only this many layers (smaller cases for profiler captures)")
+    p.add_argument("--e2e-steps", type=int, default=10)
+    p.add_argument("--no-cpu-baseline", action="store_true")
+    return p.parse_args()
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured"
+    return 6650.0, "fallback"
+
+
+def target_bits(shape):
+    """Bit mix of the workload by chunk rank: counts as the rank -> bits rule gives them."""
+    import numpy as np
+    n = shape.n_chunks
+    f8, f4, _ = shape.frac if shape.frac is not None else (1 / 3, 1 / 3, 1 / 3)
+    n8 = int(np.floor(f8 * n + 0.5))
+    n84 = int(np.floor((f8 + f4) * n + 0.5))
+    return n8, n84 - n8, n - n84
+
+
+class ClockSampler:
+    """nvidia-smi samples of SM clock and throttle reasons while the timed region runs."""
+    FIELDS = ("timestamp,index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+              "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+              "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index):
+        self.file = tempfile.NamedTemporaryFile("w+", suffix=".csv", delete=False)
+        self.proc = None
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits",
+                                          "-i", str(gpu_index), "-lms", "100"], stdout=self.file, stderr=subprocess.DEVNULL)
+        except OSError:
+            self.proc = None
+        self.t_begin = self.t_end = None
+
+    def begin(self):
+        self.t_begin = time.time()
+
+    def end(self):
+        self.t_end = time.time()
+
+    def finish(self):
+        if self.proc is not None:
+            time.sleep(0.15)
+            self.proc.terminate()
+            try:
+                self.proc.wait(timeout=5)
+            except subprocess.TimeoutExpired:
+                self.proc.kill()
+        self.file.flush()
+        self.file.seek(0)
+        rows = [r.strip().split(", ") for r in self.file.read().splitlines() if r.strip()]
+        self.file.close()
+        os.unlink(self.file.name)
+        import datetime
+        inside, every = [], []
+        for r in rows:
+            if len(r) < 10:
+                continue
+            try:
+                ts = datetime.datetime.strptime(r[0], "%Y/%m/%d %H:%M:%S.%f").timestamp()
+                rec = (float(r[2]), float(r[3]), r[6:10])
+            except ValueError:
+                continue
+            every.append(rec)
+            if self.t_begin is not None and self.t_begin - 0.05 <= ts <= self.t_end + 0.05:
+                inside.append(rec)
+        use = inside if len(inside) >= 2 else every
+        if not use:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        reasons = sorted({names[i] for rec in use for i, v in enumerate(rec[2]) if v.strip().lower() == "active"})
+        return {"sm_mhz": statistics.median(r[0] for r in use), "sm_max_mhz": use[0][1], "reasons": reasons,
+                "samples": len(use), "in_timed_region": use is inside}
+
+
+def run_reference(args):
+    """The oracle, as it stands, on the host cores: score, rank -> bits, compress, decompress of a bounded sample."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    import numpy as np
+    import torch
+    import oracle
+    from paper_2403_11805_b200 import synth
+
+    shape = synth.CONFIGS[args.workload]
+    sample_layers = min(shape.n_layers, args.layers or 8)
+    sh = shape.with_(n_layers=sample_layers)
+    W = sh.window
+    kv = synth.kv_tensor(sh).view(torch.int16).numpy().view(np.uint16)
+    q = synth.q_window(sh, W).view(torch.int16).numpy().view(np.uint16)
+    od = oracle.make_desc(sh.n_layers, sh.n_kv_heads, sh.n_q_heads, sh.head_dim, sh.n_tokens, sh.chunk_len, sh.group_size)
+    frac = sh.frac if sh.frac is not None else (1 / 3, 1 / 3, 1 / 3)
+    ids = np.arange(sh.n_chunks, dtype=np.uint32)
+    out = np.zeros(kv.size, dtype=np.uint16).reshape(kv.shape)
+
+    def step():
+        scores = oracle.chunk_tolerance(od, kv, q, W)
+        bits, _ = oracle.assign_bits(scores.astype(np.float32), frac)
+        buf, meta = oracle.compress_chunks(od, kv, ids, bits)
+        oracle.decompress_chunks(od, buf, meta, out)
+
+    steps, warmup = max(1, min(args.steps, 5)), max(1, min(args.warmup, 1))
+    for _ in range(warmup):
+        step()
+    t0 = time.perf_counter()
+    for _ in range(steps):
+        step()
+    dt = (time.perf_counter() - t0) / steps
+    value = 2 * sh.n_elements * 2 / dt / 1e9
+    sample = f"{sample_layers} of {shape.n_layers} layers of the {shape.name} context per step, all {sh.n_chunks} chunks"
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": steps,
+        "warmup": warmup, "ms_per_step": dt * 1e3, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "f32 codec decisions, f64 score", "data": "synthetic",
+        "config": {"workload": shape.name, "sample": sample},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": oracle.num_threads(), "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line))
+
+
+def cpu_baseline(shape, kv_dev, q_dev):
+    """Oracle timed on this host on a bounded sample of the same workload (rank 0, N = 1)."""
+    import numpy as np
+    import torch
+    import oracle
+
+    sample_layers = min(shape.n_layers, 8)
+    sh = shape.with_(n_layers=sample_layers)
+    W = sh.window
+    kv = kv_dev[:sample_layers].cpu().view(torch.int16).numpy().view(np.uint16)
+    q = q_dev[:sample_layers].cpu().view(torch.int16).numpy().view(np.uint16)
+    od = oracle.make_desc(sh.n_layers, sh.n_kv_heads, sh.n_q_heads, sh.head_dim, sh.n_tokens, sh.chunk_len, sh.group_size)
+    frac = sh.frac if sh.frac is not None else (1 / 3, 1 / 3, 1 / 3)
+    ids = np.arange(sh.n_chunks, dtype=np.uint32)
+    out = np.zeros(kv.size, dtype=np.uint16).reshape(kv.shape)
+    t0 = time.perf_counter()
+    scores = oracle.chunk_tolerance(od, kv, q, W)
+    bits, _ = oracle.assign_bits(scores.astype(np.float32), frac)
+    t1 = time.perf_counter()
+    buf, meta = oracle.compress_chunks(od, kv, ids, bits)
+    t2 = time.perf_counter()
+    oracle.decompress_chunks(od, buf, meta, out)
+    t3 = time.perf_counter()
+    nbytes = sh.n_elements * 2
+    return {
+        "value": 2 * nbytes / (t3 - t0) / 1e9, "unit": UNIT, "cores": oracle.num_threads(), "kind": "oracle",
+        "sample": f"{sample_layers} of {shape.n_layers} layers, all {sh.n_chunks} chunks, one pass",
+        "score_s": t1 - t0, "compress_gbs": nbytes / (t2 - t1) / 1e9, "decompress_gbs": nbytes / (t3 - t2) / 1e9,
+    }
+
+
+def run_ours(args):
+    import numpy as np
+    import torch
+    from paper_2403_11805_b200 import binding as B, synth
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the hot path has no CPU fallback")
+    torch.cuda.set_device(local_rank)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+    B.lib()
+
+    shape = synth.CONFIGS[args.workload]
+    if args.layers:
+        shape = shape.with_(n_layers=args.layers)
+    W = shape.window
+    frac = shape.frac if shape.frac is not None else (1 / 3, 1 / 3, 1 / 3)
+    # every rank owns one context of the workload (contexts are independent: no data-path collective)
+    kv = synth.kv_tensor(shape, device="cuda", context=rank)
+    q_win = synth.q_window(shape, W, device="cuda", context=rank)
+    d = B.desc_of(shape)
+    n = shape.n_chunks
+    ids = np.arange(n, dtype=np.uint32)
+    n8, n4, n2 = target_bits(shape)
+    worst_bits = np.full(n, 8, dtype=np.uint8)
+    buf = torch.empty(B.compressed_size(d, worst_bits), dtype=torch.uint8, device="cuda")
+    kv_out = torch.empty_like(kv)
+    scores = torch.empty(n, dtype=torch.float32, device="cuda")
+    scores_host = torch.empty(n, dtype=torch.float32).pin_memory()
+    ws_tol = torch.empty(B.tolerance_workspace_bytes(d, W), dtype=torch.uint8, device="cuda")
+    ws = torch.empty(B.codec_workspace_bytes(n), dtype=torch.uint8, device="cuda")
+    meta = B.new_meta(n, pinned=True)
+    stream = torch.cuda.current_stream()
+    state = {}
+
+    def step(ev=None):
+        if ev:
+            ev[0].record(stream)
+        B.chunk_tolerance(d, kv, q_win, W, scores, ws_tol)
+        scores_host.copy_(scores, non_blocking=True)
+        stream.synchronize()                     # the ranking is a host step
+        bits, _ = B.assign_bits(scores_host.numpy(), frac)
+        if ev:
+            ev[1].record(stream)
+        B.compress_chunks(d, kv, ids, bits, buf, meta, ws)
+        if ev:
+            ev[2].record(stream)
+        B.decompress_chunks(d, buf, meta, None, kv_out, ws)
+        if ev:
+            ev[3].record(stream)
+        state["bits"] = bits
+
+    def barrier():
+        torch.cuda.synchronize()
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for _ in range(max(args.warmup, 3)):
+        step()
+    assert B.codec_corrupt_count(ws) == 0
+    bits = state["bits"]
+    assert tuple(int((bits == b).sum()) for b in (8, 4, 2)) == (n8, n4, n2)
+    record_bytes = B.compressed_size(d, bits)
+
+    sampler = ClockSampler(local_rank) if rank == 0 else None
+    events = [[torch.cuda.Event(enable_timing=True) for _ in range(4)] for _ in range(args.steps)]
+    barrier()
+    if sampler:
+        sampler.begin()
+    t_wall = time.perf_counter()
+    for k in range(args.steps):
+        step(events[k])
+    barrier()
+    t_wall = time.perf_counter() - t_wall
+    if sampler:
+        sampler.end()
+    span_ms = events[0][0].elapsed_time(events[-1][3])
+    tol_ms = sum(e[0].elapsed_time(e[1]) for e in events) / args.steps
+    comp_ms = sum(e[1].elapsed_time(e[2]) for e in events) / args.steps
+    decomp_ms = sum(e[2].elapsed_time(e[3]) for e in events) / args.steps
+    ms_per_step = span_ms / args.steps
+    if dist is not None:
+        t = torch.tensor([ms_per_step, tol_ms, comp_ms, decomp_ms], dtype=torch.float64, device="cuda")
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms_per_step, tol_ms, comp_ms, decomp_ms = t.tolist()
+    kv_bytes = shape.n_elements * 2
+    value = world * 2 * kv_bytes / (ms_per_step * 1e-3) / 1e9
+
+    # ---- end to end: compress -> swap-out -> swap-in -> decompress with the pinned arena in the loop
+    arena = torch.empty(record_bytes, dtype=torch.uint8).pin_memory()
+    back = torch.empty(record_bytes, dtype=torch.uint8, device="cuda")
+    side = torch.cuda.Stream()
+    ev_c, ev_in = B.new_event(), B.new_event()
+
+    def e2e_step():
+        B.compress_chunks(d, kv, ids, bits, buf, meta, ws)
+        ev_c.record(stream)
+        stream.synchronize()                     # record sizes and checksums are final on the host
+        B.swap_out(buf, meta, arena, side_stream=side, after=ev_c)
+        B.swap_in(arena, meta, back, side_stream=side, done=ev_in)
+        stream.wait_event(ev_in)
+        B.decompress_chunks(d, back, meta, None, kv_out, ws)
+
+    for _ in range(3):
+        e2e_step()
+    assert B.codec_corrupt_count(ws) == 0
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    barrier()
+    e0.record(stream)
+    for _ in range(args.e2e_steps):
+        e2e_step()
+    e1.record(stream)
+    barrier()
+    e2e_ms = e0.elapsed_time(e1) / args.e2e_steps
+    if dist is not None:
+        t = torch.tensor([e2e_ms], dtype=torch.float64, device="cuda")
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        e2e_ms = float(t.item())
+    e2e_value = world * 2 * kv_bytes / (e2e_ms * 1e-3) / 1e9
+    clocks = sampler.finish() if sampler else None
+
+    if rank != 0:
+        if dist is not None:
+            dist.destroy_process_group()
+        return
+
+    # ---- roofline of the dominant codec kernel (algorithmic bytes per launch / measured launch time)
+    peak, peak_kind = measured_peaks()
+    algo_bytes = kv_bytes + record_bytes             # compress: fp16 read + record written; decompress: the reverse
+    k_ms = {"compress_kernel": comp_ms, "decompress_kernel": decomp_ms}
+    dominant = max(k_ms, key=k_ms.get)
+    achieved = algo_bytes / (k_ms[dominant] * 1e-3) / 1e9
+    roofline = {
+        "kernel": dominant, "bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
+        "peak_source": f"{peak_kind} copy bandwidth", "traffic": None,
+        "algorithmic_bytes_per_launch": algo_bytes,
+        "frac_of_nominal_8000": achieved / 8000.0,
+        "per_stage": {
+            "tolerance_ms": tol_ms, "compress_ms": comp_ms, "decompress_ms": decomp_ms,
+            "tolerance_gbs_of_K_read": (kv_bytes / 2) / (tol_ms * 1e-3) / 1e9,
+            "compress_algorithmic_gbs": algo_bytes / (comp_ms * 1e-3) / 1e9,
+            "decompress_algorithmic_gbs": algo_bytes / (decomp_ms * 1e-3) / 1e9,
+            "compress_fp16_gbs": kv_bytes / (comp_ms * 1e-3) / 1e9,
+            "decompress_fp16_gbs": kv_bytes / (decomp_ms * 1e-3) / 1e9,
+            "codec_only_fp16_gbs": 2 * kv_bytes / ((comp_ms + decomp_ms) * 1e-3) / 1e9,
+        },
+    }
+    line = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": max(args.warmup, 3),
+        "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "f32 (fp16 in/out, integer codes)", "data": "synthetic",
+        "config": {"workload": shape.name, "layers": shape.n_layers, "kv_heads": shape.n_kv_heads, "head_dim": shape.head_dim,
+                   "tokens": shape.n_tokens, "chunk_len": shape.chunk_len, "group_size": shape.group_size,
+                   "window": W, "bits_8_4_2": [n8, n4, n2], "contexts_per_gpu": 1,
+                   "l2": "inputs larger than L2 (fp16 KV %.0f MiB per context)" % (kv_bytes / 2 ** 20),
+                   "step": "score + rank->bits + compress + decompress of one context"},
+        "contexts_per_s": world / (ms_per_step * 1e-3),
+        "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": record_bytes, "d2h_bytes_per_step": record_bytes,
+                "ms_per_step": e2e_ms, "context_switches_per_s": world / (e2e_ms * 1e-3),
+                "host_copy_gbs_each_way": None,
+                "what": "compress -> swap-out to pinned host -> swap-in -> decompress"},
+        "gpu_launches": args.steps * 7,
+        "roofline": roofline, "clocks": clocks,
+        "wall_ms_per_step": t_wall * 1e3 / args.steps,
+    }
+    if world == 1 and not args.no_cpu_baseline:
+        line["cpu_baseline"] = cpu_baseline(shape, kv, q_win)
+    print(json.dumps(line))
+    if dist is not None:
+        dist.destroy_process_group()
+
+
+def main():
+    args = parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

@@ -26,3 +26,12 @@ def read_golden(path):
             if line:
                 rows.append([float(x) for x in line.split()])
     return rows
+
+
+@pytest.fixture(scope="session", autouse=True)
+def built_libraries():
+    """Both shared libraries are built in-tree before any test runs (nvcc cross-compiles without a GPU)."""
+    from paper_2403_11805_b200 import build as gpu_build
+    from oracle import build as oracle_build
+    oracle_build.build()
+    gpu_build.build()

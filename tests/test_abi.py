@@ -1,0 +1,113 @@
+"""The C-ABI library: it loads, exports every function the header declares, and its host-only entry points
+(sizes, rank -> bits, LCTRU order, argument checks) agree with the oracle.  No GPU needed."""
+import ctypes
+import itertools
+import os
+import re
+
+import numpy as np
+import pytest
+
+import oracle
+from paper_2403_11805_b200 import binding as B, synth
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+def declared_functions():
+    text = open(os.path.join(ROOT, "include", "llms.h")).read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    return sorted(set(re.findall(r"\b(llms_[a-z_0-9]+)\s*\(", text)))
+
+
+def test_every_declared_function_is_exported():
+    names = declared_functions()
+    assert len(names) >= 17
+    lib = ctypes.CDLL(B.LIB_PATH)
+    for name in names:
+        assert hasattr(lib, name), name
+    assert set(B._SIGNATURES) == set(names)
+
+
+def odesc(sh, mode=0):
+    return oracle.make_desc(sh.n_layers, sh.n_kv_heads, sh.n_q_heads, sh.head_dim, sh.n_tokens, sh.chunk_len,
+                            sh.group_size, mode)
+
+
+def test_record_sizes_match_oracle():
+    for sh in synth.CONFIGS.values():
+        for mode in (0, 1):
+            for b in (2, 4, 8):
+                assert B.record_layout(B.desc_of(sh, mode), b) == oracle.record_layout(odesc(sh, mode), b)
+    odd = synth.KVShape("odd", 1, 1, 1, 16, 3, 3, 16)
+    assert B.record_layout(B.desc_of(odd), 4) == oracle.record_layout(odesc(odd), 4) == (32, 256)
+    bits = [8, 4, 2, 2, 8]
+    sh = synth.CONFIGS["tiny"]
+    assert B.compressed_size(B.desc_of(sh), bits) == oracle.compressed_size(odesc(sh), bits)
+
+
+def test_assign_bits_matches_oracle_bit_for_bit():
+    rng = np.random.default_rng(0)
+    for n, frac in [(256, (1 / 3, 1 / 3, 1 / 3)), (128, (1 / 3, 1 / 3, 1 / 3)), (32, (1 / 3, 1 / 3, 1 / 3)),
+                    (512, (0.1, 0.5, 0.4)), (7, (0.5, 0.25, 0.25)), (1, (0.2, 0.3, 0.5)), (0, (1 / 3, 1 / 3, 1 / 3))]:
+        for ties in (False, True):
+            s = rng.random(n).astype(np.float32)
+            if ties:
+                s = np.round(s * 4) / 4
+            gb, go = B.assign_bits(s, frac)
+            ob, oo = oracle.assign_bits(s, frac)
+            assert np.array_equal(gb, ob) and np.array_equal(go, oo)
+    for scores in itertools.product([0.1, 0.2, 0.3], repeat=5):
+        gb, go = B.assign_bits(scores, (0.4, 0.2, 0.4))
+        ob, oo = oracle.assign_bits(scores, (0.4, 0.2, 0.4))
+        assert np.array_equal(gb, ob) and np.array_equal(go, oo)
+
+
+def test_lctru_order_matches_oracle_bit_for_bit():
+    rng = np.random.default_rng(1)
+    for n in (0, 1, 5, 64, 2048):
+        t = np.zeros(n, dtype=B.STATE_DTYPE)
+        t["ctx_id"] = rng.integers(0, 64, n)
+        t["chunk_id"] = rng.integers(0, 32, n)
+        t["bits"] = rng.choice([8, 4, 2], n)
+        t["resident"] = rng.random(n) < 0.7
+        t["locked"] = rng.random(n) < 0.2
+        t["last_access_step"] = rng.integers(0, 10, n)
+        assert np.array_equal(B.lctru_order(t), oracle.lctru_order(t.astype(oracle.STATE_DTYPE)))
+
+
+def test_argument_errors_on_the_host():
+    sh = synth.CONFIGS["tiny"]
+    d = B.desc_of(sh)
+    with pytest.raises(B.LlmsError) as e:
+        B.record_bytes(d, 3)
+    assert e.value.status == B.ERR_BAD_BITS
+    bad = B.desc_of(sh)
+    bad.n_q_heads = 3
+    with pytest.raises(B.LlmsError) as e:
+        B.record_bytes(bad, 4)
+    assert e.value.status == B.ERR_INVALID_ARG
+    with pytest.raises(B.LlmsError):
+        B.assign_bits([0.1, 0.2], (0.5, 0.6, 0.2))
+    # the codec entry points check their arguments before touching CUDA: dummy addresses are enough
+    meta = B.new_meta(2)
+    lib = B.lib()
+    ids = np.array([1, 1], dtype=np.uint32)
+    bits = np.array([8, 4], dtype=np.uint8)
+    call = lambda **kw: lib.llms_compress_chunks(
+        ctypes.addressof(kw.get("desc", d)), kw.get("kv", 4096), B._ptr(kw.get("ids", ids)), B._ptr(kw.get("bits", bits)),
+        2, kw.get("out", 8192), kw.get("out_bytes", 1 << 20), B._ptr(meta), kw.get("ws", 4096), kw.get("ws_bytes", 4096), None)
+    assert call() == B.ERR_INVALID_ARG                                   # duplicate chunk id
+    ok_ids = np.array([1, 2], dtype=np.uint32)
+    assert call(ids=np.array([1, 16], dtype=np.uint32)) == B.ERR_INVALID_ARG   # id out of range
+    assert call(ids=ok_ids, bits=np.array([8, 5], dtype=np.uint8)) == B.ERR_BAD_BITS
+    assert call(ids=ok_ids, kv=4098) == B.ERR_MISALIGNED
+    assert call(ids=ok_ids, out=8192 + 64) == B.ERR_MISALIGNED
+    assert call(ids=ok_ids, out_bytes=8704) == B.ERR_BUF_TOO_SMALL        # needs 8704 + 4608
+    assert call(ids=ok_ids, ws_bytes=32) == B.ERR_BUF_TOO_SMALL
+    d2 = B.desc_of(sh)
+    d2.group_size = 48                                                      # divides 96 but is not a power of two
+    d2.head_dim = 96
+    assert call(ids=ok_ids, desc=d2) == B.ERR_UNSUPPORTED
+    assert B.lib().llms_wait(None, 1) == B.ERR_INVALID_ARG
+    assert B.lib().llms_strerror(B.ERR_CORRUPT).decode() == "record checksum mismatch"

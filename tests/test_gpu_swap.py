@@ -1,0 +1,97 @@
+"""Swap copies over pinned host memory on a side stream: byte equality, checksums, events, the bounded wait."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2403_11805_b200 import binding as B, synth
+from gpu_helpers import bits_view, first_mismatch, odesc
+
+pytestmark = pytest.mark.gpu
+
+
+def test_round_trip_through_pinned_memory_matches_oracle():
+    sh = synth.CONFIGS["llama7b"].with_(n_layers=2, n_tokens=512)
+    kv = synth.kv_tensor(sh)
+    kv_dev = kv.cuda()
+    n = sh.n_chunks
+    ids = np.arange(n, dtype=np.uint32)
+    bits = np.array([(8, 4, 2)[i % 3] for i in range(n)], dtype=np.uint8)
+    d = B.desc_of(sh)
+    total = B.compressed_size(d, bits)
+    main, side = torch.cuda.current_stream(), torch.cuda.Stream()
+    buf = torch.empty(total, dtype=torch.uint8, device="cuda")
+    back = torch.zeros(total, dtype=torch.uint8, device="cuda")
+    arena = torch.zeros(total, dtype=torch.uint8).pin_memory()
+    meta = B.new_meta(n, pinned=True)
+    ws = torch.empty(B.codec_workspace_bytes(n), dtype=torch.uint8, device="cuda")
+    compressed, out_done, in_done = B.new_event(), B.new_event(), B.new_event()
+    B.compress_chunks(d, kv_dev, ids, bits, buf, meta, ws)
+    compressed.record(main)
+    torch.cuda.synchronize()     # meta (sizes) is final; checksums too
+    B.swap_out(buf, meta, arena, side_stream=side, after=compressed, done=out_done)
+    B.swap_in(arena, meta, back, side_stream=side, done=in_done)
+    main.wait_event(in_done)
+    out = torch.zeros_like(kv_dev)
+    B.decompress_chunks(d, back, meta, None, out, ws)
+    B.wait(in_done, 10000)
+    assert B.codec_corrupt_count(ws) == 0
+    want_buf, want_meta = oracle.compress_chunks(odesc(sh), bits_view(kv), ids, bits)
+    assert first_mismatch(arena.numpy(), want_buf) is None
+    for i in range(n):
+        rec = arena.numpy()[int(meta[i]["offset"]):int(meta[i]["offset"] + meta[i]["nbytes"])]
+        assert oracle.checksum(rec) == meta[i]["checksum"] == want_meta[i]["checksum"]
+    want = np.zeros(kv.numel(), dtype=np.uint16).reshape(kv.shape)
+    oracle.decompress_chunks(odesc(sh), want_buf, want_meta, want)
+    assert first_mismatch(bits_view(out).reshape(-1), want.reshape(-1)) is None
+
+
+def test_scattered_host_offsets():
+    sh = synth.CONFIGS["tiny"]
+    kv_dev = synth.kv_tensor(sh).cuda()
+    ids = np.array([3, 4, 9], dtype=np.uint32)
+    bits = np.array([8, 2, 4], dtype=np.uint8)
+    d = B.desc_of(sh)
+    total = B.compressed_size(d, bits)
+    buf = torch.empty(total, dtype=torch.uint8, device="cuda")
+    meta = B.new_meta(3, pinned=True)
+    ws = torch.empty(B.codec_workspace_bytes(3), dtype=torch.uint8, device="cuda")
+    B.compress_chunks(d, kv_dev, ids, bits, buf, meta, ws)
+    torch.cuda.synchronize()
+    arena = torch.full((65536,), 0x5A, dtype=torch.uint8).pin_memory()
+    offs = np.array([40960, 0, 16384], dtype=np.uint64)
+    side = torch.cuda.Stream()
+    done = B.new_event()
+    B.swap_out(buf, meta, arena, host_offsets=offs, side_stream=side, done=done)
+    B.wait(done)
+    host = buf.cpu().numpy()
+    used = np.zeros(65536, dtype=bool)
+    for i in range(3):
+        o, nb, ho = int(meta[i]["offset"]), int(meta[i]["nbytes"]), int(offs[i])
+        assert np.array_equal(arena.numpy()[ho:ho + nb], host[o:o + nb])
+        used[ho:ho + nb] = True
+    assert (arena.numpy()[~used] == 0x5A).all()
+    back = torch.zeros(total, dtype=torch.uint8, device="cuda")
+    B.swap_in(arena, meta, back, host_offsets=offs, side_stream=side, done=done)
+    B.wait(done)
+    assert torch.equal(back, buf)
+
+
+def test_wait_times_out_and_then_succeeds():
+    side = torch.cuda.Stream()
+    ev = B.new_event(side)
+    with torch.cuda.stream(side):
+        torch.cuda._sleep(int(1.0e9))       # a bounded spin of about half a second
+        ev.record(side)
+    with pytest.raises(B.LlmsError) as e:
+        B.wait(ev, 5)
+    assert e.value.status == B.ERR_TIMEOUT
+    B.wait(ev, 20000)
+
+
+def test_swap_argument_errors():
+    meta = B.new_meta(1)
+    meta[0]["nbytes"] = 100          # not a multiple of 256
+    assert B.lib().llms_swap_out(4096, meta.ctypes.data, 1, 8192, None, None, None, None) == B.ERR_MISALIGNED
+    assert B.lib().llms_swap_out(None, meta.ctypes.data, 1, 8192, None, None, None, None) == B.ERR_INVALID_ARG
+    assert B.lib().llms_swap_in(4096, None, meta.ctypes.data, 0, 8192, None, None, None) == B.OK
