@@ -244,6 +244,7 @@ def run_ours(args):
         B.compress_chunks(d, kv, ids, bits, buf, meta, ws)
         if ev:
             ev[2].record(stream)
+        stream.synchronize()                     # the records' checksums reach the host-side meta here
         B.decompress_chunks(d, buf, meta, None, kv_out, ws)
         if ev:
             ev[3].record(stream)
