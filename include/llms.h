@@ -133,6 +133,24 @@ int llms_compress_chunks(const llms_kv_desc *desc, const void *kv, const uint32_
                          const uint8_t *bits, int n, void *out_buf, uint64_t out_bytes,
                          llms_chunk_meta *meta, void *workspace, uint64_t workspace_bytes, void *stream);
 
+/* llms_compress_chunks without a workspace argument, for callers that cannot obtain device scratch:
+ * a service that handed all device memory to its KV pool at start-up (an allocation would fail, or
+ * would stall inference because cudaMalloc synchronises the device), or code running where the CUDA
+ * allocator must not be entered at all.  The paper has no counterpart to this call; it is a
+ * convenience of this library.  The chunk table lives in a fixed array inside the library image
+ * (about 37 KB, present on every GPU that loads the library until the process exits), which limits
+ * one call to LLMS_STATIC_MAX_CHUNKS chunks: a larger n returns LLMS_ERR_BUF_TOO_SMALL and nothing
+ * is launched.  No device memory is allocated or freed.  All other arguments, results and errors
+ * are those of llms_compress_chunks.
+ * The first call on each device looks up the array's device address (with that device current);
+ * make that first call outside of any stream capture.  Every call on a device uses the same array
+ * and overwrites what the previous call left in it, so two calls whose GPU work may overlap (different
+ * streams, different threads) race on it: order them on one stream or with events. */
+#define LLMS_STATIC_MAX_CHUNKS 1024
+int llms_compress_chunks_static(const llms_kv_desc *desc, const void *kv, const uint32_t *chunk_ids,
+                                const uint8_t *bits, int n, void *out_buf, uint64_t out_bytes,
+                                llms_chunk_meta *meta, void *stream);
+
 /* ------------------------------------------------------------------ swap-in: unpack + dequantize */
 
 /* Load's decompression half.  Record i (meta[i], inside `buf`) is decoded into chunk slot

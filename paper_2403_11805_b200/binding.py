@@ -48,6 +48,8 @@ _SIGNATURES = {
     "llms_codec_workspace_bytes": (C.c_int, [C.c_int, C.c_void_p]),
     "llms_compress_chunks": (C.c_int, [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_int, C.c_void_p,
                                        C.c_uint64, C.c_void_p, C.c_void_p, C.c_uint64, C.c_void_p]),
+    "llms_compress_chunks_static": (C.c_int, [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_int, C.c_void_p,
+                                              C.c_uint64, C.c_void_p, C.c_void_p]),
     "llms_decompress_chunks": (C.c_int, [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_int, C.c_void_p,
                                          C.c_void_p, C.c_uint64, C.c_void_p]),
     "llms_codec_corrupt_count": (C.c_int, [C.c_void_p, C.c_void_p, C.c_void_p]),
@@ -202,6 +204,19 @@ def compress_chunks(desc, kv, chunk_ids, bits, out_buf, meta, workspace, stream=
         C.addressof(desc), _ptr(kv), _ptr(chunk_ids), _ptr(bits), len(bits), _ptr(out_buf),
         _nbytes(out_buf) if out_bytes is None else out_bytes, _ptr(meta), _ptr(workspace),
         _nbytes(workspace) if workspace_bytes is None else workspace_bytes, _stream(stream)), "llms_compress_chunks")
+
+
+STATIC_MAX_CHUNKS = 1024
+
+
+def compress_chunks_static(desc, kv, chunk_ids, bits, out_buf, meta, stream=None, out_bytes=None):
+    """llms_compress_chunks_static: same as compress_chunks, scratch built into the library (<= 1024 chunks)."""
+    chunk_ids = np.ascontiguousarray(chunk_ids, dtype=np.uint32)
+    bits = np.ascontiguousarray(bits, dtype=np.uint8)
+    assert len(chunk_ids) == len(bits) and len(meta) >= len(bits)
+    _check(lib().llms_compress_chunks_static(
+        C.addressof(desc), _ptr(kv), _ptr(chunk_ids), _ptr(bits), len(bits), _ptr(out_buf),
+        _nbytes(out_buf) if out_bytes is None else out_bytes, _ptr(meta), _stream(stream)), "llms_compress_chunks_static")
 
 
 def decompress_chunks(desc, buf, meta, dst_chunk_ids, kv_out, workspace, stream=None, n=None, workspace_bytes=None):

@@ -419,3 +419,46 @@ extern "C" int llms_codec_corrupt_count(const void *workspace, uint32_t *n_corru
     if (n_corrupt) *n_corrupt = bad;
     return bad ? LLMS_ERR_CORRUPT : LLMS_OK;
 }
+
+// ---------------------------------------------------------------------------------------------- no-allocation variant
+
+namespace llms {
+
+constexpr uint64_t kStaticWorkspaceBytes =
+    (kWsEntriesOffset + (uint64_t)LLMS_STATIC_MAX_CHUNKS * (sizeof(ChunkEntry) + 4) + 255) / 256 * 256;
+
+// Scratch of llms_compress_chunks_static: lives in the library image, one copy on every GPU that loads it.
+static __device__ __align__(256) unsigned char g_static_workspace[kStaticWorkspaceBytes];
+
+// Device address of the array above, looked up once per device.  (In host code the array's name is only a handle
+// for the runtime; the address a kernel can use has to be asked for.)
+static int static_workspace_address(void **out)
+{
+    static void *cached[64] = {nullptr};
+    int dev = -1;
+    LLMS_CUDA_TRY(cudaGetDevice(&dev));
+    if (dev < 0 || dev >= 64) return LLMS_ERR_UNSUPPORTED;
+    if (cached[dev] == nullptr) {
+        void *p = nullptr;
+        LLMS_CUDA_TRY(cudaGetSymbolAddress(&p, g_static_workspace));
+        if (p == nullptr) return LLMS_ERR_CUDA;
+        cached[dev] = p;  // two threads racing here store the same value
+    }
+    *out = cached[dev];
+    return LLMS_OK;
+}
+
+}  // namespace llms
+
+extern "C" int llms_compress_chunks_static(const llms_kv_desc *desc, const void *kv, const uint32_t *chunk_ids,
+                                           const uint8_t *bits, int n, void *out_buf, uint64_t out_bytes,
+                                           llms_chunk_meta *meta, void *stream)
+{
+    if (n > LLMS_STATIC_MAX_CHUNKS) return LLMS_ERR_BUF_TOO_SMALL;  // the built-in scratch holds no more entries
+    void *ws = nullptr;
+    const int rc = static_workspace_address(&ws);
+    if (rc) return rc;
+    // The chunk table copied in by the call below carries zeroed checksum fields, which is all of the
+    // scratch that has to start from zero; whatever the previous call left behind is overwritten.
+    return llms_compress_chunks(desc, kv, chunk_ids, bits, n, out_buf, out_bytes, meta, ws, kStaticWorkspaceBytes, stream);
+}
