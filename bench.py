@@ -360,7 +360,7 @@ def run_ours(args):
                 "ms_per_step": e2e_ms, "context_switches_per_s": world / (e2e_ms * 1e-3),
                 "host_copy_gbs_each_way": None,
                 "what": "compress -> swap-out to pinned host -> swap-in -> decompress"},
-        "gpu_launches": args.steps * 7,
+        "gpu_launches": args.steps * 11,   # 4 score kernels, compress and decompress once per bit-width, 1 verify
         "roofline": roofline, "clocks": clocks,
         "wall_ms_per_step": t_wall * 1e3 / args.steps,
     }

@@ -1,13 +1,16 @@
 // Chunk codec kernels for sm_100a: group quantize + bit-pack (swap-out) and unpack + dequantize (swap-in).
 //
-// Work item = one slab (chunk_len*head_dim contiguous fp16 of one chunk, layer, K/V, head).  One warp
-// takes a slab at a time from a persistent grid.  A lane owns 16 consecutive elements (32 bytes of
-// fp16), so a group of G channels is G/16 neighbouring lanes: min/max take log2(G/16) xor-shuffles,
-// a lane's packed codes are 4/8/16 contiguous bytes at 2/4/8 bits, and the warp's stores are contiguous.
-// The bit-width is uniform per chunk, hence per warp.
+// Work unit = one warp pass over a slab (chunk_len*head_dim contiguous fp16 of one chunk, layer, K/V, head):
+// 2048 elements, a lane owning 64 consecutive ones as four 32-byte pieces.  A group of G >= 64 channels is
+// G/64 neighbouring lanes (min/max by xor-shuffles on a packed (min, -max) half2); smaller groups sit inside
+// a lane.  A lane's packed codes are 16/32/64 contiguous bytes at 2/4/8 bits, so every access of the warp is
+// made of whole 32-byte sectors.  Warps of a persistent grid walk the units with a stride; the loads of the
+// next unit are issued before the current one is computed (two register buffers), which keeps 128 bytes per
+// lane in flight all the time.  The bit-width is uniform per chunk, hence per warp.
 //
-// The arithmetic is fixed by the record format (see llms.h): every binary32 operation is written with a
-// round-to-nearest intrinsic so that nothing is contracted into an FMA or replaced by an approximation.
+// The arithmetic is fixed by the record format (see llms.h): every binary32 operation is a single IEEE
+// round-to-nearest operation (intrinsics, or sm_100 mixed-precision PTX whose fp16 inputs convert exactly),
+// nothing is contracted or approximated.
 #include <vector>
 
 #include "llms_internal.cuh"
@@ -16,27 +19,51 @@ namespace llms {
 
 constexpr int kWarpsPerBlock = 8;
 constexpr int kThreads = kWarpsPerBlock * 32;
-constexpr int kElemsPerLane = 16;
-constexpr int kElemsPerWarpIter = 32 * kElemsPerLane;  // 512 elements = 1 KiB of fp16
-constexpr int kUnroll = 4;                             // warp passes whose loads are issued together
+constexpr int kPieceElems = 16;                 // one 32-byte access
+constexpr int kPieces = 4;                      // pieces per lane per pass
+constexpr int kLaneElems = kPieces * kPieceElems;
+constexpr int kPassElems = 32 * kLaneElems;     // 2048 elements = 4 KiB of fp16
 
 struct CodecArgs {
     const __half *kv_in;   // compress: source
     __half *kv_out;        // decompress: destination
     uint8_t *buf;          // swap buffer (written by compress, read by decompress)
-    ChunkEntry *entries;   // n entries in the workspace
+    ChunkEntry *entries;   // n entries in the workspace (caller's order)
     uint32_t *sums;        // decompress: recomputed checksums
-    int n;
+    const uint32_t *order; // entry indices grouped by bit-width; this launch covers order[0 .. n)
+    int n;                 // chunks of this launch (all of one bit-width)
     int n_slabs;           // slabs per chunk
     int slab_elems;        // chunk_len * head_dim
     int groups_per_slab;
     int n_kv_heads;
-    int slab_major;        // 1: consecutive work items walk the listed chunks of one slab index (linear KV addresses
-                           //    when the ids are consecutive); 0: they walk the slabs of one chunk (linear record addresses)
+    int passes;            // warp passes per slab
+    uint32_t total_units;  // n * n_slabs * passes
     uint32_t codes_off;    // byte offset of the code stream in a record
     uint32_t params_bytes; // 4 * n_groups
     int64_t stride_l, stride_s, stride_h, chunk_stride;
 };
+
+// Where a unit's data is.  Units are numbered slab-major: consecutive units walk the passes of a slab, then
+// the listed chunks of one slab index, so KV addresses run linearly when the chunk ids are consecutive
+// (measured: faster than walking the slabs of one chunk, which makes the record addresses linear instead).
+struct UnitPos {
+    uint32_t i, s_idx, chunk_id, bits;
+    uint64_t rec_off;
+    int e0;                // first element of this lane inside the slab
+};
+
+__device__ __forceinline__ void decode_unit(const CodecArgs &a, uint32_t unit, int lane, UnitPos &u)
+{
+    const uint32_t item = unit / (uint32_t)a.passes;
+    const uint32_t pass = unit - item * (uint32_t)a.passes;
+    u.s_idx = item / (uint32_t)a.n;
+    u.i = a.order[item - u.s_idx * (uint32_t)a.n];
+    const uint4 head = *reinterpret_cast<const uint4 *>(a.entries + u.i);  // chunk_id, bits, offset
+    u.chunk_id = head.x;
+    u.bits = head.y;
+    u.rec_off = (uint64_t)head.z | ((uint64_t)head.w << 32);
+    u.e0 = (int)pass * kPassElems + lane * kLaneElems;
+}
 
 __device__ __forceinline__ int64_t slab_offset(const CodecArgs &a, uint32_t s_idx, uint32_t chunk)
 {
@@ -46,22 +73,31 @@ __device__ __forceinline__ int64_t slab_offset(const CodecArgs &a, uint32_t s_id
            (int64_t)chunk * a.chunk_stride;
 }
 
-__device__ __forceinline__ void item_to_chunk_slab(const CodecArgs &a, uint32_t item, uint32_t &i, uint32_t &s_idx)
-{
-    if (a.slab_major) {
-        s_idx = item / (uint32_t)a.n;
-        i = item - s_idx * (uint32_t)a.n;
-    } else {
-        i = item / (uint32_t)a.n_slabs;
-        s_idx = item - i * (uint32_t)a.n_slabs;
-    }
-}
-
 __device__ __forceinline__ __half2 as_h2(uint32_t u) { return *reinterpret_cast<__half2 *>(&u); }
 __device__ __forceinline__ uint32_t as_u32(__half2 h) { return *reinterpret_cast<uint32_t *>(&h); }
 
-// 32 bytes per lane.  WIDE: one 256-bit access (needs 32-byte alignment); otherwise two 128-bit accesses.
-// Data touched once: no L1 allocation.
+__device__ __forceinline__ void split_halves(uint32_t w, unsigned short &lo, unsigned short &hi)
+{
+    asm("mov.b32 {%0, %1}, %2;" : "=h"(lo), "=h"(hi) : "r"(w));
+}
+
+// fp32(x) + c with one rounding; x is an fp16 bit pattern (converts exactly)
+__device__ __forceinline__ float add_f32_f16(unsigned short x, float c)
+{
+    float d;
+    asm("add.rn.f32.f16 %0, %1, %2;" : "=f"(d) : "h"(x), "f"(c));
+    return d;
+}
+
+// fp32(a) * fp32(b) + c with one rounding; a, b are fp16 bit patterns
+__device__ __forceinline__ float fma_f32_f16(unsigned short x, unsigned short y, float c)
+{
+    float d;
+    asm("fma.rn.f32.f16 %0, %1, %2, %3;" : "=f"(d) : "h"(x), "h"(y), "f"(c));
+    return d;
+}
+
+// Global accesses of data that is touched once: no L1 allocation.  WIDE: one 256-bit access (32-byte aligned).
 template <bool WIDE>
 __device__ __forceinline__ void load32(const void *p, uint32_t (&w)[8])
 {
@@ -77,20 +113,60 @@ __device__ __forceinline__ void load32(const void *p, uint32_t (&w)[8])
     }
 }
 
+__device__ __forceinline__ void st256(void *p, uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t a4,
+                                      uint32_t a5, uint32_t a6, uint32_t a7)
+{
+    asm volatile("st.global.L1::no_allocate.v8.b32 [%8], {%0,%1,%2,%3,%4,%5,%6,%7};"
+                 :: "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(a4), "r"(a5), "r"(a6), "r"(a7), "l"(p) : "memory");
+}
+__device__ __forceinline__ void st128(void *p, uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3)
+{
+    asm volatile("st.global.L1::no_allocate.v4.b32 [%4], {%0,%1,%2,%3};" :: "r"(a0), "r"(a1), "r"(a2), "r"(a3), "l"(p) : "memory");
+}
+__device__ __forceinline__ void st64(void *p, uint32_t a0, uint32_t a1)
+{
+    asm volatile("st.global.L1::no_allocate.v2.b32 [%2], {%0,%1};" :: "r"(a0), "r"(a1), "l"(p) : "memory");
+}
+__device__ __forceinline__ void st32(void *p, uint32_t a0)
+{
+    asm volatile("st.global.L1::no_allocate.b32 [%1], %0;" :: "r"(a0), "l"(p) : "memory");
+}
+__device__ __forceinline__ void ld256(const void *p, uint32_t *w)
+{
+    asm volatile("ld.global.nc.L1::no_allocate.v8.b32 {%0,%1,%2,%3,%4,%5,%6,%7}, [%8];"
+                 : "=r"(w[0]), "=r"(w[1]), "=r"(w[2]), "=r"(w[3]), "=r"(w[4]), "=r"(w[5]), "=r"(w[6]), "=r"(w[7]) : "l"(p));
+}
+__device__ __forceinline__ void ld128(const void *p, uint32_t *w)
+{
+    asm volatile("ld.global.nc.L1::no_allocate.v4.b32 {%0,%1,%2,%3}, [%4];" : "=r"(w[0]), "=r"(w[1]), "=r"(w[2]), "=r"(w[3]) : "l"(p));
+}
+__device__ __forceinline__ void ld64(const void *p, uint32_t *w)
+{
+    asm volatile("ld.global.nc.L1::no_allocate.v2.b32 {%0,%1}, [%2];" : "=r"(w[0]), "=r"(w[1]) : "l"(p));
+}
+__device__ __forceinline__ void ld32(const void *p, uint32_t *w)
+{
+    asm volatile("ld.global.nc.L1::no_allocate.b32 %0, [%1];" : "=r"(w[0]) : "l"(p));
+}
+
 template <bool WIDE>
 __device__ __forceinline__ void store32(void *p, const uint32_t (&w)[8])
 {
     if constexpr (WIDE) {
-        asm volatile("st.global.L1::no_allocate.v8.b32 [%8], {%0,%1,%2,%3,%4,%5,%6,%7};"
-                     :: "r"(w[0]), "r"(w[1]), "r"(w[2]), "r"(w[3]), "r"(w[4]), "r"(w[5]), "r"(w[6]), "r"(w[7]), "l"(p)
-                     : "memory");
+        st256(p, w[0], w[1], w[2], w[3], w[4], w[5], w[6], w[7]);
     } else {
-        asm volatile("st.global.L1::no_allocate.v4.b32 [%4], {%0,%1,%2,%3};"
-                     :: "r"(w[0]), "r"(w[1]), "r"(w[2]), "r"(w[3]), "l"(p) : "memory");
-        asm volatile("st.global.L1::no_allocate.v4.b32 [%4], {%0,%1,%2,%3};"
-                     :: "r"(w[4]), "r"(w[5]), "r"(w[6]), "r"(w[7]), "l"(static_cast<char *>(p) + 16) : "memory");
+        st128(p, w[0], w[1], w[2], w[3]);
+        st128(static_cast<char *>(p) + 16, w[4], w[5], w[6], w[7]);
     }
 }
+
+// Group geometry for a lane that owns 64 consecutive elements.
+template <int G>
+struct Geo {
+    static constexpr int kLanesPerGroup = G >= kLaneElems ? G / kLaneElems : 1;
+    static constexpr int kGroupsPerLane = G >= kLaneElems ? 1 : kLaneElems / G;
+    static constexpr int kPiecesPerGroup = kPieces / kGroupsPerLane;
+};
 
 // ---------------------------------------------------------------------------------------------- quantize
 
@@ -98,25 +174,58 @@ __device__ __forceinline__ void store32(void *p, const uint32_t (&w)[8])
 // low mantissa bits: bits = 0x4B400000 + q.
 constexpr float kRoundMagic = 12582912.0f;
 constexpr uint32_t kRoundMagicBits = 0x4B400000u;
+constexpr float kMinNormalHalf = 6.103515625e-05f;
 
-// Quantize the lane's 16 values and pack them into BITS/2 words.  CLAMP is only needed when the scale is a
-// subnormal fp16 number: otherwise (x - zero) / scale cannot reach 2^BITS - 1/2.
-template <int BITS, bool CLAMP>
-__device__ __forceinline__ void quantize_pack16(const uint32_t (&w)[8], float zero, float inv, uint32_t (&out)[BITS / 2])
+struct GroupParams {
+    float neg_zero_point;  // -(minimum)
+    float inv;             // 1 / scale, or 0 when scale == 0 (every code becomes 0)
+    uint32_t word;         // scale bits | zero-point bits << 16
+    bool needs_clamp;      // scale is a subnormal fp16 number (or 0): (x - zero)/scale may pass 2^b - 1
+};
+
+// mm = (min, -max) of a group
+template <int BITS>
+__device__ __forceinline__ GroupParams group_params(__half2 mm)
 {
     constexpr float kQmax = (float)((1 << BITS) - 1);
+    // adding +0 turns a -0 minimum or maximum into +0 and changes nothing else
+    const float zero = __fadd_rn(__low2float(mm), 0.0f);
+    const float top = __fadd_rn(-__high2float(mm), 0.0f);
+    const __half scale_h = __float2half_rn(__fdiv_rn(__fsub_rn(top, zero), kQmax));
+    const float scale = __half2float(scale_h);
+    GroupParams g;
+    g.neg_zero_point = -zero;
+    g.inv = scale == 0.0f ? 0.0f : __frcp_rn(scale);
+    g.word = (uint32_t)__half_as_ushort(scale_h) | ((uint32_t)__half_as_ushort(__float2half_rn(zero)) << 16);
+    g.needs_clamp = scale < kMinNormalHalf;
+    return g;
+}
+
+// min and max of 16 values as two half2 (element-wise over the pairs)
+__device__ __forceinline__ void piece_minmax(const uint32_t (&w)[8], __half2 &mn2, __half2 &mx2)
+{
+    mn2 = as_h2(w[0]);
+    mx2 = as_h2(w[0]);
+#pragma unroll
+    for (int k = 1; k < 8; ++k) {
+        mn2 = __hmin2(mn2, as_h2(w[k]));
+        mx2 = __hmax2(mx2, as_h2(w[k]));
+    }
+}
+
+// Quantize 16 values and pack them into BITS/2 words.  No clamp: only valid when the scale is a normal fp16
+// number, where (x - zero) / scale stays below 2^BITS - 1/2.
+template <int BITS>
+__device__ __forceinline__ void quantize_piece(const uint32_t (&w)[8], float neg_zero, float inv, uint32_t (&out)[BITS / 2])
+{
     uint32_t t[16];
 #pragma unroll
     for (int k = 0; k < 8; ++k) {
-        const float2 f = __half22float2(as_h2(w[k]));
-        float v0 = __fmul_rn(__fsub_rn(f.x, zero), inv);  // >= 0: zero is the minimum
-        float v1 = __fmul_rn(__fsub_rn(f.y, zero), inv);
-        if constexpr (CLAMP) {
-            v0 = fminf(v0, kQmax);
-            v1 = fminf(v1, kQmax);
-        }
-        t[2 * k] = __float_as_uint(__fadd_rn(v0, kRoundMagic));
-        t[2 * k + 1] = __float_as_uint(__fadd_rn(v1, kRoundMagic));
+        unsigned short lo, hi;
+        split_halves(w[k], lo, hi);
+        // (x - zero) * inv, two roundings; >= 0 because zero is the minimum
+        t[2 * k] = __float_as_uint(__fadd_rn(__fmul_rn(add_f32_f16(lo, neg_zero), inv), kRoundMagic));
+        t[2 * k + 1] = __float_as_uint(__fadd_rn(__fmul_rn(add_f32_f16(hi, neg_zero), inv), kRoundMagic));
     }
     if constexpr (BITS == 8) {
 #pragma unroll
@@ -142,74 +251,112 @@ __device__ __forceinline__ void quantize_pack16(const uint32_t (&w)[8], float ze
     }
 }
 
-template <int BITS>
-__device__ __forceinline__ void store_codes(uint8_t *p, const uint32_t (&c)[BITS / 2])
+// The rare case (subnormal scale): same arithmetic plus the clamp, written for size, not speed.
+__device__ __noinline__ void quantize_piece_clamped(const uint32_t *w, float neg_zero, float inv, int bits, uint32_t *out)
 {
-    if constexpr (BITS == 8)
-        asm volatile("st.global.L1::no_allocate.v4.b32 [%4], {%0,%1,%2,%3};" :: "r"(c[0]), "r"(c[1]), "r"(c[2]), "r"(c[3]), "l"(p) : "memory");
-    else if constexpr (BITS == 4)
-        asm volatile("st.global.L1::no_allocate.v2.b32 [%2], {%0,%1};" :: "r"(c[0]), "r"(c[1]), "l"(p) : "memory");
-    else
-        asm volatile("st.global.L1::no_allocate.b32 [%1], %0;" :: "r"(c[0]), "l"(p) : "memory");
+    const float qmax = (float)((1 << bits) - 1);
+    for (int j = 0; j < bits / 2; ++j) out[j] = 0;
+    for (int k = 0; k < 16; ++k) {
+        const unsigned short x = (unsigned short)(w[k >> 1] >> ((k & 1) * 16));
+        const float v = fminf(__fmul_rn(add_f32_f16(x, neg_zero), inv), qmax);
+        const uint32_t q = (uint32_t)__float2int_rn(v);
+        out[(k * bits) >> 5] |= q << ((k * bits) & 31);
+    }
 }
 
-// One slab by one warp.  Returns this lane's share of the checksum.
-template <int BITS, int LPG, bool WIDE>
-__device__ __forceinline__ uint32_t compress_slab(const CodecArgs &a, const __half *__restrict__ src, uint8_t *__restrict__ rec,
-                                                  uint32_t s_idx, int lane)
+template <int BITS, int G, bool WIDE>
+__device__ __forceinline__ uint32_t compress_unit_bits(const CodecArgs &a, const UnitPos &u, const uint32_t (&w)[kPieces][8],
+                                                       uint8_t *__restrict__ rec, int lane)
 {
-    constexpr float kQmax = (float)((1 << BITS) - 1);
-    constexpr int kLaneBytes = kElemsPerLane * BITS / 8;
-    uint32_t *params = reinterpret_cast<uint32_t *>(rec) + (uint64_t)s_idx * a.groups_per_slab;
-    uint8_t *codes = rec + a.codes_off + (uint64_t)s_idx * a.slab_elems * BITS / 8;
-    uint32_t sum = 0;
-    for (int base = 0; base < a.slab_elems; base += kUnroll * kElemsPerWarpIter) {
-        uint32_t w[kUnroll][8];
+    using geo = Geo<G>;
+    constexpr int kPieceBytes = kPieceElems * BITS / 8;
+    // ---- group minima and maxima
+    GroupParams gp[geo::kGroupsPerLane];
+    {
+        __half2 mn2[kPieces], mx2[kPieces];
 #pragma unroll
-        for (int u = 0; u < kUnroll; ++u) {  // all loads of the block first: 128 bytes in flight per lane
-            const int e0 = base + u * kElemsPerWarpIter + lane * kElemsPerLane;
-            if (e0 < a.slab_elems) {
-                load32<WIDE>(src + e0, w[u]);
-            } else {
+        for (int j = 0; j < kPieces; ++j) piece_minmax(w[j], mn2[j], mx2[j]);
 #pragma unroll
-                for (int k = 0; k < 8; ++k) w[u][k] = 0;  // inactive lanes form whole inactive groups
-            }
-        }
+        for (int g = 0; g < geo::kGroupsPerLane; ++g) {
+            __half2 mn = mn2[g * geo::kPiecesPerGroup], mx = mx2[g * geo::kPiecesPerGroup];
 #pragma unroll
-        for (int u = 0; u < kUnroll; ++u) {
-            const int e0 = base + u * kElemsPerWarpIter + lane * kElemsPerLane;
-            if (base + u * kElemsPerWarpIter >= a.slab_elems) break;  // warp-uniform
-            const bool active = e0 < a.slab_elems;
-            // min and max of the lane's 16 values, two at a time
-            __half2 mn2 = as_h2(w[u][0]), mx2 = as_h2(w[u][0]);
-#pragma unroll
-            for (int k = 1; k < 8; ++k) {
-                mn2 = __hmin2(mn2, as_h2(w[u][k]));
-                mx2 = __hmax2(mx2, as_h2(w[u][k]));
+            for (int j = 1; j < geo::kPiecesPerGroup; ++j) {
+                mn = __hmin2(mn, mn2[g * geo::kPiecesPerGroup + j]);
+                mx = __hmax2(mx, mx2[g * geo::kPiecesPerGroup + j]);
             }
             // (min, -max) in one register: a single min per shuffle step reduces both
-            __half2 mm = __halves2half2(__hmin(__low2half(mn2), __high2half(mn2)),
-                                        __hneg(__hmax(__low2half(mx2), __high2half(mx2))));
+            __half2 mm = __halves2half2(__hmin(__low2half(mn), __high2half(mn)), __hneg(__hmax(__low2half(mx), __high2half(mx))));
 #pragma unroll
-            for (int m = LPG / 2; m > 0; m >>= 1) mm = __hmin2(mm, as_h2(__shfl_xor_sync(0xffffffffu, as_u32(mm), m)));
-            // adding +0 turns a -0 minimum or maximum into +0 and changes nothing else
-            const float zero = __fadd_rn(__low2float(mm), 0.0f);
-            const float top = __fadd_rn(-__high2float(mm), 0.0f);
-            const __half scale_h = __float2half_rn(__fdiv_rn(__fsub_rn(top, zero), kQmax));
-            const float scale = __half2float(scale_h);
-            const float inv = scale == 0.0f ? 0.0f : __frcp_rn(scale);  // inv = 0 makes every code 0
-            uint32_t c[BITS / 2];
-            if (__any_sync(0xffffffffu, scale < 6.103515625e-05f)) quantize_pack16<BITS, true>(w[u], zero, inv, c);
-            else quantize_pack16<BITS, false>(w[u], zero, inv, c);
-            if (active) {
-                store_codes<BITS>(codes + (uint32_t)(e0 / kElemsPerLane) * kLaneBytes, c);
+            for (int m = geo::kLanesPerGroup / 2; m > 0; m >>= 1)
+                mm = __hmin2(mm, as_h2(__shfl_xor_sync(0xffffffffu, as_u32(mm), m)));
+            gp[g] = group_params<BITS>(mm);
+        }
+    }
+    // ---- codes
+    uint32_t c[kPieces][BITS / 2];
+    bool any_clamp = false;
 #pragma unroll
-                for (int j = 0; j < BITS / 2; ++j) sum += c[j];
-                if ((lane & (LPG - 1)) == 0) {
-                    const uint32_t p = (uint32_t)__half_as_ushort(scale_h) | ((uint32_t)__half_as_ushort(__float2half_rn(zero)) << 16);
-                    params[e0 / (kElemsPerLane * LPG)] = p;
-                    sum += p;
-                }
+    for (int g = 0; g < geo::kGroupsPerLane; ++g) any_clamp |= gp[g].needs_clamp;
+    if (__any_sync(0xffffffffu, any_clamp)) {
+#pragma unroll
+        for (int j = 0; j < kPieces; ++j) {
+            const GroupParams &g = gp[j / geo::kPiecesPerGroup];
+            uint32_t tmp_in[8], tmp_out[4];
+#pragma unroll
+            for (int k = 0; k < 8; ++k) tmp_in[k] = w[j][k];
+            quantize_piece_clamped(tmp_in, g.neg_zero_point, g.inv, BITS, tmp_out);
+#pragma unroll
+            for (int k = 0; k < BITS / 2; ++k) c[j][k] = tmp_out[k];
+        }
+    } else {
+#pragma unroll
+        for (int j = 0; j < kPieces; ++j) {
+            const GroupParams &g = gp[j / geo::kPiecesPerGroup];
+            quantize_piece<BITS>(w[j], g.neg_zero_point, g.inv, c[j]);
+        }
+    }
+    // ---- stores
+    uint8_t *codes = rec + a.codes_off + (uint64_t)u.s_idx * a.slab_elems * BITS / 8 + (uint32_t)u.e0 * BITS / 8;
+    uint32_t *params = reinterpret_cast<uint32_t *>(rec) + (uint64_t)u.s_idx * a.groups_per_slab + (uint32_t)u.e0 / G;
+    uint32_t sum = 0;
+    const bool lane_full = u.e0 + kLaneElems <= a.slab_elems;
+    constexpr uintptr_t kLaneAlign = BITS == 2 ? 15 : 31;
+    if (lane_full && (reinterpret_cast<uintptr_t>(codes) & kLaneAlign) == 0) {
+        if constexpr (BITS == 8) {
+            st256(codes, c[0][0], c[0][1], c[0][2], c[0][3], c[1][0], c[1][1], c[1][2], c[1][3]);
+            st256(codes + 32, c[2][0], c[2][1], c[2][2], c[2][3], c[3][0], c[3][1], c[3][2], c[3][3]);
+        } else if constexpr (BITS == 4) {
+            st256(codes, c[0][0], c[0][1], c[1][0], c[1][1], c[2][0], c[2][1], c[3][0], c[3][1]);
+        } else {
+            st128(codes, c[0][0], c[1][0], c[2][0], c[3][0]);
+        }
+#pragma unroll
+        for (int j = 0; j < kPieces; ++j)
+#pragma unroll
+            for (int k = 0; k < BITS / 2; ++k) sum += c[j][k];
+    } else {
+#pragma unroll
+        for (int j = 0; j < kPieces; ++j) {
+            if (u.e0 + j * kPieceElems < a.slab_elems) {
+                if constexpr (BITS == 8) st128(codes + j * kPieceBytes, c[j][0], c[j][1], c[j][2], c[j][3]);
+                else if constexpr (BITS == 4) st64(codes + j * kPieceBytes, c[j][0], c[j][1]);
+                else st32(codes + j * kPieceBytes, c[j][0]);
+#pragma unroll
+                for (int k = 0; k < BITS / 2; ++k) sum += c[j][k];
+            }
+        }
+    }
+    if constexpr (geo::kGroupsPerLane == 1) {
+        if (u.e0 < a.slab_elems && (lane & (geo::kLanesPerGroup - 1)) == 0) {
+            st32(params, gp[0].word);
+            sum += gp[0].word;
+        }
+    } else {
+#pragma unroll
+        for (int g = 0; g < geo::kGroupsPerLane; ++g) {
+            if (u.e0 + g * G < a.slab_elems) {
+                st32(params + g, gp[g].word);
+                sum += gp[g].word;
             }
         }
     }
@@ -217,91 +364,169 @@ __device__ __forceinline__ uint32_t compress_slab(const CodecArgs &a, const __ha
 }
 
 // Zero the two padding runs of a record (after the parameter block, after the code stream).
-__device__ __forceinline__ void zero_padding(const CodecArgs &a, uint8_t *rec, const ChunkEntry &e, int lane)
+__device__ __forceinline__ void zero_padding(const CodecArgs &a, uint8_t *rec, uint32_t bits, int lane)
 {
-    for (uint32_t i = a.params_bytes + lane; i < a.codes_off; i += 32) rec[i] = 0;
-    const uint64_t codes_end = a.codes_off + (uint64_t)a.n_slabs * a.slab_elems * e.bits / 8;
-    for (uint64_t i = codes_end + lane; i < e.nbytes; i += 32) rec[i] = 0;
+    for (uint32_t k = a.params_bytes + lane; k < a.codes_off; k += 32) rec[k] = 0;
+    const uint64_t codes_end = a.codes_off + (uint64_t)a.n_slabs * a.slab_elems * bits / 8;
+    const uint64_t nbytes = (codes_end + 255) / 256 * 256;
+    for (uint64_t k = codes_end + lane; k < nbytes; k += 32) rec[k] = 0;
 }
 
-__device__ __forceinline__ ChunkEntry load_entry(const ChunkEntry *p)
+template <bool WIDE>
+__device__ __forceinline__ void load_unit(const CodecArgs &a, const UnitPos &u, uint32_t (&w)[kPieces][8])
 {
-    const uint4 lo = *reinterpret_cast<const uint4 *>(p);
-    const uint4 hi = *(reinterpret_cast<const uint4 *>(p) + 1);
-    ChunkEntry e;
-    e.chunk_id = lo.x; e.bits = lo.y;
-    e.offset = (uint64_t)lo.z | ((uint64_t)lo.w << 32);
-    e.nbytes = (uint64_t)hi.x | ((uint64_t)hi.y << 32);
-    e.n_groups = hi.z; e.checksum = hi.w;
-    return e;
+    const __half *src = a.kv_in + slab_offset(a, u.s_idx, u.chunk_id) + u.e0;
+#pragma unroll
+    for (int j = 0; j < kPieces; ++j) {
+        if (u.e0 + j * kPieceElems < a.slab_elems) {
+            load32<WIDE>(src + j * kPieceElems, w[j]);
+        } else {
+#pragma unroll
+            for (int k = 0; k < 8; ++k) w[j][k] = 0;  // pieces past the end form whole inactive groups
+        }
+    }
 }
 
-template <int LPG, bool WIDE>
-__global__ void __launch_bounds__(kThreads) compress_kernel(const CodecArgs a)
+template <int BITS, int G, bool WIDE>
+__device__ __forceinline__ void compress_unit(const CodecArgs &a, const UnitPos &u, const uint32_t (&w)[kPieces][8], int lane)
+{
+    uint8_t *rec = a.buf + u.rec_off;
+    uint32_t sum = compress_unit_bits<BITS, G, WIDE>(a, u, w, rec, lane);
+    if (u.s_idx == 0 && u.e0 < kPassElems) zero_padding(a, rec, BITS, lane);  // first pass of the chunk's first slab
+    sum = __reduce_add_sync(0xffffffffu, sum);
+    if (lane == 0) atomicAdd(&a.entries[u.i].checksum, sum);
+}
+
+// One launch per bit-width present in the call: a single code path per kernel keeps the instruction
+// working set small (with all three widths in one kernel the warps stalled on instruction fetch).
+template <int BITS, int G, bool WIDE>
+__global__ void __launch_bounds__(kThreads, 2) compress_kernel(const CodecArgs a)
 {
     const int lane = threadIdx.x & 31;
-    const uint32_t warp = blockIdx.x * kWarpsPerBlock + (threadIdx.x >> 5);
     const uint32_t n_warps = gridDim.x * kWarpsPerBlock;
-    const uint32_t total = (uint32_t)a.n * (uint32_t)a.n_slabs;
-    for (uint32_t item = warp; item < total; item += n_warps) {
-        uint32_t i, s_idx;
-        item_to_chunk_slab(a, item, i, s_idx);
-        const ChunkEntry e = load_entry(a.entries + i);
-        const __half *src = a.kv_in + slab_offset(a, s_idx, e.chunk_id);
-        uint8_t *rec = a.buf + e.offset;
-        uint32_t sum;
-        if (e.bits == 8) sum = compress_slab<8, LPG, WIDE>(a, src, rec, s_idx, lane);
-        else if (e.bits == 4) sum = compress_slab<4, LPG, WIDE>(a, src, rec, s_idx, lane);
-        else sum = compress_slab<2, LPG, WIDE>(a, src, rec, s_idx, lane);
-        if (s_idx == 0) zero_padding(a, rec, e, lane);
-        sum = __reduce_add_sync(0xffffffffu, sum);
-        if (lane == 0) atomicAdd(&a.entries[i].checksum, sum);
+    uint32_t unit = blockIdx.x * kWarpsPerBlock + (threadIdx.x >> 5);
+    if (unit >= a.total_units) return;
+    UnitPos pa, pb;
+    uint32_t wa[kPieces][8], wb[kPieces][8];
+    decode_unit(a, unit, lane, pa);
+    load_unit<WIDE>(a, pa, wa);
+    for (;;) {  // two units per trip, so that the buffers swap roles without register copies
+        bool more = a.total_units - unit > n_warps;
+        if (more) {
+            decode_unit(a, unit + n_warps, lane, pb);
+            load_unit<WIDE>(a, pb, wb);
+        }
+        compress_unit<BITS, G, WIDE>(a, pa, wa, lane);
+        if (!more) break;
+        unit += n_warps;
+        more = a.total_units - unit > n_warps;
+        if (more) {
+            decode_unit(a, unit + n_warps, lane, pa);
+            load_unit<WIDE>(a, pa, wa);
+        }
+        compress_unit<BITS, G, WIDE>(a, pb, wb, lane);
+        if (!more) break;
+        unit += n_warps;
     }
 }
 
 // ---------------------------------------------------------------------------------------------- dequantize
 
-template <int BITS>
-__device__ __forceinline__ void load_codes(const uint8_t *p, uint32_t (&c)[BITS / 2])
+// A lane's codes (kLaneElems*bits/8 bytes) and group parameters of one unit.
+template <int BITS, int G>
+__device__ __forceinline__ void load_unit_codes(const CodecArgs &a, const UnitPos &u, uint32_t (&c)[kLaneElems * BITS / 32],
+                                                uint32_t (&p)[Geo<G>::kGroupsPerLane])
 {
-    if constexpr (BITS == 8)
-        asm volatile("ld.global.nc.L1::no_allocate.v4.b32 {%0,%1,%2,%3}, [%4];" : "=r"(c[0]), "=r"(c[1]), "=r"(c[2]), "=r"(c[3]) : "l"(p));
-    else if constexpr (BITS == 4)
-        asm volatile("ld.global.nc.L1::no_allocate.v2.b32 {%0,%1}, [%2];" : "=r"(c[0]), "=r"(c[1]) : "l"(p));
-    else
-        asm volatile("ld.global.nc.L1::no_allocate.b32 %0, [%1];" : "=r"(c[0]) : "l"(p));
-}
-
-// Spread the lane's 16 codes over bytes: code e ends up in byte (e % 4) of b[e / 4] (BITS 8),
-// byte (e / 2 % 4) of b[(e % 2) + 2 * (e / 8)] (BITS 4) or byte (e / 4) of b[e % 4] (BITS 2).
-template <int BITS>
-__device__ __forceinline__ uint32_t code_as_float_bits(const uint32_t (&c)[BITS / 2], const uint32_t (&b)[4], int e)
-{
-    // 0x4B000000 | q is the binary32 number 2^23 + q
-    if constexpr (BITS == 8) return __byte_perm(c[e / 4], 0x4B000000u, 0x7650 | (e % 4));
-    else if constexpr (BITS == 4) return __byte_perm(b[(e % 2) + 2 * (e / 8)], 0x4B000000u, 0x7650 | ((e / 2) % 4));
-    else return __byte_perm(b[e % 4], 0x4B000000u, 0x7650 | (e / 4));
-}
-
-template <int BITS, bool CLAMP>
-__device__ __forceinline__ void dequantize16(const uint32_t (&c)[BITS / 2], float scale, float zero, uint32_t (&w)[8])
-{
-    uint32_t b[4] = {0, 0, 0, 0};
-    if constexpr (BITS == 4) {
-        b[0] = c[0] & 0x0F0F0F0Fu; b[1] = (c[0] >> 4) & 0x0F0F0F0Fu;
-        b[2] = c[1] & 0x0F0F0F0Fu; b[3] = (c[1] >> 4) & 0x0F0F0F0Fu;
-    } else if constexpr (BITS == 2) {
-        b[0] = c[0] & 0x03030303u; b[1] = (c[0] >> 2) & 0x03030303u;
-        b[2] = (c[0] >> 4) & 0x03030303u; b[3] = (c[0] >> 6) & 0x03030303u;
+    using geo = Geo<G>;
+    const uint8_t *rec = a.buf + u.rec_off;
+    const uint32_t *params = reinterpret_cast<const uint32_t *>(rec) + (uint64_t)u.s_idx * a.groups_per_slab + (uint32_t)u.e0 / G;
+#pragma unroll
+    for (int g = 0; g < geo::kGroupsPerLane; ++g) p[g] = (u.e0 + g * G < a.slab_elems) ? __ldg(params + g) : 0u;
+#pragma unroll
+    for (int k = 0; k < kLaneElems * BITS / 32; ++k) c[k] = 0;
+    const uint8_t *codes = rec + a.codes_off + ((uint64_t)u.s_idx * a.slab_elems + (uint32_t)u.e0) * BITS / 8;
+    const bool lane_full = u.e0 + kLaneElems <= a.slab_elems;
+    const uintptr_t addr = reinterpret_cast<uintptr_t>(codes);
+    if constexpr (BITS == 8) {
+        if (lane_full && (addr & 31) == 0) {
+            ld256(codes, c);
+            ld256(codes + 32, c + 8);
+        } else {
+#pragma unroll
+            for (int j = 0; j < kPieces; ++j)
+                if (u.e0 + j * kPieceElems < a.slab_elems) ld128(codes + j * 16, c + 4 * j);
+        }
+    } else if constexpr (BITS == 4) {
+        if (lane_full && (addr & 31) == 0) {
+            ld256(codes, c);
+        } else {
+#pragma unroll
+            for (int j = 0; j < kPieces; ++j)
+                if (u.e0 + j * kPieceElems < a.slab_elems) ld64(codes + j * 8, c + 2 * j);
+        }
+    } else {
+        if (lane_full && (addr & 15) == 0) {
+            ld128(codes, c);
+        } else {
+#pragma unroll
+            for (int j = 0; j < kPieces; ++j)
+                if (u.e0 + j * kPieceElems < a.slab_elems) ld32(codes + j * 4, c + j);
+        }
     }
+}
+
+// 16 codes -> 8 half2 holding the codes as exact fp16 integers.  0x6400 | q is the fp16 number 1024 + q.
+template <int BITS>
+__device__ __forceinline__ void codes_to_half2(const uint32_t *c, __half2 (&q)[8])
+{
+    const __half2 k1024 = as_h2(0x64006400u);
+    if constexpr (BITS == 8) {
+#pragma unroll
+        for (int m = 0; m < 4; ++m) {
+            q[2 * m] = __hsub2(as_h2(__byte_perm(c[m], 0x64646464u, 0x4140)), k1024);      // codes 4m, 4m+1
+            q[2 * m + 1] = __hsub2(as_h2(__byte_perm(c[m], 0x64646464u, 0x4342)), k1024);  // codes 4m+2, 4m+3
+        }
+    } else if constexpr (BITS == 4) {
+#pragma unroll
+        for (int m = 0; m < 2; ++m) {
+            const uint32_t even = c[m] & 0x0F0F0F0Fu;         // codes 8m + 0, 2, 4, 6 in bytes 0..3
+            const uint32_t odd = (c[m] >> 4) & 0x0F0F0F0Fu;   // codes 8m + 1, 3, 5, 7
+#pragma unroll
+            for (int b = 0; b < 4; ++b) {
+                const uint32_t pair = __byte_perm(even, odd, (b) | ((4 + b) << 8)) & 0x00FF00FFu;
+                q[4 * m + b] = __hsub2(as_h2(pair | 0x64006400u), k1024);
+            }
+        }
+    } else {
+        const uint32_t r0 = c[0] & 0x03030303u;          // codes 0, 4, 8, 12
+        const uint32_t r1 = (c[0] >> 2) & 0x03030303u;   // codes 1, 5, 9, 13
+        const uint32_t r2 = (c[0] >> 4) & 0x03030303u;   // codes 2, 6, 10, 14
+        const uint32_t r3 = (c[0] >> 6) & 0x03030303u;   // codes 3, 7, 11, 15
+#pragma unroll
+        for (int b = 0; b < 4; ++b) {
+            const uint32_t p01 = __byte_perm(r0, r1, (b) | ((4 + b) << 8)) & 0x00FF00FFu;
+            const uint32_t p23 = __byte_perm(r2, r3, (b) | ((4 + b) << 8)) & 0x00FF00FFu;
+            q[2 * b] = __hsub2(as_h2(p01 | 0x64006400u), k1024);
+            q[2 * b + 1] = __hsub2(as_h2(p23 | 0x64006400u), k1024);
+        }
+    }
+}
+
+// 16 decoded values.  q*scale is exact in binary32, so the mixed-precision fused form rounds once, as
+// multiply-then-add would.  CLAMP only when zero + (2^b - 1)*scale can pass the fp16 range (zero >= -65504 and
+// scale >= 0, so only the upper end can).
+template <int BITS, bool CLAMP>
+__device__ __forceinline__ void dequantize_piece(const uint32_t *c, unsigned short scale_h, float zero, uint32_t (&w)[8])
+{
+    __half2 q[8];
+    codes_to_half2<BITS>(c, q);
 #pragma unroll
     for (int k = 0; k < 8; ++k) {
-        const float q0 = __fsub_rn(__uint_as_float(code_as_float_bits<BITS>(c, b, 2 * k)), 8388608.0f);      // exact
-        const float q1 = __fsub_rn(__uint_as_float(code_as_float_bits<BITS>(c, b, 2 * k + 1)), 8388608.0f);
-        // q*scale is exact in binary32, so the fused form rounds once, like multiply-then-add would
-        float y0 = __fmaf_rn(q0, scale, zero);
-        float y1 = __fmaf_rn(q1, scale, zero);
-        if constexpr (CLAMP) {  // zero >= -65504 and scale >= 0: only the upper end can leave the fp16 range
+        unsigned short q0, q1;
+        split_halves(as_u32(q[k]), q0, q1);
+        float y0 = fma_f32_f16(q0, scale_h, zero);
+        float y1 = fma_f32_f16(q1, scale_h, zero);
+        if constexpr (CLAMP) {
             y0 = fminf(y0, 65504.0f);
             y1 = fminf(y1, 65504.0f);
         }
@@ -309,69 +534,86 @@ __device__ __forceinline__ void dequantize16(const uint32_t (&c)[BITS / 2], floa
     }
 }
 
-template <int BITS, int LPG, bool WIDE>
-__device__ __forceinline__ uint32_t decompress_slab(const CodecArgs &a, const uint8_t *__restrict__ rec, __half *__restrict__ dst,
-                                                    uint32_t s_idx, int lane)
+template <int BITS, int G, bool WIDE>
+__device__ __forceinline__ uint32_t decompress_unit_bits(const CodecArgs &a, const UnitPos &u, const uint32_t (&c)[kLaneElems * BITS / 32],
+                                                         const uint32_t (&p)[Geo<G>::kGroupsPerLane], __half *__restrict__ dst, int lane)
 {
+    using geo = Geo<G>;
     constexpr float kQmax = (float)((1 << BITS) - 1);
-    constexpr int kLaneBytes = kElemsPerLane * BITS / 8;
-    const uint32_t *params = reinterpret_cast<const uint32_t *>(rec) + (uint64_t)s_idx * a.groups_per_slab;
-    const uint8_t *codes = rec + a.codes_off + (uint64_t)s_idx * a.slab_elems * BITS / 8;
+    constexpr int kPieceWords = BITS / 2;
     uint32_t sum = 0;
-    for (int base = 0; base < a.slab_elems; base += kUnroll * kElemsPerWarpIter) {
-        uint32_t c[kUnroll][BITS / 2];
-        uint32_t p[kUnroll];
+    bool any_clamp = false;
 #pragma unroll
-        for (int u = 0; u < kUnroll; ++u) {
-            const int e0 = base + u * kElemsPerWarpIter + lane * kElemsPerLane;
-            if (e0 < a.slab_elems) {
-                load_codes<BITS>(codes + (uint32_t)(e0 / kElemsPerLane) * kLaneBytes, c[u]);
-                p[u] = __ldg(params + e0 / (kElemsPerLane * LPG));
-            } else {
+    for (int g = 0; g < geo::kGroupsPerLane; ++g) {
+        const float scale = __half2float(__ushort_as_half((unsigned short)(p[g] & 0xffffu)));
+        const float zero = __half2float(__ushort_as_half((unsigned short)(p[g] >> 16)));
+        any_clamp |= __fmaf_rn(kQmax, scale, zero) > 65504.0f;
+    }
+    const bool clamp = __any_sync(0xffffffffu, any_clamp);
 #pragma unroll
-                for (int j = 0; j < BITS / 2; ++j) c[u][j] = 0;
-                p[u] = 0;
-            }
+    for (int j = 0; j < kPieces; ++j) {
+        const uint32_t pw = p[j / geo::kPiecesPerGroup];
+        const unsigned short scale_h = (unsigned short)(pw & 0xffffu);
+        const float zero = __half2float(__ushort_as_half((unsigned short)(pw >> 16)));
+        uint32_t w[8];
+        if (clamp) dequantize_piece<BITS, true>(c + j * kPieceWords, scale_h, zero, w);
+        else dequantize_piece<BITS, false>(c + j * kPieceWords, scale_h, zero, w);
+        if (u.e0 + j * kPieceElems < a.slab_elems) {
+            store32<WIDE>(dst + j * kPieceElems, w);
+#pragma unroll
+            for (int k = 0; k < kPieceWords; ++k) sum += c[j * kPieceWords + k];
         }
+    }
+    if constexpr (geo::kGroupsPerLane == 1) {
+        if (u.e0 < a.slab_elems && (lane & (geo::kLanesPerGroup - 1)) == 0) sum += p[0];
+    } else {
 #pragma unroll
-        for (int u = 0; u < kUnroll; ++u) {
-            const int e0 = base + u * kElemsPerWarpIter + lane * kElemsPerLane;
-            if (base + u * kElemsPerWarpIter >= a.slab_elems) break;  // warp-uniform
-            const float scale = __half2float(__ushort_as_half((unsigned short)(p[u] & 0xffffu)));
-            const float zero = __half2float(__ushort_as_half((unsigned short)(p[u] >> 16)));
-            uint32_t w[8];
-            if (__any_sync(0xffffffffu, __fmaf_rn(kQmax, scale, zero) > 65504.0f)) dequantize16<BITS, true>(c[u], scale, zero, w);
-            else dequantize16<BITS, false>(c[u], scale, zero, w);
-            if (e0 < a.slab_elems) {
-                store32<WIDE>(dst + e0, w);
-#pragma unroll
-                for (int j = 0; j < BITS / 2; ++j) sum += c[u][j];
-                if ((lane & (LPG - 1)) == 0) sum += p[u];
-            }
-        }
+        for (int g = 0; g < geo::kGroupsPerLane; ++g)
+            if (u.e0 + g * G < a.slab_elems) sum += p[g];
     }
     return sum;
 }
 
-template <int LPG, bool WIDE>
-__global__ void __launch_bounds__(kThreads) decompress_kernel(const CodecArgs a)
+template <int BITS, int G, bool WIDE>
+__device__ __forceinline__ void decompress_unit(const CodecArgs &a, const UnitPos &u, const uint32_t (&c)[kLaneElems * BITS / 32],
+                                                const uint32_t (&p)[Geo<G>::kGroupsPerLane], int lane)
 {
+    __half *dst = a.kv_out + slab_offset(a, u.s_idx, u.chunk_id) + u.e0;
+    uint32_t sum = decompress_unit_bits<BITS, G, WIDE>(a, u, c, p, dst, lane);
+    sum = __reduce_add_sync(0xffffffffu, sum);
+    if (lane == 0) atomicAdd(&a.sums[u.i], sum);
+}
+
+template <int BITS, int G, bool WIDE>
+__global__ void __launch_bounds__(kThreads, 2) decompress_kernel(const CodecArgs a)
+{
+    using geo = Geo<G>;
     const int lane = threadIdx.x & 31;
-    const uint32_t warp = blockIdx.x * kWarpsPerBlock + (threadIdx.x >> 5);
     const uint32_t n_warps = gridDim.x * kWarpsPerBlock;
-    const uint32_t total = (uint32_t)a.n * (uint32_t)a.n_slabs;
-    for (uint32_t item = warp; item < total; item += n_warps) {
-        uint32_t i, s_idx;
-        item_to_chunk_slab(a, item, i, s_idx);
-        const ChunkEntry e = load_entry(a.entries + i);
-        const uint8_t *rec = a.buf + e.offset;
-        __half *dst = a.kv_out + slab_offset(a, s_idx, e.chunk_id);
-        uint32_t sum;
-        if (e.bits == 8) sum = decompress_slab<8, LPG, WIDE>(a, rec, dst, s_idx, lane);
-        else if (e.bits == 4) sum = decompress_slab<4, LPG, WIDE>(a, rec, dst, s_idx, lane);
-        else sum = decompress_slab<2, LPG, WIDE>(a, rec, dst, s_idx, lane);
-        sum = __reduce_add_sync(0xffffffffu, sum);
-        if (lane == 0) atomicAdd(&a.sums[i], sum);
+    uint32_t unit = blockIdx.x * kWarpsPerBlock + (threadIdx.x >> 5);
+    if (unit >= a.total_units) return;
+    UnitPos pa, pb;
+    uint32_t ca[kLaneElems * BITS / 32], cb[kLaneElems * BITS / 32];
+    uint32_t qa[geo::kGroupsPerLane], qb[geo::kGroupsPerLane];
+    decode_unit(a, unit, lane, pa);
+    load_unit_codes<BITS, G>(a, pa, ca, qa);
+    for (;;) {
+        bool more = a.total_units - unit > n_warps;
+        if (more) {
+            decode_unit(a, unit + n_warps, lane, pb);
+            load_unit_codes<BITS, G>(a, pb, cb, qb);
+        }
+        decompress_unit<BITS, G, WIDE>(a, pa, ca, qa, lane);
+        if (!more) break;
+        unit += n_warps;
+        more = a.total_units - unit > n_warps;
+        if (more) {
+            decode_unit(a, unit + n_warps, lane, pa);
+            load_unit_codes<BITS, G>(a, pa, ca, qa);
+        }
+        decompress_unit<BITS, G, WIDE>(a, pb, cb, qb, lane);
+        if (!more) break;
+        unit += n_warps;
     }
 }
 
@@ -399,10 +641,43 @@ static int fill_args(const llms_kv_desc &d, CodecArgs &a, int n, void *workspace
     a.stride_s = d.stride_s;
     a.stride_h = d.stride_h;
     a.chunk_stride = (int64_t)d.chunk_len * d.head_dim;
-    a.slab_major = 1;  // measured: linear KV addresses beat linear record addresses (decompress 0.54 vs 0.72 ms on the 7B shape)
+    a.passes = (a.slab_elems + kPassElems - 1) / kPassElems;
+    a.total_units = (uint32_t)n * (uint32_t)a.n_slabs * (uint32_t)a.passes;
     a.entries = reinterpret_cast<ChunkEntry *>(static_cast<uint8_t *>(workspace) + kWsEntriesOffset);
     a.sums = reinterpret_cast<uint32_t *>(static_cast<uint8_t *>(workspace) + ws_sums_offset(n));
+    a.order = reinterpret_cast<const uint32_t *>(static_cast<uint8_t *>(workspace) + ws_order_offset(n));
     return LLMS_OK;
+}
+
+// Entry indices grouped by bit-width (8, then 4, then 2), list order kept inside a group.
+struct BitGroups {
+    std::vector<uint32_t> order;
+    int first[3], count[3];
+};
+
+template <typename GetBits>
+static BitGroups group_by_bits(int n, GetBits bits_of)
+{
+    static const uint32_t kWidths[3] = {8, 4, 2};
+    BitGroups g;
+    g.order.reserve(n);
+    for (int k = 0; k < 3; ++k) {
+        g.first[k] = (int)g.order.size();
+        for (int i = 0; i < n; ++i)
+            if (bits_of(i) == kWidths[k]) g.order.push_back((uint32_t)i);
+        g.count[k] = (int)g.order.size() - g.first[k];
+    }
+    return g;
+}
+
+// The launch arguments of one bit-width's share of the call.
+static CodecArgs args_for_group(const CodecArgs &a, const BitGroups &g, int k)
+{
+    CodecArgs b = a;
+    b.order = a.order + g.first[k];
+    b.n = g.count[k];
+    b.total_units = (uint32_t)b.n * (uint32_t)b.n_slabs * (uint32_t)b.passes;
+    return b;
 }
 
 // Persistent grid: as many CTAs as are resident at once, or fewer when there is less work.
@@ -426,15 +701,15 @@ static bool wide_ok(const llms_kv_desc &d, const void *kv)
 }
 
 template <typename F>
-static int dispatch_lpg(int group_size, F &&f)
+static int dispatch_group(int group_size, F &&f)
 {
-    switch (group_size / kElemsPerLane) {
-    case 1: f(std::integral_constant<int, 1>()); break;
-    case 2: f(std::integral_constant<int, 2>()); break;
-    case 4: f(std::integral_constant<int, 4>()); break;
-    case 8: f(std::integral_constant<int, 8>()); break;
+    switch (group_size) {
     case 16: f(std::integral_constant<int, 16>()); break;
     case 32: f(std::integral_constant<int, 32>()); break;
+    case 64: f(std::integral_constant<int, 64>()); break;
+    case 128: f(std::integral_constant<int, 128>()); break;
+    case 256: f(std::integral_constant<int, 256>()); break;
+    case 512: f(std::integral_constant<int, 512>()); break;
     default: return LLMS_ERR_UNSUPPORTED;
     }
     return LLMS_OK;
@@ -452,7 +727,8 @@ static int check_common(const llms_kv_desc *desc, int n, const void *workspace, 
     if (workspace_bytes < ws_total(n)) return LLMS_ERR_BUF_TOO_SMALL;
     if (groups_per_chunk(*desc) * 4 > 0xffffffffull) return LLMS_ERR_UNSUPPORTED;
     if (slab_elems(*desc) > 0x7fffffff / 8) return LLMS_ERR_UNSUPPORTED;
-    if ((uint64_t)n * (uint64_t)slabs_per_chunk(*desc) > 0x7fffffffull) return LLMS_ERR_UNSUPPORTED;
+    const uint64_t passes = ((uint64_t)slab_elems(*desc) + kPassElems - 1) / kPassElems;
+    if ((uint64_t)n * (uint64_t)slabs_per_chunk(*desc) * passes > 0x7fffffffull) return LLMS_ERR_UNSUPPORTED;
     return LLMS_OK;
 }
 
@@ -498,16 +774,25 @@ extern "C" int llms_compress_chunks(const llms_kv_desc *desc, const void *kv, co
     a.kv_in = static_cast<const __half *>(kv);
     a.buf = static_cast<uint8_t *>(out_buf);
     cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const BitGroups groups = group_by_bits(n, [&](int i) { return (uint32_t)bits[i]; });
     LLMS_CUDA_TRY(cudaMemcpyAsync(a.entries, meta, (size_t)n * sizeof(ChunkEntry), cudaMemcpyHostToDevice, st));
-    const int64_t items = (int64_t)n * a.n_slabs;
+    // `groups.order` is pageable: the copy has left it by the time cudaMemcpyAsync returns
+    LLMS_CUDA_TRY(cudaMemcpyAsync(const_cast<uint32_t *>(a.order), groups.order.data(), (size_t)n * 4, cudaMemcpyHostToDevice, st));
     const bool wide = wide_ok(*desc, kv);
-    rc = dispatch_lpg(desc->group_size, [&](auto lpg) {
-        constexpr int kLpg = decltype(lpg)::value;
-        if (wide) compress_kernel<kLpg, true><<<grid_for(compress_kernel<kLpg, true>, items), kThreads, 0, st>>>(a);
-        else compress_kernel<kLpg, false><<<grid_for(compress_kernel<kLpg, false>, items), kThreads, 0, st>>>(a);
-    });
-    if (rc) return rc;
-    LLMS_CUDA_TRY(cudaGetLastError());
+    for (int k = 0; k < 3; ++k) {
+        if (groups.count[k] == 0) continue;
+        const CodecArgs b = args_for_group(a, groups, k);
+        rc = dispatch_group(desc->group_size, [&](auto g) {
+            constexpr int kG = decltype(g)::value;
+#define LLMS_LAUNCH(BITS)                                                                                               \
+    if (wide) compress_kernel<BITS, kG, true><<<grid_for(compress_kernel<BITS, kG, true>, b.total_units), kThreads, 0, st>>>(b); \
+    else compress_kernel<BITS, kG, false><<<grid_for(compress_kernel<BITS, kG, false>, b.total_units), kThreads, 0, st>>>(b)
+            if (k == 0) { LLMS_LAUNCH(8); } else if (k == 1) { LLMS_LAUNCH(4); } else { LLMS_LAUNCH(2); }
+#undef LLMS_LAUNCH
+        });
+        if (rc) return rc;
+        LLMS_CUDA_TRY(cudaGetLastError());
+    }
     LLMS_CUDA_TRY(cudaMemcpyAsync(meta, a.entries, (size_t)n * sizeof(ChunkEntry), cudaMemcpyDeviceToHost, st));
     return LLMS_OK;
 }
@@ -545,15 +830,23 @@ extern "C" int llms_decompress_chunks(const llms_kv_desc *desc, const void *buf,
     LLMS_CUDA_TRY(cudaMemcpyAsync(a.entries, staged.data(), (size_t)n * sizeof(ChunkEntry), cudaMemcpyHostToDevice, st));
     LLMS_CUDA_TRY(cudaMemsetAsync(a.sums, 0, (size_t)n * 4, st));
     LLMS_CUDA_TRY(cudaMemsetAsync(status, 0, 4, st));
-    const int64_t items = (int64_t)n * a.n_slabs;
+    const BitGroups groups = group_by_bits(n, [&](int i) { return meta[i].bits; });
+    LLMS_CUDA_TRY(cudaMemcpyAsync(const_cast<uint32_t *>(a.order), groups.order.data(), (size_t)n * 4, cudaMemcpyHostToDevice, st));
     const bool wide = wide_ok(*desc, kv_out);
-    rc = dispatch_lpg(desc->group_size, [&](auto lpg) {
-        constexpr int kLpg = decltype(lpg)::value;
-        if (wide) decompress_kernel<kLpg, true><<<grid_for(decompress_kernel<kLpg, true>, items), kThreads, 0, st>>>(a);
-        else decompress_kernel<kLpg, false><<<grid_for(decompress_kernel<kLpg, false>, items), kThreads, 0, st>>>(a);
-    });
-    if (rc) return rc;
-    LLMS_CUDA_TRY(cudaGetLastError());
+    for (int k = 0; k < 3; ++k) {
+        if (groups.count[k] == 0) continue;
+        const CodecArgs b = args_for_group(a, groups, k);
+        rc = dispatch_group(desc->group_size, [&](auto g) {
+            constexpr int kG = decltype(g)::value;
+#define LLMS_LAUNCH(BITS)                                                                                                   \
+    if (wide) decompress_kernel<BITS, kG, true><<<grid_for(decompress_kernel<BITS, kG, true>, b.total_units), kThreads, 0, st>>>(b); \
+    else decompress_kernel<BITS, kG, false><<<grid_for(decompress_kernel<BITS, kG, false>, b.total_units), kThreads, 0, st>>>(b)
+            if (k == 0) { LLMS_LAUNCH(8); } else if (k == 1) { LLMS_LAUNCH(4); } else { LLMS_LAUNCH(2); }
+#undef LLMS_LAUNCH
+        });
+        if (rc) return rc;
+        LLMS_CUDA_TRY(cudaGetLastError());
+    }
     verify_kernel<<<1, 256, 0, st>>>(a.entries, a.sums, n, status);
     LLMS_CUDA_TRY(cudaGetLastError());
     return LLMS_OK;
@@ -575,7 +868,7 @@ extern "C" int llms_codec_corrupt_count(const void *workspace, uint32_t *n_corru
 namespace llms {
 
 constexpr uint64_t kStaticWorkspaceBytes =
-    (kWsEntriesOffset + (uint64_t)LLMS_STATIC_MAX_CHUNKS * (sizeof(ChunkEntry) + 4) + 255) / 256 * 256;
+    (kWsEntriesOffset + (uint64_t)LLMS_STATIC_MAX_CHUNKS * kWsBytesPerChunk + 255) / 256 * 256;
 
 // Scratch of llms_compress_chunks_static: lives in the library image, one copy on every GPU that loads it.
 static __device__ __align__(256) unsigned char g_static_workspace[kStaticWorkspaceBytes];
