@@ -432,45 +432,36 @@ __global__ void __launch_bounds__(kThreads, 2) compress_kernel(const CodecArgs a
 
 // ---------------------------------------------------------------------------------------------- dequantize
 
-// A lane's codes (kLaneElems*bits/8 bytes) and group parameters of one unit.
-template <int BITS, int G>
-__device__ __forceinline__ void load_unit_codes(const CodecArgs &a, const UnitPos &u, uint32_t (&c)[kLaneElems * BITS / 32],
-                                                uint32_t (&p)[Geo<G>::kGroupsPerLane])
+// The decoder splits a pass differently from the encoder: piece j of lane L is elements
+// [j*512 + L*16, +16) of the pass, so that every store instruction of the warp writes 1 KiB of consecutive
+// addresses (a lane-contiguous split made each store touch 32 separate lines and ran slower).  Groups need no
+// lane cooperation here; each piece just looks its group's parameters up.
+__device__ __forceinline__ int decode_piece_elem(const UnitPos &u, int lane, int j)
 {
-    using geo = Geo<G>;
+    return (u.e0 - lane * kLaneElems) + j * (32 * kPieceElems) + lane * kPieceElems;
+}
+
+template <int BITS, int G>
+__device__ __forceinline__ void load_unit_codes(const CodecArgs &a, const UnitPos &u, int lane, uint32_t (&c)[kPieces][BITS / 2],
+                                                uint32_t (&p)[kPieces])
+{
+    constexpr int kPieceBytes = kPieceElems * BITS / 8;
     const uint8_t *rec = a.buf + u.rec_off;
-    const uint32_t *params = reinterpret_cast<const uint32_t *>(rec) + (uint64_t)u.s_idx * a.groups_per_slab + (uint32_t)u.e0 / G;
+    const uint32_t *params = reinterpret_cast<const uint32_t *>(rec) + (uint64_t)u.s_idx * a.groups_per_slab;
+    const uint8_t *codes = rec + a.codes_off + (uint64_t)u.s_idx * a.slab_elems * BITS / 8;
 #pragma unroll
-    for (int g = 0; g < geo::kGroupsPerLane; ++g) p[g] = (u.e0 + g * G < a.slab_elems) ? __ldg(params + g) : 0u;
-#pragma unroll
-    for (int k = 0; k < kLaneElems * BITS / 32; ++k) c[k] = 0;
-    const uint8_t *codes = rec + a.codes_off + ((uint64_t)u.s_idx * a.slab_elems + (uint32_t)u.e0) * BITS / 8;
-    const bool lane_full = u.e0 + kLaneElems <= a.slab_elems;
-    const uintptr_t addr = reinterpret_cast<uintptr_t>(codes);
-    if constexpr (BITS == 8) {
-        if (lane_full && (addr & 31) == 0) {
-            ld256(codes, c);
-            ld256(codes + 32, c + 8);
+    for (int j = 0; j < kPieces; ++j) {
+        const int e = decode_piece_elem(u, lane, j);
+        if (e < a.slab_elems) {
+            const uint8_t *src = codes + (uint32_t)(e / kPieceElems) * kPieceBytes;
+            if constexpr (BITS == 8) ld128(src, c[j]);
+            else if constexpr (BITS == 4) ld64(src, c[j]);
+            else ld32(src, c[j]);
+            p[j] = __ldg(params + (uint32_t)e / G);
         } else {
 #pragma unroll
-            for (int j = 0; j < kPieces; ++j)
-                if (u.e0 + j * kPieceElems < a.slab_elems) ld128(codes + j * 16, c + 4 * j);
-        }
-    } else if constexpr (BITS == 4) {
-        if (lane_full && (addr & 31) == 0) {
-            ld256(codes, c);
-        } else {
-#pragma unroll
-            for (int j = 0; j < kPieces; ++j)
-                if (u.e0 + j * kPieceElems < a.slab_elems) ld64(codes + j * 8, c + 2 * j);
-        }
-    } else {
-        if (lane_full && (addr & 15) == 0) {
-            ld128(codes, c);
-        } else {
-#pragma unroll
-            for (int j = 0; j < kPieces; ++j)
-                if (u.e0 + j * kPieceElems < a.slab_elems) ld32(codes + j * 4, c + j);
+            for (int k = 0; k < BITS / 2; ++k) c[j][k] = 0;
+            p[j] = 0;
         }
     }
 }
@@ -535,73 +526,56 @@ __device__ __forceinline__ void dequantize_piece(const uint32_t *c, unsigned sho
 }
 
 template <int BITS, int G, bool WIDE>
-__device__ __forceinline__ uint32_t decompress_unit_bits(const CodecArgs &a, const UnitPos &u, const uint32_t (&c)[kLaneElems * BITS / 32],
-                                                         const uint32_t (&p)[Geo<G>::kGroupsPerLane], __half *__restrict__ dst, int lane)
+__device__ __forceinline__ void decompress_unit(const CodecArgs &a, const UnitPos &u, const uint32_t (&c)[kPieces][BITS / 2],
+                                                const uint32_t (&p)[kPieces], int lane)
 {
-    using geo = Geo<G>;
     constexpr float kQmax = (float)((1 << BITS) - 1);
-    constexpr int kPieceWords = BITS / 2;
+    __half *dst = a.kv_out + slab_offset(a, u.s_idx, u.chunk_id);
     uint32_t sum = 0;
     bool any_clamp = false;
 #pragma unroll
-    for (int g = 0; g < geo::kGroupsPerLane; ++g) {
-        const float scale = __half2float(__ushort_as_half((unsigned short)(p[g] & 0xffffu)));
-        const float zero = __half2float(__ushort_as_half((unsigned short)(p[g] >> 16)));
+    for (int j = 0; j < kPieces; ++j) {
+        const float scale = __half2float(__ushort_as_half((unsigned short)(p[j] & 0xffffu)));
+        const float zero = __half2float(__ushort_as_half((unsigned short)(p[j] >> 16)));
         any_clamp |= __fmaf_rn(kQmax, scale, zero) > 65504.0f;
     }
     const bool clamp = __any_sync(0xffffffffu, any_clamp);
 #pragma unroll
     for (int j = 0; j < kPieces; ++j) {
-        const uint32_t pw = p[j / geo::kPiecesPerGroup];
-        const unsigned short scale_h = (unsigned short)(pw & 0xffffu);
-        const float zero = __half2float(__ushort_as_half((unsigned short)(pw >> 16)));
+        const int e = decode_piece_elem(u, lane, j);
+        const unsigned short scale_h = (unsigned short)(p[j] & 0xffffu);
+        const float zero = __half2float(__ushort_as_half((unsigned short)(p[j] >> 16)));
         uint32_t w[8];
-        if (clamp) dequantize_piece<BITS, true>(c + j * kPieceWords, scale_h, zero, w);
-        else dequantize_piece<BITS, false>(c + j * kPieceWords, scale_h, zero, w);
-        if (u.e0 + j * kPieceElems < a.slab_elems) {
-            store32<WIDE>(dst + j * kPieceElems, w);
+        if (clamp) dequantize_piece<BITS, true>(c[j], scale_h, zero, w);
+        else dequantize_piece<BITS, false>(c[j], scale_h, zero, w);
+        if (e < a.slab_elems) {
+            store32<WIDE>(dst + e, w);
 #pragma unroll
-            for (int k = 0; k < kPieceWords; ++k) sum += c[j * kPieceWords + k];
+            for (int k = 0; k < BITS / 2; ++k) sum += c[j][k];
+            if ((uint32_t)e % G == 0) sum += p[j];  // the piece that opens a group accounts for its parameter word
         }
     }
-    if constexpr (geo::kGroupsPerLane == 1) {
-        if (u.e0 < a.slab_elems && (lane & (geo::kLanesPerGroup - 1)) == 0) sum += p[0];
-    } else {
-#pragma unroll
-        for (int g = 0; g < geo::kGroupsPerLane; ++g)
-            if (u.e0 + g * G < a.slab_elems) sum += p[g];
-    }
-    return sum;
-}
-
-template <int BITS, int G, bool WIDE>
-__device__ __forceinline__ void decompress_unit(const CodecArgs &a, const UnitPos &u, const uint32_t (&c)[kLaneElems * BITS / 32],
-                                                const uint32_t (&p)[Geo<G>::kGroupsPerLane], int lane)
-{
-    __half *dst = a.kv_out + slab_offset(a, u.s_idx, u.chunk_id) + u.e0;
-    uint32_t sum = decompress_unit_bits<BITS, G, WIDE>(a, u, c, p, dst, lane);
     sum = __reduce_add_sync(0xffffffffu, sum);
     if (lane == 0) atomicAdd(&a.sums[u.i], sum);
 }
 
 template <int BITS, int G, bool WIDE>
-__global__ void __launch_bounds__(kThreads, 2) decompress_kernel(const CodecArgs a)
+__global__ void __launch_bounds__(kThreads, 3) decompress_kernel(const CodecArgs a)
 {
-    using geo = Geo<G>;
     const int lane = threadIdx.x & 31;
     const uint32_t n_warps = gridDim.x * kWarpsPerBlock;
     uint32_t unit = blockIdx.x * kWarpsPerBlock + (threadIdx.x >> 5);
     if (unit >= a.total_units) return;
     UnitPos pa, pb;
-    uint32_t ca[kLaneElems * BITS / 32], cb[kLaneElems * BITS / 32];
-    uint32_t qa[geo::kGroupsPerLane], qb[geo::kGroupsPerLane];
+    uint32_t ca[kPieces][BITS / 2], cb[kPieces][BITS / 2];
+    uint32_t qa[kPieces], qb[kPieces];
     decode_unit(a, unit, lane, pa);
-    load_unit_codes<BITS, G>(a, pa, ca, qa);
+    load_unit_codes<BITS, G>(a, pa, lane, ca, qa);
     for (;;) {
         bool more = a.total_units - unit > n_warps;
         if (more) {
             decode_unit(a, unit + n_warps, lane, pb);
-            load_unit_codes<BITS, G>(a, pb, cb, qb);
+            load_unit_codes<BITS, G>(a, pb, lane, cb, qb);
         }
         decompress_unit<BITS, G, WIDE>(a, pa, ca, qa, lane);
         if (!more) break;
@@ -609,7 +583,7 @@ __global__ void __launch_bounds__(kThreads, 2) decompress_kernel(const CodecArgs
         more = a.total_units - unit > n_warps;
         if (more) {
             decode_unit(a, unit + n_warps, lane, pa);
-            load_unit_codes<BITS, G>(a, pa, ca, qa);
+            load_unit_codes<BITS, G>(a, pa, lane, ca, qa);
         }
         decompress_unit<BITS, G, WIDE>(a, pb, cb, qb, lane);
         if (!more) break;
