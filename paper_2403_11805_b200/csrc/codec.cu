@@ -24,6 +24,29 @@ constexpr int kPieces = 4;                      // pieces per lane per pass
 constexpr int kLaneElems = kPieces * kPieceElems;
 constexpr int kPassElems = 32 * kLaneElems;     // 2048 elements = 4 KiB of fp16
 
+// Division by a launch-time constant as multiply-high and shift: exact for numerators below 2^31.
+struct FastDiv {
+    uint32_t d, mul, shr;
+    __host__ void set(uint32_t divisor)
+    {
+        d = divisor;
+        mul = 0;
+        shr = 0;
+        if (divisor > 1) {
+            uint32_t lg = 0;
+            while ((1ull << lg) < divisor) ++lg;         // ceil(log2 d)
+            const uint32_t p = 31 + lg;
+            mul = (uint32_t)(((1ull << p) + divisor - 1) / divisor);
+            shr = p - 32;
+        }
+    }
+    __device__ __forceinline__ void divmod(uint32_t x, uint32_t &q, uint32_t &r) const
+    {
+        q = d == 1 ? x : (__umulhi(x, mul) >> shr);
+        r = x - q * d;
+    }
+};
+
 struct CodecArgs {
     const __half *kv_in;   // compress: source
     __half *kv_out;        // decompress: destination
@@ -37,6 +60,7 @@ struct CodecArgs {
     int groups_per_slab;
     int n_kv_heads;
     int passes;            // warp passes per slab
+    FastDiv div_passes, div_n, div_heads;
     uint32_t total_units;  // n * n_slabs * passes
     uint32_t codes_off;    // byte offset of the code stream in a record
     uint32_t params_bytes; // 4 * n_groups
@@ -54,10 +78,10 @@ struct UnitPos {
 
 __device__ __forceinline__ void decode_unit(const CodecArgs &a, uint32_t unit, int lane, UnitPos &u)
 {
-    const uint32_t item = unit / (uint32_t)a.passes;
-    const uint32_t pass = unit - item * (uint32_t)a.passes;
-    u.s_idx = item / (uint32_t)a.n;
-    u.i = a.order[item - u.s_idx * (uint32_t)a.n];
+    uint32_t item, pass, k;
+    a.div_passes.divmod(unit, item, pass);
+    a.div_n.divmod(item, u.s_idx, k);
+    u.i = a.order[k];
     const uint4 head = *reinterpret_cast<const uint4 *>(a.entries + u.i);  // chunk_id, bits, offset
     u.chunk_id = head.x;
     u.bits = head.y;
@@ -67,8 +91,8 @@ __device__ __forceinline__ void decode_unit(const CodecArgs &a, uint32_t unit, i
 
 __device__ __forceinline__ int64_t slab_offset(const CodecArgs &a, uint32_t s_idx, uint32_t chunk)
 {
-    const uint32_t ls = s_idx / (uint32_t)a.n_kv_heads;
-    const uint32_t h = s_idx - ls * (uint32_t)a.n_kv_heads;
+    uint32_t ls, h;
+    a.div_heads.divmod(s_idx, ls, h);
     return (int64_t)(ls >> 1) * a.stride_l + (int64_t)(ls & 1) * a.stride_s + (int64_t)h * a.stride_h +
            (int64_t)chunk * a.chunk_stride;
 }
@@ -617,6 +641,9 @@ static int fill_args(const llms_kv_desc &d, CodecArgs &a, int n, void *workspace
     a.chunk_stride = (int64_t)d.chunk_len * d.head_dim;
     a.passes = (a.slab_elems + kPassElems - 1) / kPassElems;
     a.total_units = (uint32_t)n * (uint32_t)a.n_slabs * (uint32_t)a.passes;
+    a.div_passes.set((uint32_t)a.passes);
+    a.div_n.set((uint32_t)n);
+    a.div_heads.set((uint32_t)a.n_kv_heads);
     a.entries = reinterpret_cast<ChunkEntry *>(static_cast<uint8_t *>(workspace) + kWsEntriesOffset);
     a.sums = reinterpret_cast<uint32_t *>(static_cast<uint8_t *>(workspace) + ws_sums_offset(n));
     a.order = reinterpret_cast<const uint32_t *>(static_cast<uint8_t *>(workspace) + ws_order_offset(n));
@@ -651,6 +678,7 @@ static CodecArgs args_for_group(const CodecArgs &a, const BitGroups &g, int k)
     b.order = a.order + g.first[k];
     b.n = g.count[k];
     b.total_units = (uint32_t)b.n * (uint32_t)b.n_slabs * (uint32_t)b.passes;
+    b.div_n.set((uint32_t)b.n);
     return b;
 }
 
