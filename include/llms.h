@@ -163,9 +163,10 @@ int llms_decompress_chunks(const llms_kv_desc *desc, const void *buf, const llms
                            const uint32_t *dst_chunk_ids, int n, void *kv_out,
                            void *workspace, uint64_t workspace_bytes, void *stream);
 
-/* Synchronises `stream`, then returns LLMS_OK if the last llms_decompress_chunks that used this
- * workspace saw no checksum mismatch, LLMS_ERR_CORRUPT otherwise; *n_corrupt (host, may be NULL)
- * receives the count. */
+/* Synchronises `stream`, then reports on the last llms_compress_chunks or llms_decompress_chunks
+ * that used this workspace: LLMS_ERR_TIMEOUT if one of its kernels abandoned a bounded wait for a
+ * copy (its output is then incomplete), else LLMS_ERR_CORRUPT if a decoded record's checksum did
+ * not match, else LLMS_OK; *n_corrupt (host, may be NULL) receives the number of such records. */
 int llms_codec_corrupt_count(const void *workspace, uint32_t *n_corrupt, void *stream);
 
 /* ------------------------------------------------------------------ tolerance score (Eq. 1) */

@@ -53,6 +53,7 @@ struct CodecArgs {
     uint8_t *buf;          // swap buffer (written by compress, read by decompress)
     ChunkEntry *entries;   // n entries in the workspace (caller's order)
     uint32_t *sums;        // decompress: recomputed checksums
+    uint32_t *gave_up;     // second status word: warps that abandoned a bounded wait
     const uint32_t *order; // entry indices grouped by bit-width; this launch covers order[0 .. n)
     int n;                 // chunks of this launch (all of one bit-width)
     int n_slabs;           // slabs per chunk
@@ -615,6 +616,12 @@ __global__ void __launch_bounds__(kThreads, 3) decompress_kernel(const CodecArgs
     }
 }
 
+}  // namespace llms
+
+#include "codec_bulk.cuh"
+
+namespace llms {
+
 // status word = number of records whose recomputed sum differs from the expected one
 __global__ void verify_kernel(const ChunkEntry *entries, const uint32_t *sums, int n, uint32_t *status)
 {
@@ -647,6 +654,7 @@ static int fill_args(const llms_kv_desc &d, CodecArgs &a, int n, void *workspace
     a.entries = reinterpret_cast<ChunkEntry *>(static_cast<uint8_t *>(workspace) + kWsEntriesOffset);
     a.sums = reinterpret_cast<uint32_t *>(static_cast<uint8_t *>(workspace) + ws_sums_offset(n));
     a.order = reinterpret_cast<const uint32_t *>(static_cast<uint8_t *>(workspace) + ws_order_offset(n));
+    a.gave_up = static_cast<uint32_t *>(workspace) + 1;
     return LLMS_OK;
 }
 
@@ -684,10 +692,10 @@ static CodecArgs args_for_group(const CodecArgs &a, const BitGroups &g, int k)
 
 // Persistent grid: as many CTAs as are resident at once, or fewer when there is less work.
 template <typename K>
-static int grid_for(K kernel, int64_t items)
+static int grid_for(K kernel, int64_t items, size_t dyn_smem = 0)
 {
     int per_sm = 0;
-    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kernel, kThreads, 0) != cudaSuccess || per_sm <= 0) {
+    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kernel, kThreads, dyn_smem) != cudaSuccess || per_sm <= 0) {
         cudaGetLastError();
         per_sm = 2;
     }
@@ -780,19 +788,32 @@ extern "C" int llms_compress_chunks(const llms_kv_desc *desc, const void *kv, co
     LLMS_CUDA_TRY(cudaMemcpyAsync(a.entries, meta, (size_t)n * sizeof(ChunkEntry), cudaMemcpyHostToDevice, st));
     // `groups.order` is pageable: the copy has left it by the time cudaMemcpyAsync returns
     LLMS_CUDA_TRY(cudaMemcpyAsync(const_cast<uint32_t *>(a.order), groups.order.data(), (size_t)n * 4, cudaMemcpyHostToDevice, st));
+    LLMS_CUDA_TRY(cudaMemsetAsync(workspace, 0, 8, st));  // both status words
     const bool wide = wide_ok(*desc, kv);
     for (int k = 0; k < 3; ++k) {
         if (groups.count[k] == 0) continue;
         const CodecArgs b = args_for_group(a, groups, k);
+        cudaError_t attr_err = cudaSuccess;
         rc = dispatch_group(desc->group_size, [&](auto g) {
             constexpr int kG = decltype(g)::value;
+            if constexpr (kG >= kLaneElems) {
+                // groups of 64 channels and more: the bulk-copy pipeline
+#define LLMS_LAUNCH(BITS)                                                                                                      \
+    attr_err = cudaFuncSetAttribute(compress_bulk_kernel<BITS, kG>, cudaFuncAttributeMaxDynamicSharedMemorySize, kBulkSmemBytes); \
+    if (attr_err == cudaSuccess)                                                                                                \
+        compress_bulk_kernel<BITS, kG><<<grid_for(compress_bulk_kernel<BITS, kG>, b.total_units, kBulkSmemBytes), kThreads, kBulkSmemBytes, st>>>(b)
+                if (k == 0) { LLMS_LAUNCH(8); } else if (k == 1) { LLMS_LAUNCH(4); } else { LLMS_LAUNCH(2); }
+#undef LLMS_LAUNCH
+            } else {
 #define LLMS_LAUNCH(BITS)                                                                                               \
     if (wide) compress_kernel<BITS, kG, true><<<grid_for(compress_kernel<BITS, kG, true>, b.total_units), kThreads, 0, st>>>(b); \
     else compress_kernel<BITS, kG, false><<<grid_for(compress_kernel<BITS, kG, false>, b.total_units), kThreads, 0, st>>>(b)
-            if (k == 0) { LLMS_LAUNCH(8); } else if (k == 1) { LLMS_LAUNCH(4); } else { LLMS_LAUNCH(2); }
+                if (k == 0) { LLMS_LAUNCH(8); } else if (k == 1) { LLMS_LAUNCH(4); } else { LLMS_LAUNCH(2); }
 #undef LLMS_LAUNCH
+            }
         });
         if (rc) return rc;
+        LLMS_CUDA_TRY(attr_err);
         LLMS_CUDA_TRY(cudaGetLastError());
     }
     LLMS_CUDA_TRY(cudaMemcpyAsync(meta, a.entries, (size_t)n * sizeof(ChunkEntry), cudaMemcpyDeviceToHost, st));
@@ -831,7 +852,7 @@ extern "C" int llms_decompress_chunks(const llms_kv_desc *desc, const void *buf,
     // `staged` is pageable: the copy has left it by the time cudaMemcpyAsync returns
     LLMS_CUDA_TRY(cudaMemcpyAsync(a.entries, staged.data(), (size_t)n * sizeof(ChunkEntry), cudaMemcpyHostToDevice, st));
     LLMS_CUDA_TRY(cudaMemsetAsync(a.sums, 0, (size_t)n * 4, st));
-    LLMS_CUDA_TRY(cudaMemsetAsync(status, 0, 4, st));
+    LLMS_CUDA_TRY(cudaMemsetAsync(status, 0, 8, st));  // both status words
     const BitGroups groups = group_by_bits(n, [&](int i) { return meta[i].bits; });
     LLMS_CUDA_TRY(cudaMemcpyAsync(const_cast<uint32_t *>(a.order), groups.order.data(), (size_t)n * 4, cudaMemcpyHostToDevice, st));
     const bool wide = wide_ok(*desc, kv_out);
@@ -857,12 +878,13 @@ extern "C" int llms_decompress_chunks(const llms_kv_desc *desc, const void *buf,
 extern "C" int llms_codec_corrupt_count(const void *workspace, uint32_t *n_corrupt, void *stream)
 {
     if (!workspace) return LLMS_ERR_INVALID_ARG;
-    uint32_t bad = 0;
+    uint32_t status[2] = {0, 0};  // {records with a wrong checksum, warps that gave up a bounded wait}
     cudaStream_t st = static_cast<cudaStream_t>(stream);
-    LLMS_CUDA_TRY(cudaMemcpyAsync(&bad, workspace, 4, cudaMemcpyDeviceToHost, st));
+    LLMS_CUDA_TRY(cudaMemcpyAsync(status, workspace, 8, cudaMemcpyDeviceToHost, st));
     LLMS_CUDA_TRY(cudaStreamSynchronize(st));
-    if (n_corrupt) *n_corrupt = bad;
-    return bad ? LLMS_ERR_CORRUPT : LLMS_OK;
+    if (n_corrupt) *n_corrupt = status[0];
+    if (status[1]) return LLMS_ERR_TIMEOUT;
+    return status[0] ? LLMS_ERR_CORRUPT : LLMS_OK;
 }
 
 // ---------------------------------------------------------------------------------------------- no-allocation variant
