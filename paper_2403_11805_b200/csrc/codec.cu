@@ -47,6 +47,14 @@ struct FastDiv {
     }
 };
 
+// One chunk of a launch, in the order the launch walks them.
+struct UnitEntry {
+    uint32_t chunk_id;  // source / destination chunk (slot) in the KV tensor
+    uint32_t entry;     // index into the caller-ordered entry table (checksums)
+    uint64_t rec_off;   // byte offset of the record in the swap buffer
+};
+static_assert(sizeof(UnitEntry) == 16, "table layout");
+
 struct CodecArgs {
     const __half *kv_in;   // compress: source
     __half *kv_out;        // decompress: destination
@@ -55,6 +63,7 @@ struct CodecArgs {
     uint32_t *sums;        // decompress: recomputed checksums
     uint32_t *gave_up;     // second status word: warps that abandoned a bounded wait
     const uint32_t *order; // entry indices grouped by bit-width; this launch covers order[0 .. n)
+    const UnitEntry *table; // the same chunks with what a unit needs to know, one 16-byte load
     int n;                 // chunks of this launch (all of one bit-width)
     int n_slabs;           // slabs per chunk
     int slab_elems;        // chunk_len * head_dim
@@ -62,6 +71,7 @@ struct CodecArgs {
     int n_kv_heads;
     int passes;            // warp passes per slab
     FastDiv div_passes, div_n, div_heads;
+    uint32_t step_units, step_pass, step_k, step_s;  // stride between a warp's units (= warps of the grid), split by radix
     uint32_t total_units;  // n * n_slabs * passes
     uint32_t codes_off;    // byte offset of the code stream in a record
     uint32_t params_bytes; // 4 * n_groups
@@ -654,6 +664,7 @@ static int fill_args(const llms_kv_desc &d, CodecArgs &a, int n, void *workspace
     a.entries = reinterpret_cast<ChunkEntry *>(static_cast<uint8_t *>(workspace) + kWsEntriesOffset);
     a.sums = reinterpret_cast<uint32_t *>(static_cast<uint8_t *>(workspace) + ws_sums_offset(n));
     a.order = reinterpret_cast<const uint32_t *>(static_cast<uint8_t *>(workspace) + ws_order_offset(n));
+    a.table = reinterpret_cast<const UnitEntry *>(static_cast<uint8_t *>(workspace) + ws_table_offset(n));
     a.gave_up = static_cast<uint32_t *>(workspace) + 1;
     return LLMS_OK;
 }
@@ -661,11 +672,12 @@ static int fill_args(const llms_kv_desc &d, CodecArgs &a, int n, void *workspace
 // Entry indices grouped by bit-width (8, then 4, then 2), list order kept inside a group.
 struct BitGroups {
     std::vector<uint32_t> order;
+    std::vector<UnitEntry> table;
     int first[3], count[3];
 };
 
 template <typename GetBits>
-static BitGroups group_by_bits(int n, GetBits bits_of)
+static BitGroups group_by_bits(int n, const llms_chunk_meta *meta, GetBits bits_of)
 {
     static const uint32_t kWidths[3] = {8, 4, 2};
     BitGroups g;
@@ -676,6 +688,13 @@ static BitGroups group_by_bits(int n, GetBits bits_of)
             if (bits_of(i) == kWidths[k]) g.order.push_back((uint32_t)i);
         g.count[k] = (int)g.order.size() - g.first[k];
     }
+    g.table.resize(n);
+    for (int j = 0; j < n; ++j) {
+        const llms_chunk_meta &m = meta[g.order[j]];
+        g.table[j].chunk_id = m.chunk_id;
+        g.table[j].entry = g.order[j];
+        g.table[j].rec_off = m.offset;
+    }
     return g;
 }
 
@@ -684,6 +703,7 @@ static CodecArgs args_for_group(const CodecArgs &a, const BitGroups &g, int k)
 {
     CodecArgs b = a;
     b.order = a.order + g.first[k];
+    b.table = a.table + g.first[k];
     b.n = g.count[k];
     b.total_units = (uint32_t)b.n * (uint32_t)b.n_slabs * (uint32_t)b.passes;
     b.div_n.set((uint32_t)b.n);
@@ -702,6 +722,17 @@ static int grid_for(K kernel, int64_t items, size_t dyn_smem = 0)
     const int64_t want = (items + kWarpsPerBlock - 1) / kWarpsPerBlock;
     const int64_t cap = (int64_t)sm_count() * per_sm;
     return (int)(want < cap ? want : cap);
+}
+
+// The stride between a warp's units, split into (passes, chunks, slab indices).
+static CodecArgs with_grid(CodecArgs a, int grid)
+{
+    a.step_units = (uint32_t)grid * kWarpsPerBlock;
+    a.step_pass = a.step_units % (uint32_t)a.passes;
+    const uint32_t items = a.step_units / (uint32_t)a.passes;
+    a.step_k = items % (uint32_t)a.n;
+    a.step_s = items / (uint32_t)a.n;
+    return a;
 }
 
 // 256-bit accesses need every slab to start on a 32-byte boundary
@@ -784,10 +815,11 @@ extern "C" int llms_compress_chunks(const llms_kv_desc *desc, const void *kv, co
     a.kv_in = static_cast<const __half *>(kv);
     a.buf = static_cast<uint8_t *>(out_buf);
     cudaStream_t st = static_cast<cudaStream_t>(stream);
-    const BitGroups groups = group_by_bits(n, [&](int i) { return (uint32_t)bits[i]; });
+    const BitGroups groups = group_by_bits(n, meta, [&](int i) { return (uint32_t)bits[i]; });
     LLMS_CUDA_TRY(cudaMemcpyAsync(a.entries, meta, (size_t)n * sizeof(ChunkEntry), cudaMemcpyHostToDevice, st));
     // `groups.order` is pageable: the copy has left it by the time cudaMemcpyAsync returns
     LLMS_CUDA_TRY(cudaMemcpyAsync(const_cast<uint32_t *>(a.order), groups.order.data(), (size_t)n * 4, cudaMemcpyHostToDevice, st));
+    LLMS_CUDA_TRY(cudaMemcpyAsync(const_cast<UnitEntry *>(a.table), groups.table.data(), (size_t)n * sizeof(UnitEntry), cudaMemcpyHostToDevice, st));
     LLMS_CUDA_TRY(cudaMemsetAsync(workspace, 0, 8, st));  // both status words
     const bool wide = wide_ok(*desc, kv);
     for (int k = 0; k < 3; ++k) {
@@ -800,8 +832,10 @@ extern "C" int llms_compress_chunks(const llms_kv_desc *desc, const void *kv, co
                 // groups of 64 channels and more: the bulk-copy pipeline
 #define LLMS_LAUNCH(BITS)                                                                                                      \
     attr_err = cudaFuncSetAttribute(compress_bulk_kernel<BITS, kG>, cudaFuncAttributeMaxDynamicSharedMemorySize, kBulkSmemBytes); \
-    if (attr_err == cudaSuccess)                                                                                                \
-        compress_bulk_kernel<BITS, kG><<<grid_for(compress_bulk_kernel<BITS, kG>, b.total_units, kBulkSmemBytes), kThreads, kBulkSmemBytes, st>>>(b)
+    if (attr_err == cudaSuccess) {                                                                                              \
+        const int grid = grid_for(compress_bulk_kernel<BITS, kG>, b.total_units, kBulkSmemBytes);                               \
+        compress_bulk_kernel<BITS, kG><<<grid, kThreads, kBulkSmemBytes, st>>>(with_grid(b, grid));                             \
+    }
                 if (k == 0) { LLMS_LAUNCH(8); } else if (k == 1) { LLMS_LAUNCH(4); } else { LLMS_LAUNCH(2); }
 #undef LLMS_LAUNCH
             } else {
@@ -853,8 +887,9 @@ extern "C" int llms_decompress_chunks(const llms_kv_desc *desc, const void *buf,
     LLMS_CUDA_TRY(cudaMemcpyAsync(a.entries, staged.data(), (size_t)n * sizeof(ChunkEntry), cudaMemcpyHostToDevice, st));
     LLMS_CUDA_TRY(cudaMemsetAsync(a.sums, 0, (size_t)n * 4, st));
     LLMS_CUDA_TRY(cudaMemsetAsync(status, 0, 8, st));  // both status words
-    const BitGroups groups = group_by_bits(n, [&](int i) { return meta[i].bits; });
+    const BitGroups groups = group_by_bits(n, staged.data(), [&](int i) { return meta[i].bits; });
     LLMS_CUDA_TRY(cudaMemcpyAsync(const_cast<uint32_t *>(a.order), groups.order.data(), (size_t)n * 4, cudaMemcpyHostToDevice, st));
+    LLMS_CUDA_TRY(cudaMemcpyAsync(const_cast<UnitEntry *>(a.table), groups.table.data(), (size_t)n * sizeof(UnitEntry), cudaMemcpyHostToDevice, st));
     const bool wide = wide_ok(*desc, kv_out);
     for (int k = 0; k < 3; ++k) {
         if (groups.count[k] == 0) continue;
