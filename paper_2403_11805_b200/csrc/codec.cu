@@ -724,6 +724,11 @@ static int grid_for(K kernel, int64_t items, size_t dyn_smem = 0)
     return (int)(want < cap ? want : cap);
 }
 
+// Measured on the 7B-shaped context (same box, same run): register-prefetch kernel 0.561 ms, bulk-copy pipeline
+// 0.579-0.591 ms.  Both are bound by instruction issue, not by the memory path, and the pipeline spends more
+// instructions (shared-memory traffic, barrier polling, single-lane sections), so the direct kernel is used.
+constexpr bool kUseBulkCompress = false;
+
 // The stride between a warp's units, split into (passes, chunks, slab indices).
 static CodecArgs with_grid(CodecArgs a, int grid)
 {
@@ -828,7 +833,7 @@ extern "C" int llms_compress_chunks(const llms_kv_desc *desc, const void *kv, co
         cudaError_t attr_err = cudaSuccess;
         rc = dispatch_group(desc->group_size, [&](auto g) {
             constexpr int kG = decltype(g)::value;
-            if constexpr (kG >= kLaneElems) {
+            if constexpr (kUseBulkCompress && kG >= kLaneElems) {
                 // groups of 64 channels and more: the bulk-copy pipeline
 #define LLMS_LAUNCH(BITS)                                                                                                      \
     attr_err = cudaFuncSetAttribute(compress_bulk_kernel<BITS, kG>, cudaFuncAttributeMaxDynamicSharedMemorySize, kBulkSmemBytes); \
