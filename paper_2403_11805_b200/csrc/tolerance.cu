@@ -9,6 +9,8 @@
 // scores - and the ranking made from them - are reproducible bit for bit.
 #include <math.h>
 
+#include <algorithm>
+
 #include "llms_internal.cuh"
 
 namespace llms {
@@ -106,6 +108,144 @@ __global__ void __launch_bounds__(kTokThreads) logits_kernel(const TolArgs a)
                 a.pp[o] = sp;
             }
         }
+    }
+}
+
+// ------------------------------------------------------------------ the same, staged through shared memory
+//
+// For head_dim 64, 128 or 256.  A warp owns tiles of 32 consecutive tokens of one (layer, KV head).  It copies
+// a tile (32 x head_dim fp16, contiguous in memory) into shared memory with coalesced 16-byte asynchronous
+// copies (cp.async, two buffers: the next tile lands while this one is used), swizzled by XOR-ing the 16-byte
+// chunk index with the row index so that lane t can then read row t without bank conflicts.  The dot products
+// use the sm_100 mixed-precision fma (fp16 x fp16 + fp32, one rounding; the products are exact), so neither K
+// nor q is ever converted, and q stays in shared memory as fp16, read as warp-wide broadcasts: 8 fma per
+// 16-byte load.
+constexpr int kTileTokens = 32;
+constexpr int kTileWarps = 4;
+
+__device__ __forceinline__ float fma_f32_f16(unsigned short x, unsigned short y, float c)
+{
+    float d;
+    asm("fma.rn.f32.f16 %0, %1, %2, %3;" : "=f"(d) : "h"(x), "h"(y), "f"(c));
+    return d;
+}
+__device__ __forceinline__ void split_halves(uint32_t w, unsigned short &lo, unsigned short &hi)
+{
+    asm("mov.b32 {%0, %1}, %2;" : "=h"(lo), "=h"(hi) : "r"(w));
+}
+// 16-byte asynchronous copy global -> shared, bypassing L1; src_bytes = 0 fills zeros instead
+__device__ __forceinline__ void cp_async16(uint32_t dst_smem, const void *src, uint32_t src_bytes)
+{
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" :: "r"(dst_smem), "l"(src), "r"(src_bytes) : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+template <int N>
+__device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;" :: "n"(N) : "memory"); }
+
+template <int RT, int D>
+__global__ void __launch_bounds__(kTileWarps * 32) logits_tile_kernel(const TolArgs a, const int seg_len)
+{
+    constexpr int kRowBytes = D * 2, kChunks = D / 8, kTileBytes = kTileTokens * kRowBytes;
+    constexpr int kUnrollChunks = 64 / RT;                                   // 512 fma per unrolled trip
+    extern __shared__ __align__(128) unsigned char smem_raw[];
+    const int lane = threadIdx.x & 31, wib = threadIdx.x >> 5;
+    const int nr_pad = (a.NR + RT - 1) / RT * RT;                            // rows padded with zeros to whole row tiles
+    __half *q_s = reinterpret_cast<__half *>(smem_raw);                      // [nr_pad][D] fp16
+    unsigned char *tiles = smem_raw + nr_pad * kRowBytes + wib * 2 * kTileBytes;  // this warp's two buffers
+    const uint32_t tiles_s = (uint32_t)__cvta_generic_to_shared(tiles);
+
+    const int l = blockIdx.y / a.Hkv, kvh = blockIdx.y % a.Hkv;
+    const __half *q_src = a.q_win + ((int64_t)(l * a.Hq + kvh * a.rep) * a.W) * D;
+    for (int i = threadIdx.x; i < nr_pad * kChunks; i += blockDim.x)
+        reinterpret_cast<uint4 *>(q_s)[i] = i < a.NR * kChunks ? __ldg(reinterpret_cast<const uint4 *>(q_src) + i) : make_uint4(0, 0, 0, 0);
+    __syncthreads();
+
+    const __half *k_plane = a.kv + (int64_t)l * a.stride_l + (int64_t)kvh * a.stride_h;
+    const int n_tiles = (a.T + kTileTokens - 1) / kTileTokens;
+    // this block's share of the tiles, its warps taking them in turn
+    const int per_block = (n_tiles + gridDim.x - 1) / gridDim.x;
+    const int tile_begin = blockIdx.x * per_block + wib;
+    const int tile_end = min(n_tiles, (int)(blockIdx.x + 1) * per_block);
+    const int64_t row0 = (int64_t)(l * a.Hq + kvh * a.rep) * a.W;
+
+    // lane L copies chunk (i*32 + L) of the tile, i = 0 .. kChunks-1: consecutive lanes, consecutive addresses
+    auto issue_tile = [&](int tile, int buf) {
+        const __half *src = k_plane + (int64_t)tile * kTileTokens * D;
+        const int valid_rows = min(kTileTokens, a.T - tile * kTileTokens);
+#pragma unroll
+        for (int i = 0; i < kChunks; ++i) {
+            const int n = i * 32 + lane;
+            const int row = n / kChunks, c = n % kChunks;
+            const uint32_t dst = tiles_s + buf * kTileBytes + row * kRowBytes + ((c ^ (row & 7)) << 4);
+            const bool in = row < valid_rows;
+            cp_async16(dst, in ? src + n * 8 : src, in ? 16u : 0u);
+        }
+        cp_async_commit();
+    };
+
+    int buf = 0;
+    if (tile_begin < tile_end) issue_tile(tile_begin, 0);
+    for (int tile = tile_begin; tile < tile_end; tile += kTileWarps, buf ^= 1) {
+        if (tile + kTileWarps < tile_end) {
+            issue_tile(tile + kTileWarps, buf ^ 1);
+            cp_async_wait<1>();
+        } else {
+            cp_async_wait<0>();
+        }
+        __syncwarp();
+        const int t = tile * kTileTokens + lane;
+        const bool valid = t < a.T;
+        const int n_vis = min(a.W, a.T - (valid ? t : 0));
+        const float w_col = 1.0f / (float)n_vis;
+        const int seg = t / seg_len;
+        const unsigned char *my_row = tiles + buf * kTileBytes + lane * kRowBytes;
+        const int swz = (lane & 7) << 4;
+        for (int j0 = 0; j0 < a.NR; j0 += RT) {
+            float acc[RT];
+#pragma unroll
+            for (int j = 0; j < RT; ++j) acc[j] = 0.0f;
+            const __half *q_tile = q_s + j0 * D;
+#pragma unroll kUnrollChunks
+            for (int c = 0; c < kChunks; ++c) {
+                const uint4 kk = *reinterpret_cast<const uint4 *>(my_row + ((c << 4) ^ swz));
+                const uint32_t kw[4] = {kk.x, kk.y, kk.z, kk.w};
+#pragma unroll
+                for (int j = 0; j < RT; ++j) {
+                    const uint4 qq = *reinterpret_cast<const uint4 *>(q_tile + j * D + c * 8);
+                    const uint32_t qw[4] = {qq.x, qq.y, qq.z, qq.w};
+#pragma unroll
+                    for (int i = 0; i < 4; ++i) {
+                        unsigned short k0, k1, q0, q1;
+                        split_halves(kw[i], k0, k1);
+                        split_halves(qw[i], q0, q1);
+                        acc[j] = fma_f32_f16(k0, q0, acc[j]);
+                        acc[j] = fma_f32_f16(k1, q1, acc[j]);
+                    }
+                }
+            }
+#pragma unroll
+            for (int j = 0; j < RT; ++j) {
+                if (j0 + j >= a.NR) break;  // uniform
+                const int r = (j0 + j) % a.W;
+                const bool vis = valid && t <= a.T - a.W + r;
+                const float logit = vis ? acc[j] * a.inv_sqrt_d : -INFINITY;
+                float m = logit;
+                for (int s = seg_len / 2; s > 0; s >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, s));
+                const float e = vis ? expf(logit - m) : 0.0f;
+                float se = e, sp = e * w_col;
+                for (int s = seg_len / 2; s > 0; s >>= 1) {
+                    se += __shfl_xor_sync(0xffffffffu, se, s);
+                    sp += __shfl_xor_sync(0xffffffffu, sp, s);
+                }
+                if (valid && (lane & (seg_len - 1)) == 0) {
+                    const int64_t o = (row0 + j0 + j) * a.n_seg + seg;
+                    a.pm[o] = m;
+                    a.ps[o] = se;
+                    a.pp[o] = sp;
+                }
+            }
+        }
+        __syncwarp();  // the buffer is free for the copy issued two tiles from now
     }
 }
 
@@ -305,26 +445,54 @@ extern "C" int llms_chunk_tolerance(const llms_kv_desc *desc, const void *kv, co
     a.part = reinterpret_cast<float *>(ws + t.off_part);
     a.scores = scores;
     a.Y = t.Y; a.rows = t.rows;
-    const size_t q_bytes = (size_t)a.NR * a.d * sizeof(float);
-    if (q_bytes > 200 * 1024) return LLMS_ERR_UNSUPPORTED;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
-    const dim3 grid((a.T + kTokThreads - 1) / kTokThreads, a.L * a.Hkv);
     if ((unsigned)(a.L * a.Hkv) > 65535u) return LLMS_ERR_UNSUPPORTED;
+    const int rt = a.NR <= 8 ? 8 : (a.NR <= 16 ? 16 : 32);
+    const size_t tile_q_bytes = (size_t)((a.NR + rt - 1) / rt * rt) * a.d * 2;
+    const size_t tile_smem = tile_q_bytes + (size_t)kTileWarps * 2 * kTileTokens * a.d * 2;
+    if ((a.d == 64 || a.d == 128 || a.d == 256) && tile_smem <= 200 * 1024) {
+        // tiles through shared memory; enough blocks per (layer, KV head) to fill the GPU a few times over
+        const int n_tiles = (a.T + kTileTokens - 1) / kTileTokens;
+        const int pairs = a.L * a.Hkv;
+        int splits = (sm_count() * 6 + pairs - 1) / pairs;
+        splits = std::max(1, std::min(splits, (n_tiles + kTileWarps - 1) / kTileWarps));
+        const dim3 grid(splits, pairs);
+#define LLMS_LAUNCH_TILE(R, DD)                                                                                                   \
+    do {                                                                                                                          \
+        LLMS_CUDA_TRY(cudaFuncSetAttribute(logits_tile_kernel<R, DD>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)tile_smem)); \
+        logits_tile_kernel<R, DD><<<grid, kTileWarps * 32, tile_smem, st>>>(a, t.SEG);                                            \
+    } while (0)
+#define LLMS_LAUNCH_TILE_D(R)                                                       \
+    do {                                                                            \
+        if (a.d == 64) LLMS_LAUNCH_TILE(R, 64);                                     \
+        else if (a.d == 128) LLMS_LAUNCH_TILE(R, 128);                              \
+        else LLMS_LAUNCH_TILE(R, 256);                                              \
+    } while (0)
+        if (rt == 8) LLMS_LAUNCH_TILE_D(8);
+        else if (rt == 16) LLMS_LAUNCH_TILE_D(16);
+        else LLMS_LAUNCH_TILE_D(32);
+#undef LLMS_LAUNCH_TILE_D
+#undef LLMS_LAUNCH_TILE
+    } else {
+        const size_t q_bytes = (size_t)a.NR * a.d * sizeof(float);
+        if (q_bytes > 200 * 1024) return LLMS_ERR_UNSUPPORTED;
+        const dim3 grid((a.T + kTokThreads - 1) / kTokThreads, a.L * a.Hkv);
 #define LLMS_LAUNCH_LOGITS(S)                                                                                   \
     case S:                                                                                                     \
         LLMS_CUDA_TRY(cudaFuncSetAttribute(logits_kernel<S>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)q_bytes)); \
         logits_kernel<S><<<grid, kTokThreads, q_bytes, st>>>(a);                                                \
         break;
-    switch (t.SEG) {
-        LLMS_LAUNCH_LOGITS(1)
-        LLMS_LAUNCH_LOGITS(2)
-        LLMS_LAUNCH_LOGITS(4)
-        LLMS_LAUNCH_LOGITS(8)
-        LLMS_LAUNCH_LOGITS(16)
-        LLMS_LAUNCH_LOGITS(32)
-    default: return LLMS_ERR_UNSUPPORTED;
-    }
+        switch (t.SEG) {
+            LLMS_LAUNCH_LOGITS(1)
+            LLMS_LAUNCH_LOGITS(2)
+            LLMS_LAUNCH_LOGITS(4)
+            LLMS_LAUNCH_LOGITS(8)
+            LLMS_LAUNCH_LOGITS(16)
+            LLMS_LAUNCH_LOGITS(32)
+        default: return LLMS_ERR_UNSUPPORTED;
+        }
 #undef LLMS_LAUNCH_LOGITS
+    }
     LLMS_CUDA_TRY(cudaGetLastError());
     row_stats_kernel<<<(a.rows + 7) / 8, 256, 0, st>>>(a);
     LLMS_CUDA_TRY(cudaGetLastError());
