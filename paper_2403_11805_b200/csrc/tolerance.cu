@@ -111,28 +111,20 @@ __global__ void __launch_bounds__(kTokThreads) logits_kernel(const TolArgs a)
     }
 }
 
-// ------------------------------------------------------------------ the same, staged through shared memory
+// ------------------------------------------------------------------ the same on the tensor cores
 //
-// For head_dim 64, 128 or 256.  A warp owns tiles of 32 consecutive tokens of one (layer, KV head).  It copies
-// a tile (32 x head_dim fp16, contiguous in memory) into shared memory with coalesced 16-byte asynchronous
-// copies (cp.async, two buffers: the next tile lands while this one is used), swizzled by XOR-ing the 16-byte
-// chunk index with the row index so that lane t can then read row t without bank conflicts.  The dot products
-// use the sm_100 mixed-precision fma (fp16 x fp16 + fp32, one rounding; the products are exact), so neither K
-// nor q is ever converted, and q stays in shared memory as fp16, read as warp-wide broadcasts: 8 fma per
-// 16-byte load.
+// S = K q^T is a dense contraction (tokens x head_dim times head_dim x window rows): with plain fp32 fma the
+// kernel is bound by instruction issue (measured 0.56 ms for the 7B shape against 0.17 ms for reading K once),
+// so for head_dim 64, 128 and 256 it runs as warp-level matrix multiply-accumulate, m16n8k16 with fp16 inputs
+// and fp32 accumulators: 8 window rows are exactly one n-tile.  A warp owns tiles of 32 consecutive tokens of one
+// (layer, KV head).  It copies a tile (32 x head_dim fp16, contiguous in memory) into shared memory with
+// coalesced 16-byte asynchronous copies (cp.async, two buffers: the next tile lands while this one is used),
+// swizzled by XOR-ing the 16-byte chunk index with the row index so that ldmatrix reads without bank conflicts.
+// The window's query rows sit in shared memory (rows padded by 16 bytes against conflicts) and are read as B
+// fragments.  The softmax statistics are then taken straight from the accumulator fragments.
 constexpr int kTileTokens = 32;
 constexpr int kTileWarps = 4;
 
-__device__ __forceinline__ float fma_f32_f16(unsigned short x, unsigned short y, float c)
-{
-    float d;
-    asm("fma.rn.f32.f16 %0, %1, %2, %3;" : "=f"(d) : "h"(x), "h"(y), "f"(c));
-    return d;
-}
-__device__ __forceinline__ void split_halves(uint32_t w, unsigned short &lo, unsigned short &hi)
-{
-    asm("mov.b32 {%0, %1}, %2;" : "=h"(lo), "=h"(hi) : "r"(w));
-}
 // 16-byte asynchronous copy global -> shared, bypassing L1; src_bytes = 0 fills zeros instead
 __device__ __forceinline__ void cp_async16(uint32_t dst_smem, const void *src, uint32_t src_bytes)
 {
@@ -142,22 +134,66 @@ __device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commi
 template <int N>
 __device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;" :: "n"(N) : "memory"); }
 
-template <int RT, int D>
-__global__ void __launch_bounds__(kTileWarps * 32) logits_tile_kernel(const TolArgs a, const int seg_len)
+__device__ __forceinline__ void ldmatrix_x4(uint32_t addr, uint32_t (&r)[4])
+{
+    asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(addr));
+}
+__device__ __forceinline__ void mma_16816(float (&c)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1)
+{
+    asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+                 : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3]) : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
+}
+
+// Reduce the four values a lane holds for one window row (tokens mb*16 + half*8 + g, g = lane/4) over the
+// tokens of each SEG-token segment; afterwards every slot holds its segment's result.
+template <int SEG, typename Op>
+__device__ __forceinline__ void segment_reduce(float (&x)[2][2], Op op)
+{
+    if constexpr (SEG == 32) x[0][0] = op(op(x[0][0], x[0][1]), op(x[1][0], x[1][1]));
+    if constexpr (SEG == 16) {
+        x[0][0] = op(x[0][0], x[0][1]);
+        x[1][0] = op(x[1][0], x[1][1]);
+    }
+#pragma unroll
+    for (int mb = 0; mb < 2; ++mb)
+#pragma unroll
+        for (int h = 0; h < 2; ++h) {
+            if ((SEG == 32 && (mb || h)) || (SEG == 16 && h)) continue;  // folded into another slot above
+            float v = x[mb][h];
+            if constexpr (SEG >= 2) v = op(v, __shfl_xor_sync(0xffffffffu, v, 4));
+            if constexpr (SEG >= 4) v = op(v, __shfl_xor_sync(0xffffffffu, v, 8));
+            if constexpr (SEG >= 8) v = op(v, __shfl_xor_sync(0xffffffffu, v, 16));
+            x[mb][h] = v;
+        }
+    if constexpr (SEG == 32) x[0][1] = x[1][0] = x[1][1] = x[0][0];
+    if constexpr (SEG == 16) {
+        x[0][1] = x[0][0];
+        x[1][1] = x[1][0];
+    }
+}
+
+template <int SEG, int D>
+__global__ void __launch_bounds__(kTileWarps * 32) logits_mma_kernel(const TolArgs a)
 {
     constexpr int kRowBytes = D * 2, kChunks = D / 8, kTileBytes = kTileTokens * kRowBytes;
-    constexpr int kUnrollChunks = 64 / RT;                                   // 512 fma per unrolled trip
+    constexpr int kQRowBytes = kRowBytes + 16;                               // padded: B fragments read conflict-free
     extern __shared__ __align__(128) unsigned char smem_raw[];
     const int lane = threadIdx.x & 31, wib = threadIdx.x >> 5;
-    const int nr_pad = (a.NR + RT - 1) / RT * RT;                            // rows padded with zeros to whole row tiles
-    __half *q_s = reinterpret_cast<__half *>(smem_raw);                      // [nr_pad][D] fp16
-    unsigned char *tiles = smem_raw + nr_pad * kRowBytes + wib * 2 * kTileBytes;  // this warp's two buffers
+    const int g = lane >> 2, q4 = lane & 3;
+    const int n_blocks = (a.NR + 7) / 8;                                     // window rows in n-tiles of 8, zero padded
+    unsigned char *q_s = smem_raw;                                           // [n_blocks*8][kQRowBytes]
+    const int q_total = (n_blocks * 8 * kQRowBytes + 127) / 128 * 128;
+    unsigned char *tiles = smem_raw + q_total + wib * 2 * kTileBytes;        // this warp's two buffers
     const uint32_t tiles_s = (uint32_t)__cvta_generic_to_shared(tiles);
 
     const int l = blockIdx.y / a.Hkv, kvh = blockIdx.y % a.Hkv;
     const __half *q_src = a.q_win + ((int64_t)(l * a.Hq + kvh * a.rep) * a.W) * D;
-    for (int i = threadIdx.x; i < nr_pad * kChunks; i += blockDim.x)
-        reinterpret_cast<uint4 *>(q_s)[i] = i < a.NR * kChunks ? __ldg(reinterpret_cast<const uint4 *>(q_src) + i) : make_uint4(0, 0, 0, 0);
+    for (int i = threadIdx.x; i < n_blocks * 8 * kChunks; i += blockDim.x) {
+        const int row = i / kChunks, c = i % kChunks;
+        *reinterpret_cast<uint4 *>(q_s + row * kQRowBytes + c * 16) =
+            row < a.NR ? __ldg(reinterpret_cast<const uint4 *>(q_src) + i) : make_uint4(0, 0, 0, 0);
+    }
     __syncthreads();
 
     const __half *k_plane = a.kv + (int64_t)l * a.stride_l + (int64_t)kvh * a.stride_h;
@@ -183,6 +219,9 @@ __global__ void __launch_bounds__(kTileWarps * 32) logits_tile_kernel(const TolA
         cp_async_commit();
     };
 
+    // ldmatrix x4 of a 16 x 16 block: lanes 0-15 give the rows at column chunk 2*ks, lanes 16-31 at 2*ks + 1
+    const int a_row = lane & 15, a_chunk = lane >> 4;
+
     int buf = 0;
     if (tile_begin < tile_end) issue_tile(tile_begin, 0);
     for (int tile = tile_begin; tile < tile_end; tile += kTileWarps, buf ^= 1) {
@@ -193,55 +232,66 @@ __global__ void __launch_bounds__(kTileWarps * 32) logits_tile_kernel(const TolA
             cp_async_wait<0>();
         }
         __syncwarp();
-        const int t = tile * kTileTokens + lane;
-        const bool valid = t < a.T;
-        const int n_vis = min(a.W, a.T - (valid ? t : 0));
-        const float w_col = 1.0f / (float)n_vis;
-        const int seg = t / seg_len;
-        const unsigned char *my_row = tiles + buf * kTileBytes + lane * kRowBytes;
-        const int swz = (lane & 7) << 4;
-        for (int j0 = 0; j0 < a.NR; j0 += RT) {
-            float acc[RT];
+        const uint32_t tile_s = tiles_s + buf * kTileBytes;
+        for (int nb = 0; nb < n_blocks; ++nb) {
+            float acc[2][4];
 #pragma unroll
-            for (int j = 0; j < RT; ++j) acc[j] = 0.0f;
-            const __half *q_tile = q_s + j0 * D;
-#pragma unroll kUnrollChunks
-            for (int c = 0; c < kChunks; ++c) {
-                const uint4 kk = *reinterpret_cast<const uint4 *>(my_row + ((c << 4) ^ swz));
-                const uint32_t kw[4] = {kk.x, kk.y, kk.z, kk.w};
+            for (int mb = 0; mb < 2; ++mb)
 #pragma unroll
-                for (int j = 0; j < RT; ++j) {
-                    const uint4 qq = *reinterpret_cast<const uint4 *>(q_tile + j * D + c * 8);
-                    const uint32_t qw[4] = {qq.x, qq.y, qq.z, qq.w};
+                for (int i = 0; i < 4; ++i) acc[mb][i] = 0.0f;
+            const unsigned char *q_row = q_s + (nb * 8 + g) * kQRowBytes + q4 * 4;
 #pragma unroll
-                    for (int i = 0; i < 4; ++i) {
-                        unsigned short k0, k1, q0, q1;
-                        split_halves(kw[i], k0, k1);
-                        split_halves(qw[i], q0, q1);
-                        acc[j] = fma_f32_f16(k0, q0, acc[j]);
-                        acc[j] = fma_f32_f16(k1, q1, acc[j]);
-                    }
+            for (int ks = 0; ks < D / 16; ++ks) {
+                const uint32_t b0 = *reinterpret_cast<const uint32_t *>(q_row + ks * 32);
+                const uint32_t b1 = *reinterpret_cast<const uint32_t *>(q_row + ks * 32 + 16);
+#pragma unroll
+                for (int mb = 0; mb < 2; ++mb) {
+                    const int row = mb * 16 + a_row;
+                    uint32_t af[4];
+                    ldmatrix_x4(tile_s + row * kRowBytes + (((2 * ks + a_chunk) ^ (row & 7)) << 4), af);
+                    mma_16816(acc[mb], af, b0, b1);
                 }
             }
+            // acc[mb][0..1]: token mb*16 + g, window rows 2*q4, 2*q4+1;  acc[mb][2..3]: token mb*16 + 8 + g
 #pragma unroll
-            for (int j = 0; j < RT; ++j) {
-                if (j0 + j >= a.NR) break;  // uniform
-                const int r = (j0 + j) % a.W;
-                const bool vis = valid && t <= a.T - a.W + r;
-                const float logit = vis ? acc[j] * a.inv_sqrt_d : -INFINITY;
-                float m = logit;
-                for (int s = seg_len / 2; s > 0; s >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, s));
-                const float e = vis ? expf(logit - m) : 0.0f;
-                float se = e, sp = e * w_col;
-                for (int s = seg_len / 2; s > 0; s >>= 1) {
-                    se += __shfl_xor_sync(0xffffffffu, se, s);
-                    sp += __shfl_xor_sync(0xffffffffu, sp, s);
-                }
-                if (valid && (lane & (seg_len - 1)) == 0) {
-                    const int64_t o = (row0 + j0 + j) * a.n_seg + seg;
-                    a.pm[o] = m;
-                    a.ps[o] = se;
-                    a.pp[o] = sp;
+            for (int col = 0; col < 2; ++col) {
+                const int j = nb * 8 + 2 * q4 + col;       // flattened (head, window row)
+                const int r = j % a.W;
+                float lg[2][2], mx[2][2], se[2][2], sp[2][2];
+#pragma unroll
+                for (int mb = 0; mb < 2; ++mb)
+#pragma unroll
+                    for (int h = 0; h < 2; ++h) {
+                        const int t = tile * kTileTokens + mb * 16 + h * 8 + g;
+                        const bool vis = j < a.NR && t < a.T && t <= a.T - a.W + r;
+                        lg[mb][h] = vis ? acc[mb][2 * h + col] * a.inv_sqrt_d : -INFINITY;
+                        mx[mb][h] = lg[mb][h];
+                    }
+                segment_reduce<SEG>(mx, [](float x, float y) { return fmaxf(x, y); });
+#pragma unroll
+                for (int mb = 0; mb < 2; ++mb)
+#pragma unroll
+                    for (int h = 0; h < 2; ++h) {
+                        const int t = tile * kTileTokens + mb * 16 + h * 8 + g;
+                        const float e = lg[mb][h] == -INFINITY ? 0.0f : expf(lg[mb][h] - mx[mb][h]);
+                        se[mb][h] = e;
+                        sp[mb][h] = e / (float)min(a.W, max(1, a.T - t));
+                    }
+                segment_reduce<SEG>(se, [](float x, float y) { return x + y; });
+                segment_reduce<SEG>(sp, [](float x, float y) { return x + y; });
+                if (j < a.NR) {
+#pragma unroll
+                    for (int mb = 0; mb < 2; ++mb)
+#pragma unroll
+                        for (int h = 0; h < 2; ++h) {
+                            const int t = tile * kTileTokens + mb * 16 + h * 8 + g;
+                            if (t < a.T && t % SEG == 0) {   // the segment's first token writes
+                                const int64_t o = (row0 + j) * a.n_seg + t / SEG;
+                                a.pm[o] = mx[mb][h];
+                                a.ps[o] = se[mb][h];
+                                a.pp[o] = sp[mb][h];
+                            }
+                        }
                 }
             }
         }
@@ -447,32 +497,37 @@ extern "C" int llms_chunk_tolerance(const llms_kv_desc *desc, const void *kv, co
     a.Y = t.Y; a.rows = t.rows;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     if ((unsigned)(a.L * a.Hkv) > 65535u) return LLMS_ERR_UNSUPPORTED;
-    const int rt = a.NR <= 8 ? 8 : (a.NR <= 16 ? 16 : 32);
-    const size_t tile_q_bytes = (size_t)((a.NR + rt - 1) / rt * rt) * a.d * 2;
-    const size_t tile_smem = tile_q_bytes + (size_t)kTileWarps * 2 * kTileTokens * a.d * 2;
-    if ((a.d == 64 || a.d == 128 || a.d == 256) && tile_smem <= 200 * 1024) {
-        // tiles through shared memory; enough blocks per (layer, KV head) to fill the GPU a few times over
+    const size_t mma_q_bytes = ((size_t)((a.NR + 7) / 8 * 8) * (a.d * 2 + 16) + 127) / 128 * 128;
+    const size_t mma_smem = mma_q_bytes + (size_t)kTileWarps * 2 * kTileTokens * a.d * 2;
+    if ((a.d == 64 || a.d == 128 || a.d == 256) && mma_smem <= 200 * 1024) {
+        // enough blocks per (layer, KV head) to fill the GPU a few times over
         const int n_tiles = (a.T + kTileTokens - 1) / kTileTokens;
         const int pairs = a.L * a.Hkv;
         int splits = (sm_count() * 6 + pairs - 1) / pairs;
         splits = std::max(1, std::min(splits, (n_tiles + kTileWarps - 1) / kTileWarps));
         const dim3 grid(splits, pairs);
-#define LLMS_LAUNCH_TILE(R, DD)                                                                                                   \
+#define LLMS_LAUNCH_MMA(S, DD)                                                                                                    \
     do {                                                                                                                          \
-        LLMS_CUDA_TRY(cudaFuncSetAttribute(logits_tile_kernel<R, DD>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)tile_smem)); \
-        logits_tile_kernel<R, DD><<<grid, kTileWarps * 32, tile_smem, st>>>(a, t.SEG);                                            \
+        LLMS_CUDA_TRY(cudaFuncSetAttribute(logits_mma_kernel<S, DD>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)mma_smem)); \
+        logits_mma_kernel<S, DD><<<grid, kTileWarps * 32, mma_smem, st>>>(a);                                                     \
     } while (0)
-#define LLMS_LAUNCH_TILE_D(R)                                                       \
-    do {                                                                            \
-        if (a.d == 64) LLMS_LAUNCH_TILE(R, 64);                                     \
-        else if (a.d == 128) LLMS_LAUNCH_TILE(R, 128);                              \
-        else LLMS_LAUNCH_TILE(R, 256);                                              \
-    } while (0)
-        if (rt == 8) LLMS_LAUNCH_TILE_D(8);
-        else if (rt == 16) LLMS_LAUNCH_TILE_D(16);
-        else LLMS_LAUNCH_TILE_D(32);
-#undef LLMS_LAUNCH_TILE_D
-#undef LLMS_LAUNCH_TILE
+#define LLMS_LAUNCH_MMA_SEG(S)                                                      \
+    case S:                                                                         \
+        if (a.d == 64) LLMS_LAUNCH_MMA(S, 64);                                      \
+        else if (a.d == 128) LLMS_LAUNCH_MMA(S, 128);                               \
+        else LLMS_LAUNCH_MMA(S, 256);                                               \
+        break;
+        switch (t.SEG) {
+            LLMS_LAUNCH_MMA_SEG(1)
+            LLMS_LAUNCH_MMA_SEG(2)
+            LLMS_LAUNCH_MMA_SEG(4)
+            LLMS_LAUNCH_MMA_SEG(8)
+            LLMS_LAUNCH_MMA_SEG(16)
+            LLMS_LAUNCH_MMA_SEG(32)
+        default: return LLMS_ERR_UNSUPPORTED;
+        }
+#undef LLMS_LAUNCH_MMA_SEG
+#undef LLMS_LAUNCH_MMA
     } else {
         const size_t q_bytes = (size_t)a.NR * a.d * sizeof(float);
         if (q_bytes > 200 * 1024) return LLMS_ERR_UNSUPPORTED;
