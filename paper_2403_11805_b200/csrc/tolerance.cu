@@ -414,7 +414,7 @@ static int seg_len(int chunk_len)
     return s;
 }
 
-static int row_slices(int rows) { return rows >= 512 ? 16 : (rows >= 64 ? 4 : 1); }
+static int row_slices(int rows) { return rows >= 4096 ? 64 : (rows >= 512 ? 16 : (rows >= 64 ? 4 : 1)); }
 
 struct TolLayout {
     int SEG, n_seg, rows, Y;
