@@ -371,10 +371,61 @@ def run_ours(args):
         dist.destroy_process_group()
 
 
+def run_multiapp(args):
+    """Config 4: 64 contexts of 1024 tokens share a device pool of 512 chunk slots; every step serves 8 contexts that
+    are not resident (LCTRU eviction with compress + copy out, copy in + decompress).  Metric: context switches/s."""
+    import torch
+    from paper_2403_11805_b200 import binding as B, synth
+    from paper_2403_11805_b200.multiapp import MultiApp
+
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the hot path has no CPU fallback")
+    torch.cuda.set_device(int(os.environ.get("LOCAL_RANK", "0")))
+    B.lib()
+    shape = synth.CONFIGS["multiapp"]
+    if args.layers:
+        shape = shape.with_(n_layers=args.layers)
+    per_step, n_slots = 8, 512
+    app = MultiApp(shape, n_slots=n_slots, seed=shape.seed)
+    app.build()
+    for _ in range(max(args.warmup, 3)):
+        app.step(per_step)
+    steps = min(args.steps, 100)
+    sampler = ClockSampler(0)
+    out0, in0 = app.bytes_out, app.bytes_in
+    torch.cuda.synchronize()
+    sampler.begin()
+    t0 = time.perf_counter()
+    for _ in range(steps):
+        app.step(per_step)              # ends with a device synchronisation
+    dt = time.perf_counter() - t0
+    sampler.end()
+    clocks = sampler.finish()
+    chunk_bytes = shape.n_slabs * shape.chunk_len * shape.head_dim * 2
+    chunks_moved = (app.bytes_in - in0) / (sum(app.rec_bytes.values()) / 3)
+    line = {
+        "metric": "context switches/sec", "value": per_step * steps / dt, "unit": "contexts/s", "n_gpus": 1, "steps": steps,
+        "warmup": max(args.warmup, 3), "ms_per_step": dt * 1e3 / steps, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f32 (fp16 in/out, integer codes)", "data": "synthetic",
+        "config": {"workload": shape.name, "contexts": shape.n_contexts, "tokens_per_context": shape.n_tokens,
+                   "chunk_len": shape.chunk_len, "layers": shape.n_layers, "pool_slots": n_slots, "contexts_per_step": per_step,
+                   "l2": "pool of %.0f MiB, far larger than L2" % (n_slots * chunk_bytes / 2 ** 20)},
+        "e2e": {"value": per_step * steps / dt, "unit": "contexts/s",
+                "h2d_bytes_per_step": (app.bytes_in - in0) // steps, "d2h_bytes_per_step": (app.bytes_out - out0) // steps,
+                "h2d_gbs": (app.bytes_in - in0) / dt / 1e9, "d2h_gbs": (app.bytes_out - out0) / dt / 1e9,
+                "what": "LCTRU eviction (compress + copy out) and load (copy in + decompress) per step, wall clock"},
+        "fp16_gbs_through_codec": 2 * chunks_moved * chunk_bytes / dt / 1e9,
+        "gpu_launches": None, "clocks": clocks,
+    }
+    print(json.dumps(line))
+
+
 def main():
     args = parse_args()
     if args.impl == "reference":
         run_reference(args)
+    elif args.workload == "multiapp":
+        run_multiapp(args)
     else:
         run_ours(args)
 
