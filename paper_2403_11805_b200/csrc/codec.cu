@@ -501,7 +501,10 @@ __device__ __forceinline__ void load_unit_codes(const CodecArgs &a, const UnitPo
     }
 }
 
-// 16 codes -> 8 half2 holding the codes as exact fp16 integers.  0x6400 | q is the fp16 number 1024 + q.
+// 16 codes -> 8 half2 holding the codes as exact fp16 integers.  0x6400 | q is the fp16 number 1024 + q, so a
+// code only has to be moved to the low bits of a 16-bit half.  At 8 bits one byte permute places two codes; at 4
+// and 2 bits one shift and one and-or place the two codes that sit 16 bits apart.  which[e] tells where code e
+// ended up: half2 index * 2 + (0 low half, 1 high half).
 template <int BITS>
 __device__ __forceinline__ void codes_to_half2(const uint32_t *c, __half2 (&q)[8])
 {
@@ -514,28 +517,28 @@ __device__ __forceinline__ void codes_to_half2(const uint32_t *c, __half2 (&q)[8
         }
     } else if constexpr (BITS == 4) {
 #pragma unroll
-        for (int m = 0; m < 2; ++m) {
-            const uint32_t even = c[m] & 0x0F0F0F0Fu;         // codes 8m + 0, 2, 4, 6 in bytes 0..3
-            const uint32_t odd = (c[m] >> 4) & 0x0F0F0F0Fu;   // codes 8m + 1, 3, 5, 7
+        for (int m = 0; m < 2; ++m)
 #pragma unroll
-            for (int b = 0; b < 4; ++b) {
-                const uint32_t pair = __byte_perm(even, odd, (b) | ((4 + b) << 8)) & 0x00FF00FFu;
-                q[4 * m + b] = __hsub2(as_h2(pair | 0x64006400u), k1024);
-            }
-        }
+            for (int s = 0; s < 4; ++s)  // codes 8m + s (low half) and 8m + s + 4 (high half)
+                q[4 * m + s] = __hsub2(as_h2(((c[m] >> (4 * s)) & 0x000F000Fu) | 0x64006400u), k1024);
     } else {
-        const uint32_t r0 = c[0] & 0x03030303u;          // codes 0, 4, 8, 12
-        const uint32_t r1 = (c[0] >> 2) & 0x03030303u;   // codes 1, 5, 9, 13
-        const uint32_t r2 = (c[0] >> 4) & 0x03030303u;   // codes 2, 6, 10, 14
-        const uint32_t r3 = (c[0] >> 6) & 0x03030303u;   // codes 3, 7, 11, 15
 #pragma unroll
-        for (int b = 0; b < 4; ++b) {
-            const uint32_t p01 = __byte_perm(r0, r1, (b) | ((4 + b) << 8)) & 0x00FF00FFu;
-            const uint32_t p23 = __byte_perm(r2, r3, (b) | ((4 + b) << 8)) & 0x00FF00FFu;
-            q[2 * b] = __hsub2(as_h2(p01 | 0x64006400u), k1024);
-            q[2 * b + 1] = __hsub2(as_h2(p23 | 0x64006400u), k1024);
-        }
+        for (int s = 0; s < 8; ++s)      // codes s (low half) and s + 8 (high half)
+            q[s] = __hsub2(as_h2(((c[0] >> (2 * s)) & 0x00030003u) | 0x64006400u), k1024);
     }
+}
+
+// the fp16 bit pattern of code e (0..15) inside q[] as laid out above
+template <int BITS>
+__device__ __forceinline__ unsigned short code_half(const __half2 (&q)[8], int e)
+{
+    int idx, hi;
+    if constexpr (BITS == 8) { idx = e / 2; hi = e % 2; }
+    else if constexpr (BITS == 4) { idx = 4 * (e / 8) + e % 4; hi = (e % 8) / 4; }
+    else { idx = e % 8; hi = e / 8; }
+    unsigned short lo_h, hi_h;
+    split_halves(as_u32(q[idx]), lo_h, hi_h);
+    return hi ? hi_h : lo_h;
 }
 
 // 16 decoded values.  q*scale is exact in binary32, so the mixed-precision fused form rounds once, as
@@ -548,10 +551,8 @@ __device__ __forceinline__ void dequantize_piece(const uint32_t *c, unsigned sho
     codes_to_half2<BITS>(c, q);
 #pragma unroll
     for (int k = 0; k < 8; ++k) {
-        unsigned short q0, q1;
-        split_halves(as_u32(q[k]), q0, q1);
-        float y0 = fma_f32_f16(q0, scale_h, zero);
-        float y1 = fma_f32_f16(q1, scale_h, zero);
+        float y0 = fma_f32_f16(code_half<BITS>(q, 2 * k), scale_h, zero);
+        float y1 = fma_f32_f16(code_half<BITS>(q, 2 * k + 1), scale_h, zero);
         if constexpr (CLAMP) {
             y0 = fminf(y0, 65504.0f);
             y1 = fminf(y1, 65504.0f);
