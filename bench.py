@@ -46,6 +46,15 @@ def measured_peaks():
     return 6650.0, "fallback"
 
 
+# dram__bytes_read.sum + dram__bytes_write.sum of one stage (its three launches, one per bit-width) on the full
+# llama7b workload, from one ncu capture of the kernels as they are now (profiles/codec_and_score_kernels_llama7b.md).
+# Set an entry to None when its kernel changes.
+NCU_DRAM_TRAFFIC = {
+    ("llama7b", 32, "compress_kernel"): 2147632896 + 592608000,
+    ("llama7b", 32, "decompress_kernel"): 668158208 + 1962685952,
+}
+
+
 def target_bits(shape):
     """Bit mix of the workload by chunk rank: counts as the rank -> bits rule gives them."""
     import numpy as np
@@ -333,7 +342,8 @@ def run_ours(args):
     achieved = algo_bytes / (k_ms[dominant] * 1e-3) / 1e9
     roofline = {
         "kernel": dominant, "bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
-        "peak_source": f"{peak_kind} copy bandwidth", "traffic": None,
+        "peak_source": f"{peak_kind} copy bandwidth", "launches_per_stage": 3,
+        "traffic": NCU_DRAM_TRAFFIC.get((shape.name, shape.n_layers, dominant)),
         "algorithmic_bytes_per_launch": algo_bytes,
         "frac_of_nominal_8000": achieved / 8000.0,
         "per_stage": {
