@@ -224,8 +224,10 @@ def run_ours(args):
     W = shape.window
     frac = shape.frac if shape.frac is not None else (1 / 3, 1 / 3, 1 / 3)
     # every rank owns one context of the workload (contexts are independent: no data-path collective)
-    kv = synth.kv_tensor(shape, device="cuda", context=rank)
-    q_win = synth.q_window(shape, W, device="cuda", context=rank)
+    from paper_2403_11805_b200 import sharding
+    my_context = sharding.contexts_of_rank(world, rank, world)[0]
+    kv = synth.kv_tensor(shape, device="cuda", context=my_context)
+    q_win = synth.q_window(shape, W, device="cuda", context=my_context)
     d = B.desc_of(shape)
     n = shape.n_chunks
     ids = np.arange(n, dtype=np.uint32)
@@ -289,10 +291,7 @@ def run_ours(args):
     comp_ms = sum(e[1].elapsed_time(e[2]) for e in events) / args.steps
     decomp_ms = sum(e[2].elapsed_time(e[3]) for e in events) / args.steps
     ms_per_step = span_ms / args.steps
-    if dist is not None:
-        t = torch.tensor([ms_per_step, tol_ms, comp_ms, decomp_ms], dtype=torch.float64, device="cuda")
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms_per_step, tol_ms, comp_ms, decomp_ms = t.tolist()
+    ms_per_step, tol_ms, comp_ms, decomp_ms = sharding.max_over_ranks([ms_per_step, tol_ms, comp_ms, decomp_ms], dist, "cuda")
     kv_bytes = shape.n_elements * 2
     value = world * 2 * kv_bytes / (ms_per_step * 1e-3) / 1e9
 
@@ -322,10 +321,7 @@ def run_ours(args):
     e1.record(stream)
     barrier()
     e2e_ms = e0.elapsed_time(e1) / args.e2e_steps
-    if dist is not None:
-        t = torch.tensor([e2e_ms], dtype=torch.float64, device="cuda")
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        e2e_ms = float(t.item())
+    e2e_ms = sharding.max_over_ranks([e2e_ms], dist, "cuda")[0]
     e2e_value = world * 2 * kv_bytes / (e2e_ms * 1e-3) / 1e9
     clocks = sampler.finish() if sampler else None
 
