@@ -630,6 +630,7 @@ __global__ void __launch_bounds__(kThreads, 3) decompress_kernel(const CodecArgs
 }  // namespace llms
 
 #include "codec_bulk.cuh"
+#include "codec_cw.cuh"
 
 namespace llms {
 
@@ -766,7 +767,7 @@ static int check_common(const llms_kv_desc *desc, int n, const void *workspace, 
 {
     int rc = check_desc_codec(desc);
     if (rc) return rc;
-    if (desc->quant_mode != 0) return LLMS_ERR_UNSUPPORTED;
+    if (desc->quant_mode == 1 && desc->head_dim != 64 && desc->head_dim != 128 && desc->head_dim != 256) return LLMS_ERR_UNSUPPORTED;
     if (n < 0) return LLMS_ERR_INVALID_ARG;
     if (n == 0) return LLMS_OK;
     if (!workspace) return LLMS_ERR_INVALID_ARG;
@@ -832,6 +833,14 @@ extern "C" int llms_compress_chunks(const llms_kv_desc *desc, const void *kv, co
         if (groups.count[k] == 0) continue;
         const CodecArgs b = args_for_group(a, groups, k);
         cudaError_t attr_err = cudaSuccess;
+        if (desc->quant_mode == 1) {
+            const int64_t items = (int64_t)b.n * b.n_slabs;
+            if (k == 0) compress_cw_kernel<8><<<grid_for(compress_cw_kernel<8>, items), kThreads, 0, st>>>(b, desc->head_dim, desc->chunk_len);
+            else if (k == 1) compress_cw_kernel<4><<<grid_for(compress_cw_kernel<4>, items), kThreads, 0, st>>>(b, desc->head_dim, desc->chunk_len);
+            else compress_cw_kernel<2><<<grid_for(compress_cw_kernel<2>, items), kThreads, 0, st>>>(b, desc->head_dim, desc->chunk_len);
+            LLMS_CUDA_TRY(cudaGetLastError());
+            continue;
+        }
         rc = dispatch_group(desc->group_size, [&](auto g) {
             constexpr int kG = decltype(g)::value;
             if constexpr (kUseBulkCompress && kG >= kLaneElems) {
@@ -900,6 +909,14 @@ extern "C" int llms_decompress_chunks(const llms_kv_desc *desc, const void *buf,
     for (int k = 0; k < 3; ++k) {
         if (groups.count[k] == 0) continue;
         const CodecArgs b = args_for_group(a, groups, k);
+        if (desc->quant_mode == 1) {
+            const int64_t items = (int64_t)b.n * b.n_slabs;
+            if (k == 0) decompress_cw_kernel<8><<<grid_for(decompress_cw_kernel<8>, items), kThreads, 0, st>>>(b, desc->head_dim, desc->chunk_len);
+            else if (k == 1) decompress_cw_kernel<4><<<grid_for(decompress_cw_kernel<4>, items), kThreads, 0, st>>>(b, desc->head_dim, desc->chunk_len);
+            else decompress_cw_kernel<2><<<grid_for(decompress_cw_kernel<2>, items), kThreads, 0, st>>>(b, desc->head_dim, desc->chunk_len);
+            LLMS_CUDA_TRY(cudaGetLastError());
+            continue;
+        }
         rc = dispatch_group(desc->group_size, [&](auto g) {
             constexpr int kG = decltype(g)::value;
 #define LLMS_LAUNCH(BITS)                                                                                                   \

@@ -240,3 +240,72 @@ def test_full_size_sampled_chunks(name):
         t_idx = torch.arange(x.shape[0], device="cuda") // (sh.head_dim // G) % sh.n_tokens
         qmax = (2 ** chunk_bits[t_idx // CL] - 1).float()
         assert bool((err8 <= 0.5 / qmax * (1 + 2.0 ** -8) + 2.0 ** -10 * x.abs().max(1).values / (hi - lo).squeeze(1).clamp_min(1e-20)).all())
+
+
+# ----------------------------------------------------------------- channel-wise mode (quant_mode 1)
+
+CW_SHAPES = [
+    synth.CONFIGS["tiny"],                                                        # d 64: 4 lanes per column
+    synth.CONFIGS["llama7b"].with_(n_layers=1, n_tokens=256),                     # d 128
+    synth.CONFIGS["gemma2b"].with_(n_layers=2, n_tokens=160),                     # d 256, MQA
+    synth.CONFIGS["multiapp"].with_(n_layers=1, n_kv_heads=4, n_q_heads=4, n_tokens=128),   # chunk_len 32
+    synth.KVShape("cw_ragged", 2, 3, 3, 64, 53, 5, 64, seed=21),                  # chunk_len 5, tail tokens
+    synth.KVShape("cw_one_token", 1, 2, 2, 64, 4, 1, 64, seed=22),                # fewer tokens than lanes per column
+    synth.KVShape("cw_24", 1, 2, 2, 128, 100, 24, 128, seed=23),
+]
+
+
+@pytest.mark.parametrize("sh", CW_SHAPES, ids=[s.name for s in CW_SHAPES])
+def test_channel_wise_mode_matches_oracle(sh):
+    kv = synth.kv_tensor(sh)
+    rng = np.random.default_rng(5)
+    ids = rng.permutation(sh.n_chunks).astype(np.uint32)
+    bits = np.array([(8, 4, 2)[i % 3] for i in range(sh.n_chunks)], dtype=np.uint8)
+    got_buf, got_meta, buf_dev = gpu_compress(sh, kv.cuda(), ids, bits, mode=1)
+    want_buf, want_meta = oracle.compress_chunks(odesc(sh, 1), bits_view(kv), ids, bits)
+    assert first_mismatch(got_buf, want_buf) is None
+    assert_meta_equal(got_meta, want_meta)
+    out_dev = torch.full(kv.shape, float("nan"), dtype=torch.float16, device="cuda")
+    assert gpu_decompress(sh, buf_dev, got_meta, out_dev, mode=1) == 0
+    want = np.full(kv.numel(), 0x7E00, dtype=np.uint16).reshape(kv.shape)
+    oracle.decompress_chunks(odesc(sh, 1), want_buf, want_meta, want)
+    assert first_mismatch(bits_view(out_dev).reshape(-1), want.reshape(-1)) is None
+
+
+def test_channel_wise_special_values_and_outliers():
+    sh = synth.KVShape("cw_special", 1, 2, 2, 64, 64, 16, 64, seed=9)
+    kv = synth.kv_tensor(sh)
+    kv[0, 0, 0, 0:16, 3] = 2.5                       # a constant channel: scale 0, reproduced exactly
+    kv[0, 0, 0, 0:16, 4] = torch.tensor([-0.0, 0.0] * 8).half()
+    kv[0, 0, 0, 0:16, 5] = torch.linspace(-6e-7, 6e-7, 16).half()   # subnormal scale: the clamped path
+    kv[0, 0, 0, 0, 6] = 65504.0
+    kv[0, 0, 0, 1, 6] = -65504.0                     # decode saturates
+    ids = np.arange(sh.n_chunks, dtype=np.uint32)
+    for b in (8, 4, 2):
+        bits = np.full(sh.n_chunks, b, dtype=np.uint8)
+        got_buf, got_meta, buf_dev = gpu_compress(sh, kv.cuda(), ids, bits, mode=1)
+        want_buf, want_meta = oracle.compress_chunks(odesc(sh, 1), bits_view(kv), ids, bits)
+        assert first_mismatch(got_buf, want_buf) is None
+        assert_meta_equal(got_meta, want_meta)
+        out_dev = torch.zeros_like(kv, device="cuda")
+        assert gpu_decompress(sh, buf_dev, got_meta, out_dev, mode=1) == 0
+        want = np.zeros(kv.numel(), dtype=np.uint16).reshape(kv.shape)
+        oracle.decompress_chunks(odesc(sh, 1), want_buf, want_meta, want)
+        assert first_mismatch(bits_view(out_dev).reshape(-1), want.reshape(-1)) is None
+        assert torch.equal(out_dev[0, 0, 0, 0:16, 3].cpu(), kv[0, 0, 0, 0:16, 3])
+        assert bool(torch.isfinite(out_dev.float()).all())
+
+
+def test_channel_wise_outlier_channels_cost_less_error_than_token_groups():
+    # the two 10x outlier channels of K stretch every token group's range; channel-wise groups isolate them
+    sh = synth.CONFIGS["llama7b"].with_(n_layers=1, n_tokens=256)
+    kv = synth.kv_tensor(sh)
+    ids = np.arange(sh.n_chunks, dtype=np.uint32)
+    bits = np.full(sh.n_chunks, 4, dtype=np.uint8)
+    err = {}
+    for mode in (0, 1):
+        _, meta, buf_dev = gpu_compress(sh, kv.cuda(), ids, bits, mode=mode)
+        out_dev = torch.zeros_like(kv, device="cuda")
+        assert gpu_decompress(sh, buf_dev, meta, out_dev, mode=mode) == 0
+        err[mode] = float((out_dev.cpu().float() - kv.float())[:, 0].pow(2).mean())     # K half
+    assert err[1] < err[0]
