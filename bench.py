@@ -35,6 +35,9 @@ def parse_args():
     p.add_argument("--layers", type=int, default=0, help="use only this many layers (smaller cases for profiler captures)")
     p.add_argument("--e2e-steps", type=int, default=10)
     p.add_argument("--no-cpu-baseline", action="store_true")
+    p.add_argument("--quant-mode", type=int, default=0, choices=[0, 1],
+                   help="0: groups of group_size channels of one token (the metric's setting); 1: one group per channel "
+                        "across the chunk's tokens")
     return p.parse_args()
 
 
@@ -228,7 +231,7 @@ def run_ours(args):
     my_context = sharding.contexts_of_rank(world, rank, world)[0]
     kv = synth.kv_tensor(shape, device="cuda", context=my_context)
     q_win = synth.q_window(shape, W, device="cuda", context=my_context)
-    d = B.desc_of(shape)
+    d = B.desc_of(shape, quant_mode=args.quant_mode)
     n = shape.n_chunks
     ids = np.arange(n, dtype=np.uint32)
     n8, n4, n2 = target_bits(shape)
@@ -339,7 +342,7 @@ def run_ours(args):
     roofline = {
         "kernel": dominant, "bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
         "peak_source": f"{peak_kind} copy bandwidth", "launches_per_stage": 3,
-        "traffic": NCU_DRAM_TRAFFIC.get((shape.name, shape.n_layers, dominant)),
+        "traffic": NCU_DRAM_TRAFFIC.get((shape.name, shape.n_layers, dominant)) if args.quant_mode == 0 else None,
         "algorithmic_bytes_per_launch": algo_bytes,
         "frac_of_nominal_8000": achieved / 8000.0,
         "per_stage": {
@@ -358,7 +361,7 @@ def run_ours(args):
         "dtype": "f32 (fp16 in/out, integer codes)", "data": "synthetic",
         "config": {"workload": shape.name, "layers": shape.n_layers, "kv_heads": shape.n_kv_heads, "head_dim": shape.head_dim,
                    "tokens": shape.n_tokens, "chunk_len": shape.chunk_len, "group_size": shape.group_size,
-                   "window": W, "bits_8_4_2": [n8, n4, n2], "contexts_per_gpu": 1,
+                   "window": W, "bits_8_4_2": [n8, n4, n2], "contexts_per_gpu": 1, "quant_mode": args.quant_mode,
                    "l2": "inputs larger than L2 (fp16 KV %.0f MiB per context)" % (kv_bytes / 2 ** 20),
                    "step": "score + rank->bits + compress + decompress of one context"},
         "contexts_per_s": world / (ms_per_step * 1e-3),
@@ -370,7 +373,7 @@ def run_ours(args):
         "roofline": roofline, "clocks": clocks,
         "wall_ms_per_step": t_wall * 1e3 / args.steps,
     }
-    if world == 1 and not args.no_cpu_baseline:
+    if world == 1 and not args.no_cpu_baseline and args.quant_mode == 0:
         line["cpu_baseline"] = cpu_baseline(shape, kv, q_win)
     print(json.dumps(line))
     if dist is not None:
