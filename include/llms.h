@@ -197,6 +197,15 @@ int llms_chunk_tolerance_from_probs(const llms_kv_desc *desc, const float *probs
  * floor((f8+f4)*n + 1/2) get 4, the rest 2 - low density means high tolerance means fewer bits. */
 int llms_assign_bits(const float *scores, int n, const float frac[3], uint8_t *bits_out, uint32_t *order_out);
 
+/* Eq. 3: the shares of chunks per level that maximise the context's information under a global average
+ * ratio, for the levels {8/8, 4/8, 2/8} (Sec. 3.2: one free variable is left).  A chunk at level w keeps
+ * weight ratio_w of its density (reading of the garbled 1/ratio_w; see the format notes of the build).
+ * ratio_global in [0.25, 1] is relative to 8 bits: f8 + f4/2 + f2/4 = ratio_global, hence
+ * f2 = 2*f8 + 2 - 4*ratio_global.  Every count n8 of 8-bit chunks is tried on the density-ordered list
+ * (n2 = floor(2*n8 + (2 - 4*ratio_global)*n + 1/2), n4 the rest); the best wins, the smaller n8 on a tie.
+ * frac_out = {n8, n4, n2} / n, ready for llms_assign_bits.  scores: host, n > 0 values. */
+int llms_optimize_thresholds(const float *scores, int n, float ratio_global, float frac_out[3]);
+
 /* Sec. 3.4 (ii): eviction order over the rows that are resident and not locked - the 8-bit
  * sub-queue first, then 4, then 2 ("heavy chunks first"), least recently used first inside a
  * sub-queue, ties by (ctx_id, chunk_id).  order_out (n entries) receives row indices; the return

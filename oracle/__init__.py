@@ -204,6 +204,15 @@ def assign_bits(scores, frac):
     return bits, order
 
 
+def optimize_thresholds(scores, ratio_global):
+    """-> (frac float32[3], counts int[3]) for the levels 8 / 4 / 2 bits."""
+    s = np.ascontiguousarray(scores, dtype=np.float32)
+    frac = (C.c_float * 3)()
+    counts = (C.c_int * 3)()
+    _check(lib().orc_optimize_thresholds(_ptr(s), int(s.size), C.c_float(ratio_global), frac, counts), "optimize_thresholds")
+    return np.array(list(frac), dtype=np.float32), list(counts)
+
+
 def lctru_order(table):
     t = np.ascontiguousarray(table, dtype=STATE_DTYPE)
     order = np.empty(max(len(t), 1), dtype=np.uint32)

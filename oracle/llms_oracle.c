@@ -530,6 +530,54 @@ int orc_assign_bits(const float *scores, int n, const float frac[3], uint8_t *bi
     return ORC_OK;
 }
 
+/* ------------------------------------------------------ Eq. 3: thresholds */
+
+/* Thresholds of Eq. 2 chosen as Eq. 3 asks: maximise the context's information
+ *   ctxInfo = sum over levels w of weight_w * (sum of D_i of the chunks at level w)
+ * under a global average ratio, for the three levels {8/8, 4/8, 2/8} (Sec. 3.2: with three levels
+ * one free variable is left).  Reading: weight_w = ratio_w (a chunk kept at more bits keeps more
+ * of its information); the printed 1/ratio_w would reward compressing the densest chunks most.
+ * With shares f8 + f4 + f2 = 1 and f8 + f4/2 + f2/4 = R:  f2 = 2*f8 + 2 - 4R.
+ * Chunks are taken in density order (as in orc_assign_bits); for every count n8 = 0..n the count
+ * n2 = floor(2*n8 + (2 - 4R)*n + 1/2) follows, n4 is the rest, and with prefix sums
+ * P[k] = D(rank 0) + ... + D(rank k-1) (added in that order, binary64)
+ *   ctxInfo(n8) = P[n8] + (P[n-n2] - P[n8])/2 + (P[n] - P[n-n2])/4.
+ * The largest wins, the smaller n8 on a tie.  counts_out = {n8, n4, n2}; frac_out = counts / n. */
+int orc_optimize_thresholds(const float *scores, int n, float ratio_global, float frac_out[3], int counts_out[3])
+{
+    if (n <= 0 || !scores) return ORC_ERR_ARG;
+    const double R = (double)ratio_global;
+    if (!(R >= 0.25 && R <= 1.0)) return ORC_ERR_ARG;
+    uint32_t *ord = (uint32_t *)malloc(sizeof(uint32_t) * (size_t)n);
+    double *P = (double *)malloc(sizeof(double) * (size_t)(n + 1));
+    for (int i = 0; i < n; ++i) ord[i] = (uint32_t)i;
+    for (int i = 1; i < n; ++i) {
+        uint32_t k = ord[i];
+        int j = i - 1;
+        while (j >= 0 && scores[ord[j]] < scores[k]) { ord[j + 1] = ord[j]; --j; }
+        ord[j + 1] = k;
+    }
+    P[0] = 0.0;
+    for (int k = 0; k < n; ++k) P[k + 1] = P[k] + (double)scores[ord[k]];
+    int best8 = -1, best2 = 0;
+    double best = 0.0;
+    for (int n8 = 0; n8 <= n; ++n8) {
+        const double x = 2.0 * n8 + (2.0 - 4.0 * R) * n;
+        const long n2 = (long)floor(x + 0.5);
+        if (n2 < 0 || n8 + n2 > n) continue;
+        const double info = P[n8] + (P[n - n2] - P[n8]) / 2.0 + (P[n] - P[n - n2]) / 4.0;
+        if (best8 < 0 || info > best) { best8 = n8; best2 = (int)n2; best = info; }
+    }
+    free(ord);
+    free(P);
+    if (best8 < 0) return ORC_ERR_ARG;
+    counts_out[0] = best8;
+    counts_out[1] = n - best8 - best2;
+    counts_out[2] = best2;
+    for (int w = 0; w < 3; ++w) frac_out[w] = (float)((double)counts_out[w] / (double)n);
+    return ORC_OK;
+}
+
 /* ------------------------------------------------------------- LCTRU order */
 
 static int lctru_before(const orc_chunk_state *a, const orc_chunk_state *b)

@@ -59,6 +59,7 @@ _SIGNATURES = {
     "llms_chunk_tolerance_from_probs": (C.c_int, [C.c_void_p, C.c_void_p, C.c_int, C.c_void_p, C.c_void_p,
                                                   C.c_uint64, C.c_void_p]),
     "llms_assign_bits": (C.c_int, [C.c_void_p, C.c_int, C.c_void_p, C.c_void_p, C.c_void_p]),
+    "llms_optimize_thresholds": (C.c_int, [C.c_void_p, C.c_int, C.c_float, C.c_void_p]),
     "llms_lctru_order": (C.c_int, [C.c_void_p, C.c_int, C.c_void_p]),
     "llms_swap_out": (C.c_int, [C.c_void_p, C.c_void_p, C.c_int, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p,
                                 C.c_void_p]),
@@ -257,6 +258,13 @@ def assign_bits(scores, frac):
     order = np.empty(s.size, dtype=np.uint32)
     _check(lib().llms_assign_bits(_ptr(s), int(s.size), _ptr(f), _ptr(bits), _ptr(order)), "llms_assign_bits")
     return bits, order
+
+
+def optimize_thresholds(scores, ratio_global):
+    s = np.ascontiguousarray(scores, dtype=np.float32)
+    frac = np.zeros(3, dtype=np.float32)
+    _check(lib().llms_optimize_thresholds(_ptr(s), int(s.size), float(ratio_global), _ptr(frac)), "llms_optimize_thresholds")
+    return frac
 
 
 def lctru_order(table):

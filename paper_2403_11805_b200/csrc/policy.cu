@@ -26,6 +26,37 @@ extern "C" int llms_assign_bits(const float *scores, int n, const float frac[3],
     return LLMS_OK;
 }
 
+extern "C" int llms_optimize_thresholds(const float *scores, int n, float ratio_global, float frac_out[3])
+{
+    if (n <= 0 || !scores || !frac_out) return LLMS_ERR_INVALID_ARG;
+    const double R = (double)ratio_global;
+    if (!(R >= 0.25 && R <= 1.0)) return LLMS_ERR_INVALID_ARG;
+    std::vector<uint32_t> order(n);
+    std::iota(order.begin(), order.end(), 0u);
+    std::stable_sort(order.begin(), order.end(), [&](uint32_t a, uint32_t b) { return scores[a] > scores[b]; });
+    // prefix[k] = density of the k densest chunks, added in rank order
+    std::vector<double> prefix(n + 1, 0.0);
+    for (int k = 0; k < n; ++k) prefix[k + 1] = prefix[k] + (double)scores[order[k]];
+    long best8 = -1, best2 = 0;
+    double best = 0.0;
+    for (long n8 = 0; n8 <= n; ++n8) {
+        // shares: f8 + f4 + f2 = 1 and f8 + f4/2 + f2/4 = R  =>  f2 = 2 f8 + 2 - 4R
+        const long n2 = (long)std::floor(2.0 * n8 + (2.0 - 4.0 * R) * n + 0.5);
+        if (n2 < 0 || n8 + n2 > n) continue;
+        const double info = prefix[n8] + (prefix[n - n2] - prefix[n8]) / 2.0 + (prefix[n] - prefix[n - n2]) / 4.0;
+        if (best8 < 0 || info > best) {
+            best8 = n8;
+            best2 = n2;
+            best = info;
+        }
+    }
+    if (best8 < 0) return LLMS_ERR_INVALID_ARG;
+    frac_out[0] = (float)((double)best8 / n);
+    frac_out[1] = (float)((double)(n - best8 - best2) / n);
+    frac_out[2] = (float)((double)best2 / n);
+    return LLMS_OK;
+}
+
 extern "C" int llms_lctru_order(const llms_chunk_state *table, int n, uint32_t *order_out)
 {
     if (n < 0 || (n > 0 && (!table || !order_out))) return LLMS_ERR_INVALID_ARG;

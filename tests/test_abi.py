@@ -63,6 +63,25 @@ def test_assign_bits_matches_oracle_bit_for_bit():
         assert np.array_equal(gb, ob) and np.array_equal(go, oo)
 
 
+def test_optimize_thresholds_matches_oracle_bit_for_bit():
+    rng = np.random.default_rng(2)
+    for n in (1, 2, 5, 32, 256, 512):
+        for R in (0.5, 0.3, 0.8, 1.0, 0.25):
+            for ties in (False, True):
+                s = (rng.random(n) ** 3).astype(np.float32)
+                if ties:
+                    s = np.round(s * 4) / 4
+                try:
+                    want, _ = oracle.optimize_thresholds(s, R)
+                except RuntimeError:                   # no integer split meets the ratio (tiny n): both refuse
+                    with pytest.raises(B.LlmsError):
+                        B.optimize_thresholds(s, R)
+                    continue
+                assert np.array_equal(B.optimize_thresholds(s, R).view(np.uint32), want.view(np.uint32))
+    with pytest.raises(B.LlmsError):
+        B.optimize_thresholds([0.1, 0.2], 0.2)
+
+
 def test_lctru_order_matches_oracle_bit_for_bit():
     rng = np.random.default_rng(1)
     for n in (0, 1, 5, 64, 2048):

@@ -90,3 +90,49 @@ def test_lctru_is_the_unique_sorted_permutation():
         for a, b in zip(order, order[1:]):         # every adjacent pair respects the precedence
             ra, rb = rows[a], rows[b]
             assert (-ra[2], ra[5], ra[0], ra[1]) < (-rb[2], rb[5], rb[0], rb[1])
+
+
+# ----------------------------------------------------------------- Eq. 3: thresholds
+
+def test_thresholds_uniform_density_means_uniform_bits():
+    # every chunk equally dense: nothing is gained by moving bits around, the tie goes to n8 = 0 -> all 4-bit
+    frac, counts = oracle.optimize_thresholds([0.25] * 12, 0.5)
+    assert counts == [0, 12, 0] and frac.tolist() == [0.0, 1.0, 0.0]
+
+
+def test_thresholds_one_dominant_chunk():
+    # one chunk carries all the density: it alone keeps 8 bits, paid for by two chunks at 2 bits (f2 = 2 f8 at 50%)
+    frac, counts = oracle.optimize_thresholds([0.001] * 5 + [0.9] + [0.001] * 6, 0.5)
+    assert counts == [1, 9, 2]
+
+
+def test_thresholds_closed_form_relation_and_achieved_ratio():
+    rng = np.random.default_rng(4)
+    for n in (3, 16, 32, 256, 511):
+        for R in (0.5, 0.4, 0.7, 0.25, 1.0):
+            s = rng.random(n) ** 3
+            frac, (n8, n4, n2) = oracle.optimize_thresholds(s, R)
+            assert n8 + n4 + n2 == n and min(n8, n4, n2) >= 0
+            assert n2 == int(np.floor(2 * n8 + (2 - 4 * np.float64(np.float32(R))) * n + 0.5))
+            assert abs((n8 + n4 / 2 + n2 / 4) / n - R) <= 1 / (8 * n) + 1e-7
+            bits, _ = oracle.assign_bits(s, frac)          # the shares reproduce the counts
+            assert [int((bits == b).sum()) for b in (8, 4, 2)] == [n8, n4, n2]
+
+
+def test_thresholds_brute_force_over_all_level_assignments():
+    # every assignment of levels to chunks (not only rank-ordered ones) whose counts obey the ratio rule
+    rng = np.random.default_rng(9)
+    for n in (4, 6, 7):
+        for _ in range(6):
+            s = (rng.random(n) ** 2).astype(np.float32)
+            _, (n8, n4, n2) = oracle.optimize_thresholds(s, 0.5)
+            order = np.argsort(-s, kind="stable")
+            got = s[order[:n8]].sum(dtype=np.float64) + s[order[n8:n8 + n4]].sum(dtype=np.float64) / 2 \
+                + s[order[n8 + n4:]].sum(dtype=np.float64) / 4
+            best = -1.0
+            for levels in itertools.product((1.0, 0.5, 0.25), repeat=n):
+                c8, c2 = levels.count(1.0), levels.count(0.25)
+                if c2 != 2 * c8:                      # f2 = 2 f8 at a 50% global ratio
+                    continue
+                best = max(best, float(np.dot(np.array(levels), s.astype(np.float64))))
+            assert got == pytest.approx(best, rel=1e-12)
