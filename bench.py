@@ -35,6 +35,7 @@ def parse_args():
     p.add_argument("--layers", type=int, default=0, help="use only this many layers (smaller cases for profiler captures)")
     p.add_argument("--e2e-steps", type=int, default=10)
     p.add_argument("--no-cpu-baseline", action="store_true")
+    p.add_argument("--aot", action="store_true", help="multiapp: swap served contexts out ahead of time (Sec. 3.4 i)")
     p.add_argument("--quant-mode", type=int, default=0, choices=[0, 1],
                    help="0: groups of group_size channels of one token (the metric's setting); 1: one group per channel "
                         "across the chunk's tokens")
@@ -419,7 +420,7 @@ def run_multiapp(args):
     if args.layers:
         shape = shape.with_(n_layers=args.layers)
     per_step, n_slots = 8, 512
-    app = MultiApp(shape, n_slots=n_slots, seed=shape.seed)
+    app = MultiApp(shape, n_slots=n_slots, seed=shape.seed, aot=args.aot)
     app.build()
     for _ in range(max(args.warmup, 3)):
         app.step(per_step)
@@ -448,6 +449,8 @@ def run_multiapp(args):
                 "h2d_gbs": (app.bytes_in - in0) / dt / 1e9, "d2h_gbs": (app.bytes_out - out0) / dt / 1e9,
                 "what": "LCTRU eviction (compress + copy out) and load (copy in + decompress) per step, wall clock"},
         "fp16_gbs_through_codec": 2 * chunks_moved * chunk_bytes / dt / 1e9,
+        "aot_swap_out": bool(args.aot),
+        "switch_latency_ms": statistics.mean(app.ready_ms[-steps:]),   # step start until the 8 working sets are resident
         "gpu_launches": None, "clocks": clocks,
     }
     print(json.dumps(line))

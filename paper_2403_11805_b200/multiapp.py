@@ -17,9 +17,11 @@ from . import synth
 
 
 class MultiApp:
-    def __init__(self, shape, n_slots, frac=(1 / 3, 1 / 3, 1 / 3), seed=1, log_ops=False):
-        """shape: synth.KVShape of ONE context (n_contexts of them); n_slots: device pool size in chunks."""
-        self.shape, self.n_slots, self.frac, self.seed = shape, n_slots, frac, seed
+    def __init__(self, shape, n_slots, frac=(1 / 3, 1 / 3, 1 / 3), seed=1, log_ops=False, aot=False):
+        """shape: synth.KVShape of ONE context (n_contexts of them); n_slots: device pool size in chunks.
+        aot: swap the served contexts out ahead of time, when the call returns (Sec. 3.4 i), so that a later
+        Reclaim of their chunks costs nothing."""
+        self.shape, self.n_slots, self.frac, self.seed, self.aot = shape, n_slots, frac, seed, aot
         self.n_ctx, self.cpc = shape.n_contexts, shape.n_chunks       # contexts, chunks per context
         self.desc_ctx = B.desc_of(shape)
         self.desc_pool = B.desc_of(shape, n_tokens=n_slots * shape.chunk_len)
@@ -36,6 +38,8 @@ class MultiApp:
         self.slot = np.full(n, -1, dtype=np.int64)
         self.free = list(range(n_slots - 1, -1, -1))
         self.checksum = np.zeros(n, dtype=np.uint32)
+        self.clean = np.zeros(n, dtype=bool)      # the record in the arena matches what sits in the slot
+        self.ready_ms = []                        # per step: time until the served contexts were resident
         self.arena_off = np.zeros(n, dtype=np.uint64)
         self.step_no = 0
         self.ops = [] if log_ops else None        # ("evict"|"load", row, slot) in execution order
@@ -136,8 +140,21 @@ class MultiApp:
 
     # ------------------------------------------------------------------ Reclaim and Load
     def _evict(self, rows):
-        """Reclaim: quantize + pack the chunks in `rows` out of their slots, copy the records to the arena."""
+        """Reclaim: chunks whose record in the arena is still valid are simply dropped; the others are
+        quantized + packed out of their slots and their records copied to the arena first."""
         rows = np.asarray(rows)
+        for r in rows[self.clean[rows]]:
+            s = int(self.slot[r])
+            if self.ops is not None:
+                self.ops.append(("drop", int(r), s))
+            self.free.append(s)
+            self.slot[r] = -1
+            self.table["resident"][r] = 0
+        self._write_back(rows[~self.clean[rows]], release=True)
+
+    def _write_back(self, rows, release):
+        """Quantize + pack the chunks in `rows` and copy their records to the arena; release=True frees the
+        slots (Reclaim), release=False leaves the chunks resident (ahead-of-time swap-out)."""
         for r0 in range(0, len(rows), self.cpc):
             part = rows[r0:r0 + self.cpc]
             slots = self.slot[part].astype(np.uint32)
@@ -154,10 +171,14 @@ class MultiApp:
             self.bytes_out += int(sum(self.rec_bytes[int(b)] for b in bits))
             for r, s in zip(part, slots):
                 if self.ops is not None:
-                    self.ops.append(("evict", int(r), int(s)))
-                self.free.append(int(s))
-            self.slot[part] = -1
-            self.table["resident"][part] = 0
+                    self.ops.append(("evict" if release else "aot", int(r), int(s)))
+                if release:
+                    self.free.append(int(s))
+            if release:
+                self.slot[part] = -1
+                self.table["resident"][part] = 0
+            else:
+                self.clean[part] = True
 
     def _load(self, rows):
         """Load: copy the records of the chunks in `rows` from the arena, unpack + dequantize into free slots."""
@@ -186,6 +207,7 @@ class MultiApp:
             self.bytes_in += int(sizes.sum())
             self.slot[part] = slots
             self.table["resident"][part] = 1
+            self.clean[part] = True
             if self.ops is not None:
                 self.ops.extend(("load", int(r), int(s)) for r, s in zip(part, slots))
 
@@ -218,6 +240,9 @@ class MultiApp:
     def step(self, k=8):
         """Serve k contexts: lock, evict in LCTRU order as far as needed, load, touch, unlock."""
         self.step_no += 1
+        if not hasattr(self, "_ev_t0"):
+            self._ev_t0, self._ev_ready = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        self._ev_t0.record(self.main)
         ctxs = self.draw_contexts(k)
         locked_rows = np.concatenate([np.arange(c * self.cpc, (c + 1) * self.cpc) for c in ctxs])
         self.table["locked"][locked_rows] = 1            # working-set lock
@@ -235,8 +260,13 @@ class MultiApp:
             if len(missing):
                 self._load(missing)
             self.table["last_access_step"][rows] = self.step_no
+        self._ev_ready.record(self.main)                 # the working sets are resident: inference could start
+        self.clean[locked_rows] = False                  # a served context counts as modified by its call
+        if self.aot:
+            self._write_back(locked_rows, release=False)
         self.table["locked"][locked_rows] = 0
         self._end_of_step()
+        self.ready_ms.append(self._ev_t0.elapsed_time(self._ev_ready))
         return ctxs
 
     def context_kv(self, c):

@@ -12,14 +12,20 @@ from gpu_helpers import bits_view, odesc
 pytestmark = pytest.mark.gpu
 
 
-def test_multiapp_history_matches_oracle_replay():
+@pytest.mark.parametrize("aot", [False, True], ids=["reclaim", "aot"])
+def test_multiapp_history_matches_oracle_replay(aot):
     sh = synth.KVShape("apps", 2, 4, 4, 64, 128, 32, 64, window=8, seed=1, n_contexts=10)   # 4 chunks per context
-    app = MultiApp(sh, n_slots=12, seed=1, log_ops=True)        # room for 3 contexts
+    app = MultiApp(sh, n_slots=12, seed=1, log_ops=True, aot=aot)   # room for 3 contexts
     app.keep_sources = True
     app.build()
     served = [app.step(k=2) for _ in range(12)]
     assert all(len(s) == 2 for s in served)
     assert app.bytes_out > 0 and app.bytes_in > 0
+    kinds = {op for op, _, _ in app.ops}
+    if aot:   # everything that leaves was written back when its call returned: Reclaim never compresses
+        assert "aot" in kinds and "drop" in kinds and "evict" not in kinds
+    else:
+        assert "evict" in kinds and "aot" not in kinds
 
     # (1) every eviction order is the oracle's order for the same table
     assert len(app.orders) > 5
@@ -54,9 +60,13 @@ def test_multiapp_history_matches_oracle_replay():
             out = np.zeros((sh.n_layers, 2, sh.n_kv_heads, CL, sh.head_dim), dtype=np.uint16)
             oracle.decompress_chunks(od_one, buf, meta, out)
             pool[slot] = out
-        else:
+        elif op == "drop":
+            pool.pop(slot)
+        else:   # "evict" frees the slot after writing the record, "aot" writes it and stays
             bits = int(app.table["bits"][row])
-            arena[row] = oracle.compress_chunks(od_one, pool.pop(slot), [0], [bits])
+            arena[row] = oracle.compress_chunks(od_one, pool[slot], [0], [bits])
+            if op == "evict":
+                pool.pop(slot)
     host_arena = app.arena.numpy()
     for row, (buf, meta) in arena.items():
         off = int(app.arena_off[row])
@@ -80,7 +90,7 @@ def test_multiapp_locked_contexts_are_never_evicted():
         before = len(app.ops)
         ctxs = app.step(k=2)
         rows_served = {c * app.cpc + i for c in ctxs for i in range(app.cpc)}
-        evicted = {row for op, row, _ in app.ops[before:] if op == "evict"}
+        evicted = {row for op, row, _ in app.ops[before:] if op in ("evict", "drop")}
         assert not (evicted & rows_served)
         for c in ctxs:
             assert app.table["resident"][c * app.cpc:(c + 1) * app.cpc].all()
