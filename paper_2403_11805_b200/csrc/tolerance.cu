@@ -233,6 +233,18 @@ __global__ void __launch_bounds__(kTileWarps * 32) logits_mma_kernel(const TolAr
         }
         __syncwarp();
         const uint32_t tile_s = tiles_s + buf * kTileBytes;
+        // this lane's four tokens of the tile and their column weights 1/n_vis
+        int t_tok[2][2];
+        float w_tok[2][2];
+#pragma unroll
+        for (int mb = 0; mb < 2; ++mb)
+#pragma unroll
+            for (int h = 0; h < 2; ++h) {
+                t_tok[mb][h] = tile * kTileTokens + mb * 16 + h * 8 + g;
+                w_tok[mb][h] = 1.0f / (float)min(a.W, max(1, a.T - t_tok[mb][h]));
+            }
+        const bool tail_tile = tile * kTileTokens + kTileTokens > a.T - a.W + 1;
+        const float inv_w = 1.0f / (float)a.W;
         for (int nb = 0; nb < n_blocks; ++nb) {
             float acc[2][4];
 #pragma unroll
@@ -257,14 +269,13 @@ __global__ void __launch_bounds__(kTileWarps * 32) logits_mma_kernel(const TolAr
             for (int col = 0; col < 2; ++col) {
                 const int j = nb * 8 + 2 * q4 + col;       // flattened (head, window row)
                 const int r = j % a.W;
+                const int last_col = j < a.NR ? a.T - a.W + r : -1;   // last token this row sees
                 float lg[2][2], mx[2][2], se[2][2], sp[2][2];
 #pragma unroll
                 for (int mb = 0; mb < 2; ++mb)
 #pragma unroll
                     for (int h = 0; h < 2; ++h) {
-                        const int t = tile * kTileTokens + mb * 16 + h * 8 + g;
-                        const bool vis = j < a.NR && t < a.T && t <= a.T - a.W + r;
-                        lg[mb][h] = vis ? acc[mb][2 * h + col] * a.inv_sqrt_d : -INFINITY;
+                        lg[mb][h] = t_tok[mb][h] <= last_col ? acc[mb][2 * h + col] * a.inv_sqrt_d : -INFINITY;
                         mx[mb][h] = lg[mb][h];
                     }
                 segment_reduce<SEG>(mx, [](float x, float y) { return fmaxf(x, y); });
@@ -272,19 +283,26 @@ __global__ void __launch_bounds__(kTileWarps * 32) logits_mma_kernel(const TolAr
                 for (int mb = 0; mb < 2; ++mb)
 #pragma unroll
                     for (int h = 0; h < 2; ++h) {
-                        const int t = tile * kTileTokens + mb * 16 + h * 8 + g;
-                        const float e = lg[mb][h] == -INFINITY ? 0.0f : expf(lg[mb][h] - mx[mb][h]);
+                        // exp2-based exponential: relative error of a few 1e-6 for the arguments met here
+                        const float e = lg[mb][h] == -INFINITY ? 0.0f : __expf(lg[mb][h] - mx[mb][h]);
                         se[mb][h] = e;
-                        sp[mb][h] = e / (float)min(a.W, max(1, a.T - t));
+                        sp[mb][h] = e * w_tok[mb][h];
                     }
                 segment_reduce<SEG>(se, [](float x, float y) { return x + y; });
-                segment_reduce<SEG>(sp, [](float x, float y) { return x + y; });
+                if (tail_tile) {   // 1/n_vis varies inside the tile only among the last W columns
+                    segment_reduce<SEG>(sp, [](float x, float y) { return x + y; });
+                } else {
+#pragma unroll
+                    for (int mb = 0; mb < 2; ++mb)
+#pragma unroll
+                        for (int h = 0; h < 2; ++h) sp[mb][h] = se[mb][h] * inv_w;
+                }
                 if (j < a.NR) {
 #pragma unroll
                     for (int mb = 0; mb < 2; ++mb)
 #pragma unroll
                         for (int h = 0; h < 2; ++h) {
-                            const int t = tile * kTileTokens + mb * 16 + h * 8 + g;
+                            const int t = t_tok[mb][h];
                             if (t < a.T && t % SEG == 0) {   // the segment's first token writes
                                 const int64_t o = (row0 + j) * a.n_seg + t / SEG;
                                 a.pm[o] = mx[mb][h];
