@@ -123,7 +123,8 @@ __global__ void __launch_bounds__(kTokThreads) logits_kernel(const TolArgs a)
 // The window's query rows sit in shared memory (rows padded by 16 bytes against conflicts) and are read as B
 // fragments.  The softmax statistics are then taken straight from the accumulator fragments.
 constexpr int kTileTokens = 32;
-constexpr int kTileWarps = 4;
+constexpr int kTileWarps = 8;
+constexpr int kTileBuffers = 1;   // per warp; with 1 the other warps of the SM cover a warp's copy latency
 
 // 16-byte asynchronous copy global -> shared, bypassing L1; src_bytes = 0 fills zeros instead
 __device__ __forceinline__ void cp_async16(uint32_t dst_smem, const void *src, uint32_t src_bytes)
@@ -184,7 +185,7 @@ __global__ void __launch_bounds__(kTileWarps * 32) logits_mma_kernel(const TolAr
     const int n_blocks = (a.NR + 7) / 8;                                     // window rows in n-tiles of 8, zero padded
     unsigned char *q_s = smem_raw;                                           // [n_blocks*8][kQRowBytes]
     const int q_total = (n_blocks * 8 * kQRowBytes + 127) / 128 * 128;
-    unsigned char *tiles = smem_raw + q_total + wib * 2 * kTileBytes;        // this warp's two buffers
+    unsigned char *tiles = smem_raw + q_total + wib * kTileBuffers * kTileBytes;   // this warp's buffers
     const uint32_t tiles_s = (uint32_t)__cvta_generic_to_shared(tiles);
 
     const int l = blockIdx.y / a.Hkv, kvh = blockIdx.y % a.Hkv;
@@ -223,9 +224,12 @@ __global__ void __launch_bounds__(kTileWarps * 32) logits_mma_kernel(const TolAr
     const int a_row = lane & 15, a_chunk = lane >> 4;
 
     int buf = 0;
-    if (tile_begin < tile_end) issue_tile(tile_begin, 0);
-    for (int tile = tile_begin; tile < tile_end; tile += kTileWarps, buf ^= 1) {
-        if (tile + kTileWarps < tile_end) {
+    if (kTileBuffers == 2 && tile_begin < tile_end) issue_tile(tile_begin, 0);
+    for (int tile = tile_begin; tile < tile_end; tile += kTileWarps, buf ^= (kTileBuffers - 1)) {
+        if (kTileBuffers == 1) {
+            issue_tile(tile, 0);
+            cp_async_wait<0>();
+        } else if (tile + kTileWarps < tile_end) {
             issue_tile(tile + kTileWarps, buf ^ 1);
             cp_async_wait<1>();
         } else {
@@ -516,7 +520,7 @@ extern "C" int llms_chunk_tolerance(const llms_kv_desc *desc, const void *kv, co
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     if ((unsigned)(a.L * a.Hkv) > 65535u) return LLMS_ERR_UNSUPPORTED;
     const size_t mma_q_bytes = ((size_t)((a.NR + 7) / 8 * 8) * (a.d * 2 + 16) + 127) / 128 * 128;
-    const size_t mma_smem = mma_q_bytes + (size_t)kTileWarps * 2 * kTileTokens * a.d * 2;
+    const size_t mma_smem = mma_q_bytes + (size_t)kTileWarps * kTileBuffers * kTileTokens * a.d * 2;
     if ((a.d == 64 || a.d == 128 || a.d == 256) && mma_smem <= 200 * 1024) {
         // enough blocks per (layer, KV head) to fill the GPU a few times over
         const int n_tiles = (a.T + kTileTokens - 1) / kTileTokens;
