@@ -11,6 +11,8 @@
 // The arithmetic is fixed by the record format (see llms.h): every binary32 operation is a single IEEE
 // round-to-nearest operation (intrinsics, or sm_100 mixed-precision PTX whose fp16 inputs convert exactly),
 // nothing is contracted or approximated.
+#include <string.h>
+
 #include <vector>
 
 #include "llms_internal.cuh"
@@ -700,6 +702,18 @@ static BitGroups group_by_bits(int n, const llms_chunk_meta *meta, GetBits bits_
     return g;
 }
 
+// One host-to-device copy sets the workspace up: zeroed status words, the entries, the unit table, the order.
+static int upload_tables(void *workspace, const llms_chunk_meta *entries, const BitGroups &g, int n, cudaStream_t st)
+{
+    std::vector<uint8_t> image(ws_sums_offset(n), 0);
+    memcpy(image.data() + kWsEntriesOffset, entries, (size_t)n * sizeof(ChunkEntry));
+    memcpy(image.data() + ws_table_offset(n), g.table.data(), (size_t)n * sizeof(UnitEntry));
+    memcpy(image.data() + ws_order_offset(n), g.order.data(), (size_t)n * 4);
+    // `image` is pageable: the copy has left it by the time cudaMemcpyAsync returns
+    LLMS_CUDA_TRY(cudaMemcpyAsync(workspace, image.data(), image.size(), cudaMemcpyHostToDevice, st));
+    return LLMS_OK;
+}
+
 // The launch arguments of one bit-width's share of the call.
 static CodecArgs args_for_group(const CodecArgs &a, const BitGroups &g, int k)
 {
@@ -823,11 +837,8 @@ extern "C" int llms_compress_chunks(const llms_kv_desc *desc, const void *kv, co
     a.buf = static_cast<uint8_t *>(out_buf);
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     const BitGroups groups = group_by_bits(n, meta, [&](int i) { return (uint32_t)bits[i]; });
-    LLMS_CUDA_TRY(cudaMemcpyAsync(a.entries, meta, (size_t)n * sizeof(ChunkEntry), cudaMemcpyHostToDevice, st));
-    // `groups.order` is pageable: the copy has left it by the time cudaMemcpyAsync returns
-    LLMS_CUDA_TRY(cudaMemcpyAsync(const_cast<uint32_t *>(a.order), groups.order.data(), (size_t)n * 4, cudaMemcpyHostToDevice, st));
-    LLMS_CUDA_TRY(cudaMemcpyAsync(const_cast<UnitEntry *>(a.table), groups.table.data(), (size_t)n * sizeof(UnitEntry), cudaMemcpyHostToDevice, st));
-    LLMS_CUDA_TRY(cudaMemsetAsync(workspace, 0, 8, st));  // both status words
+    rc = upload_tables(workspace, meta, groups, n, st);
+    if (rc) return rc;
     const bool wide = wide_ok(*desc, kv);
     for (int k = 0; k < 3; ++k) {
         if (groups.count[k] == 0) continue;
@@ -898,13 +909,10 @@ extern "C" int llms_decompress_chunks(const llms_kv_desc *desc, const void *buf,
     a.buf = const_cast<uint8_t *>(static_cast<const uint8_t *>(buf));
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     uint32_t *status = static_cast<uint32_t *>(workspace);
-    // `staged` is pageable: the copy has left it by the time cudaMemcpyAsync returns
-    LLMS_CUDA_TRY(cudaMemcpyAsync(a.entries, staged.data(), (size_t)n * sizeof(ChunkEntry), cudaMemcpyHostToDevice, st));
     LLMS_CUDA_TRY(cudaMemsetAsync(a.sums, 0, (size_t)n * 4, st));
-    LLMS_CUDA_TRY(cudaMemsetAsync(status, 0, 8, st));  // both status words
     const BitGroups groups = group_by_bits(n, staged.data(), [&](int i) { return meta[i].bits; });
-    LLMS_CUDA_TRY(cudaMemcpyAsync(const_cast<uint32_t *>(a.order), groups.order.data(), (size_t)n * 4, cudaMemcpyHostToDevice, st));
-    LLMS_CUDA_TRY(cudaMemcpyAsync(const_cast<UnitEntry *>(a.table), groups.table.data(), (size_t)n * sizeof(UnitEntry), cudaMemcpyHostToDevice, st));
+    rc = upload_tables(workspace, staged.data(), groups, n, st);
+    if (rc) return rc;
     const bool wide = wide_ok(*desc, kv_out);
     for (int k = 0; k < 3; ++k) {
         if (groups.count[k] == 0) continue;

@@ -51,13 +51,13 @@ struct ChunkEntry {          // same bytes as llms_chunk_meta
 static_assert(sizeof(ChunkEntry) == sizeof(llms_chunk_meta) && sizeof(ChunkEntry) == 32, "meta layout");
 
 // Workspace of the codec calls:
-// [two status words, padded to 16 bytes][n entries][n 16-byte unit-table rows][n recomputed sums]
-// [n entry indices grouped by bit-width].
+// [two status words, padded to 16 bytes][n entries][n 16-byte unit-table rows][n entry indices grouped by
+// bit-width][n recomputed sums].  Everything up to the sums is written by one host-to-device copy per call.
 constexpr uint64_t kWsEntriesOffset = 16;
 constexpr uint64_t kWsBytesPerChunk = sizeof(ChunkEntry) + 16 + 4 + 4;
 inline uint64_t ws_table_offset(int n) { return kWsEntriesOffset + (uint64_t)n * sizeof(ChunkEntry); }
-inline uint64_t ws_sums_offset(int n) { return ws_table_offset(n) + (uint64_t)n * 16; }
-inline uint64_t ws_order_offset(int n) { return ws_sums_offset(n) + (uint64_t)n * 4; }
+inline uint64_t ws_order_offset(int n) { return ws_table_offset(n) + (uint64_t)n * 16; }
+inline uint64_t ws_sums_offset(int n) { return ws_order_offset(n) + (uint64_t)n * 4; }
 inline uint64_t ws_total(int n) { return round_up(kWsEntriesOffset + (uint64_t)n * kWsBytesPerChunk, 16); }
 
 }  // namespace llms
