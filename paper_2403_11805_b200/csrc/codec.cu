@@ -25,6 +25,7 @@ constexpr int kPieceElems = 16;                 // one 32-byte access
 constexpr int kPieces = 4;                      // pieces per lane per pass
 constexpr int kLaneElems = kPieces * kPieceElems;
 constexpr int kPassElems = 32 * kLaneElems;     // 2048 elements = 4 KiB of fp16
+constexpr uint32_t kPrefetchAhead = 3;          // compress: units ahead of the current one that are pulled into L2
 
 // Division by a launch-time constant as multiply-high and shift: exact for numerators below 2^31.
 struct FastDiv {
@@ -424,6 +425,19 @@ __device__ __forceinline__ void load_unit(const CodecArgs &a, const UnitPos &u, 
     }
 }
 
+// Ask for a unit's KV bytes to be brought into L2 (one bulk prefetch by one lane): the register loads of that
+// unit, issued one unit later, then find them there instead of waiting for DRAM.
+__device__ __forceinline__ void prefetch_unit_l2(const CodecArgs &a, uint32_t unit, int lane)
+{
+    UnitPos u;
+    decode_unit(a, unit, 0, u);
+    if (lane == 0) {
+        const __half *src = a.kv_in + slab_offset(a, u.s_idx, u.chunk_id) + u.e0;
+        const uint32_t bytes = (uint32_t)min(kPassElems, a.slab_elems - u.e0) * 2;
+        asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" :: "l"(src), "r"(bytes) : "memory");
+    }
+}
+
 template <int BITS, int G, bool WIDE>
 __device__ __forceinline__ void compress_unit(const CodecArgs &a, const UnitPos &u, const uint32_t (&w)[kPieces][8], int lane)
 {
@@ -453,6 +467,7 @@ __global__ void __launch_bounds__(kThreads, 2) compress_kernel(const CodecArgs a
             decode_unit(a, unit + n_warps, lane, pb);
             load_unit<WIDE>(a, pb, wb);
         }
+        if (a.total_units - unit > kPrefetchAhead * n_warps) prefetch_unit_l2(a, unit + kPrefetchAhead * n_warps, lane);
         compress_unit<BITS, G, WIDE>(a, pa, wa, lane);
         if (!more) break;
         unit += n_warps;
@@ -461,6 +476,7 @@ __global__ void __launch_bounds__(kThreads, 2) compress_kernel(const CodecArgs a
             decode_unit(a, unit + n_warps, lane, pa);
             load_unit<WIDE>(a, pa, wa);
         }
+        if (a.total_units - unit > kPrefetchAhead * n_warps) prefetch_unit_l2(a, unit + kPrefetchAhead * n_warps, lane);
         compress_unit<BITS, G, WIDE>(a, pb, wb, lane);
         if (!more) break;
         unit += n_warps;
