@@ -411,19 +411,50 @@ __device__ __forceinline__ void zero_padding(const CodecArgs &a, uint8_t *rec, u
     for (uint64_t k = codes_end + lane; k < nbytes; k += 32) rec[k] = 0;
 }
 
+// The unit is fetched so that every load instruction of the warp reads 1 KiB of consecutive bytes (piece j of
+// lane L = elements [j*512 + L*16, +16) of the pass): measured on this part, a stream read with 128 consecutive
+// bytes per lane tops out near 5.6 TB/s, one with consecutive lanes on consecutive 32 bytes near 6.9 TB/s.
 template <bool WIDE>
-__device__ __forceinline__ void load_unit(const CodecArgs &a, const UnitPos &u, uint32_t (&w)[kPieces][8])
+__device__ __forceinline__ void load_unit(const CodecArgs &a, const UnitPos &u, int lane, uint32_t (&w)[kPieces][8])
 {
-    const __half *src = a.kv_in + slab_offset(a, u.s_idx, u.chunk_id) + u.e0;
+    const int pass_e0 = u.e0 - lane * kLaneElems;
+    const __half *src = a.kv_in + slab_offset(a, u.s_idx, u.chunk_id) + pass_e0 + lane * kPieceElems;
 #pragma unroll
     for (int j = 0; j < kPieces; ++j) {
-        if (u.e0 + j * kPieceElems < a.slab_elems) {
-            load32<WIDE>(src + j * kPieceElems, w[j]);
+        if (pass_e0 + j * (32 * kPieceElems) + lane * kPieceElems < a.slab_elems) {
+            load32<WIDE>(src + j * (32 * kPieceElems), w[j]);
         } else {
 #pragma unroll
-            for (int k = 0; k < 8; ++k) w[j][k] = 0;  // pieces past the end form whole inactive groups
+            for (int k = 0; k < 8; ++k) w[j][k] = 0;  // past the end of the slab: whole inactive groups
         }
     }
+}
+
+// ... and brought to the layout the arithmetic wants (lane L holds elements [L*64, +64) of the pass) through the
+// warp's patch of shared memory.  Rows of 128 bytes are padded to 144: both the 32-byte-per-lane writes and the
+// 128-byte-per-lane reads are then free of bank conflicts.
+constexpr int kTransposeRowBytes = 128 + 16;
+constexpr int kTransposeBytes = 32 * kTransposeRowBytes;
+
+__device__ __forceinline__ void to_lane_contiguous(uint32_t (&w)[kPieces][8], unsigned char *patch, int lane)
+{
+#pragma unroll
+    for (int j = 0; j < kPieces; ++j) {
+        // piece j of this lane = 16-byte chunks 64j + 2L and 64j + 2L + 1 of the unit; chunk n -> row n/8, column n%8
+        unsigned char *dst = patch + (8 * j + (lane >> 2)) * kTransposeRowBytes + (lane & 3) * 32;
+        *reinterpret_cast<uint4 *>(dst) = make_uint4(w[j][0], w[j][1], w[j][2], w[j][3]);
+        *reinterpret_cast<uint4 *>(dst + 16) = make_uint4(w[j][4], w[j][5], w[j][6], w[j][7]);
+    }
+    __syncwarp();
+    const unsigned char *row = patch + lane * kTransposeRowBytes;
+#pragma unroll
+    for (int j = 0; j < kPieces; ++j) {
+        const uint4 lo = *reinterpret_cast<const uint4 *>(row + j * 32);
+        const uint4 hi = *reinterpret_cast<const uint4 *>(row + j * 32 + 16);
+        w[j][0] = lo.x; w[j][1] = lo.y; w[j][2] = lo.z; w[j][3] = lo.w;
+        w[j][4] = hi.x; w[j][5] = hi.y; w[j][6] = hi.z; w[j][7] = hi.w;
+    }
+    __syncwarp();  // the patch is free for the next unit
 }
 
 // Ask for a unit's KV bytes to be brought into L2 (one bulk prefetch by one lane): the register loads of that
@@ -458,26 +489,30 @@ __global__ void __launch_bounds__(kThreads, 2) compress_kernel(const CodecArgs a
     const uint32_t n_warps = gridDim.x * kWarpsPerBlock;
     uint32_t unit = blockIdx.x * kWarpsPerBlock + (threadIdx.x >> 5);
     if (unit >= a.total_units) return;
+    __shared__ __align__(16) unsigned char patches[kWarpsPerBlock][kTransposeBytes];
+    unsigned char *patch = patches[threadIdx.x >> 5];
     UnitPos pa, pb;
     uint32_t wa[kPieces][8], wb[kPieces][8];
     decode_unit(a, unit, lane, pa);
-    load_unit<WIDE>(a, pa, wa);
+    load_unit<WIDE>(a, pa, lane, wa);
     for (;;) {  // two units per trip, so that the buffers swap roles without register copies
         bool more = a.total_units - unit > n_warps;
         if (more) {
             decode_unit(a, unit + n_warps, lane, pb);
-            load_unit<WIDE>(a, pb, wb);
+            load_unit<WIDE>(a, pb, lane, wb);
         }
         if (a.total_units - unit > kPrefetchAhead * n_warps) prefetch_unit_l2(a, unit + kPrefetchAhead * n_warps, lane);
+        to_lane_contiguous(wa, patch, lane);
         compress_unit<BITS, G, WIDE>(a, pa, wa, lane);
         if (!more) break;
         unit += n_warps;
         more = a.total_units - unit > n_warps;
         if (more) {
             decode_unit(a, unit + n_warps, lane, pa);
-            load_unit<WIDE>(a, pa, wa);
+            load_unit<WIDE>(a, pa, lane, wa);
         }
         if (a.total_units - unit > kPrefetchAhead * n_warps) prefetch_unit_l2(a, unit + kPrefetchAhead * n_warps, lane);
+        to_lane_contiguous(wb, patch, lane);
         compress_unit<BITS, G, WIDE>(a, pb, wb, lane);
         if (!more) break;
         unit += n_warps;
