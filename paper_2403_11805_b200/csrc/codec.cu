@@ -25,7 +25,7 @@ constexpr int kPieceElems = 16;                 // one 32-byte access
 constexpr int kPieces = 4;                      // pieces per lane per pass
 constexpr int kLaneElems = kPieces * kPieceElems;
 constexpr int kPassElems = 32 * kLaneElems;     // 2048 elements = 4 KiB of fp16
-constexpr uint32_t kPrefetchAhead = 2;          // units ahead of the current one that are pulled into L2 (measured: 2 -> 0.521 ms,
+constexpr uint32_t kPrefetchAhead = 2;          // compress: units ahead that are pulled into L2 (measured: 2 -> 0.521 ms,
                                                 // 3 -> 0.535, 5 -> 0.59, 8 -> 0.79 for compress on the 7B shape)
 
 // Division by a launch-time constant as multiply-high and shift: exact for numerators below 2^31.
@@ -649,19 +649,6 @@ __device__ __forceinline__ void decompress_unit(const CodecArgs &a, const UnitPo
     if (lane == 0) atomicAdd(&a.sums[u.i], sum);
 }
 
-template <int BITS>
-__device__ __forceinline__ void prefetch_codes_l2(const CodecArgs &a, uint32_t unit, int lane)
-{
-    UnitPos u;
-    decode_unit(a, unit, 0, u);
-    if (lane == 0) {
-        const uint8_t *codes = a.buf + u.rec_off + a.codes_off + ((uint64_t)u.s_idx * a.slab_elems + (uint32_t)u.e0) * BITS / 8;
-        const uint32_t bytes = ((uint32_t)min(kPassElems, a.slab_elems - u.e0) * BITS / 8) & ~15u;
-        if (bytes && (reinterpret_cast<uintptr_t>(codes) & 15) == 0)
-            asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" :: "l"(codes), "r"(bytes) : "memory");
-    }
-}
-
 template <int BITS, int G, bool WIDE>
 __global__ void __launch_bounds__(kThreads, 3) decompress_kernel(const CodecArgs a)
 {
@@ -680,7 +667,6 @@ __global__ void __launch_bounds__(kThreads, 3) decompress_kernel(const CodecArgs
             decode_unit(a, unit + n_warps, lane, pb);
             load_unit_codes<BITS, G>(a, pb, lane, cb, qb);
         }
-        if (a.total_units - unit > kPrefetchAhead * n_warps) prefetch_codes_l2<BITS>(a, unit + kPrefetchAhead * n_warps, lane);
         decompress_unit<BITS, G, WIDE>(a, pa, ca, qa, lane);
         if (!more) break;
         unit += n_warps;
@@ -689,7 +675,6 @@ __global__ void __launch_bounds__(kThreads, 3) decompress_kernel(const CodecArgs
             decode_unit(a, unit + n_warps, lane, pa);
             load_unit_codes<BITS, G>(a, pa, lane, ca, qa);
         }
-        if (a.total_units - unit > kPrefetchAhead * n_warps) prefetch_codes_l2<BITS>(a, unit + kPrefetchAhead * n_warps, lane);
         decompress_unit<BITS, G, WIDE>(a, pb, cb, qb, lane);
         if (!more) break;
         unit += n_warps;
