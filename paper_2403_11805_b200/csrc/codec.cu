@@ -524,29 +524,47 @@ __global__ void __launch_bounds__(kThreads, 2) compress_kernel(const CodecArgs a
 // The decoder splits a pass differently from the encoder: piece j of lane L is elements
 // [j*512 + L*16, +16) of the pass, so that every store instruction of the warp writes 1 KiB of consecutive
 // addresses (a lane-contiguous split made each store touch 32 separate lines and ran slower).  Groups need no
-// lane cooperation here; each piece just looks its group's parameters up.
-__device__ __forceinline__ int decode_piece_elem(const UnitPos &u, int lane, int j)
+// lane cooperation here; each piece just looks its group's parameters up.  Everything a piece needs sits at a
+// compile-time distance from piece 0 (512 elements, 512/G groups), so a unit's addresses are computed once.
+constexpr int kPieceStride = 32 * kPieceElems;  // elements between a lane's pieces
+
+struct DecodePos {
+    uint32_t i;              // entry index (checksum slot)
+    int room;                // slab elements from this lane's piece 0 to the end of the slab (<= 0: none)
+    const uint8_t *codes;    // piece 0: packed codes
+    const uint32_t *params;  // piece 0: parameter word of its group
+    __half *dst;             // piece 0: destination
+};
+
+template <int BITS, int G>
+__device__ __forceinline__ void decode_unit_for_decoder(const CodecArgs &a, uint32_t unit, int lane, DecodePos &u)
 {
-    return (u.e0 - lane * kLaneElems) + j * (32 * kPieceElems) + lane * kPieceElems;
+    static_assert(kPieceStride % G == 0 || G % kPieceStride == 0, "groups and pieces nest");
+    uint32_t item, pass, s_idx, k;
+    a.div_passes.divmod(unit, item, pass);
+    a.div_n.divmod(item, s_idx, k);
+    const uint4 t = *reinterpret_cast<const uint4 *>(a.table + k);  // chunk_id, entry, record offset
+    u.i = t.y;
+    const uint32_t e = pass * kPassElems + lane * kPieceElems;      // piece 0 inside the slab
+    u.room = a.slab_elems - (int)e;
+    const uint8_t *rec = a.buf + ((uint64_t)t.z | ((uint64_t)t.w << 32));
+    u.params = reinterpret_cast<const uint32_t *>(rec) + (s_idx * (uint32_t)a.groups_per_slab + e / G);
+    u.codes = rec + a.codes_off + ((uint64_t)s_idx * a.slab_elems + e) * BITS / 8;
+    u.dst = a.kv_out + slab_offset(a, s_idx, t.x) + e;
 }
 
 template <int BITS, int G>
-__device__ __forceinline__ void load_unit_codes(const CodecArgs &a, const UnitPos &u, int lane, uint32_t (&c)[kPieces][BITS / 2],
-                                                uint32_t (&p)[kPieces])
+__device__ __forceinline__ void load_unit_codes(const DecodePos &u, uint32_t (&c)[kPieces][BITS / 2], uint32_t (&p)[kPieces])
 {
-    constexpr int kPieceBytes = kPieceElems * BITS / 8;
-    const uint8_t *rec = a.buf + u.rec_off;
-    const uint32_t *params = reinterpret_cast<const uint32_t *>(rec) + (uint64_t)u.s_idx * a.groups_per_slab;
-    const uint8_t *codes = rec + a.codes_off + (uint64_t)u.s_idx * a.slab_elems * BITS / 8;
+    constexpr int kStrideBytes = kPieceStride * BITS / 8;
 #pragma unroll
     for (int j = 0; j < kPieces; ++j) {
-        const int e = decode_piece_elem(u, lane, j);
-        if (e < a.slab_elems) {
-            const uint8_t *src = codes + (uint32_t)(e / kPieceElems) * kPieceBytes;
+        if (u.room > j * kPieceStride) {
+            const uint8_t *src = u.codes + j * kStrideBytes;
             if constexpr (BITS == 8) ld128(src, c[j]);
             else if constexpr (BITS == 4) ld64(src, c[j]);
             else ld32(src, c[j]);
-            p[j] = __ldg(params + (uint32_t)e / G);
+            p[j] = __ldg(u.params + j * (kPieceStride / G));
         } else {
 #pragma unroll
             for (int k = 0; k < BITS / 2; ++k) c[j][k] = 0;
@@ -595,55 +613,46 @@ __device__ __forceinline__ unsigned short code_half(const __half2 (&q)[8], int e
     return hi ? hi_h : lo_h;
 }
 
+// Two binary32 values -> packed fp16, round to nearest even, magnitudes above 65504 become +-65504: the clamp
+// and the conversion of the decode rule in one instruction.
+__device__ __forceinline__ uint32_t pack_half2_clamped(float lo, float hi)
+{
+    uint32_t w;
+    asm("cvt.rn.satfinite.f16x2.f32 %0, %1, %2;" : "=r"(w) : "f"(hi), "f"(lo));
+    return w;
+}
+
 // 16 decoded values.  q*scale is exact in binary32, so the mixed-precision fused form rounds once, as
-// multiply-then-add would.  CLAMP only when zero + (2^b - 1)*scale can pass the fp16 range (zero >= -65504 and
-// scale >= 0, so only the upper end can).
-template <int BITS, bool CLAMP>
+// multiply-then-add would.
+template <int BITS>
 __device__ __forceinline__ void dequantize_piece(const uint32_t *c, unsigned short scale_h, float zero, uint32_t (&w)[8])
 {
     __half2 q[8];
     codes_to_half2<BITS>(c, q);
 #pragma unroll
-    for (int k = 0; k < 8; ++k) {
-        float y0 = fma_f32_f16(code_half<BITS>(q, 2 * k), scale_h, zero);
-        float y1 = fma_f32_f16(code_half<BITS>(q, 2 * k + 1), scale_h, zero);
-        if constexpr (CLAMP) {
-            y0 = fminf(y0, 65504.0f);
-            y1 = fminf(y1, 65504.0f);
-        }
-        w[k] = as_u32(__floats2half2_rn(y0, y1));
-    }
+    for (int k = 0; k < 8; ++k)
+        w[k] = pack_half2_clamped(fma_f32_f16(code_half<BITS>(q, 2 * k), scale_h, zero),
+                                  fma_f32_f16(code_half<BITS>(q, 2 * k + 1), scale_h, zero));
 }
 
 template <int BITS, int G, bool WIDE>
-__device__ __forceinline__ void decompress_unit(const CodecArgs &a, const UnitPos &u, const uint32_t (&c)[kPieces][BITS / 2],
+__device__ __forceinline__ void decompress_unit(const CodecArgs &a, const DecodePos &u, const uint32_t (&c)[kPieces][BITS / 2],
                                                 const uint32_t (&p)[kPieces], int lane)
 {
-    constexpr float kQmax = (float)((1 << BITS) - 1);
-    __half *dst = a.kv_out + slab_offset(a, u.s_idx, u.chunk_id);
+    // a lane's pieces all sit at the same place inside their groups: either every one opens a group or none does
+    const bool opens_group = (lane * kPieceElems) % G == 0;
     uint32_t sum = 0;
-    bool any_clamp = false;
 #pragma unroll
     for (int j = 0; j < kPieces; ++j) {
-        const float scale = __half2float(__ushort_as_half((unsigned short)(p[j] & 0xffffu)));
-        const float zero = __half2float(__ushort_as_half((unsigned short)(p[j] >> 16)));
-        any_clamp |= __fmaf_rn(kQmax, scale, zero) > 65504.0f;
-    }
-    const bool clamp = __any_sync(0xffffffffu, any_clamp);
-#pragma unroll
-    for (int j = 0; j < kPieces; ++j) {
-        const int e = decode_piece_elem(u, lane, j);
         const unsigned short scale_h = (unsigned short)(p[j] & 0xffffu);
         const float zero = __half2float(__ushort_as_half((unsigned short)(p[j] >> 16)));
         uint32_t w[8];
-        if (clamp) dequantize_piece<BITS, true>(c[j], scale_h, zero, w);
-        else dequantize_piece<BITS, false>(c[j], scale_h, zero, w);
-        if (e < a.slab_elems) {
-            store32<WIDE>(dst + e, w);
+        dequantize_piece<BITS>(c[j], scale_h, zero, w);
+        if (u.room > j * kPieceStride) store32<WIDE>(u.dst + j * kPieceStride, w);
+        // pieces past the end of the slab were loaded as zeros and add nothing
 #pragma unroll
-            for (int k = 0; k < BITS / 2; ++k) sum += c[j][k];
-            if ((uint32_t)e % G == 0) sum += p[j];  // the piece that opens a group accounts for its parameter word
-        }
+        for (int k = 0; k < BITS / 2; ++k) sum += c[j][k];
+        if (opens_group) sum += p[j];  // the piece that opens a group accounts for its parameter word
     }
     sum = __reduce_add_sync(0xffffffffu, sum);
     if (lane == 0) atomicAdd(&a.sums[u.i], sum);
@@ -656,24 +665,24 @@ __global__ void __launch_bounds__(kThreads, 3) decompress_kernel(const CodecArgs
     const uint32_t n_warps = gridDim.x * kWarpsPerBlock;
     uint32_t unit = blockIdx.x * kWarpsPerBlock + (threadIdx.x >> 5);
     if (unit >= a.total_units) return;
-    UnitPos pa, pb;
+    DecodePos pa, pb;
     uint32_t ca[kPieces][BITS / 2], cb[kPieces][BITS / 2];
     uint32_t qa[kPieces], qb[kPieces];
-    decode_unit(a, unit, lane, pa);
-    load_unit_codes<BITS, G>(a, pa, lane, ca, qa);
+    decode_unit_for_decoder<BITS, G>(a, unit, lane, pa);
+    load_unit_codes<BITS, G>(pa, ca, qa);
     for (;;) {
         bool more = a.total_units - unit > n_warps;
         if (more) {
-            decode_unit(a, unit + n_warps, lane, pb);
-            load_unit_codes<BITS, G>(a, pb, lane, cb, qb);
+            decode_unit_for_decoder<BITS, G>(a, unit + n_warps, lane, pb);
+            load_unit_codes<BITS, G>(pb, cb, qb);
         }
         decompress_unit<BITS, G, WIDE>(a, pa, ca, qa, lane);
         if (!more) break;
         unit += n_warps;
         more = a.total_units - unit > n_warps;
         if (more) {
-            decode_unit(a, unit + n_warps, lane, pa);
-            load_unit_codes<BITS, G>(a, pa, lane, ca, qa);
+            decode_unit_for_decoder<BITS, G>(a, unit + n_warps, lane, pa);
+            load_unit_codes<BITS, G>(pa, ca, qa);
         }
         decompress_unit<BITS, G, WIDE>(a, pb, cb, qb, lane);
         if (!more) break;
