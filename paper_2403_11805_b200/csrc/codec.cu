@@ -1,12 +1,18 @@
 // Chunk codec kernels for sm_100a: group quantize + bit-pack (swap-out) and unpack + dequantize (swap-in).
 //
 // Work unit = one warp pass over a slab (chunk_len*head_dim contiguous fp16 of one chunk, layer, K/V, head):
-// 2048 elements, a lane owning 64 consecutive ones as four 32-byte pieces.  A group of G >= 64 channels is
-// G/64 neighbouring lanes (min/max by xor-shuffles on a packed (min, -max) half2); smaller groups sit inside
-// a lane.  A lane's packed codes are 16/32/64 contiguous bytes at 2/4/8 bits, so every access of the warp is
-// made of whole 32-byte sectors.  Warps of a persistent grid walk the units with a stride; the loads of the
-// next unit are issued before the current one is computed (two register buffers), which keeps 128 bytes per
-// lane in flight all the time.  The bit-width is uniform per chunk, hence per warp.
+// 2048 elements.  Warps of a persistent grid walk the units with a stride; the loads of the next unit are
+// issued before the current one is computed (register buffers), and the bit-width is uniform per launch.
+//
+// Encoder: every load instruction of a warp reads 1 KiB of consecutive bytes (piece j of lane L = elements
+// j*512 + L*16; with 128 consecutive bytes per lane instead, a streaming probe reached 5.6 instead of 6.9 TB/s);
+// the unit is then transposed through padded shared memory so that a lane owns 64 consecutive elements.  A
+// group of G >= 64 channels is G/64 neighbouring lanes (min/max by xor-shuffles on a packed (min, -max) half2);
+// smaller groups sit inside a lane.  A lane's packed codes are 16/32/64 contiguous bytes at 2/4/8 bits.  The
+// unit two strides ahead is pulled into L2 by a bulk prefetch.
+//
+// Decoder: keeps the interleaved split for its stores (1 KiB of consecutive bytes per store instruction) and
+// needs no lane cooperation: each piece looks its group's parameters up.
 //
 // The arithmetic is fixed by the record format (see llms.h): every binary32 operation is a single IEEE
 // round-to-nearest operation (intrinsics, or sm_100 mixed-precision PTX whose fp16 inputs convert exactly),
@@ -658,35 +664,45 @@ __device__ __forceinline__ void decompress_unit(const CodecArgs &a, const Decode
     if (lane == 0) atomicAdd(&a.sums[u.i], sum);
 }
 
+// Units whose loads are in flight per warp, the one being decoded included, and resident CTAs per SM.  Measured
+// on the 7B shape (decompress stage, ms): depth 2 with 3 CTAs 0.555, depth 3 with 3 CTAs 0.561-0.565, depth 3 or 4
+// with 2 CTAs 0.555-0.557, depth 4 with 3 CTAs 0.62-0.63 (spills), 4 CTAs 0.60: the stage is bound by the write
+// path, not by load latency.
+constexpr int kDecodeDepth = 2;
+constexpr int kDecodeBlocksPerSm = 3;
+
 template <int BITS, int G, bool WIDE>
-__global__ void __launch_bounds__(kThreads, 3) decompress_kernel(const CodecArgs a)
+__global__ void __launch_bounds__(kThreads, kDecodeBlocksPerSm) decompress_kernel(const CodecArgs a)
 {
+    constexpr int D = kDecodeDepth;
     const int lane = threadIdx.x & 31;
     const uint32_t n_warps = gridDim.x * kWarpsPerBlock;
     uint32_t unit = blockIdx.x * kWarpsPerBlock + (threadIdx.x >> 5);
     if (unit >= a.total_units) return;
-    DecodePos pa, pb;
-    uint32_t ca[kPieces][BITS / 2], cb[kPieces][BITS / 2];
-    uint32_t qa[kPieces], qb[kPieces];
-    decode_unit_for_decoder<BITS, G>(a, unit, lane, pa);
-    load_unit_codes<BITS, G>(pa, ca, qa);
+    DecodePos pos[D];
+    uint32_t c[D][kPieces][BITS / 2], p[D][kPieces];
+#pragma unroll
+    for (int s = 0; s < D - 1; ++s) {
+        const uint32_t ahead = unit + s * n_warps;
+        if (ahead < a.total_units) {
+            decode_unit_for_decoder<BITS, G>(a, ahead, lane, pos[s]);
+            load_unit_codes<BITS, G>(pos[s], c[s], p[s]);
+        }
+    }
     for (;;) {
-        bool more = a.total_units - unit > n_warps;
-        if (more) {
-            decode_unit_for_decoder<BITS, G>(a, unit + n_warps, lane, pb);
-            load_unit_codes<BITS, G>(pb, cb, qb);
+#pragma unroll
+        for (int s = 0; s < D; ++s) {
+            // ring slot s holds the current unit; the slot freed last takes the unit D-1 strides ahead
+            const int fill = (s + D - 1) % D;
+            const uint32_t ahead = unit + (D - 1) * n_warps;
+            if (ahead < a.total_units) {
+                decode_unit_for_decoder<BITS, G>(a, ahead, lane, pos[fill]);
+                load_unit_codes<BITS, G>(pos[fill], c[fill], p[fill]);
+            }
+            decompress_unit<BITS, G, WIDE>(a, pos[s], c[s], p[s], lane);
+            unit += n_warps;
+            if (unit >= a.total_units) return;
         }
-        decompress_unit<BITS, G, WIDE>(a, pa, ca, qa, lane);
-        if (!more) break;
-        unit += n_warps;
-        more = a.total_units - unit > n_warps;
-        if (more) {
-            decode_unit_for_decoder<BITS, G>(a, unit + n_warps, lane, pa);
-            load_unit_codes<BITS, G>(pa, ca, qa);
-        }
-        decompress_unit<BITS, G, WIDE>(a, pb, cb, qb, lane);
-        if (!more) break;
-        unit += n_warps;
     }
 }
 
