@@ -426,7 +426,7 @@ def run_multiapp(args):
         app.step(per_step)
     steps = min(args.steps, 100)
     sampler = ClockSampler(0)
-    out0, in0 = app.bytes_out, app.bytes_in
+    out0, in0, launches0 = app.bytes_out, app.bytes_in, app.kernel_launches
     torch.cuda.synchronize()
     sampler.begin()
     t0 = time.perf_counter()
@@ -451,7 +451,7 @@ def run_multiapp(args):
         "fp16_gbs_through_codec": 2 * chunks_moved * chunk_bytes / dt / 1e9,
         "aot_swap_out": bool(args.aot),
         "switch_latency_ms": statistics.mean(app.ready_ms[-steps:]),   # step start until the 8 working sets are resident
-        "gpu_launches": None, "clocks": clocks,
+        "gpu_launches": app.kernel_launches - launches0, "clocks": clocks,
     }
     print(json.dumps(line))
 

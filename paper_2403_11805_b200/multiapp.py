@@ -47,6 +47,7 @@ class MultiApp:
         self._pending = []                        # (meta, rows) of compress calls whose checksums are not read yet
         self._draw = 0
         self.bytes_out = self.bytes_in = 0
+        self.kernel_launches = 0                  # codec kernels launched (one per bit-width present, plus the checksum check)
 
     # ------------------------------------------------------------------ set-up (untimed)
     def build(self):
@@ -169,6 +170,7 @@ class MultiApp:
                        after=self.ev_compressed[k], done=self.ev_stage_out_free[k], n=len(part))
             self._pending.append((meta, part))
             self.bytes_out += int(sum(self.rec_bytes[int(b)] for b in bits))
+            self.kernel_launches += len(set(bits.tolist()))
             for r, s in zip(part, slots):
                 if self.ops is not None:
                     self.ops.append(("evict" if release else "aot", int(r), int(s)))
@@ -205,6 +207,7 @@ class MultiApp:
             self.ev_stage_in_free[k].record(self.main)
             self._used_ws.append(ws)
             self.bytes_in += int(sizes.sum())
+            self.kernel_launches += len(set(bits.tolist())) + 1
             self.slot[part] = slots
             self.table["resident"][part] = 1
             self.clean[part] = True
