@@ -35,6 +35,8 @@ def parse_args():
     p.add_argument("--layers", type=int, default=0, help="use only this many layers (smaller cases for profiler captures)")
     p.add_argument("--e2e-steps", type=int, default=10)
     p.add_argument("--no-cpu-baseline", action="store_true")
+    p.add_argument("--no-layerwise", dest="layerwise", action="store_false",
+                   help="skip the layer-wise swap timing (records split per layer, Sec. 4: first layer ready / all layers ready)")
     p.add_argument("--aot", action="store_true", help="multiapp: swap served contexts out ahead of time (Sec. 3.4 i)")
     p.add_argument("--quant-mode", type=int, default=0, choices=[0, 1],
                    help="0: groups of group_size channels of one token (the metric's setting); 1: one group per channel "
@@ -350,6 +352,50 @@ def run_ours(args):
     e2e_serial_ms = time_e2e(make_plan(n))
     e2e_ms = time_e2e(make_plan(e2e_batch))
     e2e_value = world * 2 * kv_bytes / (e2e_ms * 1e-3) / 1e9
+
+    # ---- layer-wise load (Sec. 4): records split per layer; how soon is the first layer usable, when the last
+    layerwise = None
+    if args.e2e_steps > 0 and args.layerwise:
+        from paper_2403_11805_b200.layerwise import LayerwiseContext
+        p_ = make_plan(n)[0]                         # the whole context as one batch, for comparison
+        B.compress_chunks(d, kv, p_["ids"], p_["bits"], buf, p_["meta"], p_["ws"])
+        arena.copy_(buf[:record_bytes], non_blocking=True)
+        torch.cuda.synchronize()
+        whole = []
+        for it in range(3 + args.e2e_steps):
+            w0, w1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            w0.record(stream)
+            p_["ev_out"].record(stream)
+            B.swap_in(arena, p_["meta"], back, side_stream=side_in, after=p_["ev_out"], done=p_["ev_in"], n=n)
+            stream.wait_event(p_["ev_in"])
+            B.decompress_chunks(d, back, p_["meta"], None, kv_out, p_["ws"])
+            w1.record(stream)
+            torch.cuda.synchronize()
+            if it >= 3:
+                whole.append(w0.elapsed_time(w1))
+        del back, arena
+        lw = LayerwiseContext(shape, bits, quant_mode=args.quant_mode)
+        first, last, out_ms = [], [], []
+        for it in range(3 + args.e2e_steps):
+            o0, o1, i0 = (torch.cuda.Event(enable_timing=True) for _ in range(3))
+            o0.record(stream)
+            lw.swap_out(kv)
+            lw.side_out.synchronize()
+            o1.record(stream)
+            torch.cuda.synchronize()
+            i0.record(stream)
+            lw.swap_in(kv_out)
+            torch.cuda.synchronize()
+            if it >= 3:
+                out_ms.append(o0.elapsed_time(o1))
+                first.append(i0.elapsed_time(lw.ready[0]))
+                last.append(i0.elapsed_time(lw.ready[-1]))
+        assert lw.corrupt_count() == 0
+        layerwise = {"first_layer_ready_ms": sharding.max_over_ranks([statistics.median(first)], dist, "cuda")[0],
+                     "all_layers_ready_ms": sharding.max_over_ranks([statistics.median(last)], dist, "cuda")[0],
+                     "swap_out_ms": sharding.max_over_ranks([statistics.median(out_ms)], dist, "cuda")[0],
+                     "records": "one per (layer, chunk); a layer's records travel as one copy",
+                     "whole_context_load_ms": sharding.max_over_ranks([statistics.median(whole)], dist, "cuda")[0]}
     clocks = sampler.finish() if sampler else None
 
     if rank != 0:
@@ -393,7 +439,8 @@ def run_ours(args):
                 "ms_per_step": e2e_ms, "context_switches_per_s": world / (e2e_ms * 1e-3),
                 "host_copy_gbs_each_way": record_bytes / (e2e_ms * 1e-3) / 1e9,
                 "serial_ms_per_step": e2e_serial_ms, "batch_chunks": e2e_batch,
-                "what": "compress -> swap-out to pinned host -> swap-in -> decompress, pipelined in batches of chunks"},
+                "what": "compress -> swap-out to pinned host -> swap-in -> decompress, pipelined in batches of chunks",
+                "layerwise_load": layerwise},
         "gpu_launches": args.steps * 11,   # 4 score kernels, compress and decompress once per bit-width, 1 verify
         "roofline": roofline, "clocks": clocks,
         "wall_ms_per_step": t_wall * 1e3 / args.steps,
