@@ -33,6 +33,7 @@ def parse_args():
     p.add_argument("--impl", default="ours", choices=["ours", "reference"])
     p.add_argument("--workload", default="llama7b", help="a key of synth.CONFIGS (single-context workloads)")
     p.add_argument("--layers", type=int, default=0, help="use only this many layers (smaller cases for profiler captures)")
+    p.add_argument("--chunk-len", type=int, default=0, help="override the workload's tokens per chunk (chunk-size sweep, Sec. 5.4)")
     p.add_argument("--e2e-steps", type=int, default=10)
     p.add_argument("--no-cpu-baseline", action="store_true")
     p.add_argument("--no-layerwise", dest="layerwise", action="store_false",
@@ -227,6 +228,8 @@ def run_ours(args):
     shape = synth.CONFIGS[args.workload]
     if args.layers:
         shape = shape.with_(n_layers=args.layers)
+    if args.chunk_len:
+        shape = shape.with_(chunk_len=args.chunk_len)
     W = shape.window
     frac = shape.frac if shape.frac is not None else (1 / 3, 1 / 3, 1 / 3)
     # every rank owns one context of the workload (contexts are independent: no data-path collective)

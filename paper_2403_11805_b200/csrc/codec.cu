@@ -92,7 +92,7 @@ struct CodecArgs {
 // the listed chunks of one slab index, so KV addresses run linearly when the chunk ids are consecutive
 // (measured: faster than walking the slabs of one chunk, which makes the record addresses linear instead).
 struct UnitPos {
-    uint32_t i, s_idx, chunk_id, bits;
+    uint32_t i, k, s_idx, chunk_id, bits;  // i: entry index (caller's order), k: position in this launch's list
     uint64_t rec_off;
     int e0;                // first element of this lane inside the slab
 };
@@ -102,6 +102,7 @@ __device__ __forceinline__ void decode_unit(const CodecArgs &a, uint32_t unit, i
     uint32_t item, pass, k;
     a.div_passes.divmod(unit, item, pass);
     a.div_n.divmod(item, u.s_idx, k);
+    u.k = k;
     u.i = a.order[k];
     const uint4 head = *reinterpret_cast<const uint4 *>(a.entries + u.i);  // chunk_id, bits, offset
     u.chunk_id = head.x;
@@ -212,6 +213,29 @@ struct Geo {
     static constexpr int kGroupsPerLane = G >= kLaneElems ? 1 : kLaneElems / G;
     static constexpr int kPiecesPerGroup = kPieces / kGroupsPerLane;
 };
+
+// Record checksums are sums of 32-bit words, so partial sums may be added in any order.  A launch with few
+// chunks would send every unit's partial sum to the same few addresses (measured: with 5 chunks per launch the
+// same-address atomics made the kernels up to twice as slow), so a CTA first adds them up in shared memory,
+// one slot per chunk of the launch, and sends one atomic per chunk when it ends.  Launches with more chunks than
+// slots add straight to global memory, where that many addresses do not collide.
+constexpr int kSumSlots = 1024;
+
+__device__ __forceinline__ void cta_sums_clear(uint32_t *slots, int n)
+{
+    if (n <= kSumSlots)
+        for (int k = threadIdx.x; k < n; k += kThreads) slots[k] = 0;
+    __syncthreads();
+}
+
+__device__ __forceinline__ void unit_sum_add(uint32_t *slots, int n, uint32_t k, uint32_t *global_slot, uint32_t sum, int lane)
+{
+    sum = __reduce_add_sync(0xffffffffu, sum);
+    if (lane == 0) {
+        if (n <= kSumSlots) atomicAdd(&slots[k], sum);
+        else atomicAdd(global_slot, sum);
+    }
+}
 
 // ---------------------------------------------------------------------------------------------- quantize
 
@@ -341,7 +365,8 @@ __device__ __forceinline__ uint32_t compress_unit_bits(const CodecArgs &a, const
     uint32_t c[kPieces][BITS / 2];
     bool any_clamp = false;
 #pragma unroll
-    for (int g = 0; g < geo::kGroupsPerLane; ++g) any_clamp |= gp[g].needs_clamp;
+    for (int g = 0; g < geo::kGroupsPerLane; ++g)  // groups past the end of the slab (loaded as zeros) do not count
+        any_clamp |= gp[g].needs_clamp && u.e0 + (geo::kGroupsPerLane > 1 ? g * G : 0) < a.slab_elems;
     if (__any_sync(0xffffffffu, any_clamp)) {
 #pragma unroll
         for (int j = 0; j < kPieces; ++j) {
@@ -477,13 +502,13 @@ __device__ __forceinline__ void prefetch_unit_l2(const CodecArgs &a, uint32_t un
 }
 
 template <int BITS, int G, bool WIDE>
-__device__ __forceinline__ void compress_unit(const CodecArgs &a, const UnitPos &u, const uint32_t (&w)[kPieces][8], int lane)
+__device__ __forceinline__ void compress_unit(const CodecArgs &a, const UnitPos &u, const uint32_t (&w)[kPieces][8], int lane,
+                                              uint32_t *sum_slots)
 {
     uint8_t *rec = a.buf + u.rec_off;
-    uint32_t sum = compress_unit_bits<BITS, G, WIDE>(a, u, w, rec, lane);
+    const uint32_t sum = compress_unit_bits<BITS, G, WIDE>(a, u, w, rec, lane);
     if (u.s_idx == 0 && u.e0 < kPassElems) zero_padding(a, rec, BITS, lane);  // first pass of the chunk's first slab
-    sum = __reduce_add_sync(0xffffffffu, sum);
-    if (lane == 0) atomicAdd(&a.entries[u.i].checksum, sum);
+    unit_sum_add(sum_slots, a.n, u.k, &a.entries[u.i].checksum, sum, lane);
 }
 
 // One launch per bit-width present in the call: a single code path per kernel keeps the instruction
@@ -494,35 +519,42 @@ __global__ void __launch_bounds__(kThreads, 2) compress_kernel(const CodecArgs a
     const int lane = threadIdx.x & 31;
     const uint32_t n_warps = gridDim.x * kWarpsPerBlock;
     uint32_t unit = blockIdx.x * kWarpsPerBlock + (threadIdx.x >> 5);
-    if (unit >= a.total_units) return;
     __shared__ __align__(16) unsigned char patches[kWarpsPerBlock][kTransposeBytes];
-    unsigned char *patch = patches[threadIdx.x >> 5];
-    UnitPos pa, pb;
-    uint32_t wa[kPieces][8], wb[kPieces][8];
-    decode_unit(a, unit, lane, pa);
-    load_unit<WIDE>(a, pa, lane, wa);
-    for (;;) {  // two units per trip, so that the buffers swap roles without register copies
-        bool more = a.total_units - unit > n_warps;
-        if (more) {
-            decode_unit(a, unit + n_warps, lane, pb);
-            load_unit<WIDE>(a, pb, lane, wb);
+    __shared__ uint32_t sum_slots[kSumSlots];
+    cta_sums_clear(sum_slots, a.n);
+    if (unit < a.total_units) {
+        unsigned char *patch = patches[threadIdx.x >> 5];
+        UnitPos pa, pb;
+        uint32_t wa[kPieces][8], wb[kPieces][8];
+        decode_unit(a, unit, lane, pa);
+        load_unit<WIDE>(a, pa, lane, wa);
+        for (;;) {  // two units per trip, so that the buffers swap roles without register copies
+            bool more = a.total_units - unit > n_warps;
+            if (more) {
+                decode_unit(a, unit + n_warps, lane, pb);
+                load_unit<WIDE>(a, pb, lane, wb);
+            }
+            if (a.total_units - unit > kPrefetchAhead * n_warps) prefetch_unit_l2(a, unit + kPrefetchAhead * n_warps, lane);
+            to_lane_contiguous(wa, patch, lane);
+            compress_unit<BITS, G, WIDE>(a, pa, wa, lane, sum_slots);
+            if (!more) break;
+            unit += n_warps;
+            more = a.total_units - unit > n_warps;
+            if (more) {
+                decode_unit(a, unit + n_warps, lane, pa);
+                load_unit<WIDE>(a, pa, lane, wa);
+            }
+            if (a.total_units - unit > kPrefetchAhead * n_warps) prefetch_unit_l2(a, unit + kPrefetchAhead * n_warps, lane);
+            to_lane_contiguous(wb, patch, lane);
+            compress_unit<BITS, G, WIDE>(a, pb, wb, lane, sum_slots);
+            if (!more) break;
+            unit += n_warps;
         }
-        if (a.total_units - unit > kPrefetchAhead * n_warps) prefetch_unit_l2(a, unit + kPrefetchAhead * n_warps, lane);
-        to_lane_contiguous(wa, patch, lane);
-        compress_unit<BITS, G, WIDE>(a, pa, wa, lane);
-        if (!more) break;
-        unit += n_warps;
-        more = a.total_units - unit > n_warps;
-        if (more) {
-            decode_unit(a, unit + n_warps, lane, pa);
-            load_unit<WIDE>(a, pa, lane, wa);
-        }
-        if (a.total_units - unit > kPrefetchAhead * n_warps) prefetch_unit_l2(a, unit + kPrefetchAhead * n_warps, lane);
-        to_lane_contiguous(wb, patch, lane);
-        compress_unit<BITS, G, WIDE>(a, pb, wb, lane);
-        if (!more) break;
-        unit += n_warps;
     }
+    __syncthreads();
+    if (a.n <= kSumSlots)
+        for (int k = threadIdx.x; k < a.n; k += kThreads)
+            if (sum_slots[k]) atomicAdd(&a.entries[a.order[k]].checksum, sum_slots[k]);
 }
 
 // ---------------------------------------------------------------------------------------------- dequantize
@@ -535,7 +567,7 @@ __global__ void __launch_bounds__(kThreads, 2) compress_kernel(const CodecArgs a
 constexpr int kPieceStride = 32 * kPieceElems;  // elements between a lane's pieces
 
 struct DecodePos {
-    uint32_t i;              // entry index (checksum slot)
+    uint32_t i, k;           // entry index (checksum slot); position in this launch's list
     int room;                // slab elements from this lane's piece 0 to the end of the slab (<= 0: none)
     const uint8_t *codes;    // piece 0: packed codes
     const uint32_t *params;  // piece 0: parameter word of its group
@@ -551,6 +583,7 @@ __device__ __forceinline__ void decode_unit_for_decoder(const CodecArgs &a, uint
     a.div_n.divmod(item, s_idx, k);
     const uint4 t = *reinterpret_cast<const uint4 *>(a.table + k);  // chunk_id, entry, record offset
     u.i = t.y;
+    u.k = k;
     const uint32_t e = pass * kPassElems + lane * kPieceElems;      // piece 0 inside the slab
     u.room = a.slab_elems - (int)e;
     const uint8_t *rec = a.buf + ((uint64_t)t.z | ((uint64_t)t.w << 32));
@@ -643,7 +676,7 @@ __device__ __forceinline__ void dequantize_piece(const uint32_t *c, unsigned sho
 
 template <int BITS, int G, bool WIDE>
 __device__ __forceinline__ void decompress_unit(const CodecArgs &a, const DecodePos &u, const uint32_t (&c)[kPieces][BITS / 2],
-                                                const uint32_t (&p)[kPieces], int lane)
+                                                const uint32_t (&p)[kPieces], int lane, uint32_t *sum_slots)
 {
     // a lane's pieces all sit at the same place inside their groups: either every one opens a group or none does
     const bool opens_group = (lane * kPieceElems) % G == 0;
@@ -660,8 +693,7 @@ __device__ __forceinline__ void decompress_unit(const CodecArgs &a, const Decode
         for (int k = 0; k < BITS / 2; ++k) sum += c[j][k];
         if (opens_group) sum += p[j];  // the piece that opens a group accounts for its parameter word
     }
-    sum = __reduce_add_sync(0xffffffffu, sum);
-    if (lane == 0) atomicAdd(&a.sums[u.i], sum);
+    unit_sum_add(sum_slots, a.n, u.k, &a.sums[u.i], sum, lane);
 }
 
 // Units whose loads are in flight per warp, the one being decoded included, and resident CTAs per SM.  Measured
@@ -678,32 +710,40 @@ __global__ void __launch_bounds__(kThreads, kDecodeBlocksPerSm) decompress_kerne
     const int lane = threadIdx.x & 31;
     const uint32_t n_warps = gridDim.x * kWarpsPerBlock;
     uint32_t unit = blockIdx.x * kWarpsPerBlock + (threadIdx.x >> 5);
-    if (unit >= a.total_units) return;
-    DecodePos pos[D];
-    uint32_t c[D][kPieces][BITS / 2], p[D][kPieces];
+    __shared__ uint32_t sum_slots[kSumSlots];
+    cta_sums_clear(sum_slots, a.n);
+    if (unit < a.total_units) {
+        DecodePos pos[D];
+        uint32_t c[D][kPieces][BITS / 2], p[D][kPieces];
 #pragma unroll
-    for (int s = 0; s < D - 1; ++s) {
-        const uint32_t ahead = unit + s * n_warps;
-        if (ahead < a.total_units) {
-            decode_unit_for_decoder<BITS, G>(a, ahead, lane, pos[s]);
-            load_unit_codes<BITS, G>(pos[s], c[s], p[s]);
-        }
-    }
-    for (;;) {
-#pragma unroll
-        for (int s = 0; s < D; ++s) {
-            // ring slot s holds the current unit; the slot freed last takes the unit D-1 strides ahead
-            const int fill = (s + D - 1) % D;
-            const uint32_t ahead = unit + (D - 1) * n_warps;
+        for (int s = 0; s < D - 1; ++s) {
+            const uint32_t ahead = unit + s * n_warps;
             if (ahead < a.total_units) {
-                decode_unit_for_decoder<BITS, G>(a, ahead, lane, pos[fill]);
-                load_unit_codes<BITS, G>(pos[fill], c[fill], p[fill]);
+                decode_unit_for_decoder<BITS, G>(a, ahead, lane, pos[s]);
+                load_unit_codes<BITS, G>(pos[s], c[s], p[s]);
             }
-            decompress_unit<BITS, G, WIDE>(a, pos[s], c[s], p[s], lane);
-            unit += n_warps;
-            if (unit >= a.total_units) return;
+        }
+        for (bool done = false; !done;) {
+#pragma unroll
+            for (int s = 0; s < D; ++s) {
+                if (done) break;
+                // ring slot s holds the current unit; the slot freed last takes the unit D-1 strides ahead
+                const int fill = (s + D - 1) % D;
+                const uint32_t ahead = unit + (D - 1) * n_warps;
+                if (ahead < a.total_units) {
+                    decode_unit_for_decoder<BITS, G>(a, ahead, lane, pos[fill]);
+                    load_unit_codes<BITS, G>(pos[fill], c[fill], p[fill]);
+                }
+                decompress_unit<BITS, G, WIDE>(a, pos[s], c[s], p[s], lane, sum_slots);
+                unit += n_warps;
+                done = unit >= a.total_units;
+            }
         }
     }
+    __syncthreads();
+    if (a.n <= kSumSlots)
+        for (int k = threadIdx.x; k < a.n; k += kThreads)
+            if (sum_slots[k]) atomicAdd(&a.sums[a.table[k].entry], sum_slots[k]);
 }
 
 }  // namespace llms
