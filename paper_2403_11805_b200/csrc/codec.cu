@@ -697,11 +697,11 @@ __device__ __forceinline__ void decompress_unit(const CodecArgs &a, const Decode
 }
 
 // Units whose loads are in flight per warp, the one being decoded included, and resident CTAs per SM.  Measured
-// on the 7B shape (decompress stage, ms): depth 2 with 3 CTAs 0.555, depth 3 with 3 CTAs 0.561-0.565, depth 3 or 4
-// with 2 CTAs 0.555-0.557, depth 4 with 3 CTAs 0.62-0.63 (spills), 4 CTAs 0.60: the stage is bound by the write
-// path, not by load latency.
+// on the 7B shape (decompress stage, ms; depth x CTAs): 2x2 0.516-0.519, 4x1 0.513-0.514, 6x1 0.515, 2x3 0.535,
+// 3x2 0.534-0.537, 4x2 0.539, 2x4 0.539, 3x3 0.549, 2x1 0.583: the store-heavy stream runs best with 8 to 16
+// warps per SM as long as 32 or more units are in flight.
 constexpr int kDecodeDepth = 2;
-constexpr int kDecodeBlocksPerSm = 3;
+constexpr int kDecodeBlocksPerSm = 2;
 
 template <int BITS, int G, bool WIDE>
 __global__ void __launch_bounds__(kThreads, kDecodeBlocksPerSm) decompress_kernel(const CodecArgs a)
@@ -855,6 +855,15 @@ static int grid_for(K kernel, int64_t items, size_t dyn_smem = 0)
     const int64_t want = (items + kWarpsPerBlock - 1) / kWarpsPerBlock;
     const int64_t cap = (int64_t)sm_count() * per_sm;
     return (int)(want < cap ? want : cap);
+}
+
+// The decoder's grid: never more CTAs per SM than it was tuned for, whatever the register count allows.
+template <typename K>
+static int decode_grid(K kernel, int64_t items)
+{
+    const int cap = sm_count() * kDecodeBlocksPerSm;
+    const int grid = grid_for(kernel, items);
+    return grid < cap ? grid : cap;
 }
 
 // Measured on the 7B-shaped context (same box, same run): register-prefetch kernel 0.561 ms, bulk-copy pipeline
@@ -1045,8 +1054,8 @@ extern "C" int llms_decompress_chunks(const llms_kv_desc *desc, const void *buf,
         rc = dispatch_group(desc->group_size, [&](auto g) {
             constexpr int kG = decltype(g)::value;
 #define LLMS_LAUNCH(BITS)                                                                                                   \
-    if (wide) decompress_kernel<BITS, kG, true><<<grid_for(decompress_kernel<BITS, kG, true>, b.total_units), kThreads, 0, st>>>(b); \
-    else decompress_kernel<BITS, kG, false><<<grid_for(decompress_kernel<BITS, kG, false>, b.total_units), kThreads, 0, st>>>(b)
+    if (wide) decompress_kernel<BITS, kG, true><<<decode_grid(decompress_kernel<BITS, kG, true>, b.total_units), kThreads, 0, st>>>(b); \
+    else decompress_kernel<BITS, kG, false><<<decode_grid(decompress_kernel<BITS, kG, false>, b.total_units), kThreads, 0, st>>>(b)
             if (k == 0) { LLMS_LAUNCH(8); } else if (k == 1) { LLMS_LAUNCH(4); } else { LLMS_LAUNCH(2); }
 #undef LLMS_LAUNCH
         });
