@@ -34,6 +34,11 @@ constexpr int kPassElems = 32 * kLaneElems;     // 2048 elements = 4 KiB of fp16
 constexpr uint32_t kPrefetchAhead = 2;          // compress: units ahead that are pulled into L2 (measured: 2 -> 0.521 ms,
                                                 // 3 -> 0.535, 5 -> 0.59, 8 -> 0.79 for compress on the 7B shape)
 
+// Measured on the 7B-shaped context (same box, same run): register-prefetch kernel 0.561 ms, bulk-copy pipeline
+// 0.579-0.591 ms.  Both are bound by instruction issue, not by the memory path, and the pipeline spends more
+// instructions (shared-memory traffic, barrier polling, single-lane sections), so the direct kernel is used.
+constexpr bool kUseBulkCompress = false;
+
 // Division by a launch-time constant as multiply-high and shift: exact for numerators below 2^31.
 struct FastDiv {
     uint32_t d, mul, shr;
@@ -79,7 +84,12 @@ struct CodecArgs {
     int slab_elems;        // chunk_len * head_dim
     int groups_per_slab;
     int n_kv_heads;
-    int passes;            // warp passes per slab
+    int passes;            // warp passes per slab (1 when packed)
+    int unit_rows;         // slabs per chunk, or, packed, units per chunk
+    int packed;            // 1: slabs shorter than a pass, a unit covers slabs_per_unit whole slabs (see UnitPos)
+    int slab_shift;        // packed: log2(slab_elems)
+    int slabs_per_unit;    // packed: kPassElems / slab_elems
+    uint32_t chunk_elems;  // n_slabs * slab_elems
     FastDiv div_passes, div_n, div_heads;
     uint32_t step_units, step_pass, step_k, step_s;  // stride between a warp's units (= warps of the grid), split by radix
     uint32_t total_units;  // n * n_slabs * passes
@@ -91,24 +101,41 @@ struct CodecArgs {
 // Where a unit's data is.  Units are numbered slab-major: consecutive units walk the passes of a slab, then
 // the listed chunks of one slab index, so KV addresses run linearly when the chunk ids are consecutive
 // (measured: faster than walking the slabs of one chunk, which makes the record addresses linear instead).
+//
+// Packed units: when a slab is shorter than a pass (small chunk_len * head_dim) and divides it, a unit covers
+// kPassElems / slab_elems consecutive slabs of one chunk instead of a mostly empty pass of one.  In the record
+// those slabs are adjacent (codes and parameters are stored in slab order), so s_idx and e0 below keep their
+// meaning for every record offset, with e0 running past the end of slab s_idx; only the KV addresses have to be
+// looked up slab by slab.
 struct UnitPos {
     uint32_t i, k, s_idx, chunk_id, bits;  // i: entry index (caller's order), k: position in this launch's list
     uint64_t rec_off;
-    int e0;                // first element of this lane inside the slab
+    int e0;                // first element of this lane, counted from the start of slab s_idx
+    int limit;             // elements of this unit that exist, counted from the unit's first element
 };
 
+template <bool PACKED>
 __device__ __forceinline__ void decode_unit(const CodecArgs &a, uint32_t unit, int lane, UnitPos &u)
 {
     uint32_t item, pass, k;
     a.div_passes.divmod(unit, item, pass);
-    a.div_n.divmod(item, u.s_idx, k);
+    uint32_t row;
+    a.div_n.divmod(item, row, k);
     u.k = k;
     u.i = a.order[k];
     const uint4 head = *reinterpret_cast<const uint4 *>(a.entries + u.i);  // chunk_id, bits, offset
     u.chunk_id = head.x;
     u.bits = head.y;
     u.rec_off = (uint64_t)head.z | ((uint64_t)head.w << 32);
-    u.e0 = (int)pass * kPassElems + lane * kLaneElems;
+    if constexpr (PACKED) {
+        u.s_idx = row * (uint32_t)a.slabs_per_unit;
+        u.e0 = lane * kLaneElems;
+        u.limit = (int)min((uint32_t)kPassElems, a.chunk_elems - row * kPassElems);
+    } else {
+        u.s_idx = row;
+        u.e0 = (int)pass * kPassElems + lane * kLaneElems;
+        u.limit = min(kPassElems, a.slab_elems - (int)pass * kPassElems);
+    }
 }
 
 __device__ __forceinline__ int64_t slab_offset(const CodecArgs &a, uint32_t s_idx, uint32_t chunk)
@@ -117,6 +144,14 @@ __device__ __forceinline__ int64_t slab_offset(const CodecArgs &a, uint32_t s_id
     a.div_heads.divmod(s_idx, ls, h);
     return (int64_t)(ls >> 1) * a.stride_l + (int64_t)(ls & 1) * a.stride_s + (int64_t)h * a.stride_h +
            (int64_t)chunk * a.chunk_stride;
+}
+
+// KV offset of element v of a unit (v counted from the unit's first element)
+template <bool PACKED>
+__device__ __forceinline__ int64_t unit_elem_offset(const CodecArgs &a, uint32_t s_idx, uint32_t chunk, int pass_e0, int v)
+{
+    if constexpr (PACKED) return slab_offset(a, s_idx + (uint32_t)(v >> a.slab_shift), chunk) + (v & (a.slab_elems - 1));
+    return slab_offset(a, s_idx, chunk) + pass_e0 + v;
 }
 
 __device__ __forceinline__ __half2 as_h2(uint32_t u) { return *reinterpret_cast<__half2 *>(&u); }
@@ -339,6 +374,7 @@ __device__ __forceinline__ uint32_t compress_unit_bits(const CodecArgs &a, const
 {
     using geo = Geo<G>;
     constexpr int kPieceBytes = kPieceElems * BITS / 8;
+    const int le0 = lane * kLaneElems;  // this lane's first element inside the unit
     // ---- group minima and maxima
     GroupParams gp[geo::kGroupsPerLane];
     {
@@ -366,7 +402,7 @@ __device__ __forceinline__ uint32_t compress_unit_bits(const CodecArgs &a, const
     bool any_clamp = false;
 #pragma unroll
     for (int g = 0; g < geo::kGroupsPerLane; ++g)  // groups past the end of the slab (loaded as zeros) do not count
-        any_clamp |= gp[g].needs_clamp && u.e0 + (geo::kGroupsPerLane > 1 ? g * G : 0) < a.slab_elems;
+        any_clamp |= gp[g].needs_clamp && le0 + (geo::kGroupsPerLane > 1 ? g * G : 0) < u.limit;
     if (__any_sync(0xffffffffu, any_clamp)) {
 #pragma unroll
         for (int j = 0; j < kPieces; ++j) {
@@ -389,7 +425,7 @@ __device__ __forceinline__ uint32_t compress_unit_bits(const CodecArgs &a, const
     uint8_t *codes = rec + a.codes_off + (uint64_t)u.s_idx * a.slab_elems * BITS / 8 + (uint32_t)u.e0 * BITS / 8;
     uint32_t *params = reinterpret_cast<uint32_t *>(rec) + (uint64_t)u.s_idx * a.groups_per_slab + (uint32_t)u.e0 / G;
     uint32_t sum = 0;
-    const bool lane_full = u.e0 + kLaneElems <= a.slab_elems;
+    const bool lane_full = le0 + kLaneElems <= u.limit;
     constexpr uintptr_t kLaneAlign = BITS == 2 ? 15 : 31;
     if (lane_full && (reinterpret_cast<uintptr_t>(codes) & kLaneAlign) == 0) {
         if constexpr (BITS == 8) {
@@ -407,7 +443,7 @@ __device__ __forceinline__ uint32_t compress_unit_bits(const CodecArgs &a, const
     } else {
 #pragma unroll
         for (int j = 0; j < kPieces; ++j) {
-            if (u.e0 + j * kPieceElems < a.slab_elems) {
+            if (le0 + j * kPieceElems < u.limit) {
                 if constexpr (BITS == 8) st128(codes + j * kPieceBytes, c[j][0], c[j][1], c[j][2], c[j][3]);
                 else if constexpr (BITS == 4) st64(codes + j * kPieceBytes, c[j][0], c[j][1]);
                 else st32(codes + j * kPieceBytes, c[j][0]);
@@ -417,14 +453,14 @@ __device__ __forceinline__ uint32_t compress_unit_bits(const CodecArgs &a, const
         }
     }
     if constexpr (geo::kGroupsPerLane == 1) {
-        if (u.e0 < a.slab_elems && (lane & (geo::kLanesPerGroup - 1)) == 0) {
+        if (le0 < u.limit && (lane & (geo::kLanesPerGroup - 1)) == 0) {
             st32(params, gp[0].word);
             sum += gp[0].word;
         }
     } else {
 #pragma unroll
         for (int g = 0; g < geo::kGroupsPerLane; ++g) {
-            if (u.e0 + g * G < a.slab_elems) {
+            if (le0 + g * G < u.limit) {
                 st32(params + g, gp[g].word);
                 sum += gp[g].word;
             }
@@ -445,18 +481,18 @@ __device__ __forceinline__ void zero_padding(const CodecArgs &a, uint8_t *rec, u
 // The unit is fetched so that every load instruction of the warp reads 1 KiB of consecutive bytes (piece j of
 // lane L = elements [j*512 + L*16, +16) of the pass): measured on this part, a stream read with 128 consecutive
 // bytes per lane tops out near 5.6 TB/s, one with consecutive lanes on consecutive 32 bytes near 6.9 TB/s.
-template <bool WIDE>
+template <bool WIDE, bool PACKED>
 __device__ __forceinline__ void load_unit(const CodecArgs &a, const UnitPos &u, int lane, uint32_t (&w)[kPieces][8])
 {
     const int pass_e0 = u.e0 - lane * kLaneElems;
-    const __half *src = a.kv_in + slab_offset(a, u.s_idx, u.chunk_id) + pass_e0 + lane * kPieceElems;
 #pragma unroll
     for (int j = 0; j < kPieces; ++j) {
-        if (pass_e0 + j * (32 * kPieceElems) + lane * kPieceElems < a.slab_elems) {
-            load32<WIDE>(src + j * (32 * kPieceElems), w[j]);
+        const int v = j * (32 * kPieceElems) + lane * kPieceElems;
+        if (v < u.limit) {
+            load32<WIDE>(a.kv_in + unit_elem_offset<PACKED>(a, u.s_idx, u.chunk_id, pass_e0, v), w[j]);
         } else {
 #pragma unroll
-            for (int k = 0; k < 8; ++k) w[j][k] = 0;  // past the end of the slab: whole inactive groups
+            for (int k = 0; k < 8; ++k) w[j][k] = 0;  // past the end: whole inactive groups
         }
     }
 }
@@ -490,14 +526,19 @@ __device__ __forceinline__ void to_lane_contiguous(uint32_t (&w)[kPieces][8], un
 
 // Ask for a unit's KV bytes to be brought into L2 (one bulk prefetch by one lane): the register loads of that
 // unit, issued one unit later, then find them there instead of waiting for DRAM.
+template <bool PACKED>
 __device__ __forceinline__ void prefetch_unit_l2(const CodecArgs &a, uint32_t unit, int lane)
 {
     UnitPos u;
-    decode_unit(a, unit, 0, u);
-    if (lane == 0) {
+    decode_unit<PACKED>(a, unit, 0, u);
+    if constexpr (PACKED) {  // one prefetch per slab of the unit
+        if (lane < a.slabs_per_unit && lane * a.slab_elems < u.limit) {
+            const __half *src = a.kv_in + slab_offset(a, u.s_idx + lane, u.chunk_id);
+            asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" :: "l"(src), "r"((uint32_t)a.slab_elems * 2) : "memory");
+        }
+    } else if (lane == 0) {
         const __half *src = a.kv_in + slab_offset(a, u.s_idx, u.chunk_id) + u.e0;
-        const uint32_t bytes = (uint32_t)min(kPassElems, a.slab_elems - u.e0) * 2;
-        asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" :: "l"(src), "r"(bytes) : "memory");
+        asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" :: "l"(src), "r"((uint32_t)u.limit * 2) : "memory");
     }
 }
 
@@ -513,7 +554,7 @@ __device__ __forceinline__ void compress_unit(const CodecArgs &a, const UnitPos 
 
 // One launch per bit-width present in the call: a single code path per kernel keeps the instruction
 // working set small (with all three widths in one kernel the warps stalled on instruction fetch).
-template <int BITS, int G, bool WIDE>
+template <int BITS, int G, bool WIDE, bool PACKED>
 __global__ void __launch_bounds__(kThreads, 2) compress_kernel(const CodecArgs a)
 {
     const int lane = threadIdx.x & 31;
@@ -526,25 +567,25 @@ __global__ void __launch_bounds__(kThreads, 2) compress_kernel(const CodecArgs a
         unsigned char *patch = patches[threadIdx.x >> 5];
         UnitPos pa, pb;
         uint32_t wa[kPieces][8], wb[kPieces][8];
-        decode_unit(a, unit, lane, pa);
-        load_unit<WIDE>(a, pa, lane, wa);
+        decode_unit<PACKED>(a, unit, lane, pa);
+        load_unit<WIDE, PACKED>(a, pa, lane, wa);
         for (;;) {  // two units per trip, so that the buffers swap roles without register copies
             bool more = a.total_units - unit > n_warps;
             if (more) {
-                decode_unit(a, unit + n_warps, lane, pb);
-                load_unit<WIDE>(a, pb, lane, wb);
+                decode_unit<PACKED>(a, unit + n_warps, lane, pb);
+                load_unit<WIDE, PACKED>(a, pb, lane, wb);
             }
-            if (a.total_units - unit > kPrefetchAhead * n_warps) prefetch_unit_l2(a, unit + kPrefetchAhead * n_warps, lane);
+            if (a.total_units - unit > kPrefetchAhead * n_warps) prefetch_unit_l2<PACKED>(a, unit + kPrefetchAhead * n_warps, lane);
             to_lane_contiguous(wa, patch, lane);
             compress_unit<BITS, G, WIDE>(a, pa, wa, lane, sum_slots);
             if (!more) break;
             unit += n_warps;
             more = a.total_units - unit > n_warps;
             if (more) {
-                decode_unit(a, unit + n_warps, lane, pa);
-                load_unit<WIDE>(a, pa, lane, wa);
+                decode_unit<PACKED>(a, unit + n_warps, lane, pa);
+                load_unit<WIDE, PACKED>(a, pa, lane, wa);
             }
-            if (a.total_units - unit > kPrefetchAhead * n_warps) prefetch_unit_l2(a, unit + kPrefetchAhead * n_warps, lane);
+            if (a.total_units - unit > kPrefetchAhead * n_warps) prefetch_unit_l2<PACKED>(a, unit + kPrefetchAhead * n_warps, lane);
             to_lane_contiguous(wb, patch, lane);
             compress_unit<BITS, G, WIDE>(a, pb, wb, lane, sum_slots);
             if (!more) break;
@@ -568,28 +609,39 @@ constexpr int kPieceStride = 32 * kPieceElems;  // elements between a lane's pie
 
 struct DecodePos {
     uint32_t i, k;           // entry index (checksum slot); position in this launch's list
-    int room;                // slab elements from this lane's piece 0 to the end of the slab (<= 0: none)
+    int room;                // elements from this lane's piece 0 to the end of the unit's data (<= 0: none)
     const uint8_t *codes;    // piece 0: packed codes
     const uint32_t *params;  // piece 0: parameter word of its group
-    __half *dst;             // piece 0: destination
+    uint32_t s_idx, chunk_id;  // destination: first slab of the unit, chunk slot
+    int pass_e0;             // first element of the unit inside slab s_idx (0 when packed)
 };
 
-template <int BITS, int G>
+template <int BITS, int G, bool PACKED>
 __device__ __forceinline__ void decode_unit_for_decoder(const CodecArgs &a, uint32_t unit, int lane, DecodePos &u)
 {
     static_assert(kPieceStride % G == 0 || G % kPieceStride == 0, "groups and pieces nest");
-    uint32_t item, pass, s_idx, k;
+    uint32_t item, pass, row, k;
     a.div_passes.divmod(unit, item, pass);
-    a.div_n.divmod(item, s_idx, k);
+    a.div_n.divmod(item, row, k);
     const uint4 t = *reinterpret_cast<const uint4 *>(a.table + k);  // chunk_id, entry, record offset
     u.i = t.y;
     u.k = k;
-    const uint32_t e = pass * kPassElems + lane * kPieceElems;      // piece 0 inside the slab
-    u.room = a.slab_elems - (int)e;
+    u.chunk_id = t.x;
+    int limit;
+    if constexpr (PACKED) {
+        u.s_idx = row * (uint32_t)a.slabs_per_unit;
+        u.pass_e0 = 0;
+        limit = (int)min((uint32_t)kPassElems, a.chunk_elems - row * kPassElems);
+    } else {
+        u.s_idx = row;
+        u.pass_e0 = (int)pass * kPassElems;
+        limit = a.slab_elems - u.pass_e0;
+    }
+    u.room = limit - lane * kPieceElems;
+    const uint32_t e = (uint32_t)u.pass_e0 + lane * kPieceElems;    // piece 0, counted from the start of slab s_idx
     const uint8_t *rec = a.buf + ((uint64_t)t.z | ((uint64_t)t.w << 32));
-    u.params = reinterpret_cast<const uint32_t *>(rec) + (s_idx * (uint32_t)a.groups_per_slab + e / G);
-    u.codes = rec + a.codes_off + ((uint64_t)s_idx * a.slab_elems + e) * BITS / 8;
-    u.dst = a.kv_out + slab_offset(a, s_idx, t.x) + e;
+    u.params = reinterpret_cast<const uint32_t *>(rec) + (u.s_idx * (uint32_t)a.groups_per_slab + e / G);
+    u.codes = rec + a.codes_off + ((uint64_t)u.s_idx * a.slab_elems + e) * BITS / 8;
 }
 
 template <int BITS, int G>
@@ -674,7 +726,7 @@ __device__ __forceinline__ void dequantize_piece(const uint32_t *c, unsigned sho
                                   fma_f32_f16(code_half<BITS>(q, 2 * k + 1), scale_h, zero));
 }
 
-template <int BITS, int G, bool WIDE>
+template <int BITS, int G, bool WIDE, bool PACKED>
 __device__ __forceinline__ void decompress_unit(const CodecArgs &a, const DecodePos &u, const uint32_t (&c)[kPieces][BITS / 2],
                                                 const uint32_t (&p)[kPieces], int lane, uint32_t *sum_slots)
 {
@@ -687,7 +739,8 @@ __device__ __forceinline__ void decompress_unit(const CodecArgs &a, const Decode
         const float zero = __half2float(__ushort_as_half((unsigned short)(p[j] >> 16)));
         uint32_t w[8];
         dequantize_piece<BITS>(c[j], scale_h, zero, w);
-        if (u.room > j * kPieceStride) store32<WIDE>(u.dst + j * kPieceStride, w);
+        if (u.room > j * kPieceStride)
+            store32<WIDE>(a.kv_out + unit_elem_offset<PACKED>(a, u.s_idx, u.chunk_id, u.pass_e0, j * kPieceStride + lane * kPieceElems), w);
         // pieces past the end of the slab were loaded as zeros and add nothing
 #pragma unroll
         for (int k = 0; k < BITS / 2; ++k) sum += c[j][k];
@@ -703,7 +756,7 @@ __device__ __forceinline__ void decompress_unit(const CodecArgs &a, const Decode
 constexpr int kDecodeDepth = 2;
 constexpr int kDecodeBlocksPerSm = 2;
 
-template <int BITS, int G, bool WIDE>
+template <int BITS, int G, bool WIDE, bool PACKED>
 __global__ void __launch_bounds__(kThreads, kDecodeBlocksPerSm) decompress_kernel(const CodecArgs a)
 {
     constexpr int D = kDecodeDepth;
@@ -719,7 +772,7 @@ __global__ void __launch_bounds__(kThreads, kDecodeBlocksPerSm) decompress_kerne
         for (int s = 0; s < D - 1; ++s) {
             const uint32_t ahead = unit + s * n_warps;
             if (ahead < a.total_units) {
-                decode_unit_for_decoder<BITS, G>(a, ahead, lane, pos[s]);
+                decode_unit_for_decoder<BITS, G, PACKED>(a, ahead, lane, pos[s]);
                 load_unit_codes<BITS, G>(pos[s], c[s], p[s]);
             }
         }
@@ -731,10 +784,10 @@ __global__ void __launch_bounds__(kThreads, kDecodeBlocksPerSm) decompress_kerne
                 const int fill = (s + D - 1) % D;
                 const uint32_t ahead = unit + (D - 1) * n_warps;
                 if (ahead < a.total_units) {
-                    decode_unit_for_decoder<BITS, G>(a, ahead, lane, pos[fill]);
+                    decode_unit_for_decoder<BITS, G, PACKED>(a, ahead, lane, pos[fill]);
                     load_unit_codes<BITS, G>(pos[fill], c[fill], p[fill]);
                 }
-                decompress_unit<BITS, G, WIDE>(a, pos[s], c[s], p[s], lane, sum_slots);
+                decompress_unit<BITS, G, WIDE, PACKED>(a, pos[s], c[s], p[s], lane, sum_slots);
                 unit += n_warps;
                 done = unit >= a.total_units;
             }
@@ -764,7 +817,7 @@ __global__ void verify_kernel(const ChunkEntry *entries, const uint32_t *sums, i
 
 // ---------------------------------------------------------------------------------------------- host side
 
-static int fill_args(const llms_kv_desc &d, CodecArgs &a, int n, void *workspace)
+static int fill_args(const llms_kv_desc &d, CodecArgs &a, int n, void *workspace, bool wide)
 {
     a.n = n;
     a.n_slabs = (int)slabs_per_chunk(d);
@@ -777,8 +830,22 @@ static int fill_args(const llms_kv_desc &d, CodecArgs &a, int n, void *workspace
     a.stride_s = d.stride_s;
     a.stride_h = d.stride_h;
     a.chunk_stride = (int64_t)d.chunk_len * d.head_dim;
-    a.passes = (a.slab_elems + kPassElems - 1) / kPassElems;
-    a.total_units = (uint32_t)n * (uint32_t)a.n_slabs * (uint32_t)a.passes;
+    a.chunk_elems = (uint32_t)a.n_slabs * (uint32_t)a.slab_elems;
+    // slabs shorter than a pass: whole slabs are packed into a unit (only with 256-bit accesses; the bulk-copy
+    // and channel-wise kernels keep their own walk over slabs)
+    a.packed = wide && d.quant_mode == 0 && !kUseBulkCompress && a.slab_elems < kPassElems && kPassElems % a.slab_elems == 0 &&
+               a.slab_elems % kLaneElems == 0;
+    if (a.packed) {
+        a.passes = 1;
+        a.slabs_per_unit = kPassElems / a.slab_elems;
+        a.slab_shift = 0;
+        while ((1 << a.slab_shift) < a.slab_elems) ++a.slab_shift;
+        a.unit_rows = (int)((a.chunk_elems + kPassElems - 1) / kPassElems);
+    } else {
+        a.passes = (a.slab_elems + kPassElems - 1) / kPassElems;
+        a.unit_rows = a.n_slabs;
+    }
+    a.total_units = (uint32_t)n * (uint32_t)a.unit_rows * (uint32_t)a.passes;
     a.div_passes.set((uint32_t)a.passes);
     a.div_n.set((uint32_t)n);
     a.div_heads.set((uint32_t)a.n_kv_heads);
@@ -838,7 +905,7 @@ static CodecArgs args_for_group(const CodecArgs &a, const BitGroups &g, int k)
     b.order = a.order + g.first[k];
     b.table = a.table + g.first[k];
     b.n = g.count[k];
-    b.total_units = (uint32_t)b.n * (uint32_t)b.n_slabs * (uint32_t)b.passes;
+    b.total_units = (uint32_t)b.n * (uint32_t)b.unit_rows * (uint32_t)b.passes;
     b.div_n.set((uint32_t)b.n);
     return b;
 }
@@ -866,10 +933,6 @@ static int decode_grid(K kernel, int64_t items)
     return grid < cap ? grid : cap;
 }
 
-// Measured on the 7B-shaped context (same box, same run): register-prefetch kernel 0.561 ms, bulk-copy pipeline
-// 0.579-0.591 ms.  Both are bound by instruction issue, not by the memory path, and the pipeline spends more
-// instructions (shared-memory traffic, barrier polling, single-lane sections), so the direct kernel is used.
-constexpr bool kUseBulkCompress = false;
 
 // The stride between a warp's units, split into (passes, chunks, slab indices).
 static CodecArgs with_grid(CodecArgs a, int grid)
@@ -958,14 +1021,14 @@ extern "C" int llms_compress_chunks(const llms_kv_desc *desc, const void *kv, co
         off += nb;
     }
     CodecArgs a{};
-    fill_args(*desc, a, n, workspace);
+    const bool wide = wide_ok(*desc, kv);
+    fill_args(*desc, a, n, workspace, wide);
     a.kv_in = static_cast<const __half *>(kv);
     a.buf = static_cast<uint8_t *>(out_buf);
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     const BitGroups groups = group_by_bits(n, meta, [&](int i) { return (uint32_t)bits[i]; });
     rc = upload_tables(workspace, meta, groups, n, st);
     if (rc) return rc;
-    const bool wide = wide_ok(*desc, kv);
     for (int k = 0; k < 3; ++k) {
         if (groups.count[k] == 0) continue;
         const CodecArgs b = args_for_group(a, groups, k);
@@ -992,8 +1055,9 @@ extern "C" int llms_compress_chunks(const llms_kv_desc *desc, const void *kv, co
 #undef LLMS_LAUNCH
             } else {
 #define LLMS_LAUNCH(BITS)                                                                                               \
-    if (wide) compress_kernel<BITS, kG, true><<<grid_for(compress_kernel<BITS, kG, true>, b.total_units), kThreads, 0, st>>>(b); \
-    else compress_kernel<BITS, kG, false><<<grid_for(compress_kernel<BITS, kG, false>, b.total_units), kThreads, 0, st>>>(b)
+    if (b.packed) compress_kernel<BITS, kG, true, true><<<grid_for(compress_kernel<BITS, kG, true, true>, b.total_units), kThreads, 0, st>>>(b); \
+    else if (wide) compress_kernel<BITS, kG, true, false><<<grid_for(compress_kernel<BITS, kG, true, false>, b.total_units), kThreads, 0, st>>>(b); \
+    else compress_kernel<BITS, kG, false, false><<<grid_for(compress_kernel<BITS, kG, false, false>, b.total_units), kThreads, 0, st>>>(b)
                 if (k == 0) { LLMS_LAUNCH(8); } else if (k == 1) { LLMS_LAUNCH(4); } else { LLMS_LAUNCH(2); }
 #undef LLMS_LAUNCH
             }
@@ -1030,7 +1094,8 @@ extern "C" int llms_decompress_chunks(const llms_kv_desc *desc, const void *buf,
         staged[i].chunk_id = dst;
     }
     CodecArgs a{};
-    fill_args(*desc, a, n, workspace);
+    const bool wide = wide_ok(*desc, kv_out);
+    fill_args(*desc, a, n, workspace, wide);
     a.kv_out = static_cast<__half *>(kv_out);
     a.buf = const_cast<uint8_t *>(static_cast<const uint8_t *>(buf));
     cudaStream_t st = static_cast<cudaStream_t>(stream);
@@ -1039,7 +1104,6 @@ extern "C" int llms_decompress_chunks(const llms_kv_desc *desc, const void *buf,
     const BitGroups groups = group_by_bits(n, staged.data(), [&](int i) { return meta[i].bits; });
     rc = upload_tables(workspace, staged.data(), groups, n, st);
     if (rc) return rc;
-    const bool wide = wide_ok(*desc, kv_out);
     for (int k = 0; k < 3; ++k) {
         if (groups.count[k] == 0) continue;
         const CodecArgs b = args_for_group(a, groups, k);
@@ -1054,8 +1118,9 @@ extern "C" int llms_decompress_chunks(const llms_kv_desc *desc, const void *buf,
         rc = dispatch_group(desc->group_size, [&](auto g) {
             constexpr int kG = decltype(g)::value;
 #define LLMS_LAUNCH(BITS)                                                                                                   \
-    if (wide) decompress_kernel<BITS, kG, true><<<decode_grid(decompress_kernel<BITS, kG, true>, b.total_units), kThreads, 0, st>>>(b); \
-    else decompress_kernel<BITS, kG, false><<<decode_grid(decompress_kernel<BITS, kG, false>, b.total_units), kThreads, 0, st>>>(b)
+    if (b.packed) decompress_kernel<BITS, kG, true, true><<<decode_grid(decompress_kernel<BITS, kG, true, true>, b.total_units), kThreads, 0, st>>>(b); \
+    else if (wide) decompress_kernel<BITS, kG, true, false><<<decode_grid(decompress_kernel<BITS, kG, true, false>, b.total_units), kThreads, 0, st>>>(b); \
+    else decompress_kernel<BITS, kG, false, false><<<decode_grid(decompress_kernel<BITS, kG, false, false>, b.total_units), kThreads, 0, st>>>(b)
             if (k == 0) { LLMS_LAUNCH(8); } else if (k == 1) { LLMS_LAUNCH(4); } else { LLMS_LAUNCH(2); }
 #undef LLMS_LAUNCH
         });
