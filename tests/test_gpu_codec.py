@@ -91,6 +91,27 @@ def test_every_group_size_and_ragged_shapes(G):
         check_decompress(sh, kv, buf_dev, meta, want_buf)
 
 
+@pytest.mark.parametrize("CL,d,G,L,H", [
+    (1, 64, 64, 1, 1),       # slab of 64 elements, 2 slabs per chunk: one unit, mostly empty
+    (1, 128, 32, 3, 5),      # 30 slabs of 128: 1.9 units per chunk, ragged last unit, four groups per slab
+    (2, 128, 128, 2, 3),     # slabs of 256
+    (4, 128, 64, 2, 5),      # slabs of 512: one load instruction per slab
+    (8, 128, 128, 3, 3),     # slabs of 1024: 18 slabs = 9 units
+    (16, 64, 16, 1, 3),      # head_dim 64 at the paper's chunk size, groups inside a lane
+    (4, 256, 256, 1, 3),     # slabs of 1024 from a wide head
+])
+def test_slabs_shorter_than_a_warp_pass(CL, d, G, L, H):
+    """Short slabs are packed several to a unit; KV addresses then change slab inside a unit."""
+    sh = synth.KVShape("short", L, H, H, d, CL * 11 + (CL - 1), CL, G, seed=CL + d + G)   # tail tokens unless CL == 1
+    kv = synth.kv_tensor(sh)
+    rng = np.random.default_rng(CL * d)
+    ids = rng.permutation(sh.n_chunks)[:9].astype(np.uint32)
+    bits = np.array([(2, 8, 4)[i % 3] for i in range(len(ids))], dtype=np.uint8)
+    kv_dev, buf_dev, meta, want_buf = check_compress(sh, kv, ids, bits)
+    check_decompress(sh, kv, buf_dev, meta, want_buf)
+    check_decompress(sh, kv, buf_dev, meta, want_buf, dst_ids=np.arange(2, 11, dtype=np.uint32))
+
+
 def test_padding_is_written_and_compared():
     # 2 slabs * 3 tokens * 1 group = 6 groups -> 24 parameter bytes -> 8 zero bytes before the codes,
     # and 144/288 code bytes -> tail padding up to 256/512
