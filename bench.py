@@ -35,6 +35,7 @@ def parse_args():
     p.add_argument("--layers", type=int, default=0, help="use only this many layers (smaller cases for profiler captures)")
     p.add_argument("--chunk-len", type=int, default=0, help="override the workload's tokens per chunk (chunk-size sweep, Sec. 5.4)")
     p.add_argument("--e2e-steps", type=int, default=10)
+    p.add_argument("--e2e-batches", type=int, default=8, help="batches of chunks the pipelined round trip is cut into")
     p.add_argument("--no-cpu-baseline", action="store_true")
     p.add_argument("--no-layerwise", dest="layerwise", action="store_false",
                    help="skip the layer-wise swap timing (records split per layer, Sec. 4: first layer ready / all layers ready)")
@@ -351,7 +352,7 @@ def run_ours(args):
         barrier()
         return sharding.max_over_ranks([e0.elapsed_time(e1) / args.e2e_steps], dist, "cuda")[0]
 
-    e2e_batch = max(1, n // 8)
+    e2e_batch = max(1, n // max(1, args.e2e_batches))
     e2e_serial_ms = time_e2e(make_plan(n))
     e2e_ms = time_e2e(make_plan(e2e_batch))
     e2e_value = world * 2 * kv_bytes / (e2e_ms * 1e-3) / 1e9

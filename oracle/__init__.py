@@ -204,6 +204,17 @@ def assign_bits(scores, frac):
     return bits, order
 
 
+def assign_levels(scores, frac, levels):
+    """Eq. 2 for a level set {top, middle, low}, e.g. (8, 4, 2) or (4, 2, 1)."""
+    s = np.ascontiguousarray(scores, dtype=np.float32)
+    f = (C.c_float * 3)(*[float(x) for x in frac])
+    lv = (C.c_uint8 * 3)(*[int(x) for x in levels])
+    bits = np.empty(s.size, dtype=np.uint8)
+    order = np.empty(s.size, dtype=np.uint32)
+    _check(lib().orc_assign_levels(_ptr(s), int(s.size), f, lv, _ptr(bits), _ptr(order)), "assign_levels")
+    return bits, order
+
+
 def optimize_thresholds(scores, ratio_global):
     """-> (frac float32[3], counts int[3]) for the levels 8 / 4 / 2 bits."""
     s = np.ascontiguousarray(scores, dtype=np.float32)

@@ -156,7 +156,7 @@ static uint64_t round_up(uint64_t x, uint64_t a) { return (x + a - 1) / a * a; }
 int orc_record_layout(const orc_kv_desc *d, int bits, uint64_t *codes_off, uint64_t *nbytes)
 {
     if (!desc_ok(d)) return ORC_ERR_ARG;
-    if (bits != 2 && bits != 4 && bits != 8) return ORC_ERR_BITS;
+    if (bits != 1 && bits != 2 && bits != 4 && bits != 8) return ORC_ERR_BITS;
     uint64_t ng = groups_per_chunk(d);
     uint64_t n_elem = (uint64_t)n_slabs(d) * d->chunk_len * d->head_dim;
     if ((n_elem * bits) % 8) return ORC_ERR_ARG;
@@ -500,12 +500,18 @@ int orc_chunk_tolerance(const orc_kv_desc *d, const uint16_t *kv, const uint16_t
 /* ------------------------------------------------------ Eq. 2: rank -> bits */
 
 /* order_out: chunk indices by density, most informative first (ties: lower
- * index first).  The first n8 keep 8 bits, the next n4 get 4, the rest 2:
- * low density = high tolerance = fewer bits.  Counts round to nearest:
- *   n8 = floor(f8*n + 1/2), n8 + n4 = floor((f8+f4)*n + 1/2). */
-int orc_assign_bits(const float *scores, int n, const float frac[3], uint8_t *bits_out, uint32_t *order_out)
+ * index first).  levels = {top, middle, low} bit-widths, e.g. {8, 4, 2}, or
+ * {4, 2, 1} atop a 4-bit base (Sec. 3.2).  The first n_top chunks keep the top
+ * level, the next n_mid get the middle one, the rest the low one: low density =
+ * high tolerance = fewer bits.  Counts round to nearest:
+ *   n_top = floor(f_top*n + 1/2), n_top + n_mid = floor((f_top+f_mid)*n + 1/2). */
+int orc_assign_levels(const float *scores, int n, const float frac[3], const uint8_t levels[3], uint8_t *bits_out,
+                      uint32_t *order_out)
 {
-    if (n < 0 || !frac) return ORC_ERR_ARG;
+    if (n < 0 || !frac || !levels) return ORC_ERR_ARG;
+    for (int w = 0; w < 3; ++w)
+        if (levels[w] != 1 && levels[w] != 2 && levels[w] != 4 && levels[w] != 8) return ORC_ERR_BITS;
+    if (!(levels[0] > levels[1] && levels[1] > levels[2])) return ORC_ERR_ARG;
     double f8 = frac[0], f4 = frac[1], f2 = frac[2];
     if (f8 < 0 || f4 < 0 || f2 < 0 || fabs(f8 + f4 + f2 - 1.0) > 1e-3) return ORC_ERR_ARG;
     uint32_t *ord = (uint32_t *)malloc(sizeof(uint32_t) * (size_t)(n > 0 ? n : 1));
@@ -522,12 +528,19 @@ int orc_assign_bits(const float *scores, int n, const float frac[3], uint8_t *bi
     if (n84 > n) n84 = n;
     if (n84 < n8) n84 = n8;
     for (int r = 0; r < n; ++r) {
-        uint8_t b = r < n8 ? 8 : (r < n84 ? 4 : 2);
+        uint8_t b = r < n8 ? levels[0] : (r < n84 ? levels[1] : levels[2]);
         bits_out[ord[r]] = b;
         if (order_out) order_out[r] = ord[r];
     }
     free(ord);
     return ORC_OK;
+}
+
+/* Eq. 2 with the levels of the paper's experiments, {8, 4, 2}. */
+int orc_assign_bits(const float *scores, int n, const float frac[3], uint8_t *bits_out, uint32_t *order_out)
+{
+    static const uint8_t k842[3] = {8, 4, 2};
+    return orc_assign_levels(scores, n, frac, k842, bits_out, order_out);
 }
 
 /* ------------------------------------------------------ Eq. 3: thresholds */

@@ -152,7 +152,7 @@ def test_subnormal_scale_clamps_codes():
 
 # ----------------------------------------------------------------- invariants on random groups
 
-@pytest.mark.parametrize("bits", [2, 4, 8])
+@pytest.mark.parametrize("bits", [1, 2, 4, 8])
 @pytest.mark.parametrize("G", [16, 64, 128])
 def test_quantizer_invariants(bits, G):
     rng = np.random.default_rng(bits * 1000 + G)
@@ -179,16 +179,40 @@ def test_quantizer_invariants(bits, G):
 
 def test_pack_unpack_every_byte_value():
     # each byte is b-bit fields, field k at bits [k*b, (k+1)*b): check against the definition, all 256 bytes
-    for bits in (2, 4, 8):
+    for bits in (1, 2, 4, 8):
         per = 8 // bits
         for byte in range(256):
             fields = [(byte >> (k * bits)) & ((1 << bits) - 1) for k in range(per)]
             assert oracle.pack_codes(np.array(fields, dtype=np.uint8), bits).tolist() == [byte]
             assert oracle.unpack_codes(np.array([byte], dtype=np.uint8), per, bits).tolist() == fields
     rng = np.random.default_rng(0)
-    for bits in (2, 4, 8):
+    for bits in (1, 2, 4, 8):
         q = rng.integers(0, 1 << bits, 4096).astype(np.uint8)
         assert np.array_equal(oracle.unpack_codes(oracle.pack_codes(q, bits), q.size, bits), q)
+    # one bit per code is numpy's own little-endian bit packing
+    q = rng.integers(0, 2, 1000).astype(np.uint8)
+    assert np.array_equal(oracle.pack_codes(q, 1), np.packbits(q, bitorder="little"))
+
+
+def test_group_b1_is_a_threshold_at_the_midpoint():
+    # Sec. 3.2: atop a 4-bit base the levels are 4, 2 and 1 bits.  One bit: scale = max - min, zero = min, and a
+    # value becomes 1 when (x - min) / scale rounds to 1: above one half, the tie at exactly one half goes to 0 (even)
+    x = h([0.0, 1.0, 0.25, 0.5, 0.75, 0.5009765625, 0.49951171875])
+    sc, ze, codes = oracle.quantize_group(x, 1)
+    assert (sc, ze) == (0x3C00, 0x0000)
+    assert codes.tolist() == [0, 1, 0, 0, 1, 1, 0]
+    assert [oracle.dequantize_one(sc, ze, q) for q in (0, 1)] == [0x0000, 0x3C00]
+    # shifted and scaled: the two decoded values are the minimum and (to fp16 accuracy) the maximum
+    rng = np.random.default_rng(5)
+    for _ in range(200):
+        x = h(rng.standard_normal(32) * 3 + rng.uniform(-5, 5))
+        xv = hval(x)
+        sc, ze, codes = oracle.quantize_group(x, 1)
+        lo, hi = hval([oracle.dequantize_one(sc, ze, 0)])[0], hval([oracle.dequantize_one(sc, ze, 1)])[0]
+        assert lo == xv.min() and abs(hi - xv.max()) <= 2.0 ** -10 * max(abs(xv.max()), xv.max() - xv.min())
+        mid = (xv.min() + xv.max()) / 2
+        clear = np.abs(xv - mid) > 2.0 ** -9 * (xv.max() - xv.min())     # away from the rounding of the midpoint
+        assert np.array_equal(codes[clear], (xv[clear] > mid).astype(np.uint8))
 
 
 def test_dequantize_closed_form():
@@ -222,6 +246,9 @@ def test_record_sizes_closed_form():
     for name, sizes in want.items():
         d = desc_of(synth.CONFIGS[name])
         assert tuple(oracle.record_bytes(d, b) for b in (8, 4, 2)) == sizes
+    # one bit per element: 128 KiB of parameters + 2^25 elements / 8 for a 7B-shaped chunk, 1536 + 128 bytes for tiny
+    assert oracle.record_bytes(desc_of(synth.CONFIGS["llama7b"]), 1) == 128 * 1024 + 2 ** 19
+    assert oracle.record_bytes(desc_of(synth.CONFIGS["tiny"]), 1) == 1536
     # whole 7B-shaped context at 85/86/85 chunks of 8/4/2 bits: 629 MiB against 2048 MiB of fp16
     d = desc_of(synth.CONFIGS["llama7b"])
     total = oracle.compressed_size(d, [8] * 85 + [4] * 86 + [2] * 85)
@@ -247,8 +274,8 @@ def test_compress_chunks_places_groups_where_the_layout_says(quant_mode):
     shape = synth.KVShape("t", 2, 2, 2, 32, 40, 8, 16, seed=5)     # 5 chunks, ragged: T = 40
     kv = synth.kv_tensor(shape).numpy().view(np.uint16)            # [L,2,H,T,d]
     d = desc_of(shape, quant_mode)
-    ids = [3, 0, 4]
-    bits = [4, 8, 2]
+    ids = [3, 0, 4, 1]
+    bits = [4, 8, 2, 1]
     buf, meta = oracle.compress_chunks(d, kv, ids, bits)
     L, H, CL, D, G = shape.n_layers, shape.n_kv_heads, shape.chunk_len, shape.head_dim, shape.group_size
     off = 0

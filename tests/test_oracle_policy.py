@@ -48,6 +48,21 @@ def test_assign_bits_counts(n, frac, want):
     assert tuple(int((bits == b).sum()) for b in (8, 4, 2)) == want
 
 
+def test_assign_levels_other_level_sets():
+    # atop a 4-bit base the further levels are 2 and 1 bits (Sec. 3.2): same ranks, other widths
+    scores = [0.9, 0.1, 0.5, 0.8, 0.2, 0.4]
+    bits, order = oracle.assign_levels(scores, (1 / 3, 1 / 3, 1 / 3), (4, 2, 1))
+    assert bits.tolist() == [4, 1, 2, 4, 1, 2] and order.tolist() == [0, 3, 2, 5, 4, 1]
+    rng = np.random.default_rng(11)
+    s = rng.random(200)
+    b842, o842 = oracle.assign_bits(s, (0.2, 0.5, 0.3))
+    b421, o421 = oracle.assign_levels(s, (0.2, 0.5, 0.3), (4, 2, 1))
+    assert np.array_equal(o842, o421) and np.array_equal(b842, 2 * b421)
+    for bad in ((4, 4, 2), (2, 4, 8), (8, 3, 1)):
+        with pytest.raises(RuntimeError):
+            oracle.assign_levels(s, (0.2, 0.5, 0.3), bad)
+
+
 def test_global_ratio_of_the_paper_setting():
     # levels {8/8, 4/8, 2/8} with shares f8, f4, f2 = 2*f8 give the paper's 50% global ratio when
     # f8 + f4/2 + f2/4 = 1/2; the tertile split gives (1 + 1/2 + 1/4)/3 = 58.3% of the 8-bit size
@@ -82,7 +97,7 @@ def test_lctru_is_the_unique_sorted_permutation():
     rng = np.random.default_rng(7)
     for _ in range(50):
         n = int(rng.integers(1, 9))
-        rows = [(int(rng.integers(0, 3)), i, int(rng.choice([8, 4, 2])), int(rng.random() < 0.8),
+        rows = [(int(rng.integers(0, 3)), i, int(rng.choice([8, 4, 2, 1])), int(rng.random() < 0.8),
                  int(rng.random() < 0.2), int(rng.integers(0, 4))) for i in range(n)]
         order = oracle.lctru_order(make_table(rows)).tolist()
         eligible = [i for i, r in enumerate(rows) if r[3] and not r[4]]
