@@ -204,6 +204,7 @@ void orc_quantize_group(const uint16_t *x, int64_t step, int n, int bits,
     volatile float range = mx - mn;
     volatile float sc32 = range / (float)qmax;
     *scale_h = orc_f32_to_f16(sc32);
+    if (*scale_h == 0x7C00) *scale_h = 0x7BFF; /* a range above 65504 (possible at 1 bit only) keeps the largest finite scale */
     *zero_h = mn_h;
     /* Q3 */
     float s = orc_f16_to_f32(*scale_h);

@@ -194,6 +194,17 @@ def test_pack_unpack_every_byte_value():
     assert np.array_equal(oracle.pack_codes(q, 1), np.packbits(q, bitorder="little"))
 
 
+def test_group_b1_range_beyond_fp16_keeps_a_finite_scale():
+    # max - min = 125504 is not an fp16 number: the scale saturates at 65504 instead of becoming infinite,
+    # codes are rint((x - min) / 65504) clamped to 1, and both decoded values are finite
+    x = h([-60000.0, 65504.0, 0.0, -27000.0, -27500.0, 30000.0])
+    sc, ze, codes = oracle.quantize_group(x, 1)
+    assert (sc, ze) == (0x7BFF, int(h([-60000.0])[0]))
+    assert codes.tolist() == [0, 1, 1, 1, 0, 1]          # (x + 60000) / 65504 = 0, 1.92, 0.916, 0.504, 0.496, 1.37
+    assert hval([oracle.dequantize_one(sc, ze, 0)])[0] == -60000.0
+    assert hval([oracle.dequantize_one(sc, ze, 1)])[0] == 5504.0
+
+
 def test_group_b1_is_a_threshold_at_the_midpoint():
     # Sec. 3.2: atop a 4-bit base the levels are 4, 2 and 1 bits.  One bit: scale = max - min, zero = min, and a
     # value becomes 1 when (x - min) / scale rounds to 1: above one half, the tie at exactly one half goes to 0 (even)
