@@ -34,6 +34,7 @@ def parse_args():
     p.add_argument("--workload", default="llama7b", help="a key of synth.CONFIGS (single-context workloads)")
     p.add_argument("--layers", type=int, default=0, help="use only this many layers (smaller cases for profiler captures)")
     p.add_argument("--chunk-len", type=int, default=0, help="override the workload's tokens per chunk (chunk-size sweep, Sec. 5.4)")
+    p.add_argument("--levels", default="8,4,2", help="bit-widths of the three levels, top first (Sec. 3.2: 8,4,2 or 4,2,1)")
     p.add_argument("--e2e-steps", type=int, default=10)
     p.add_argument("--e2e-batches", type=int, default=8, help="batches of chunks the pipelined round trip is cut into")
     p.add_argument("--no-cpu-baseline", action="store_true")
@@ -61,6 +62,9 @@ NCU_DRAM_TRAFFIC = {
     ("llama7b", 32, "compress_kernel"): 2147838464 + 590607104,
     ("llama7b", 32, "decompress_kernel"): 669177856 + 1960866304,
 }
+
+
+LEVELS = (8, 4, 2)      # set from --levels
 
 
 def target_bits(shape):
@@ -153,7 +157,7 @@ def run_reference(args):
 
     def step():
         scores = oracle.chunk_tolerance(od, kv, q, W)
-        bits, _ = oracle.assign_bits(scores.astype(np.float32), frac)
+        bits, _ = oracle.assign_levels(scores.astype(np.float32), frac, LEVELS)
         buf, meta = oracle.compress_chunks(od, kv, ids, bits)
         oracle.decompress_chunks(od, buf, meta, out)
 
@@ -195,7 +199,7 @@ def cpu_baseline(shape, kv_dev, q_dev):
     out = np.zeros(kv.size, dtype=np.uint16).reshape(kv.shape)
     t0 = time.perf_counter()
     scores = oracle.chunk_tolerance(od, kv, q, W)
-    bits, _ = oracle.assign_bits(scores.astype(np.float32), frac)
+    bits, _ = oracle.assign_levels(scores.astype(np.float32), frac, LEVELS)
     t1 = time.perf_counter()
     buf, meta = oracle.compress_chunks(od, kv, ids, bits)
     t2 = time.perf_counter()
@@ -259,7 +263,7 @@ def run_ours(args):
         B.chunk_tolerance(d, kv, q_win, W, scores, ws_tol)
         scores_host.copy_(scores, non_blocking=True)
         stream.synchronize()                     # the ranking is a host step
-        bits, _ = B.assign_bits(scores_host.numpy(), frac)
+        bits, _ = B.assign_levels(scores_host.numpy(), frac, LEVELS)
         if ev:
             ev[1].record(stream)
         B.compress_chunks(d, kv, ids, bits, buf, meta, ws)
@@ -281,7 +285,7 @@ def run_ours(args):
         step()
     assert B.codec_corrupt_count(ws) == 0
     bits = state["bits"]
-    assert tuple(int((bits == b).sum()) for b in (8, 4, 2)) == (n8, n4, n2)
+    assert tuple(int((bits == b).sum()) for b in LEVELS) == (n8, n4, n2)
     record_bytes = B.compressed_size(d, bits)
 
     sampler = ClockSampler(local_rank) if rank == 0 else None
@@ -416,7 +420,8 @@ def run_ours(args):
     roofline = {
         "kernel": dominant, "bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
         "peak_source": f"{peak_kind} copy bandwidth", "launches_per_stage": 3,
-        "traffic": NCU_DRAM_TRAFFIC.get((shape.name, shape.n_layers, dominant)) if args.quant_mode == 0 else None,
+        "traffic": (NCU_DRAM_TRAFFIC.get((shape.name, shape.n_layers, dominant))
+                    if args.quant_mode == 0 and LEVELS == (8, 4, 2) and not args.chunk_len else None),
         "algorithmic_bytes_per_launch": algo_bytes,
         "frac_of_nominal_8000": achieved / 8000.0,
         "per_stage": {
@@ -435,7 +440,7 @@ def run_ours(args):
         "dtype": "f32 (fp16 in/out, integer codes)", "data": "synthetic",
         "config": {"workload": shape.name, "layers": shape.n_layers, "kv_heads": shape.n_kv_heads, "head_dim": shape.head_dim,
                    "tokens": shape.n_tokens, "chunk_len": shape.chunk_len, "group_size": shape.group_size,
-                   "window": W, "bits_8_4_2": [n8, n4, n2], "contexts_per_gpu": 1, "quant_mode": args.quant_mode,
+                   "window": W, "levels": list(LEVELS), "chunks_per_level": [n8, n4, n2], "contexts_per_gpu": 1, "quant_mode": args.quant_mode,
                    "l2": "inputs larger than L2 (fp16 KV %.0f MiB per context)" % (kv_bytes / 2 ** 20),
                    "step": "score + rank->bits + compress + decompress of one context"},
         "contexts_per_s": world / (ms_per_step * 1e-3),
@@ -508,7 +513,10 @@ def run_multiapp(args):
 
 
 def main():
+    global LEVELS
     args = parse_args()
+    LEVELS = tuple(int(x) for x in args.levels.split(","))
+    assert len(LEVELS) == 3
     if args.impl == "reference":
         run_reference(args)
     elif args.workload == "multiapp":

@@ -42,7 +42,7 @@
  * quant_mode 1: a group is one channel of one slab across the chunk's tokens
  * (group index = s_idx*head_dim + c), the paper's "channel-wise" wording.
  * Per group, in binary32 with IEEE round-to-nearest and no fused operations:
- *     zero = min x (stored as +0 when it is a zero);  scale = fp16((max x - min x) / (2^b - 1));
+ *     zero = min x (stored as +0 when it is a zero);  scale = fp16((max x - min x) / (2^b - 1)), 65504 if larger;
  *     code = min(2^b - 1, rint((x - zero) * (1 / scale)))  (ties to even; all codes 0 when scale == 0);
  *     decoded value = fp16(clamp(zero + code*scale, -65504, 65504)).
  * Inputs must be finite.
@@ -59,7 +59,7 @@ extern "C" {
 typedef enum llms_status {
     LLMS_OK = 0,
     LLMS_ERR_INVALID_ARG = -1,   /* null pointer, non-positive size, id out of range, duplicate chunk id */
-    LLMS_ERR_BAD_BITS = -2,      /* a bit-width other than 2, 4, 8 */
+    LLMS_ERR_BAD_BITS = -2,      /* a bit-width other than 1, 2, 4, 8 */
     LLMS_ERR_MISALIGNED = -3,    /* pointer, stride or offset not aligned as required */
     LLMS_ERR_BUF_TOO_SMALL = -4, /* output buffer or workspace smaller than needed */
     LLMS_ERR_CUDA = -5,          /* a CUDA runtime call failed (see llms_last_cuda_error) */
@@ -81,7 +81,7 @@ typedef struct llms_kv_desc {
 /* One record of a swap buffer: where it is and what is in it (32 bytes). */
 typedef struct llms_chunk_meta {
     uint32_t chunk_id;  /* chunk (slot) the record was made from */
-    uint32_t bits;      /* 2, 4 or 8 */
+    uint32_t bits;      /* 1, 2, 4 or 8 */
     uint64_t offset;    /* byte offset of the record in its swap buffer, multiple of 256 */
     uint64_t nbytes;    /* record size, multiple of 256 */
     uint32_t n_groups;
@@ -119,7 +119,7 @@ int llms_codec_workspace_bytes(int n, uint64_t *nbytes);
  * down in out_buf at the running offset (records in list order, each 256-byte aligned).
  *   kv         device, fp16, 16-byte aligned, read only
  *   chunk_ids  host, n distinct ids < floor(n_tokens/chunk_len)
- *   bits       host, n values from {2, 4, 8}
+ *   bits       host, n values from {1, 2, 4, 8} (1 only with quant_mode 0: LLMS_ERR_UNSUPPORTED otherwise)
  *   out_buf    device, 256-byte aligned, out_bytes >= llms_compressed_size(...); every byte of
  *              every record, padding included, is written
  *   meta       host, n entries, filled before return except `checksum`, which the device
@@ -196,6 +196,14 @@ int llms_chunk_tolerance_from_probs(const llms_kv_desc *desc, const float *probs
  * the first n8 = floor(f8*n + 1/2) chunks of that order keep 8 bits, up to
  * floor((f8+f4)*n + 1/2) get 4, the rest 2 - low density means high tolerance means fewer bits. */
 int llms_assign_bits(const float *scores, int n, const float frac[3], uint8_t *bits_out, uint32_t *order_out);
+
+/* Eq. 2 for another level set (Sec. 3.2: the method is not tied to 8/4/2 - atop a 4-bit cache it offers 2 and
+ * 1 bit).  levels = {top, middle, low} bit-widths from {8, 4, 2, 1}, strictly decreasing; frac = the shares
+ * of chunks per level, in that order; everything else as llms_assign_bits, which is this call with
+ * levels {8, 4, 2}.  llms_optimize_thresholds serves any set whose widths halve from level to level
+ * ({8,4,2}, {4,2,1}): its ratio_global is relative to the top level. */
+int llms_assign_levels(const float *scores, int n, const float frac[3], const uint8_t levels[3],
+                       uint8_t *bits_out, uint32_t *order_out);
 
 /* Eq. 3: the shares of chunks per level that maximise the context's information under a global average
  * ratio, for the levels {8/8, 4/8, 2/8} (Sec. 3.2: one free variable is left).  A chunk at level w keeps

@@ -59,6 +59,7 @@ _SIGNATURES = {
     "llms_chunk_tolerance_from_probs": (C.c_int, [C.c_void_p, C.c_void_p, C.c_int, C.c_void_p, C.c_void_p,
                                                   C.c_uint64, C.c_void_p]),
     "llms_assign_bits": (C.c_int, [C.c_void_p, C.c_int, C.c_void_p, C.c_void_p, C.c_void_p]),
+    "llms_assign_levels": (C.c_int, [C.c_void_p, C.c_int, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]),
     "llms_optimize_thresholds": (C.c_int, [C.c_void_p, C.c_int, C.c_float, C.c_void_p]),
     "llms_lctru_order": (C.c_int, [C.c_void_p, C.c_int, C.c_void_p]),
     "llms_swap_out": (C.c_int, [C.c_void_p, C.c_void_p, C.c_int, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p,
@@ -257,6 +258,18 @@ def assign_bits(scores, frac):
     bits = np.empty(s.size, dtype=np.uint8)
     order = np.empty(s.size, dtype=np.uint32)
     _check(lib().llms_assign_bits(_ptr(s), int(s.size), _ptr(f), _ptr(bits), _ptr(order)), "llms_assign_bits")
+    return bits, order
+
+
+def assign_levels(scores, frac, levels):
+    """Eq. 2 for a level set {top, middle, low}, e.g. (4, 2, 1)."""
+    s = np.ascontiguousarray(scores, dtype=np.float32)
+    f = np.asarray(frac, dtype=np.float32)
+    lv = np.asarray(levels, dtype=np.uint8)
+    assert f.size == 3 and lv.size == 3
+    bits = np.empty(s.size, dtype=np.uint8)
+    order = np.empty(s.size, dtype=np.uint32)
+    _check(lib().llms_assign_levels(_ptr(s), int(s.size), _ptr(f), _ptr(lv), _ptr(bits), _ptr(order)), "llms_assign_levels")
     return bits, order
 
 

@@ -31,6 +31,8 @@ constexpr int kPieceElems = 16;                 // one 32-byte access
 constexpr int kPieces = 4;                      // pieces per lane per pass
 constexpr int kLaneElems = kPieces * kPieceElems;
 constexpr int kPassElems = 32 * kLaneElems;     // 2048 elements = 4 KiB of fp16
+// 32-bit words that hold the packed codes of one piece; at 1 bit a piece is the low half of one word
+__host__ __device__ constexpr int piece_words(int bits) { return bits >= 2 ? bits / 2 : 1; }
 constexpr uint32_t kPrefetchAhead = 2;          // compress: units ahead that are pulled into L2 (measured: 2 -> 0.521 ms,
                                                 // 3 -> 0.535, 5 -> 0.59, 8 -> 0.79 for compress on the 7B shape)
 
@@ -212,6 +214,16 @@ __device__ __forceinline__ void st32(void *p, uint32_t a0)
 {
     asm volatile("st.global.L1::no_allocate.b32 [%1], %0;" :: "r"(a0), "l"(p) : "memory");
 }
+__device__ __forceinline__ void st16(void *p, uint32_t a0)
+{
+    asm volatile("st.global.L1::no_allocate.b16 [%1], %0;" :: "h"((unsigned short)a0), "l"(p) : "memory");
+}
+__device__ __forceinline__ void ld16(const void *p, uint32_t *w)
+{
+    unsigned short v;
+    asm volatile("ld.global.nc.L1::no_allocate.b16 %0, [%1];" : "=h"(v) : "l"(p));
+    w[0] = v;
+}
 __device__ __forceinline__ void ld256(const void *p, uint32_t *w)
 {
     asm volatile("ld.global.nc.L1::no_allocate.v8.b32 {%0,%1,%2,%3,%4,%5,%6,%7}, [%8];"
@@ -295,7 +307,10 @@ __device__ __forceinline__ GroupParams group_params(__half2 mm)
     // adding +0 turns a -0 minimum or maximum into +0 and changes nothing else
     const float zero = __fadd_rn(__low2float(mm), 0.0f);
     const float top = __fadd_rn(-__high2float(mm), 0.0f);
-    const __half scale_h = __float2half_rn(__fdiv_rn(__fsub_rn(top, zero), kQmax));
+    // a range above 65504 (possible at 1 bit only) keeps the largest finite scale
+    unsigned short scale_bits;
+    asm("cvt.rn.satfinite.f16.f32 %0, %1;" : "=h"(scale_bits) : "f"(__fdiv_rn(__fsub_rn(top, zero), kQmax)));
+    const __half scale_h = __ushort_as_half(scale_bits);
     const float scale = __half2float(scale_h);
     GroupParams g;
     g.neg_zero_point = -zero;
@@ -320,7 +335,7 @@ __device__ __forceinline__ void piece_minmax(const uint32_t (&w)[8], __half2 &mn
 // Quantize 16 values and pack them into BITS/2 words.  No clamp: only valid when the scale is a normal fp16
 // number, where (x - zero) / scale stays below 2^BITS - 1/2.
 template <int BITS>
-__device__ __forceinline__ void quantize_piece(const uint32_t (&w)[8], float neg_zero, float inv, uint32_t (&out)[BITS / 2])
+__device__ __forceinline__ void quantize_piece(const uint32_t (&w)[8], float neg_zero, float inv, uint32_t (&out)[piece_words(BITS)])
 {
     uint32_t t[16];
 #pragma unroll
@@ -340,13 +355,13 @@ __device__ __forceinline__ void quantize_piece(const uint32_t (&w)[8], float neg
         }
     } else {
         // sum of (magic + q_k) << (k*BITS), minus the magic's share: arithmetic mod 2^32, one shift-add per code
-        constexpr int kPerWord = 32 / BITS;
+        constexpr int kPerWord = BITS >= 2 ? 32 / BITS : 16;
         uint32_t ones = 0;
 #pragma unroll
         for (int k = 0; k < kPerWord; ++k) ones += 1u << (k * BITS);
         const uint32_t bias = kRoundMagicBits * ones;
 #pragma unroll
-        for (int j = 0; j < BITS / 2; ++j) {
+        for (int j = 0; j < piece_words(BITS); ++j) {
             uint32_t acc = 0u - bias;
 #pragma unroll
             for (int k = 0; k < kPerWord; ++k) acc += t[j * kPerWord + k] << (k * BITS);
@@ -359,7 +374,7 @@ __device__ __forceinline__ void quantize_piece(const uint32_t (&w)[8], float neg
 __device__ __noinline__ void quantize_piece_clamped(const uint32_t *w, float neg_zero, float inv, int bits, uint32_t *out)
 {
     const float qmax = (float)((1 << bits) - 1);
-    for (int j = 0; j < bits / 2; ++j) out[j] = 0;
+    for (int j = 0; j < piece_words(bits); ++j) out[j] = 0;
     for (int k = 0; k < 16; ++k) {
         const unsigned short x = (unsigned short)(w[k >> 1] >> ((k & 1) * 16));
         const float v = fminf(__fmul_rn(add_f32_f16(x, neg_zero), inv), qmax);
@@ -398,7 +413,7 @@ __device__ __forceinline__ uint32_t compress_unit_bits(const CodecArgs &a, const
         }
     }
     // ---- codes
-    uint32_t c[kPieces][BITS / 2];
+    uint32_t c[kPieces][piece_words(BITS)];
     bool any_clamp = false;
 #pragma unroll
     for (int g = 0; g < geo::kGroupsPerLane; ++g)  // groups past the end of the slab (loaded as zeros) do not count
@@ -412,7 +427,7 @@ __device__ __forceinline__ uint32_t compress_unit_bits(const CodecArgs &a, const
             for (int k = 0; k < 8; ++k) tmp_in[k] = w[j][k];
             quantize_piece_clamped(tmp_in, g.neg_zero_point, g.inv, BITS, tmp_out);
 #pragma unroll
-            for (int k = 0; k < BITS / 2; ++k) c[j][k] = tmp_out[k];
+            for (int k = 0; k < piece_words(BITS); ++k) c[j][k] = tmp_out[k];
         }
     } else {
 #pragma unroll
@@ -426,29 +441,40 @@ __device__ __forceinline__ uint32_t compress_unit_bits(const CodecArgs &a, const
     uint32_t *params = reinterpret_cast<uint32_t *>(rec) + (uint64_t)u.s_idx * a.groups_per_slab + (uint32_t)u.e0 / G;
     uint32_t sum = 0;
     const bool lane_full = le0 + kLaneElems <= u.limit;
-    constexpr uintptr_t kLaneAlign = BITS == 2 ? 15 : 31;
+    constexpr uintptr_t kLaneAlign = BITS == 1 ? 7 : BITS == 2 ? 15 : 31;
     if (lane_full && (reinterpret_cast<uintptr_t>(codes) & kLaneAlign) == 0) {
         if constexpr (BITS == 8) {
             st256(codes, c[0][0], c[0][1], c[0][2], c[0][3], c[1][0], c[1][1], c[1][2], c[1][3]);
             st256(codes + 32, c[2][0], c[2][1], c[2][2], c[2][3], c[3][0], c[3][1], c[3][2], c[3][3]);
         } else if constexpr (BITS == 4) {
             st256(codes, c[0][0], c[0][1], c[1][0], c[1][1], c[2][0], c[2][1], c[3][0], c[3][1]);
-        } else {
+        } else if constexpr (BITS == 2) {
             st128(codes, c[0][0], c[1][0], c[2][0], c[3][0]);
+        } else {
+            st64(codes, c[0][0] | (c[1][0] << 16), c[2][0] | (c[3][0] << 16));
         }
+        if constexpr (BITS == 1) {
+            sum = c[0][0] + (c[1][0] << 16) + c[2][0] + (c[3][0] << 16);
+        } else {
 #pragma unroll
-        for (int j = 0; j < kPieces; ++j)
+            for (int j = 0; j < kPieces; ++j)
 #pragma unroll
-            for (int k = 0; k < BITS / 2; ++k) sum += c[j][k];
+                for (int k = 0; k < piece_words(BITS); ++k) sum += c[j][k];
+        }
     } else {
 #pragma unroll
         for (int j = 0; j < kPieces; ++j) {
             if (le0 + j * kPieceElems < u.limit) {
                 if constexpr (BITS == 8) st128(codes + j * kPieceBytes, c[j][0], c[j][1], c[j][2], c[j][3]);
                 else if constexpr (BITS == 4) st64(codes + j * kPieceBytes, c[j][0], c[j][1]);
-                else st32(codes + j * kPieceBytes, c[j][0]);
+                else if constexpr (BITS == 2) st32(codes + j * kPieceBytes, c[j][0]);
+                else st16(codes + j * kPieceBytes, c[j][0]);
+                if constexpr (BITS == 1) {  // half a word: which half follows from the address (records are 256-byte aligned)
+                    sum += c[j][0] << ((reinterpret_cast<uintptr_t>(codes + j * kPieceBytes) & 2) * 8);
+                } else {
 #pragma unroll
-                for (int k = 0; k < BITS / 2; ++k) sum += c[j][k];
+                    for (int k = 0; k < piece_words(BITS); ++k) sum += c[j][k];
+                }
             }
         }
     }
@@ -645,7 +671,7 @@ __device__ __forceinline__ void decode_unit_for_decoder(const CodecArgs &a, uint
 }
 
 template <int BITS, int G>
-__device__ __forceinline__ void load_unit_codes(const DecodePos &u, uint32_t (&c)[kPieces][BITS / 2], uint32_t (&p)[kPieces])
+__device__ __forceinline__ void load_unit_codes(const DecodePos &u, uint32_t (&c)[kPieces][piece_words(BITS)], uint32_t (&p)[kPieces])
 {
     constexpr int kStrideBytes = kPieceStride * BITS / 8;
 #pragma unroll
@@ -654,11 +680,12 @@ __device__ __forceinline__ void load_unit_codes(const DecodePos &u, uint32_t (&c
             const uint8_t *src = u.codes + j * kStrideBytes;
             if constexpr (BITS == 8) ld128(src, c[j]);
             else if constexpr (BITS == 4) ld64(src, c[j]);
-            else ld32(src, c[j]);
+            else if constexpr (BITS == 2) ld32(src, c[j]);
+            else ld16(src, c[j]);
             p[j] = __ldg(u.params + j * (kPieceStride / G));
         } else {
 #pragma unroll
-            for (int k = 0; k < BITS / 2; ++k) c[j][k] = 0;
+            for (int k = 0; k < piece_words(BITS); ++k) c[j][k] = 0;
             p[j] = 0;
         }
     }
@@ -684,10 +711,15 @@ __device__ __forceinline__ void codes_to_half2(const uint32_t *c, __half2 (&q)[8
 #pragma unroll
             for (int s = 0; s < 4; ++s)  // codes 8m + s (low half) and 8m + s + 4 (high half)
                 q[4 * m + s] = __hsub2(as_h2(((c[m] >> (4 * s)) & 0x000F000Fu) | 0x64006400u), k1024);
-    } else {
+    } else if constexpr (BITS == 2) {
 #pragma unroll
         for (int s = 0; s < 8; ++s)      // codes s (low half) and s + 8 (high half)
             q[s] = __hsub2(as_h2(((c[0] >> (2 * s)) & 0x00030003u) | 0x64006400u), k1024);
+    } else {
+        const uint32_t z = (c[0] & 0xFFu) | ((c[0] & 0xFF00u) << 8);  // codes 0..7 in the low half, 8..15 in the high half
+#pragma unroll
+        for (int s = 0; s < 8; ++s)      // codes s (low half) and s + 8 (high half)
+            q[s] = __hsub2(as_h2(((z >> s) & 0x00010001u) | 0x64006400u), k1024);
     }
 }
 
@@ -727,7 +759,7 @@ __device__ __forceinline__ void dequantize_piece(const uint32_t *c, unsigned sho
 }
 
 template <int BITS, int G, bool WIDE, bool PACKED>
-__device__ __forceinline__ void decompress_unit(const CodecArgs &a, const DecodePos &u, const uint32_t (&c)[kPieces][BITS / 2],
+__device__ __forceinline__ void decompress_unit(const CodecArgs &a, const DecodePos &u, const uint32_t (&c)[kPieces][piece_words(BITS)],
                                                 const uint32_t (&p)[kPieces], int lane, uint32_t *sum_slots)
 {
     // a lane's pieces all sit at the same place inside their groups: either every one opens a group or none does
@@ -742,8 +774,12 @@ __device__ __forceinline__ void decompress_unit(const CodecArgs &a, const Decode
         if (u.room > j * kPieceStride)
             store32<WIDE>(a.kv_out + unit_elem_offset<PACKED>(a, u.s_idx, u.chunk_id, u.pass_e0, j * kPieceStride + lane * kPieceElems), w);
         // pieces past the end of the slab were loaded as zeros and add nothing
+        if constexpr (BITS == 1) {  // a piece is half of a record word; the pieces of a lane all sit in the same half
+            sum += c[j][0] << ((reinterpret_cast<uintptr_t>(u.codes) & 2) * 8);
+        } else {
 #pragma unroll
-        for (int k = 0; k < BITS / 2; ++k) sum += c[j][k];
+            for (int k = 0; k < piece_words(BITS); ++k) sum += c[j][k];
+        }
         if (opens_group) sum += p[j];  // the piece that opens a group accounts for its parameter word
     }
     unit_sum_add(sum_slots, a.n, u.k, &a.sums[u.i], sum, lane);
@@ -767,7 +803,7 @@ __global__ void __launch_bounds__(kThreads, kDecodeBlocksPerSm) decompress_kerne
     cta_sums_clear(sum_slots, a.n);
     if (unit < a.total_units) {
         DecodePos pos[D];
-        uint32_t c[D][kPieces][BITS / 2], p[D][kPieces];
+        uint32_t c[D][kPieces][piece_words(BITS)], p[D][kPieces];
 #pragma unroll
         for (int s = 0; s < D - 1; ++s) {
             const uint32_t ahead = unit + s * n_warps;
@@ -858,19 +894,20 @@ static int fill_args(const llms_kv_desc &d, CodecArgs &a, int n, void *workspace
 }
 
 // Entry indices grouped by bit-width (8, then 4, then 2), list order kept inside a group.
+constexpr int kNumWidths = 4;
 struct BitGroups {
     std::vector<uint32_t> order;
     std::vector<UnitEntry> table;
-    int first[3], count[3];
+    int first[kNumWidths], count[kNumWidths];
 };
 
 template <typename GetBits>
 static BitGroups group_by_bits(int n, const llms_chunk_meta *meta, GetBits bits_of)
 {
-    static const uint32_t kWidths[3] = {8, 4, 2};
+    static const uint32_t kWidths[kNumWidths] = {8, 4, 2, 1};
     BitGroups g;
     g.order.reserve(n);
-    for (int k = 0; k < 3; ++k) {
+    for (int k = 0; k < kNumWidths; ++k) {
         g.first[k] = (int)g.order.size();
         for (int i = 0; i < n; ++i)
             if (bits_of(i) == kWidths[k]) g.order.push_back((uint32_t)i);
@@ -1003,6 +1040,7 @@ extern "C" int llms_compress_chunks(const llms_kv_desc *desc, const void *kv, co
         uint64_t nb;
         rc = llms_record_bytes(desc, bits[i], &nb);
         if (rc) return rc;
+        if (bits[i] == 1 && desc->quant_mode == 1) return LLMS_ERR_UNSUPPORTED;  // the channel-wise kernels stop at 2 bits
         if (chunk_ids[i] >= nc || seen[chunk_ids[i]]) return LLMS_ERR_INVALID_ARG;
         seen[chunk_ids[i]] = 1;
         off += nb;
@@ -1029,7 +1067,7 @@ extern "C" int llms_compress_chunks(const llms_kv_desc *desc, const void *kv, co
     const BitGroups groups = group_by_bits(n, meta, [&](int i) { return (uint32_t)bits[i]; });
     rc = upload_tables(workspace, meta, groups, n, st);
     if (rc) return rc;
-    for (int k = 0; k < 3; ++k) {
+    for (int k = 0; k < kNumWidths; ++k) {
         if (groups.count[k] == 0) continue;
         const CodecArgs b = args_for_group(a, groups, k);
         cudaError_t attr_err = cudaSuccess;
@@ -1051,14 +1089,14 @@ extern "C" int llms_compress_chunks(const llms_kv_desc *desc, const void *kv, co
         const int grid = grid_for(compress_bulk_kernel<BITS, kG>, b.total_units, kBulkSmemBytes);                               \
         compress_bulk_kernel<BITS, kG><<<grid, kThreads, kBulkSmemBytes, st>>>(with_grid(b, grid));                             \
     }
-                if (k == 0) { LLMS_LAUNCH(8); } else if (k == 1) { LLMS_LAUNCH(4); } else { LLMS_LAUNCH(2); }
+                if (k == 0) { LLMS_LAUNCH(8); } else if (k == 1) { LLMS_LAUNCH(4); } else if (k == 2) { LLMS_LAUNCH(2); } else { attr_err = cudaErrorNotSupported; }
 #undef LLMS_LAUNCH
             } else {
 #define LLMS_LAUNCH(BITS)                                                                                               \
     if (b.packed) compress_kernel<BITS, kG, true, true><<<grid_for(compress_kernel<BITS, kG, true, true>, b.total_units), kThreads, 0, st>>>(b); \
     else if (wide) compress_kernel<BITS, kG, true, false><<<grid_for(compress_kernel<BITS, kG, true, false>, b.total_units), kThreads, 0, st>>>(b); \
     else compress_kernel<BITS, kG, false, false><<<grid_for(compress_kernel<BITS, kG, false, false>, b.total_units), kThreads, 0, st>>>(b)
-                if (k == 0) { LLMS_LAUNCH(8); } else if (k == 1) { LLMS_LAUNCH(4); } else { LLMS_LAUNCH(2); }
+                if (k == 0) { LLMS_LAUNCH(8); } else if (k == 1) { LLMS_LAUNCH(4); } else if (k == 2) { LLMS_LAUNCH(2); } else { LLMS_LAUNCH(1); }
 #undef LLMS_LAUNCH
             }
         });
@@ -1086,6 +1124,7 @@ extern "C" int llms_decompress_chunks(const llms_kv_desc *desc, const void *buf,
         uint64_t nb;
         rc = llms_record_bytes(desc, (int)meta[i].bits, &nb);
         if (rc) return rc;
+        if (meta[i].bits == 1 && desc->quant_mode == 1) return LLMS_ERR_UNSUPPORTED;
         if (meta[i].nbytes != nb || meta[i].n_groups != (uint32_t)groups_per_chunk(*desc)) return LLMS_ERR_INVALID_ARG;
         if (meta[i].offset % 256) return LLMS_ERR_MISALIGNED;
         const uint32_t dst = dst_chunk_ids ? dst_chunk_ids[i] : meta[i].chunk_id;
@@ -1104,7 +1143,7 @@ extern "C" int llms_decompress_chunks(const llms_kv_desc *desc, const void *buf,
     const BitGroups groups = group_by_bits(n, staged.data(), [&](int i) { return meta[i].bits; });
     rc = upload_tables(workspace, staged.data(), groups, n, st);
     if (rc) return rc;
-    for (int k = 0; k < 3; ++k) {
+    for (int k = 0; k < kNumWidths; ++k) {
         if (groups.count[k] == 0) continue;
         const CodecArgs b = args_for_group(a, groups, k);
         if (desc->quant_mode == 1) {
@@ -1121,7 +1160,7 @@ extern "C" int llms_decompress_chunks(const llms_kv_desc *desc, const void *buf,
     if (b.packed) decompress_kernel<BITS, kG, true, true><<<decode_grid(decompress_kernel<BITS, kG, true, true>, b.total_units), kThreads, 0, st>>>(b); \
     else if (wide) decompress_kernel<BITS, kG, true, false><<<decode_grid(decompress_kernel<BITS, kG, true, false>, b.total_units), kThreads, 0, st>>>(b); \
     else decompress_kernel<BITS, kG, false, false><<<decode_grid(decompress_kernel<BITS, kG, false, false>, b.total_units), kThreads, 0, st>>>(b)
-            if (k == 0) { LLMS_LAUNCH(8); } else if (k == 1) { LLMS_LAUNCH(4); } else { LLMS_LAUNCH(2); }
+            if (k == 0) { LLMS_LAUNCH(8); } else if (k == 1) { LLMS_LAUNCH(4); } else if (k == 2) { LLMS_LAUNCH(2); } else { LLMS_LAUNCH(1); }
 #undef LLMS_LAUNCH
         });
         if (rc) return rc;

@@ -63,7 +63,7 @@ extern "C" const char *llms_strerror(int status)
     switch (status) {
     case LLMS_OK: return "ok";
     case LLMS_ERR_INVALID_ARG: return "invalid argument";
-    case LLMS_ERR_BAD_BITS: return "bit-width must be 2, 4 or 8";
+    case LLMS_ERR_BAD_BITS: return "bit-width must be 1, 2, 4 or 8";
     case LLMS_ERR_MISALIGNED: return "pointer, stride or offset is not aligned as required";
     case LLMS_ERR_BUF_TOO_SMALL: return "buffer or workspace too small";
     case LLMS_ERR_CUDA: return "CUDA runtime error";

@@ -37,7 +37,7 @@ inline uint64_t groups_per_chunk(const llms_kv_desc &d) { return (uint64_t)slabs
 int check_desc(const llms_kv_desc *d);
 // Shape + alignment checks for the codec kernels (vector loads need 16-byte aligned slabs).
 int check_desc_codec(const llms_kv_desc *d);
-inline int check_bits(int b) { return (b == 2 || b == 4 || b == 8) ? LLMS_OK : LLMS_ERR_BAD_BITS; }
+inline int check_bits(int b) { return (b == 1 || b == 2 || b == 4 || b == 8) ? LLMS_OK : LLMS_ERR_BAD_BITS; }
 
 // Number of SMs of the current device (cached per device).
 int sm_count();

@@ -6,24 +6,34 @@
 
 #include "llms_internal.cuh"
 
-extern "C" int llms_assign_bits(const float *scores, int n, const float frac[3], uint8_t *bits_out, uint32_t *order_out)
+extern "C" int llms_assign_levels(const float *scores, int n, const float frac[3], const uint8_t levels[3],
+                                  uint8_t *bits_out, uint32_t *order_out)
 {
-    if (n < 0 || !frac || (n > 0 && (!scores || !bits_out))) return LLMS_ERR_INVALID_ARG;
-    const double f8 = frac[0], f4 = frac[1], f2 = frac[2];
-    if (!(f8 >= 0) || !(f4 >= 0) || !(f2 >= 0) || std::fabs(f8 + f4 + f2 - 1.0) > 1e-3) return LLMS_ERR_INVALID_ARG;
+    if (n < 0 || !frac || !levels || (n > 0 && (!scores || !bits_out))) return LLMS_ERR_INVALID_ARG;
+    for (int w = 0; w < 3; ++w)
+        if (llms::check_bits(levels[w])) return LLMS_ERR_BAD_BITS;
+    if (!(levels[0] > levels[1] && levels[1] > levels[2])) return LLMS_ERR_INVALID_ARG;
+    const double f_top = frac[0], f_mid = frac[1], f_low = frac[2];
+    if (!(f_top >= 0) || !(f_mid >= 0) || !(f_low >= 0) || std::fabs(f_top + f_mid + f_low - 1.0) > 1e-3) return LLMS_ERR_INVALID_ARG;
     std::vector<uint32_t> order(n);
     std::iota(order.begin(), order.end(), 0u);
     // densest first; equal densities keep index order
     std::stable_sort(order.begin(), order.end(), [&](uint32_t a, uint32_t b) { return scores[a] > scores[b]; });
-    long n8 = (long)std::floor(f8 * n + 0.5);
-    long n84 = (long)std::floor((f8 + f4) * n + 0.5);
-    n8 = std::min<long>(n8, n);
-    n84 = std::max(std::min<long>(n84, n), n8);
+    long n_top = (long)std::floor(f_top * n + 0.5);
+    long n_top_mid = (long)std::floor((f_top + f_mid) * n + 0.5);
+    n_top = std::min<long>(n_top, n);
+    n_top_mid = std::max(std::min<long>(n_top_mid, n), n_top);
     for (long r = 0; r < n; ++r) {
-        bits_out[order[r]] = r < n8 ? 8 : (r < n84 ? 4 : 2);
+        bits_out[order[r]] = r < n_top ? levels[0] : (r < n_top_mid ? levels[1] : levels[2]);
         if (order_out) order_out[r] = order[r];
     }
     return LLMS_OK;
+}
+
+extern "C" int llms_assign_bits(const float *scores, int n, const float frac[3], uint8_t *bits_out, uint32_t *order_out)
+{
+    static const uint8_t kLevels[3] = {8, 4, 2};
+    return llms_assign_levels(scores, n, frac, kLevels, bits_out, order_out);
 }
 
 extern "C" int llms_optimize_thresholds(const float *scores, int n, float ratio_global, float frac_out[3])

@@ -37,7 +37,7 @@ def odesc(sh, mode=0):
 def test_record_sizes_match_oracle():
     for sh in synth.CONFIGS.values():
         for mode in (0, 1):
-            for b in (2, 4, 8):
+            for b in (1, 2, 4, 8):
                 assert B.record_layout(B.desc_of(sh, mode), b) == oracle.record_layout(odesc(sh, mode), b)
     odd = synth.KVShape("odd", 1, 1, 1, 16, 3, 3, 16)
     assert B.record_layout(B.desc_of(odd), 4) == oracle.record_layout(odesc(odd), 4) == (32, 256)
@@ -61,6 +61,20 @@ def test_assign_bits_matches_oracle_bit_for_bit():
         gb, go = B.assign_bits(scores, (0.4, 0.2, 0.4))
         ob, oo = oracle.assign_bits(scores, (0.4, 0.2, 0.4))
         assert np.array_equal(gb, ob) and np.array_equal(go, oo)
+
+
+def test_assign_levels_matches_oracle_bit_for_bit():
+    rng = np.random.default_rng(1)
+    for levels in ((8, 4, 2), (4, 2, 1), (8, 2, 1), (8, 4, 1)):
+        for n, frac in [(256, (1 / 3, 1 / 3, 1 / 3)), (37, (0.1, 0.5, 0.4)), (1, (0.2, 0.3, 0.5)), (0, (1 / 3, 1 / 3, 1 / 3))]:
+            s = np.round(rng.random(n).astype(np.float32) * 8) / 8
+            gb, go = B.assign_levels(s, frac, levels)
+            ob, oo = oracle.assign_levels(s, frac, levels)
+            assert np.array_equal(gb, ob) and np.array_equal(go, oo)
+    for bad, status in (((4, 4, 2), B.ERR_INVALID_ARG), ((2, 4, 8), B.ERR_INVALID_ARG), ((8, 3, 1), B.ERR_BAD_BITS)):
+        with pytest.raises(B.LlmsError) as e:
+            B.assign_levels([0.5, 0.25], (0.5, 0.25, 0.25), bad)
+        assert e.value.status == status
 
 
 def test_optimize_thresholds_matches_oracle_bit_for_bit():
@@ -88,7 +102,7 @@ def test_lctru_order_matches_oracle_bit_for_bit():
         t = np.zeros(n, dtype=B.STATE_DTYPE)
         t["ctx_id"] = rng.integers(0, 64, n)
         t["chunk_id"] = rng.integers(0, 32, n)
-        t["bits"] = rng.choice([8, 4, 2], n)
+        t["bits"] = rng.choice([8, 4, 2, 1], n)
         t["resident"] = rng.random(n) < 0.7
         t["locked"] = rng.random(n) < 0.2
         t["last_access_step"] = rng.integers(0, 10, n)
@@ -124,6 +138,8 @@ def test_argument_errors_on_the_host():
     assert call(ids=ok_ids, out=8192 + 64) == B.ERR_MISALIGNED
     assert call(ids=ok_ids, out_bytes=8704) == B.ERR_BUF_TOO_SMALL        # needs 8704 + 4608
     assert call(ids=ok_ids, ws_bytes=32) == B.ERR_BUF_TOO_SMALL
+    d1 = B.desc_of(sh, 1)                                                   # channel-wise mode stops at 2 bits
+    assert call(ids=ok_ids, desc=d1, bits=np.array([8, 1], dtype=np.uint8)) == B.ERR_UNSUPPORTED
     d2 = B.desc_of(sh)
     d2.group_size = 48                                                      # divides 96 but is not a power of two
     d2.head_dim = 96

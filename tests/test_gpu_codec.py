@@ -112,6 +112,50 @@ def test_slabs_shorter_than_a_warp_pass(CL, d, G, L, H):
     check_decompress(sh, kv, buf_dev, meta, want_buf, dst_ids=np.arange(2, 11, dtype=np.uint32))
 
 
+@pytest.mark.parametrize("shape", [
+    ("tiny", None),
+    ("g128", (2, 3, 3, 128, 100, 16, 128)),     # whole passes
+    ("ragged", (2, 3, 3, 96, 50, 24, 32)),      # slab of 2304 elements: ragged second pass
+    ("odd", (1, 1, 1, 16, 25, 5, 16)),          # slab of 80 elements: 10-byte code runs, pieces on either half of a word
+    ("short", (2, 5, 5, 128, 40, 4, 64)),       # packed units
+])
+def test_one_bit_level(shape):
+    """Level set {4, 2, 1} (Sec. 3.2): records with 1-bit chunks among the others, bit for bit against the oracle."""
+    name, dims = shape
+    sh = synth.CONFIGS["tiny"] if dims is None else synth.KVShape(name, *dims, seed=17)
+    kv = synth.kv_tensor(sh)
+    ids = np.arange(sh.n_chunks)
+    bits = np.array([(1, 4, 2, 1, 8)[i % 5] for i in range(sh.n_chunks)], dtype=np.uint8)
+    kv_dev, buf_dev, meta, want_buf = check_compress(sh, kv, ids, bits)
+    out = check_decompress(sh, kv, buf_dev, meta, want_buf)
+    # a 1-bit group decodes to its minimum or (to fp16 accuracy) its maximum
+    x, y = kv.double(), out.cpu().double()
+    CL, G = sh.chunk_len, sh.group_size
+    for cid in ids[bits == 1][:3]:
+        xs = x[..., cid * CL:(cid + 1) * CL, :].reshape(-1, G)
+        ys = y[..., cid * CL:(cid + 1) * CL, :].reshape(-1, G)
+        lo, hi = xs.min(1, keepdim=True).values, xs.max(1, keepdim=True).values
+        tol = 2.0 ** -10 * torch.maximum(hi.abs(), hi - lo) + 1e-12
+        assert bool((((ys - lo).abs() <= 1e-12) | ((ys - hi).abs() <= tol)).all())
+    bits1 = np.ones(sh.n_chunks, dtype=np.uint8)
+    kv_dev, buf_dev, meta, want_buf = check_compress(sh, kv, ids, bits1)
+    check_decompress(sh, kv, buf_dev, meta, want_buf)
+
+
+def test_one_bit_special_values():
+    sh = synth.KVShape("special1", 1, 2, 2, 64, 64, 16, 64, seed=9)
+    kv = synth.kv_tensor(sh)
+    kv[0, 0, 0, 0:16] = 2.5                        # constant: scale 0
+    kv[0, 0, 0, 17, :] = torch.linspace(-6e-7, 6e-7, 64).half()   # subnormal scale: the clamped path
+    kv[0, 0, 0, 18, 0] = 65504.0                   # range 125504 is beyond fp16: the scale saturates at 65504
+    kv[0, 0, 0, 18, 1] = -60000.0
+    kv[0, 0, 0, 19, :] = torch.tensor([0.0, 1.0, 0.5, 0.25] * 16).half()      # the tie at one half goes to 0
+    ids = np.arange(sh.n_chunks)
+    bits = np.ones(sh.n_chunks, dtype=np.uint8)
+    kv_dev, buf_dev, meta, want_buf = check_compress(sh, kv, ids, bits)
+    check_decompress(sh, kv, buf_dev, meta, want_buf)
+
+
 def test_padding_is_written_and_compared():
     # 2 slabs * 3 tokens * 1 group = 6 groups -> 24 parameter bytes -> 8 zero bytes before the codes,
     # and 144/288 code bytes -> tail padding up to 256/512
