@@ -19,6 +19,9 @@
 // nothing is contracted or approximated.
 #include <string.h>
 
+#include <map>
+#include <mutex>
+#include <utility>
 #include <vector>
 
 #include "llms_internal.cuh"
@@ -510,12 +513,14 @@ __device__ __forceinline__ void zero_padding(const CodecArgs &a, uint8_t *rec, u
 template <bool WIDE, bool PACKED>
 __device__ __forceinline__ void load_unit(const CodecArgs &a, const UnitPos &u, int lane, uint32_t (&w)[kPieces][8])
 {
-    const int pass_e0 = u.e0 - lane * kLaneElems;
+    const __half *src0 = nullptr;  // piece 0 when the unit lies inside one slab
+    if constexpr (!PACKED) src0 = a.kv_in + slab_offset(a, u.s_idx, u.chunk_id) + (u.e0 - lane * kLaneElems) + lane * kPieceElems;
 #pragma unroll
     for (int j = 0; j < kPieces; ++j) {
         const int v = j * (32 * kPieceElems) + lane * kPieceElems;
         if (v < u.limit) {
-            load32<WIDE>(a.kv_in + unit_elem_offset<PACKED>(a, u.s_idx, u.chunk_id, pass_e0, v), w[j]);
+            if constexpr (PACKED) load32<WIDE>(a.kv_in + unit_elem_offset<true>(a, u.s_idx, u.chunk_id, 0, v), w[j]);
+            else load32<WIDE>(src0 + j * (32 * kPieceElems), w[j]);
         } else {
 #pragma unroll
             for (int k = 0; k < 8; ++k) w[j][k] = 0;  // past the end: whole inactive groups
@@ -764,6 +769,8 @@ __device__ __forceinline__ void decompress_unit(const CodecArgs &a, const Decode
 {
     // a lane's pieces all sit at the same place inside their groups: either every one opens a group or none does
     const bool opens_group = (lane * kPieceElems) % G == 0;
+    __half *dst0 = nullptr;  // piece 0 when the unit lies inside one slab
+    if constexpr (!PACKED) dst0 = a.kv_out + slab_offset(a, u.s_idx, u.chunk_id) + u.pass_e0 + lane * kPieceElems;
     uint32_t sum = 0;
 #pragma unroll
     for (int j = 0; j < kPieces; ++j) {
@@ -771,8 +778,12 @@ __device__ __forceinline__ void decompress_unit(const CodecArgs &a, const Decode
         const float zero = __half2float(__ushort_as_half((unsigned short)(p[j] >> 16)));
         uint32_t w[8];
         dequantize_piece<BITS>(c[j], scale_h, zero, w);
-        if (u.room > j * kPieceStride)
-            store32<WIDE>(a.kv_out + unit_elem_offset<PACKED>(a, u.s_idx, u.chunk_id, u.pass_e0, j * kPieceStride + lane * kPieceElems), w);
+        if (u.room > j * kPieceStride) {
+            if constexpr (PACKED)
+                store32<WIDE>(a.kv_out + unit_elem_offset<true>(a, u.s_idx, u.chunk_id, 0, j * kPieceStride + lane * kPieceElems), w);
+            else
+                store32<WIDE>(dst0 + j * kPieceStride, w);
+        }
         // pieces past the end of the slab were loaded as zeros and add nothing
         if constexpr (BITS == 1) {  // a piece is half of a record word; the pieces of a lane all sit in the same half
             sum += c[j][0] << ((reinterpret_cast<uintptr_t>(u.codes) & 2) * 8);
@@ -792,43 +803,47 @@ __device__ __forceinline__ void decompress_unit(const CodecArgs &a, const Decode
 constexpr int kDecodeDepth = 2;
 constexpr int kDecodeBlocksPerSm = 2;
 
+// The units of one warp, start to finish.
+template <int BITS, int G, bool WIDE, bool PACKED>
+__device__ __forceinline__ void decompress_warp(const CodecArgs &a, uint32_t unit, uint32_t n_warps, int lane, uint32_t *sum_slots)
+{
+    constexpr int D = kDecodeDepth;
+    DecodePos pos[D];
+    uint32_t c[D][kPieces][piece_words(BITS)], p[D][kPieces];
+#pragma unroll
+    for (int s = 0; s < D - 1; ++s) {
+        const uint32_t ahead = unit + s * n_warps;
+        if (ahead < a.total_units) {
+            decode_unit_for_decoder<BITS, G, PACKED>(a, ahead, lane, pos[s]);
+            load_unit_codes<BITS, G>(pos[s], c[s], p[s]);
+        }
+    }
+    for (;;) {
+#pragma unroll
+        for (int s = 0; s < D; ++s) {
+            // ring slot s holds the current unit; the slot freed last takes the unit D-1 strides ahead
+            const int fill = (s + D - 1) % D;
+            const uint32_t ahead = unit + (D - 1) * n_warps;
+            if (ahead < a.total_units) {
+                decode_unit_for_decoder<BITS, G, PACKED>(a, ahead, lane, pos[fill]);
+                load_unit_codes<BITS, G>(pos[fill], c[fill], p[fill]);
+            }
+            decompress_unit<BITS, G, WIDE, PACKED>(a, pos[s], c[s], p[s], lane, sum_slots);
+            unit += n_warps;
+            if (unit >= a.total_units) return;
+        }
+    }
+}
+
 template <int BITS, int G, bool WIDE, bool PACKED>
 __global__ void __launch_bounds__(kThreads, kDecodeBlocksPerSm) decompress_kernel(const CodecArgs a)
 {
-    constexpr int D = kDecodeDepth;
     const int lane = threadIdx.x & 31;
     const uint32_t n_warps = gridDim.x * kWarpsPerBlock;
-    uint32_t unit = blockIdx.x * kWarpsPerBlock + (threadIdx.x >> 5);
+    const uint32_t unit = blockIdx.x * kWarpsPerBlock + (threadIdx.x >> 5);
     __shared__ uint32_t sum_slots[kSumSlots];
     cta_sums_clear(sum_slots, a.n);
-    if (unit < a.total_units) {
-        DecodePos pos[D];
-        uint32_t c[D][kPieces][piece_words(BITS)], p[D][kPieces];
-#pragma unroll
-        for (int s = 0; s < D - 1; ++s) {
-            const uint32_t ahead = unit + s * n_warps;
-            if (ahead < a.total_units) {
-                decode_unit_for_decoder<BITS, G, PACKED>(a, ahead, lane, pos[s]);
-                load_unit_codes<BITS, G>(pos[s], c[s], p[s]);
-            }
-        }
-        for (bool done = false; !done;) {
-#pragma unroll
-            for (int s = 0; s < D; ++s) {
-                if (done) break;
-                // ring slot s holds the current unit; the slot freed last takes the unit D-1 strides ahead
-                const int fill = (s + D - 1) % D;
-                const uint32_t ahead = unit + (D - 1) * n_warps;
-                if (ahead < a.total_units) {
-                    decode_unit_for_decoder<BITS, G, PACKED>(a, ahead, lane, pos[fill]);
-                    load_unit_codes<BITS, G>(pos[fill], c[fill], p[fill]);
-                }
-                decompress_unit<BITS, G, WIDE, PACKED>(a, pos[s], c[s], p[s], lane, sum_slots);
-                unit += n_warps;
-                done = unit >= a.total_units;
-            }
-        }
-    }
+    if (unit < a.total_units) decompress_warp<BITS, G, WIDE, PACKED>(a, unit, n_warps, lane, sum_slots);
     __syncthreads();
     if (a.n <= kSumSlots)
         for (int k = threadIdx.x; k < a.n; k += kThreads)
@@ -923,10 +938,12 @@ static BitGroups group_by_bits(int n, const llms_chunk_meta *meta, GetBits bits_
     return g;
 }
 
-// One host-to-device copy sets the workspace up: zeroed status words, the entries, the unit table, the order.
-static int upload_tables(void *workspace, const llms_chunk_meta *entries, const BitGroups &g, int n, cudaStream_t st)
+// One host-to-device copy sets the workspace up: zeroed status words, the entries, the unit table, the order and,
+// for the decoder, the zeroed checksum accumulators behind them.
+static int upload_tables(void *workspace, const llms_chunk_meta *entries, const BitGroups &g, int n, bool zero_sums,
+                         cudaStream_t st)
 {
-    std::vector<uint8_t> image(ws_sums_offset(n), 0);
+    std::vector<uint8_t> image(ws_sums_offset(n) + (zero_sums ? (size_t)n * 4 : 0), 0);
     memcpy(image.data() + kWsEntriesOffset, entries, (size_t)n * sizeof(ChunkEntry));
     memcpy(image.data() + ws_table_offset(n), g.table.data(), (size_t)n * sizeof(UnitEntry));
     memcpy(image.data() + ws_order_offset(n), g.order.data(), (size_t)n * 4);
@@ -951,10 +968,25 @@ static CodecArgs args_for_group(const CodecArgs &a, const BitGroups &g, int k)
 template <typename K>
 static int grid_for(K kernel, int64_t items, size_t dyn_smem = 0)
 {
+    // the occupancy of a kernel does not change: asked once per kernel and device
+    static std::mutex lock;
+    static std::map<std::pair<const void *, int>, int> known;
+    int dev = 0;
+    cudaGetDevice(&dev);
+    const std::pair<const void *, int> key(reinterpret_cast<const void *>(kernel), dev);
     int per_sm = 0;
-    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kernel, kThreads, dyn_smem) != cudaSuccess || per_sm <= 0) {
-        cudaGetLastError();
-        per_sm = 2;
+    {
+        std::lock_guard<std::mutex> guard(lock);
+        auto it = known.find(key);
+        if (it != known.end()) per_sm = it->second;
+    }
+    if (per_sm == 0) {
+        if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kernel, kThreads, dyn_smem) != cudaSuccess || per_sm <= 0) {
+            cudaGetLastError();
+            per_sm = 2;
+        }
+        std::lock_guard<std::mutex> guard(lock);
+        known[key] = per_sm;
     }
     const int64_t want = (items + kWarpsPerBlock - 1) / kWarpsPerBlock;
     const int64_t cap = (int64_t)sm_count() * per_sm;
@@ -1065,7 +1097,7 @@ extern "C" int llms_compress_chunks(const llms_kv_desc *desc, const void *kv, co
     a.buf = static_cast<uint8_t *>(out_buf);
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     const BitGroups groups = group_by_bits(n, meta, [&](int i) { return (uint32_t)bits[i]; });
-    rc = upload_tables(workspace, meta, groups, n, st);
+    rc = upload_tables(workspace, meta, groups, n, false, st);
     if (rc) return rc;
     for (int k = 0; k < kNumWidths; ++k) {
         if (groups.count[k] == 0) continue;
@@ -1139,9 +1171,8 @@ extern "C" int llms_decompress_chunks(const llms_kv_desc *desc, const void *buf,
     a.buf = const_cast<uint8_t *>(static_cast<const uint8_t *>(buf));
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     uint32_t *status = static_cast<uint32_t *>(workspace);
-    LLMS_CUDA_TRY(cudaMemsetAsync(a.sums, 0, (size_t)n * 4, st));
     const BitGroups groups = group_by_bits(n, staged.data(), [&](int i) { return meta[i].bits; });
-    rc = upload_tables(workspace, staged.data(), groups, n, st);
+    rc = upload_tables(workspace, staged.data(), groups, n, true, st);
     if (rc) return rc;
     for (int k = 0; k < kNumWidths; ++k) {
         if (groups.count[k] == 0) continue;
