@@ -175,6 +175,57 @@ __device__ __forceinline__ void segment_reduce(float (&x)[2][2], Op op)
     }
 }
 
+// Softmax statistics of one n-tile (8 flattened window rows) from the accumulator fragments of a 32-token tile.
+// TAIL: the tile reaches into the last W columns, where rows stop seeing tokens and 1/n_vis varies; everywhere
+// else every row sees every token of the tile and the column weight is 1/W, so masks and weighted sums drop out.
+template <int SEG, bool TAIL>
+__device__ __forceinline__ void tile_statistics(const TolArgs &a, const float (&acc)[2][4], int nb, int q4, const int *last_col_s,
+                                                const int (&t_tok)[2][2], const float (&w_tok)[2][2], const bool (&opens)[2][2],
+                                                int64_t row0)
+{
+    const float inv_w = 1.0f / (float)a.W;
+#pragma unroll
+    for (int col = 0; col < 2; ++col) {
+        const int j = nb * 8 + 2 * q4 + col;       // flattened (head, window row)
+        const int last_col = last_col_s[j];        // last token this row sees; -1 for the zero padding rows
+        float lg[2][2], mx[2][2], se[2][2], sp[2][2];
+#pragma unroll
+        for (int mb = 0; mb < 2; ++mb)
+#pragma unroll
+            for (int h = 0; h < 2; ++h) {
+                lg[mb][h] = acc[mb][2 * h + col] * a.inv_sqrt_d;
+                if constexpr (TAIL) lg[mb][h] = t_tok[mb][h] <= last_col ? lg[mb][h] : -INFINITY;
+                mx[mb][h] = lg[mb][h];
+            }
+        segment_reduce<SEG>(mx, [](float x, float y) { return fmaxf(x, y); });
+#pragma unroll
+        for (int mb = 0; mb < 2; ++mb)
+#pragma unroll
+            for (int h = 0; h < 2; ++h) {
+                // exp2-based exponential: relative error of a few 1e-6 for the arguments met here
+                float e = __expf(lg[mb][h] - mx[mb][h]);
+                if constexpr (TAIL) e = lg[mb][h] == -INFINITY ? 0.0f : e;
+                se[mb][h] = e;
+                if constexpr (TAIL) sp[mb][h] = e * w_tok[mb][h];
+            }
+        segment_reduce<SEG>(se, [](float x, float y) { return x + y; });
+        if constexpr (TAIL) segment_reduce<SEG>(sp, [](float x, float y) { return x + y; });
+        if (last_col >= 0) {
+#pragma unroll
+            for (int mb = 0; mb < 2; ++mb)
+#pragma unroll
+                for (int h = 0; h < 2; ++h) {
+                    if (opens[mb][h]) {   // the segment's first token writes
+                        const int64_t o = (row0 + j) * a.n_seg + t_tok[mb][h] / SEG;
+                        a.pm[o] = mx[mb][h];
+                        a.ps[o] = se[mb][h];
+                        a.pp[o] = TAIL ? sp[mb][h] : se[mb][h] * inv_w;
+                    }
+                }
+        }
+    }
+}
+
 template <int SEG, int D>
 __global__ void __launch_bounds__(kTileWarps * 32) logits_mma_kernel(const TolArgs a)
 {
@@ -186,7 +237,9 @@ __global__ void __launch_bounds__(kTileWarps * 32) logits_mma_kernel(const TolAr
     const int n_blocks = (a.NR + 7) / 8;                                     // window rows in n-tiles of 8, zero padded
     unsigned char *q_s = smem_raw;                                           // [n_blocks*8][kQRowBytes]
     const int q_total = (n_blocks * 8 * kQRowBytes + 127) / 128 * 128;
-    unsigned char *tiles = smem_raw + q_total + wib * kTileBuffers * kTileBytes;   // this warp's buffers
+    int *last_col_s = reinterpret_cast<int *>(smem_raw + q_total);           // [n_blocks*8]: last token a row sees
+    const int lc_total = (n_blocks * 8 * 4 + 127) / 128 * 128;
+    unsigned char *tiles = smem_raw + q_total + lc_total + wib * kTileBuffers * kTileBytes;   // this warp's buffers
     const uint32_t tiles_s = (uint32_t)__cvta_generic_to_shared(tiles);
 
     const int l = blockIdx.y / a.Hkv, kvh = blockIdx.y % a.Hkv;
@@ -196,6 +249,7 @@ __global__ void __launch_bounds__(kTileWarps * 32) logits_mma_kernel(const TolAr
         *reinterpret_cast<uint4 *>(q_s + row * kQRowBytes + c * 16) =
             row < a.NR ? __ldg(reinterpret_cast<const uint4 *>(q_src) + i) : make_uint4(0, 0, 0, 0);
     }
+    for (int j = threadIdx.x; j < n_blocks * 8; j += blockDim.x) last_col_s[j] = j < a.NR ? a.T - a.W + j % a.W : -1;
     __syncthreads();
 
     const __half *k_plane = a.kv + (int64_t)l * a.stride_l + (int64_t)kvh * a.stride_h;
@@ -238,18 +292,19 @@ __global__ void __launch_bounds__(kTileWarps * 32) logits_mma_kernel(const TolAr
         }
         __syncwarp();
         const uint32_t tile_s = tiles_s + buf * kTileBytes;
-        // this lane's four tokens of the tile and their column weights 1/n_vis
+        // this lane's four tokens of the tile, their column weights 1/n_vis, and whether they open a segment
         int t_tok[2][2];
         float w_tok[2][2];
+        bool opens[2][2];
 #pragma unroll
         for (int mb = 0; mb < 2; ++mb)
 #pragma unroll
             for (int h = 0; h < 2; ++h) {
                 t_tok[mb][h] = tile * kTileTokens + mb * 16 + h * 8 + g;
                 w_tok[mb][h] = 1.0f / (float)min(a.W, max(1, a.T - t_tok[mb][h]));
+                opens[mb][h] = t_tok[mb][h] < a.T && t_tok[mb][h] % SEG == 0;
             }
         const bool tail_tile = tile * kTileTokens + kTileTokens > a.T - a.W + 1;
-        const float inv_w = 1.0f / (float)a.W;
         for (int nb = 0; nb < n_blocks; ++nb) {
             float acc[2][4];
 #pragma unroll
@@ -270,53 +325,8 @@ __global__ void __launch_bounds__(kTileWarps * 32) logits_mma_kernel(const TolAr
                 }
             }
             // acc[mb][0..1]: token mb*16 + g, window rows 2*q4, 2*q4+1;  acc[mb][2..3]: token mb*16 + 8 + g
-#pragma unroll
-            for (int col = 0; col < 2; ++col) {
-                const int j = nb * 8 + 2 * q4 + col;       // flattened (head, window row)
-                const int r = j % a.W;
-                const int last_col = j < a.NR ? a.T - a.W + r : -1;   // last token this row sees
-                float lg[2][2], mx[2][2], se[2][2], sp[2][2];
-#pragma unroll
-                for (int mb = 0; mb < 2; ++mb)
-#pragma unroll
-                    for (int h = 0; h < 2; ++h) {
-                        lg[mb][h] = t_tok[mb][h] <= last_col ? acc[mb][2 * h + col] * a.inv_sqrt_d : -INFINITY;
-                        mx[mb][h] = lg[mb][h];
-                    }
-                segment_reduce<SEG>(mx, [](float x, float y) { return fmaxf(x, y); });
-#pragma unroll
-                for (int mb = 0; mb < 2; ++mb)
-#pragma unroll
-                    for (int h = 0; h < 2; ++h) {
-                        // exp2-based exponential: relative error of a few 1e-6 for the arguments met here
-                        const float e = lg[mb][h] == -INFINITY ? 0.0f : __expf(lg[mb][h] - mx[mb][h]);
-                        se[mb][h] = e;
-                        sp[mb][h] = e * w_tok[mb][h];
-                    }
-                segment_reduce<SEG>(se, [](float x, float y) { return x + y; });
-                if (tail_tile) {   // 1/n_vis varies inside the tile only among the last W columns
-                    segment_reduce<SEG>(sp, [](float x, float y) { return x + y; });
-                } else {
-#pragma unroll
-                    for (int mb = 0; mb < 2; ++mb)
-#pragma unroll
-                        for (int h = 0; h < 2; ++h) sp[mb][h] = se[mb][h] * inv_w;
-                }
-                if (j < a.NR) {
-#pragma unroll
-                    for (int mb = 0; mb < 2; ++mb)
-#pragma unroll
-                        for (int h = 0; h < 2; ++h) {
-                            const int t = t_tok[mb][h];
-                            if (t < a.T && t % SEG == 0) {   // the segment's first token writes
-                                const int64_t o = (row0 + j) * a.n_seg + t / SEG;
-                                a.pm[o] = mx[mb][h];
-                                a.ps[o] = se[mb][h];
-                                a.pp[o] = sp[mb][h];
-                            }
-                        }
-                }
-            }
+            if (tail_tile) tile_statistics<SEG, true>(a, acc, nb, q4, last_col_s, t_tok, w_tok, opens, row0);
+            else tile_statistics<SEG, false>(a, acc, nb, q4, last_col_s, t_tok, w_tok, opens, row0);
         }
         __syncwarp();  // the buffer is free for the copy issued two tiles from now
     }
@@ -520,7 +530,8 @@ extern "C" int llms_chunk_tolerance(const llms_kv_desc *desc, const void *kv, co
     a.Y = t.Y; a.rows = t.rows;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     if ((unsigned)(a.L * a.Hkv) > 65535u) return LLMS_ERR_UNSUPPORTED;
-    const size_t mma_q_bytes = ((size_t)((a.NR + 7) / 8 * 8) * (a.d * 2 + 16) + 127) / 128 * 128;
+    const size_t mma_q_bytes = ((size_t)((a.NR + 7) / 8 * 8) * (a.d * 2 + 16) + 127) / 128 * 128 +
+                               ((size_t)((a.NR + 7) / 8 * 8) * 4 + 127) / 128 * 128;   // query rows + each row's last visible token
     const size_t mma_smem = mma_q_bytes + (size_t)kTileWarps * kTileBuffers * kTileTokens * a.d * 2;
     if ((a.d == 64 || a.d == 128 || a.d == 256) && mma_smem <= 200 * 1024) {
         // enough blocks per (layer, KV head) to fill the GPU a few times over
