@@ -231,5 +231,10 @@ def lctru_order(table):
     return order[:m].copy()
 
 
+def set_num_threads(n):
+    """Threads the oracle's slab loops may use from now on (for timing it single-threaded)."""
+    lib().orc_set_num_threads(int(n))
+
+
 def num_threads():
     return lib().orc_num_threads()

@@ -619,6 +619,16 @@ int orc_lctru_order(const orc_chunk_state *table, int n, uint32_t *order_out)
     return m;
 }
 
+/* Timing aid for the CPU baseline (not part of the method): threads the slab loops may use. */
+void orc_set_num_threads(int n)
+{
+#ifdef _OPENMP
+    if (n > 0) omp_set_num_threads(n);
+#else
+    (void)n;
+#endif
+}
+
 int orc_num_threads(void)
 {
 #ifdef _OPENMP
