@@ -224,6 +224,17 @@ def optimize_thresholds(scores, ratio_global):
     return np.array(list(frac), dtype=np.float32), list(counts)
 
 
+def optimize_thresholds_levels(scores, ratio_global, levels):
+    """-> (frac float32[3], counts int[3]) for a level set {top, middle, low}."""
+    s = np.ascontiguousarray(scores, dtype=np.float32)
+    frac = (C.c_float * 3)()
+    counts = (C.c_int * 3)()
+    lv = (C.c_uint8 * 3)(*[int(x) for x in levels])
+    _check(lib().orc_optimize_thresholds_levels(_ptr(s), int(s.size), C.c_float(ratio_global), lv, frac, counts),
+           "optimize_thresholds_levels")
+    return np.array(list(frac), dtype=np.float32), list(counts)
+
+
 def lctru_order(table):
     t = np.ascontiguousarray(table, dtype=STATE_DTYPE)
     order = np.empty(max(len(t), 1), dtype=np.uint32)

@@ -557,11 +557,31 @@ int orc_assign_bits(const float *scores, int n, const float frac[3], uint8_t *bi
  * P[k] = D(rank 0) + ... + D(rank k-1) (added in that order, binary64)
  *   ctxInfo(n8) = P[n8] + (P[n-n2] - P[n8])/2 + (P[n] - P[n-n2])/4.
  * The largest wins, the smaller n8 on a tie.  counts_out = {n8, n4, n2}; frac_out = counts / n. */
+int orc_optimize_thresholds_levels(const float *scores, int n, float ratio_global, const uint8_t levels[3],
+                                   float frac_out[3], int counts_out[3]);
+
 int orc_optimize_thresholds(const float *scores, int n, float ratio_global, float frac_out[3], int counts_out[3])
 {
-    if (n <= 0 || !scores) return ORC_ERR_ARG;
+    static const uint8_t k842[3] = {8, 4, 2};
+    return orc_optimize_thresholds_levels(scores, n, ratio_global, k842, frac_out, counts_out);
+}
+
+/* The same for any level set {top, middle, low} of bit-widths (Sec. 3.2: the levels are a parameter).  With
+ * r1 = middle/top and r2 = low/top the two conditions f0 + f1 + f2 = 1 and f0 + r1*f1 + r2*f2 = R leave
+ *   f2 = ((1 - r1)*f0 + r1 - R) / (r1 - r2),
+ * so n_low = floor(((1 - r1)*n_top + (r1 - R)*n) / (r1 - r2) + 1/2) for every n_top = 0..n, and
+ *   ctxInfo(n_top) = P[n_top] + r1*(P[n-n_low] - P[n_top]) + r2*(P[n] - P[n-n_low]).
+ * R in [r2, 1].  For {8, 4, 2} this is the formula above, term by term. */
+int orc_optimize_thresholds_levels(const float *scores, int n, float ratio_global, const uint8_t levels[3],
+                                   float frac_out[3], int counts_out[3])
+{
+    if (n <= 0 || !scores || !levels) return ORC_ERR_ARG;
+    for (int w = 0; w < 3; ++w)
+        if (levels[w] != 1 && levels[w] != 2 && levels[w] != 4 && levels[w] != 8) return ORC_ERR_BITS;
+    if (!(levels[0] > levels[1] && levels[1] > levels[2])) return ORC_ERR_ARG;
+    const double r1 = (double)levels[1] / (double)levels[0], r2 = (double)levels[2] / (double)levels[0];
     const double R = (double)ratio_global;
-    if (!(R >= 0.25 && R <= 1.0)) return ORC_ERR_ARG;
+    if (!(R >= r2 && R <= 1.0)) return ORC_ERR_ARG;
     uint32_t *ord = (uint32_t *)malloc(sizeof(uint32_t) * (size_t)n);
     double *P = (double *)malloc(sizeof(double) * (size_t)(n + 1));
     for (int i = 0; i < n; ++i) ord[i] = (uint32_t)i;
@@ -573,21 +593,21 @@ int orc_optimize_thresholds(const float *scores, int n, float ratio_global, floa
     }
     P[0] = 0.0;
     for (int k = 0; k < n; ++k) P[k + 1] = P[k] + (double)scores[ord[k]];
-    int best8 = -1, best2 = 0;
+    int best_top = -1, best_low = 0;
     double best = 0.0;
-    for (int n8 = 0; n8 <= n; ++n8) {
-        const double x = 2.0 * n8 + (2.0 - 4.0 * R) * n;
-        const long n2 = (long)floor(x + 0.5);
-        if (n2 < 0 || n8 + n2 > n) continue;
-        const double info = P[n8] + (P[n - n2] - P[n8]) / 2.0 + (P[n] - P[n - n2]) / 4.0;
-        if (best8 < 0 || info > best) { best8 = n8; best2 = (int)n2; best = info; }
+    for (int n_top = 0; n_top <= n; ++n_top) {
+        const double x = ((1.0 - r1) * n_top + (r1 - R) * n) / (r1 - r2);
+        const long n_low = (long)floor(x + 0.5);
+        if (n_low < 0 || n_top + n_low > n) continue;
+        const double info = P[n_top] + (P[n - n_low] - P[n_top]) * r1 + (P[n] - P[n - n_low]) * r2;
+        if (best_top < 0 || info > best) { best_top = n_top; best_low = (int)n_low; best = info; }
     }
     free(ord);
     free(P);
-    if (best8 < 0) return ORC_ERR_ARG;
-    counts_out[0] = best8;
-    counts_out[1] = n - best8 - best2;
-    counts_out[2] = best2;
+    if (best_top < 0) return ORC_ERR_ARG;
+    counts_out[0] = best_top;
+    counts_out[1] = n - best_top - best_low;
+    counts_out[2] = best_low;
     for (int w = 0; w < 3; ++w) frac_out[w] = (float)((double)counts_out[w] / (double)n);
     return ORC_OK;
 }

@@ -151,3 +151,55 @@ def test_thresholds_brute_force_over_all_level_assignments():
                     continue
                 best = max(best, float(np.dot(np.array(levels), s.astype(np.float64))))
             assert got == pytest.approx(best, rel=1e-12)
+
+
+@pytest.mark.parametrize("levels", [(8, 4, 2), (4, 2, 1), (8, 2, 1), (8, 4, 1)])
+def test_thresholds_for_other_level_sets(levels):
+    b0, b1, b2 = levels
+    r1, r2 = b1 / b0, b2 / b0
+    rng = np.random.default_rng(b0 * 100 + b1 * 10 + b2)
+    # counts obey the ratio rule and reproduce through the rank -> bits rule; the ratio is met to half a chunk step
+    for n in (5, 32, 257):
+        for R in (0.5, 0.3, 0.8, r2, 1.0):
+            s = (rng.random(n) ** 3).astype(np.float32)
+            try:
+                frac, (c0, c1, c2) = oracle.optimize_thresholds_levels(s, R, levels)
+            except RuntimeError:
+                assert n == 5                               # only so few chunks can leave a ratio without any count triple
+                continue
+            assert c0 + c1 + c2 == n and min(c0, c1, c2) >= 0
+            Rd = np.float64(np.float32(R))
+            assert c2 == int(np.floor(((1 - r1) * c0 + (r1 - Rd) * n) / (r1 - r2) + 0.5))
+            assert abs((c0 + r1 * c1 + r2 * c2) / n - R) <= (r1 - r2) / (2 * n) + 1e-7
+            bits, _ = oracle.assign_levels(s, frac, levels)
+            assert [int((bits == b).sum()) for b in levels] == [c0, c1, c2]
+    # brute force over every assignment of levels to chunks whose counts obey the rule
+    for n in (4, 6, 7):
+        for R in (0.5, 0.4):
+            s = (rng.random(n) ** 2).astype(np.float32)
+            try:
+                _, (c0, c1, c2) = oracle.optimize_thresholds_levels(s, R, levels)
+            except RuntimeError:
+                continue                                    # no count triple meets this ratio for so few chunks
+            order = np.argsort(-s, kind="stable")
+            sd = s.astype(np.float64)
+            got = sd[order[:c0]].sum() + r1 * sd[order[c0:c0 + c1]].sum() + r2 * sd[order[c0 + c1:]].sum()
+            Rd = np.float64(np.float32(R))
+            best = -1.0
+            for assign in itertools.product((0, 1, 2), repeat=n):
+                k0, k2 = assign.count(0), assign.count(2)
+                if k2 != int(np.floor(((1 - r1) * k0 + (r1 - Rd) * n) / (r1 - r2) + 0.5)):
+                    continue
+                w = np.array([(1.0, r1, r2)[a] for a in assign])
+                best = max(best, float(np.dot(w, sd)))
+            assert got == pytest.approx(best, rel=1e-12)
+
+
+def test_thresholds_levels_842_is_the_original_rule():
+    rng = np.random.default_rng(3)
+    for n in (3, 16, 255):
+        for R in (0.5, 0.4, 0.7, 0.25, 1.0):
+            s = rng.random(n).astype(np.float32) ** 2
+            a = oracle.optimize_thresholds(s, R)
+            b = oracle.optimize_thresholds_levels(s, R, (8, 4, 2))
+            assert a[1] == b[1] and np.array_equal(a[0], b[0])
