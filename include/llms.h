@@ -200,8 +200,7 @@ int llms_assign_bits(const float *scores, int n, const float frac[3], uint8_t *b
 /* Eq. 2 for another level set (Sec. 3.2: the method is not tied to 8/4/2 - atop a 4-bit cache it offers 2 and
  * 1 bit).  levels = {top, middle, low} bit-widths from {8, 4, 2, 1}, strictly decreasing; frac = the shares
  * of chunks per level, in that order; everything else as llms_assign_bits, which is this call with
- * levels {8, 4, 2}.  llms_optimize_thresholds serves any set whose widths halve from level to level
- * ({8,4,2}, {4,2,1}): its ratio_global is relative to the top level. */
+ * levels {8, 4, 2}; llms_optimize_thresholds_levels finds the shares for such a set. */
 int llms_assign_levels(const float *scores, int n, const float frac[3], const uint8_t levels[3],
                        uint8_t *bits_out, uint32_t *order_out);
 
@@ -213,6 +212,15 @@ int llms_assign_levels(const float *scores, int n, const float frac[3], const ui
  * (n2 = floor(2*n8 + (2 - 4*ratio_global)*n + 1/2), n4 the rest); the best wins, the smaller n8 on a tie.
  * frac_out = {n8, n4, n2} / n, ready for llms_assign_bits.  scores: host, n > 0 values. */
 int llms_optimize_thresholds(const float *scores, int n, float ratio_global, float frac_out[3]);
+
+/* Eq. 3 for any level set {top, middle, low} (strictly decreasing bit-widths from {8, 4, 2, 1}).  With
+ * r1 = middle/top and r2 = low/top, ratio_global in [r2, 1] is relative to the top level:
+ * f_top + r1*f_mid + r2*f_low = ratio_global, hence f_low = ((1 - r1)*f_top + r1 - ratio_global) / (r1 - r2);
+ * n_low = floor(that * n + 1/2) for every count n_top, weights 1, r1, r2, the best wins, the smaller n_top on a
+ * tie.  LLMS_ERR_INVALID_ARG when no count triple meets the ratio (possible for a handful of chunks only).
+ * llms_optimize_thresholds is this call with levels {8, 4, 2}. */
+int llms_optimize_thresholds_levels(const float *scores, int n, float ratio_global, const uint8_t levels[3],
+                                    float frac_out[3]);
 
 /* Sec. 3.4 (ii): eviction order over the rows that are resident and not locked - the 8-bit
  * sub-queue first, then 4, then 2 ("heavy chunks first"), least recently used first inside a

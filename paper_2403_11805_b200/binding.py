@@ -61,6 +61,7 @@ _SIGNATURES = {
     "llms_assign_bits": (C.c_int, [C.c_void_p, C.c_int, C.c_void_p, C.c_void_p, C.c_void_p]),
     "llms_assign_levels": (C.c_int, [C.c_void_p, C.c_int, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]),
     "llms_optimize_thresholds": (C.c_int, [C.c_void_p, C.c_int, C.c_float, C.c_void_p]),
+    "llms_optimize_thresholds_levels": (C.c_int, [C.c_void_p, C.c_int, C.c_float, C.c_void_p, C.c_void_p]),
     "llms_lctru_order": (C.c_int, [C.c_void_p, C.c_int, C.c_void_p]),
     "llms_swap_out": (C.c_int, [C.c_void_p, C.c_void_p, C.c_int, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p,
                                 C.c_void_p]),
@@ -277,6 +278,16 @@ def optimize_thresholds(scores, ratio_global):
     s = np.ascontiguousarray(scores, dtype=np.float32)
     frac = np.zeros(3, dtype=np.float32)
     _check(lib().llms_optimize_thresholds(_ptr(s), int(s.size), float(ratio_global), _ptr(frac)), "llms_optimize_thresholds")
+    return frac
+
+
+def optimize_thresholds_levels(scores, ratio_global, levels):
+    s = np.ascontiguousarray(scores, dtype=np.float32)
+    lv = np.asarray(levels, dtype=np.uint8)
+    assert lv.size == 3
+    frac = np.zeros(3, dtype=np.float32)
+    _check(lib().llms_optimize_thresholds_levels(_ptr(s), int(s.size), float(ratio_global), _ptr(lv), _ptr(frac)),
+           "llms_optimize_thresholds_levels")
     return frac
 
 

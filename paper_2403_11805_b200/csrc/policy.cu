@@ -36,35 +36,47 @@ extern "C" int llms_assign_bits(const float *scores, int n, const float frac[3],
     return llms_assign_levels(scores, n, frac, kLevels, bits_out, order_out);
 }
 
-extern "C" int llms_optimize_thresholds(const float *scores, int n, float ratio_global, float frac_out[3])
+extern "C" int llms_optimize_thresholds_levels(const float *scores, int n, float ratio_global, const uint8_t levels[3],
+                                               float frac_out[3])
 {
-    if (n <= 0 || !scores || !frac_out) return LLMS_ERR_INVALID_ARG;
+    if (n <= 0 || !scores || !levels || !frac_out) return LLMS_ERR_INVALID_ARG;
+    for (int w = 0; w < 3; ++w)
+        if (llms::check_bits(levels[w])) return LLMS_ERR_BAD_BITS;
+    if (!(levels[0] > levels[1] && levels[1] > levels[2])) return LLMS_ERR_INVALID_ARG;
+    // a chunk at the middle / low level keeps r1 / r2 of the top level's bytes, and of its density's weight
+    const double r1 = (double)levels[1] / (double)levels[0], r2 = (double)levels[2] / (double)levels[0];
     const double R = (double)ratio_global;
-    if (!(R >= 0.25 && R <= 1.0)) return LLMS_ERR_INVALID_ARG;
+    if (!(R >= r2 && R <= 1.0)) return LLMS_ERR_INVALID_ARG;
     std::vector<uint32_t> order(n);
     std::iota(order.begin(), order.end(), 0u);
     std::stable_sort(order.begin(), order.end(), [&](uint32_t a, uint32_t b) { return scores[a] > scores[b]; });
     // prefix[k] = density of the k densest chunks, added in rank order
     std::vector<double> prefix(n + 1, 0.0);
     for (int k = 0; k < n; ++k) prefix[k + 1] = prefix[k] + (double)scores[order[k]];
-    long best8 = -1, best2 = 0;
+    long best_top = -1, best_low = 0;
     double best = 0.0;
-    for (long n8 = 0; n8 <= n; ++n8) {
-        // shares: f8 + f4 + f2 = 1 and f8 + f4/2 + f2/4 = R  =>  f2 = 2 f8 + 2 - 4R
-        const long n2 = (long)std::floor(2.0 * n8 + (2.0 - 4.0 * R) * n + 0.5);
-        if (n2 < 0 || n8 + n2 > n) continue;
-        const double info = prefix[n8] + (prefix[n - n2] - prefix[n8]) / 2.0 + (prefix[n] - prefix[n - n2]) / 4.0;
-        if (best8 < 0 || info > best) {
-            best8 = n8;
-            best2 = n2;
+    for (long n_top = 0; n_top <= n; ++n_top) {
+        // shares: f0 + f1 + f2 = 1 and f0 + r1 f1 + r2 f2 = R  =>  f2 = ((1 - r1) f0 + r1 - R) / (r1 - r2)
+        const long n_low = (long)std::floor(((1.0 - r1) * n_top + (r1 - R) * n) / (r1 - r2) + 0.5);
+        if (n_low < 0 || n_top + n_low > n) continue;
+        const double info = prefix[n_top] + (prefix[n - n_low] - prefix[n_top]) * r1 + (prefix[n] - prefix[n - n_low]) * r2;
+        if (best_top < 0 || info > best) {
+            best_top = n_top;
+            best_low = n_low;
             best = info;
         }
     }
-    if (best8 < 0) return LLMS_ERR_INVALID_ARG;
-    frac_out[0] = (float)((double)best8 / n);
-    frac_out[1] = (float)((double)(n - best8 - best2) / n);
-    frac_out[2] = (float)((double)best2 / n);
+    if (best_top < 0) return LLMS_ERR_INVALID_ARG;
+    frac_out[0] = (float)((double)best_top / n);
+    frac_out[1] = (float)((double)(n - best_top - best_low) / n);
+    frac_out[2] = (float)((double)best_low / n);
     return LLMS_OK;
+}
+
+extern "C" int llms_optimize_thresholds(const float *scores, int n, float ratio_global, float frac_out[3])
+{
+    static const uint8_t kLevels[3] = {8, 4, 2};
+    return llms_optimize_thresholds_levels(scores, n, ratio_global, kLevels, frac_out);
 }
 
 extern "C" int llms_lctru_order(const llms_chunk_state *table, int n, uint32_t *order_out)

@@ -96,6 +96,23 @@ def test_optimize_thresholds_matches_oracle_bit_for_bit():
         B.optimize_thresholds([0.1, 0.2], 0.2)
 
 
+def test_optimize_thresholds_levels_matches_oracle_bit_for_bit():
+    rng = np.random.default_rng(8)
+    for levels in ((8, 4, 2), (4, 2, 1), (8, 2, 1), (8, 4, 1)):
+        for n in (6, 32, 256, 1000):
+            for R in (0.5, 0.35, 0.8, levels[2] / levels[0], 1.0):
+                s = (rng.random(n) ** 3).astype(np.float32)
+                try:
+                    want, _ = oracle.optimize_thresholds_levels(s, R, levels)
+                except RuntimeError:
+                    with pytest.raises(B.LlmsError):
+                        B.optimize_thresholds_levels(s, R, levels)
+                    continue
+                assert np.array_equal(B.optimize_thresholds_levels(s, R, levels), want)
+    with pytest.raises(B.LlmsError):
+        B.optimize_thresholds_levels([0.1, 0.2, 0.3], 0.1, (8, 4, 2))       # below the low level's ratio
+
+
 def test_lctru_order_matches_oracle_bit_for_bit():
     rng = np.random.default_rng(1)
     for n in (0, 1, 5, 64, 2048):
