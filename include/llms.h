@@ -119,7 +119,7 @@ int llms_codec_workspace_bytes(int n, uint64_t *nbytes);
  * down in out_buf at the running offset (records in list order, each 256-byte aligned).
  *   kv         device, fp16, 16-byte aligned, read only
  *   chunk_ids  host, n distinct ids < floor(n_tokens/chunk_len)
- *   bits       host, n values from {1, 2, 4, 8} (1 only with quant_mode 0: LLMS_ERR_UNSUPPORTED otherwise)
+ *   bits       host, n values from {1, 2, 4, 8}
  *   out_buf    device, 256-byte aligned, out_bytes >= llms_compressed_size(...); every byte of
  *              every record, padding included, is written
  *   meta       host, n entries, filled before return except `checksum`, which the device

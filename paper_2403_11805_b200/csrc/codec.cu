@@ -1072,7 +1072,6 @@ extern "C" int llms_compress_chunks(const llms_kv_desc *desc, const void *kv, co
         uint64_t nb;
         rc = llms_record_bytes(desc, bits[i], &nb);
         if (rc) return rc;
-        if (bits[i] == 1 && desc->quant_mode == 1) return LLMS_ERR_UNSUPPORTED;  // the channel-wise kernels stop at 2 bits
         if (chunk_ids[i] >= nc || seen[chunk_ids[i]]) return LLMS_ERR_INVALID_ARG;
         seen[chunk_ids[i]] = 1;
         off += nb;
@@ -1107,7 +1106,8 @@ extern "C" int llms_compress_chunks(const llms_kv_desc *desc, const void *kv, co
             const int64_t items = (int64_t)b.n * b.n_slabs;
             if (k == 0) compress_cw_kernel<8><<<grid_for(compress_cw_kernel<8>, items), kThreads, 0, st>>>(b, desc->head_dim, desc->chunk_len);
             else if (k == 1) compress_cw_kernel<4><<<grid_for(compress_cw_kernel<4>, items), kThreads, 0, st>>>(b, desc->head_dim, desc->chunk_len);
-            else compress_cw_kernel<2><<<grid_for(compress_cw_kernel<2>, items), kThreads, 0, st>>>(b, desc->head_dim, desc->chunk_len);
+            else if (k == 2) compress_cw_kernel<2><<<grid_for(compress_cw_kernel<2>, items), kThreads, 0, st>>>(b, desc->head_dim, desc->chunk_len);
+            else compress_cw_kernel<1><<<grid_for(compress_cw_kernel<1>, items), kThreads, 0, st>>>(b, desc->head_dim, desc->chunk_len);
             LLMS_CUDA_TRY(cudaGetLastError());
             continue;
         }
@@ -1156,7 +1156,6 @@ extern "C" int llms_decompress_chunks(const llms_kv_desc *desc, const void *buf,
         uint64_t nb;
         rc = llms_record_bytes(desc, (int)meta[i].bits, &nb);
         if (rc) return rc;
-        if (meta[i].bits == 1 && desc->quant_mode == 1) return LLMS_ERR_UNSUPPORTED;
         if (meta[i].nbytes != nb || meta[i].n_groups != (uint32_t)groups_per_chunk(*desc)) return LLMS_ERR_INVALID_ARG;
         if (meta[i].offset % 256) return LLMS_ERR_MISALIGNED;
         const uint32_t dst = dst_chunk_ids ? dst_chunk_ids[i] : meta[i].chunk_id;
@@ -1181,7 +1180,8 @@ extern "C" int llms_decompress_chunks(const llms_kv_desc *desc, const void *buf,
             const int64_t items = (int64_t)b.n * b.n_slabs;
             if (k == 0) decompress_cw_kernel<8><<<grid_for(decompress_cw_kernel<8>, items), kThreads, 0, st>>>(b, desc->head_dim, desc->chunk_len);
             else if (k == 1) decompress_cw_kernel<4><<<grid_for(decompress_cw_kernel<4>, items), kThreads, 0, st>>>(b, desc->head_dim, desc->chunk_len);
-            else decompress_cw_kernel<2><<<grid_for(decompress_cw_kernel<2>, items), kThreads, 0, st>>>(b, desc->head_dim, desc->chunk_len);
+            else if (k == 2) decompress_cw_kernel<2><<<grid_for(decompress_cw_kernel<2>, items), kThreads, 0, st>>>(b, desc->head_dim, desc->chunk_len);
+            else decompress_cw_kernel<1><<<grid_for(decompress_cw_kernel<1>, items), kThreads, 0, st>>>(b, desc->head_dim, desc->chunk_len);
             LLMS_CUDA_TRY(cudaGetLastError());
             continue;
         }

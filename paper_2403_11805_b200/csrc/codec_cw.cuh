@@ -6,7 +6,7 @@
 // chunks; a lane owns one column (8 channels) for every (32 / columns)-th token, so a warp instruction still
 // touches consecutive addresses.  Pass 1 takes the column minima and maxima (packed half2, then xor-shuffles over
 // the lanes that share a column); pass 2 reads the slab again (it is in L1/L2 by then), quantizes each value with
-// its own channel's parameters and packs 8 codes per lane and token.  head_dim 64, 128 or 256.
+// its own channel's parameters and packs 8 codes per lane and token (8, 4, 2 bytes or 1 byte).  head_dim 64, 128 or 256.
 #pragma once
 
 namespace llms {
@@ -123,9 +123,12 @@ __global__ void __launch_bounds__(kThreads) compress_cw_kernel(const CodecArgs a
                 if constexpr (BITS == 4) {
                     st32(dst, acc);
                     sum += acc;
-                } else {
-                    asm volatile("st.global.L1::no_allocate.b16 [%1], %0;" :: "h"((unsigned short)acc), "l"(dst) : "memory");
+                } else if constexpr (BITS == 2) {
+                    st16(dst, acc);
                     sum += acc << ((geo.col & 1) * 16);  // its half of the record's 32-bit word
+                } else {
+                    asm volatile("st.global.L1::no_allocate.b8 [%1], %0;" :: "r"(acc), "l"(dst) : "memory");
+                    sum += acc << ((geo.col & 3) * 8);   // its byte of the record's 32-bit word
                 }
             }
         }
@@ -178,11 +181,12 @@ __global__ void __launch_bounds__(kThreads) decompress_cw_kernel(const CodecArgs
             } else if constexpr (BITS == 4) {
                 ld32(src, c);
                 sum += c[0];
-            } else {
-                unsigned short v;
-                asm volatile("ld.global.nc.L1::no_allocate.b16 %0, [%1];" : "=h"(v) : "l"(src));
-                c[0] = v;
+            } else if constexpr (BITS == 2) {
+                ld16(src, c);
                 sum += c[0] << ((geo.col & 1) * 16);
+            } else {
+                asm volatile("ld.global.nc.L1::no_allocate.u8 %0, [%1];" : "=r"(c[0]) : "l"(src));
+                sum += c[0] << ((geo.col & 3) * 8);
             }
             // the 8 codes as exact fp16 integers (0x6400 | q = 1024 + q), in channel order
             const __half2 k1024 = as_h2(0x64006400u);
@@ -194,8 +198,10 @@ __global__ void __launch_bounds__(kThreads) decompress_cw_kernel(const CodecArgs
                 q[3] = __hsub2(as_h2(__byte_perm(c[1], 0x64646464u, 0x4342)), k1024);
             } else {
                 // codes 0..3 in the low 16 bits, codes 4..7 in the high 16 bits (at 4 bits they already are)
-                const uint32_t z = BITS == 4 ? c[0] : ((c[0] & 0xFFu) | ((c[0] & 0xFF00u) << 8));
-                constexpr uint32_t kMask = BITS == 4 ? 0x000F000Fu : 0x00030003u;
+                const uint32_t z = BITS == 4 ? c[0]
+                                   : BITS == 2 ? ((c[0] & 0xFFu) | ((c[0] & 0xFF00u) << 8))
+                                               : ((c[0] & 0xFu) | ((c[0] & 0xF0u) << 12));
+                constexpr uint32_t kMask = BITS == 4 ? 0x000F000Fu : BITS == 2 ? 0x00030003u : 0x00010001u;
 #pragma unroll
                 for (int s = 0; s < 4; ++s)  // codes s (low half) and s + 4 (high half)
                     q[s] = __hsub2(as_h2(((z >> (BITS * s)) & kMask) | 0x64006400u), k1024);

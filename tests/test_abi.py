@@ -155,8 +155,6 @@ def test_argument_errors_on_the_host():
     assert call(ids=ok_ids, out=8192 + 64) == B.ERR_MISALIGNED
     assert call(ids=ok_ids, out_bytes=8704) == B.ERR_BUF_TOO_SMALL        # needs 8704 + 4608
     assert call(ids=ok_ids, ws_bytes=32) == B.ERR_BUF_TOO_SMALL
-    d1 = B.desc_of(sh, 1)                                                   # channel-wise mode stops at 2 bits
-    assert call(ids=ok_ids, desc=d1, bits=np.array([8, 1], dtype=np.uint8)) == B.ERR_UNSUPPORTED
     d2 = B.desc_of(sh)
     d2.group_size = 48                                                      # divides 96 but is not a power of two
     d2.head_dim = 96

@@ -325,7 +325,7 @@ def test_channel_wise_mode_matches_oracle(sh):
     kv = synth.kv_tensor(sh)
     rng = np.random.default_rng(5)
     ids = rng.permutation(sh.n_chunks).astype(np.uint32)
-    bits = np.array([(8, 4, 2)[i % 3] for i in range(sh.n_chunks)], dtype=np.uint8)
+    bits = np.array([(8, 4, 2, 1)[i % 4] for i in range(sh.n_chunks)], dtype=np.uint8)
     got_buf, got_meta, buf_dev = gpu_compress(sh, kv.cuda(), ids, bits, mode=1)
     want_buf, want_meta = oracle.compress_chunks(odesc(sh, 1), bits_view(kv), ids, bits)
     assert first_mismatch(got_buf, want_buf) is None
@@ -346,7 +346,7 @@ def test_channel_wise_special_values_and_outliers():
     kv[0, 0, 0, 0, 6] = 65504.0
     kv[0, 0, 0, 1, 6] = -65504.0                     # decode saturates
     ids = np.arange(sh.n_chunks, dtype=np.uint32)
-    for b in (8, 4, 2):
+    for b in (8, 4, 2, 1):
         bits = np.full(sh.n_chunks, b, dtype=np.uint8)
         got_buf, got_meta, buf_dev = gpu_compress(sh, kv.cuda(), ids, bits, mode=1)
         want_buf, want_meta = oracle.compress_chunks(odesc(sh, 1), bits_view(kv), ids, bits)
