@@ -993,6 +993,32 @@ static int grid_for(K kernel, int64_t items, size_t dyn_smem = 0)
     return (int)(want < cap ? want : cap);
 }
 
+// Channel-wise launches: slabs of 4, 8 or 16 tokens per lane (the paper's 16-token chunks at head_dim 64, 128, 256)
+// take the kernels that hold the slab in registers, anything else the two-pass ones.
+template <int BITS>
+static void launch_compress_cw(const CodecArgs &b, int head_dim, int chunk_len, cudaStream_t st)
+{
+    const int64_t items = (int64_t)b.n * b.n_slabs;
+    const int lpc = 32 / (head_dim / 8);
+    const int tok = chunk_len % lpc == 0 ? chunk_len / lpc : 0;
+    if (tok == 4) compress_cw_reg_kernel<BITS, 4><<<grid_for(compress_cw_reg_kernel<BITS, 4>, items), kThreads, 0, st>>>(b, head_dim);
+    else if (tok == 8) compress_cw_reg_kernel<BITS, 8><<<grid_for(compress_cw_reg_kernel<BITS, 8>, items), kThreads, 0, st>>>(b, head_dim);
+    else if (tok == 16) compress_cw_reg_kernel<BITS, 16><<<grid_for(compress_cw_reg_kernel<BITS, 16>, items), kThreads, 0, st>>>(b, head_dim);
+    else compress_cw_kernel<BITS><<<grid_for(compress_cw_kernel<BITS>, items), kThreads, 0, st>>>(b, head_dim, chunk_len);
+}
+
+template <int BITS>
+static void launch_decompress_cw(const CodecArgs &b, int head_dim, int chunk_len, cudaStream_t st)
+{
+    const int64_t items = (int64_t)b.n * b.n_slabs;
+    const int lpc = 32 / (head_dim / 8);
+    const int tok = chunk_len % lpc == 0 ? chunk_len / lpc : 0;
+    if (tok == 4) decompress_cw_reg_kernel<BITS, 4><<<grid_for(decompress_cw_reg_kernel<BITS, 4>, items), kThreads, 0, st>>>(b, head_dim);
+    else if (tok == 8) decompress_cw_reg_kernel<BITS, 8><<<grid_for(decompress_cw_reg_kernel<BITS, 8>, items), kThreads, 0, st>>>(b, head_dim);
+    else if (tok == 16) decompress_cw_reg_kernel<BITS, 16><<<grid_for(decompress_cw_reg_kernel<BITS, 16>, items), kThreads, 0, st>>>(b, head_dim);
+    else decompress_cw_kernel<BITS><<<grid_for(decompress_cw_kernel<BITS>, items), kThreads, 0, st>>>(b, head_dim, chunk_len);
+}
+
 // The decoder's grid: never more CTAs per SM than it was tuned for, whatever the register count allows.
 template <typename K>
 static int decode_grid(K kernel, int64_t items)
@@ -1103,11 +1129,10 @@ extern "C" int llms_compress_chunks(const llms_kv_desc *desc, const void *kv, co
         const CodecArgs b = args_for_group(a, groups, k);
         cudaError_t attr_err = cudaSuccess;
         if (desc->quant_mode == 1) {
-            const int64_t items = (int64_t)b.n * b.n_slabs;
-            if (k == 0) compress_cw_kernel<8><<<grid_for(compress_cw_kernel<8>, items), kThreads, 0, st>>>(b, desc->head_dim, desc->chunk_len);
-            else if (k == 1) compress_cw_kernel<4><<<grid_for(compress_cw_kernel<4>, items), kThreads, 0, st>>>(b, desc->head_dim, desc->chunk_len);
-            else if (k == 2) compress_cw_kernel<2><<<grid_for(compress_cw_kernel<2>, items), kThreads, 0, st>>>(b, desc->head_dim, desc->chunk_len);
-            else compress_cw_kernel<1><<<grid_for(compress_cw_kernel<1>, items), kThreads, 0, st>>>(b, desc->head_dim, desc->chunk_len);
+            if (k == 0) launch_compress_cw<8>(b, desc->head_dim, desc->chunk_len, st);
+            else if (k == 1) launch_compress_cw<4>(b, desc->head_dim, desc->chunk_len, st);
+            else if (k == 2) launch_compress_cw<2>(b, desc->head_dim, desc->chunk_len, st);
+            else launch_compress_cw<1>(b, desc->head_dim, desc->chunk_len, st);
             LLMS_CUDA_TRY(cudaGetLastError());
             continue;
         }
@@ -1177,11 +1202,10 @@ extern "C" int llms_decompress_chunks(const llms_kv_desc *desc, const void *buf,
         if (groups.count[k] == 0) continue;
         const CodecArgs b = args_for_group(a, groups, k);
         if (desc->quant_mode == 1) {
-            const int64_t items = (int64_t)b.n * b.n_slabs;
-            if (k == 0) decompress_cw_kernel<8><<<grid_for(decompress_cw_kernel<8>, items), kThreads, 0, st>>>(b, desc->head_dim, desc->chunk_len);
-            else if (k == 1) decompress_cw_kernel<4><<<grid_for(decompress_cw_kernel<4>, items), kThreads, 0, st>>>(b, desc->head_dim, desc->chunk_len);
-            else if (k == 2) decompress_cw_kernel<2><<<grid_for(decompress_cw_kernel<2>, items), kThreads, 0, st>>>(b, desc->head_dim, desc->chunk_len);
-            else decompress_cw_kernel<1><<<grid_for(decompress_cw_kernel<1>, items), kThreads, 0, st>>>(b, desc->head_dim, desc->chunk_len);
+            if (k == 0) launch_decompress_cw<8>(b, desc->head_dim, desc->chunk_len, st);
+            else if (k == 1) launch_decompress_cw<4>(b, desc->head_dim, desc->chunk_len, st);
+            else if (k == 2) launch_decompress_cw<2>(b, desc->head_dim, desc->chunk_len, st);
+            else launch_decompress_cw<1>(b, desc->head_dim, desc->chunk_len, st);
             LLMS_CUDA_TRY(cudaGetLastError());
             continue;
         }
