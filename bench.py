@@ -275,16 +275,17 @@ def run_ours(args):
     stream = torch.cuda.current_stream()
     state = {}
 
+    frac_a = np.asarray(frac, dtype=np.float32)
+    levels_a = np.asarray(LEVELS, dtype=np.uint8)
+    bits = np.zeros(n, dtype=np.uint8)
+
     def step(ev=None):
         if ev:
             ev[0].record(stream)
-        B.chunk_tolerance(d, kv, q_win, W, scores, ws_tol)
-        scores_host.copy_(scores, non_blocking=True)
-        stream.synchronize()                     # the ranking is a host step
-        bits, _ = B.assign_levels(scores_host.numpy(), frac, LEVELS)
-        if ev:
-            ev[1].record(stream)
-        B.compress_chunks(d, kv, ids, bits, buf, meta, ws)
+        # score -> (scores to the host, ranking: a host step) -> levels -> records, as one library call;
+        # the event sits behind the score kernels and the copy of the scores
+        B.compress_context(d, kv, q_win, W, frac_a, levels_a, scores, scores_host, bits, buf, meta, ws_tol, ws,
+                           after_scores=ev[1] if ev else None)
         if ev:
             ev[2].record(stream)
         stream.synchronize()                     # the records' checksums reach the host-side meta here
@@ -308,6 +309,8 @@ def run_ours(args):
 
     sampler = ClockSampler(local_rank) if rank == 0 else None
     events = [[torch.cuda.Event(enable_timing=True) for _ in range(4)] for _ in range(args.steps)]
+    for e in events:
+        e[1].record(stream)                      # the library records this one: give it its handle first
     barrier()
     if sampler:
         sampler.begin()

@@ -228,6 +228,26 @@ int llms_optimize_thresholds_levels(const float *scores, int n, float ratio_glob
  * value is their count, or a negative status. */
 int llms_lctru_order(const llms_chunk_state *table, int n, uint32_t *order_out);
 
+/* ------------------------------------------------------------------ a whole context in one call */
+
+/* The compression half of swapping a context out (Sec. 3.2, "Compressing chunks": density of every
+ * chunk, its rank, its level, then quantization) as one call: llms_chunk_tolerance on K and the query
+ * window, the scores copied to the host, llms_assign_levels, then llms_compress_chunks over all chunks
+ * in index order (chunk_ids 0 .. n-1).  Results are those of the three calls made one after the other;
+ * what this call saves is the host time between them, during which the stream would sit empty.
+ * The ranking is a host step: the call synchronises `stream` once, after the scores' copy.
+ *   scores_dev   device fp32 [n_chunks];  scores_host  host fp32 [n_chunks] (pinned for a truly asynchronous copy)
+ *   bits_out     host, n_chunks bytes: the level each chunk got
+ *   after_scores optional cudaEvent_t, recorded on `stream` behind the score kernels and the scores' copy
+ *   everything else as in the three calls. */
+int llms_compress_context(const llms_kv_desc *desc, const void *kv, const void *q_win, int W,
+                          const float frac[3], const uint8_t levels[3],
+                          float *scores_dev, float *scores_host, uint8_t *bits_out,
+                          void *out_buf, uint64_t out_bytes, llms_chunk_meta *meta,
+                          void *tolerance_workspace, uint64_t tolerance_workspace_bytes,
+                          void *codec_workspace, uint64_t codec_workspace_bytes,
+                          void *after_scores, void *stream);
+
 /* ------------------------------------------------------------------ swap copies */
 
 /* Copy n records between a device swap buffer and a pinned host arena on `side_stream`

@@ -62,6 +62,9 @@ _SIGNATURES = {
     "llms_assign_levels": (C.c_int, [C.c_void_p, C.c_int, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]),
     "llms_optimize_thresholds": (C.c_int, [C.c_void_p, C.c_int, C.c_float, C.c_void_p]),
     "llms_optimize_thresholds_levels": (C.c_int, [C.c_void_p, C.c_int, C.c_float, C.c_void_p, C.c_void_p]),
+    "llms_compress_context": (C.c_int, [C.c_void_p, C.c_void_p, C.c_void_p, C.c_int, C.c_void_p, C.c_void_p, C.c_void_p,
+                                        C.c_void_p, C.c_void_p, C.c_void_p, C.c_uint64, C.c_void_p, C.c_void_p, C.c_uint64,
+                                        C.c_void_p, C.c_uint64, C.c_void_p, C.c_void_p]),
     "llms_lctru_order": (C.c_int, [C.c_void_p, C.c_int, C.c_void_p]),
     "llms_swap_out": (C.c_int, [C.c_void_p, C.c_void_p, C.c_int, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p,
                                 C.c_void_p]),
@@ -296,6 +299,19 @@ def lctru_order(table):
     order = np.empty(max(len(t), 1), dtype=np.uint32)
     m = _check(lib().llms_lctru_order(_ptr(t), len(t), _ptr(order)), "llms_lctru_order")
     return order[:m].copy()
+
+
+# ----------------------------------------------------------------------------- a whole context
+
+def compress_context(desc, kv, q_win, W, frac, levels, scores_dev, scores_host, bits_out, out_buf, meta,
+                     tolerance_workspace, codec_workspace, after_scores=None, stream=None):
+    """llms_compress_context: scores, levels and records of every chunk in one call (synchronises the stream once).
+    frac: float32[3], levels: uint8[3], bits_out: uint8[n_chunks] numpy arrays; scores_host: pinned fp32 tensor."""
+    assert frac.dtype == np.float32 and levels.dtype == np.uint8 and bits_out.dtype == np.uint8
+    _check(lib().llms_compress_context(
+        C.addressof(desc), _ptr(kv), _ptr(q_win), int(W), _ptr(frac), _ptr(levels), _ptr(scores_dev), _ptr(scores_host),
+        _ptr(bits_out), _ptr(out_buf), _nbytes(out_buf), _ptr(meta), _ptr(tolerance_workspace), _nbytes(tolerance_workspace),
+        _ptr(codec_workspace), _nbytes(codec_workspace), _event(after_scores), _stream(stream)), "llms_compress_context")
 
 
 # ----------------------------------------------------------------------------- swap

@@ -1093,27 +1093,30 @@ extern "C" int llms_compress_chunks(const llms_kv_desc *desc, const void *kv, co
     if (!aligned(kv, 16) || !aligned(out_buf, 256)) return LLMS_ERR_MISALIGNED;
     const uint32_t nc = (uint32_t)n_chunks(*desc);
     std::vector<uint8_t> seen(nc, 0);
+    uint64_t bytes_at[9] = {0};  // record size per bit-width, looked up once each
     uint64_t off = 0;
     for (int i = 0; i < n; ++i) {
-        uint64_t nb;
-        rc = llms_record_bytes(desc, bits[i], &nb);
-        if (rc) return rc;
+        const uint8_t b = bits[i];
+        if (b > 8) return LLMS_ERR_BAD_BITS;
+        if (bytes_at[b] == 0) {
+            rc = llms_record_bytes(desc, b, &bytes_at[b]);
+            if (rc) return rc;
+        }
         if (chunk_ids[i] >= nc || seen[chunk_ids[i]]) return LLMS_ERR_INVALID_ARG;
         seen[chunk_ids[i]] = 1;
-        off += nb;
+        off += bytes_at[b];
     }
     if (off > out_bytes) return LLMS_ERR_BUF_TOO_SMALL;
+    const uint32_t n_groups = (uint32_t)groups_per_chunk(*desc);
     off = 0;
     for (int i = 0; i < n; ++i) {
-        uint64_t nb;
-        llms_record_bytes(desc, bits[i], &nb);
         meta[i].chunk_id = chunk_ids[i];
         meta[i].bits = bits[i];
         meta[i].offset = off;
-        meta[i].nbytes = nb;
-        meta[i].n_groups = (uint32_t)groups_per_chunk(*desc);
+        meta[i].nbytes = bytes_at[bits[i]];
+        meta[i].n_groups = n_groups;
         meta[i].checksum = 0;  // the kernel accumulates into the device copy
-        off += nb;
+        off += bytes_at[bits[i]];
     }
     CodecArgs a{};
     const bool wide = wide_ok(*desc, kv);
@@ -1177,11 +1180,16 @@ extern "C" int llms_decompress_chunks(const llms_kv_desc *desc, const void *buf,
     const uint32_t nc = (uint32_t)n_chunks(*desc);
     std::vector<uint8_t> seen(nc, 0);
     std::vector<llms_chunk_meta> staged(meta, meta + n);
+    uint64_t bytes_at[9] = {0};  // record size per bit-width, looked up once each
+    const uint32_t n_groups = (uint32_t)groups_per_chunk(*desc);
     for (int i = 0; i < n; ++i) {
-        uint64_t nb;
-        rc = llms_record_bytes(desc, (int)meta[i].bits, &nb);
-        if (rc) return rc;
-        if (meta[i].nbytes != nb || meta[i].n_groups != (uint32_t)groups_per_chunk(*desc)) return LLMS_ERR_INVALID_ARG;
+        const uint32_t b = meta[i].bits;
+        if (b > 8) return LLMS_ERR_BAD_BITS;
+        if (bytes_at[b] == 0) {
+            rc = llms_record_bytes(desc, (int)b, &bytes_at[b]);
+            if (rc) return rc;
+        }
+        if (meta[i].nbytes != bytes_at[b] || meta[i].n_groups != n_groups) return LLMS_ERR_INVALID_ARG;
         if (meta[i].offset % 256) return LLMS_ERR_MISALIGNED;
         const uint32_t dst = dst_chunk_ids ? dst_chunk_ids[i] : meta[i].chunk_id;
         if (dst >= nc || seen[dst]) return LLMS_ERR_INVALID_ARG;

@@ -100,3 +100,29 @@ extern "C" int llms_lctru_order(const llms_chunk_state *table, int n, uint32_t *
     });
     return m;
 }
+
+// Score -> levels -> records for all chunks of a context: the three calls a swap-out makes, without the host
+// round trips between them.
+extern "C" int llms_compress_context(const llms_kv_desc *desc, const void *kv, const void *q_win, int W,
+                                     const float frac[3], const uint8_t levels[3],
+                                     float *scores_dev, float *scores_host, uint8_t *bits_out,
+                                     void *out_buf, uint64_t out_bytes, llms_chunk_meta *meta,
+                                     void *tolerance_workspace, uint64_t tolerance_workspace_bytes,
+                                     void *codec_workspace, uint64_t codec_workspace_bytes,
+                                     void *after_scores, void *stream)
+{
+    if (!desc || !scores_dev || !scores_host || !bits_out) return LLMS_ERR_INVALID_ARG;
+    int rc = llms_chunk_tolerance(desc, kv, q_win, W, scores_dev, tolerance_workspace, tolerance_workspace_bytes, stream);
+    if (rc) return rc;
+    const int n = (int)llms::n_chunks(*desc);
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    LLMS_CUDA_TRY(cudaMemcpyAsync(scores_host, scores_dev, (size_t)n * sizeof(float), cudaMemcpyDeviceToHost, st));
+    if (after_scores) LLMS_CUDA_TRY(cudaEventRecord(static_cast<cudaEvent_t>(after_scores), st));
+    LLMS_CUDA_TRY(cudaStreamSynchronize(st));
+    rc = llms_assign_levels(scores_host, n, frac, levels, bits_out, nullptr);
+    if (rc) return rc;
+    std::vector<uint32_t> ids(n);
+    std::iota(ids.begin(), ids.end(), 0u);
+    return llms_compress_chunks(desc, kv, ids.data(), bits_out, n, out_buf, out_bytes, meta, codec_workspace,
+                                codec_workspace_bytes, stream);
+}

@@ -1,0 +1,70 @@
+"""llms_compress_context (scores, levels and records of a whole context in one call): the same bytes as the
+three calls made one after the other, and as the oracle run on the scores the GPU produced."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2403_11805_b200 import binding as B, synth
+from gpu_helpers import assert_meta_equal, bits_view, first_mismatch, odesc
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.mark.parametrize("levels,frac", [((8, 4, 2), (1 / 3, 1 / 3, 1 / 3)), ((4, 2, 1), (0.2, 0.5, 0.3))])
+def test_compress_context_equals_the_separate_calls_and_the_oracle(levels, frac):
+    sh = synth.KVShape("ctx", 3, 2, 4, 64, 208, 16, 64, seed=13)          # 13 chunks, GQA
+    W = sh.window
+    kv, q = synth.kv_tensor(sh), synth.q_window(sh, W)
+    kv_dev, q_dev = kv.cuda(), q.cuda()
+    d = B.desc_of(sh)
+    n = sh.n_chunks
+    frac_a, levels_a = np.asarray(frac, dtype=np.float32), np.asarray(levels, dtype=np.uint8)
+
+    # one call
+    scores_dev = torch.empty(n, dtype=torch.float32, device="cuda")
+    scores_host = torch.empty(n, dtype=torch.float32).pin_memory()
+    bits = np.zeros(n, dtype=np.uint8)
+    total = B.compressed_size(d, np.full(n, levels[0], np.uint8))
+    buf = torch.zeros(total, dtype=torch.uint8, device="cuda")
+    meta = B.new_meta(n, pinned=True)
+    ws_t = torch.empty(B.tolerance_workspace_bytes(d, W), dtype=torch.uint8, device="cuda")
+    ws_c = torch.empty(B.codec_workspace_bytes(n), dtype=torch.uint8, device="cuda")
+    before, after = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    after.record()                                                        # creates the handle the library records
+    torch.cuda.synchronize()
+    before.record()
+    B.compress_context(d, kv_dev, q_dev, W, frac_a, levels_a, scores_dev, scores_host, bits, buf, meta, ws_t, ws_c,
+                       after_scores=after)
+    torch.cuda.synchronize()
+    assert before.elapsed_time(after) > 0                                 # recorded behind the score kernels
+
+    # the three calls
+    scores2 = torch.empty(n, dtype=torch.float32, device="cuda")
+    B.chunk_tolerance(d, kv_dev, q_dev, W, scores2, ws_t)
+    s2 = scores2.cpu().numpy()
+    assert np.array_equal(s2, scores_host.numpy())                        # scores are reproducible bit for bit
+    bits2, _ = B.assign_levels(s2, frac, levels)
+    assert np.array_equal(bits, bits2)
+    buf2 = torch.zeros(total, dtype=torch.uint8, device="cuda")
+    meta2 = B.new_meta(n, pinned=True)
+    B.compress_chunks(d, kv_dev, np.arange(n, dtype=np.uint32), bits2, buf2, meta2, ws_c)
+    torch.cuda.synchronize()
+    used = int(meta["offset"][-1] + meta["nbytes"][-1])
+    assert torch.equal(buf[:used], buf2[:used])
+    assert_meta_equal(meta, meta2)
+
+    # the oracle, on the GPU's scores (fp32 scores can flip near-ties against fp64 ones)
+    obits, _ = oracle.assign_levels(s2, frac, levels)
+    assert np.array_equal(bits, obits)
+    want_buf, want_meta = oracle.compress_chunks(odesc(sh), bits_view(kv), np.arange(n), obits)
+    assert first_mismatch(buf[:used].cpu().numpy(), want_buf) is None
+    assert_meta_equal(meta, want_meta)
+
+
+def test_compress_context_argument_errors():
+    sh = synth.CONFIGS["tiny"]
+    d = B.desc_of(sh)
+    rc = B.lib().llms_compress_context(None, None, None, 8, None, None, None, None, None, None, 0, None, None, 0, None, 0,
+                                       None, None)
+    assert rc == B.ERR_INVALID_ARG
