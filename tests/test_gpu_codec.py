@@ -156,6 +156,17 @@ def test_one_bit_special_values():
     check_decompress(sh, kv, buf_dev, meta, want_buf)
 
 
+def test_more_chunks_in_a_launch_than_checksum_slots():
+    """Above 1024 chunks of one bit-width a launch adds its checksums straight to global memory."""
+    sh = synth.KVShape("many", 1, 2, 2, 64, 2 * 1300, 2, 64, seed=23)      # 1300 chunks of 2 tokens
+    kv = synth.kv_tensor(sh)
+    ids = np.arange(sh.n_chunks)
+    bits = np.full(sh.n_chunks, 4, dtype=np.uint8)
+    bits[::50] = 8
+    kv_dev, buf_dev, meta, want_buf = check_compress(sh, kv, ids, bits)
+    check_decompress(sh, kv, buf_dev, meta, want_buf)
+
+
 def test_padding_is_written_and_compared():
     # 2 slabs * 3 tokens * 1 group = 6 groups -> 24 parameter bytes -> 8 zero bytes before the codes,
     # and 144/288 code bytes -> tail padding up to 256/512
