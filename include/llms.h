@@ -158,7 +158,12 @@ int llms_compress_chunks_static(const llms_kv_desc *desc, const void *kv, const 
  * are not touched.  While decoding, each record's checksum is recomputed; the number of
  * records whose sum differs from meta[i].checksum is left in the workspace and can be read
  * with llms_codec_corrupt_count (decoded values of such a record are still written).
- *   buf        device, 256-byte aligned;  meta, dst_chunk_ids  host;  kv_out  device fp16 */
+ *   buf        device, 256-byte aligned;  meta, dst_chunk_ids  host;  kv_out  device fp16
+ * Sizes, offsets and bit-widths are read from meta when the call is made.  The expected checksums are too,
+ * unless meta lies in page-locked (pinned) host memory: then the device reads meta[i].checksum itself, when
+ * the check runs on `stream`.  A decompress call may therefore follow, on the same stream and without a
+ * synchronisation in between, the llms_compress_chunks call that is still producing those checksums into
+ * the same pinned array; the host must neither free nor change the array until the stream has passed the call. */
 int llms_decompress_chunks(const llms_kv_desc *desc, const void *buf, const llms_chunk_meta *meta,
                            const uint32_t *dst_chunk_ids, int n, void *kv_out,
                            void *workspace, uint64_t workspace_bytes, void *stream);

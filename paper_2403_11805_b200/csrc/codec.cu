@@ -857,11 +857,15 @@ __global__ void __launch_bounds__(kThreads, kDecodeBlocksPerSm) decompress_kerne
 
 namespace llms {
 
-// status word = number of records whose recomputed sum differs from the expected one
-__global__ void verify_kernel(const ChunkEntry *entries, const uint32_t *sums, int n, uint32_t *status)
+// status word = number of records whose recomputed sum differs from the expected one.  live_meta: the caller's
+// meta array when it lies in page-locked host memory the device can read (the expected sums are then taken now, in
+// stream order, not when the call was made); else NULL and the copies uploaded with the call are used.
+__global__ void verify_kernel(const ChunkEntry *entries, const uint32_t *sums, int n, uint32_t *status,
+                              const llms_chunk_meta *live_meta)
 {
     uint32_t bad = 0;
-    for (int i = threadIdx.x; i < n; i += blockDim.x) bad += (sums[i] != entries[i].checksum);
+    for (int i = threadIdx.x; i < n; i += blockDim.x)
+        bad += (sums[i] != (live_meta ? *reinterpret_cast<const volatile uint32_t *>(&live_meta[i].checksum) : entries[i].checksum));
     bad = __reduce_add_sync(0xffffffffu, bad);
     if ((threadIdx.x & 31) == 0 && bad) atomicAdd(status, bad);
 }
@@ -1229,7 +1233,16 @@ extern "C" int llms_decompress_chunks(const llms_kv_desc *desc, const void *buf,
         if (rc) return rc;
         LLMS_CUDA_TRY(cudaGetLastError());
     }
-    verify_kernel<<<1, 256, 0, st>>>(a.entries, a.sums, n, status);
+    // expected sums in stream order when the device can read the caller's meta (see llms.h)
+    const llms_chunk_meta *live_meta = nullptr;
+    {
+        cudaPointerAttributes attr;
+        if (cudaPointerGetAttributes(&attr, meta) == cudaSuccess && attr.type == cudaMemoryTypeHost && attr.devicePointer)
+            live_meta = static_cast<const llms_chunk_meta *>(attr.devicePointer);
+        else
+            cudaGetLastError();
+    }
+    verify_kernel<<<1, 256, 0, st>>>(a.entries, a.sums, n, status, live_meta);
     LLMS_CUDA_TRY(cudaGetLastError());
     return LLMS_OK;
 }

@@ -234,6 +234,41 @@ def test_corrupted_record_is_reported():
     assert B.lib().llms_codec_corrupt_count(ws.data_ptr(), None, torch.cuda.current_stream().cuda_stream) == B.ERR_CORRUPT
 
 
+def test_pinned_meta_gives_stream_ordered_checksums():
+    """With meta in pinned host memory the expected checksums are read by the device when the check runs: the decode
+    call may follow the encode call on the same stream with no synchronisation in between."""
+    sh = synth.CONFIGS["gemma2b"].with_(n_layers=4)
+    kv = synth.kv_tensor(sh)
+    kv_dev = kv.cuda()
+    d = B.desc_of(sh)
+    n = sh.n_chunks
+    ids = np.arange(n, dtype=np.uint32)
+    bits = np.array([(8, 4, 2, 1)[i % 4] for i in range(n)], dtype=np.uint8)
+    buf = torch.empty(B.compressed_size(d, bits), dtype=torch.uint8, device="cuda")
+    ws_c = torch.empty(B.codec_workspace_bytes(n), dtype=torch.uint8, device="cuda")
+    ws_d = torch.empty(B.codec_workspace_bytes(n), dtype=torch.uint8, device="cuda")
+    meta = B.new_meta(n, pinned=True)
+    out = torch.full(kv.shape, float("nan"), dtype=torch.float16, device="cuda")
+    for _ in range(3):                                   # checksums of the call before never stand in: meta is zeroed
+        meta["checksum"] = 0
+        B.compress_chunks(d, kv_dev, ids, bits, buf, meta, ws_c)
+        B.decompress_chunks(d, buf, meta, None, out, ws_d)     # no synchronisation: the checksums are still on their way
+        assert B.codec_corrupt_count(ws_d) == 0
+    want_buf, want_meta = oracle.compress_chunks(odesc(sh), bits_view(kv), ids, bits)
+    assert_meta_equal(meta, want_meta)
+    want = np.zeros(kv.numel(), dtype=np.uint16).reshape(kv.shape)
+    oracle.decompress_chunks(odesc(sh), want_buf, want_meta, want)
+    assert first_mismatch(bits_view(out).reshape(-1), want.reshape(-1)) is None
+    # a wrong expectation in the pinned array is reported, and so is a damaged record
+    meta["checksum"][5] ^= 1
+    B.decompress_chunks(d, buf, meta, None, out, ws_d)
+    assert B.codec_corrupt_count(ws_d) == 1
+    meta["checksum"][5] ^= 1
+    buf[int(meta[7]["offset"]) + 1000] ^= 0x04
+    B.decompress_chunks(d, buf, meta, None, out, ws_d)
+    assert B.codec_corrupt_count(ws_d) == 1
+
+
 def test_recompression_is_stable():
     # decode(encode(x)) encoded again at the same width gives the same codes whenever the scale is unchanged
     sh = synth.CONFIGS["tiny"]
