@@ -290,7 +290,7 @@ def run_ours(args):
         if ev:
             ev[2].record(stream)
         # meta is pinned: the expected checksums are read by the device in stream order, no synchronisation here
-        B.decompress_chunks(d, buf, meta, None, kv_out, ws_dec)
+        B.decompress_chunks_ordered(d, buf, meta, None, kv_out, ws_dec)
         if ev:
             ev[3].record(stream)
         state["bits"] = bits

@@ -159,14 +159,20 @@ int llms_compress_chunks_static(const llms_kv_desc *desc, const void *kv, const 
  * records whose sum differs from meta[i].checksum is left in the workspace and can be read
  * with llms_codec_corrupt_count (decoded values of such a record are still written).
  *   buf        device, 256-byte aligned;  meta, dst_chunk_ids  host;  kv_out  device fp16
- * Sizes, offsets and bit-widths are read from meta when the call is made.  The expected checksums are too,
- * unless meta lies in page-locked (pinned) host memory: then the device reads meta[i].checksum itself, when
- * the check runs on `stream`.  A decompress call may therefore follow, on the same stream and without a
- * synchronisation in between, the llms_compress_chunks call that is still producing those checksums into
- * the same pinned array; the host must neither free nor change the array until the stream has passed the call. */
+ * Everything in meta, the expected checksums included, is read when the call is made. */
 int llms_decompress_chunks(const llms_kv_desc *desc, const void *buf, const llms_chunk_meta *meta,
                            const uint32_t *dst_chunk_ids, int n, void *kv_out,
                            void *workspace, uint64_t workspace_bytes, void *stream);
+
+/* The same with the expected checksums taken in stream order: meta must lie in page-locked (pinned) host
+ * memory (else LLMS_ERR_INVALID_ARG); sizes, offsets and bit-widths are read when the call is made, but
+ * meta[i].checksum is read by the device itself when the check runs on `stream`.  Such a call may follow,
+ * on the same stream and without a synchronisation in between, the llms_compress_chunks call that is still
+ * producing those checksums into the same array.  The host must neither free nor change the array (a new
+ * llms_compress_chunks into it changes it) until the stream has passed this call. */
+int llms_decompress_chunks_ordered(const llms_kv_desc *desc, const void *buf, const llms_chunk_meta *meta,
+                                   const uint32_t *dst_chunk_ids, int n, void *kv_out,
+                                   void *workspace, uint64_t workspace_bytes, void *stream);
 
 /* Synchronises `stream`, then reports on the last llms_compress_chunks or llms_decompress_chunks
  * that used this workspace: LLMS_ERR_TIMEOUT if one of its kernels abandoned a bounded wait for a

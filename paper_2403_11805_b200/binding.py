@@ -52,6 +52,8 @@ _SIGNATURES = {
                                               C.c_uint64, C.c_void_p, C.c_void_p]),
     "llms_decompress_chunks": (C.c_int, [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_int, C.c_void_p,
                                          C.c_void_p, C.c_uint64, C.c_void_p]),
+    "llms_decompress_chunks_ordered": (C.c_int, [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_int, C.c_void_p,
+                                         C.c_void_p, C.c_uint64, C.c_void_p]),
     "llms_codec_corrupt_count": (C.c_int, [C.c_void_p, C.c_void_p, C.c_void_p]),
     "llms_tolerance_workspace_bytes": (C.c_int, [C.c_void_p, C.c_int, C.c_void_p]),
     "llms_chunk_tolerance": (C.c_int, [C.c_void_p, C.c_void_p, C.c_void_p, C.c_int, C.c_void_p, C.c_void_p,
@@ -231,6 +233,15 @@ def decompress_chunks(desc, buf, meta, dst_chunk_ids, kv_out, workspace, stream=
     _check(lib().llms_decompress_chunks(
         C.addressof(desc), _ptr(buf), _ptr(meta), _ptr(ids), n, _ptr(kv_out), _ptr(workspace),
         _nbytes(workspace) if workspace_bytes is None else workspace_bytes, _stream(stream)), "llms_decompress_chunks")
+
+
+def decompress_chunks_ordered(desc, buf, meta, dst_chunk_ids, kv_out, workspace, stream=None, n=None, workspace_bytes=None):
+    """llms_decompress_chunks_ordered: meta pinned; its checksums are read by the device in stream order."""
+    ids = None if dst_chunk_ids is None else np.ascontiguousarray(dst_chunk_ids, dtype=np.uint32)
+    n = len(meta) if n is None else n
+    _check(lib().llms_decompress_chunks_ordered(
+        C.addressof(desc), _ptr(buf), _ptr(meta), _ptr(ids), n, _ptr(kv_out), _ptr(workspace),
+        _nbytes(workspace) if workspace_bytes is None else workspace_bytes, _stream(stream)), "llms_decompress_chunks_ordered")
 
 
 def codec_corrupt_count(workspace, stream=None):

@@ -1172,15 +1172,25 @@ extern "C" int llms_compress_chunks(const llms_kv_desc *desc, const void *kv, co
     return LLMS_OK;
 }
 
-extern "C" int llms_decompress_chunks(const llms_kv_desc *desc, const void *buf, const llms_chunk_meta *meta,
-                                      const uint32_t *dst_chunk_ids, int n, void *kv_out,
-                                      void *workspace, uint64_t workspace_bytes, void *stream)
+// live_checksums: the expected sums are read from the caller's pinned meta array by the device, in stream order
+static int decompress_chunks(const llms_kv_desc *desc, const void *buf, const llms_chunk_meta *meta,
+                             const uint32_t *dst_chunk_ids, int n, void *kv_out, void *workspace,
+                             uint64_t workspace_bytes, void *stream, bool live_checksums)
 {
     int rc = check_common(desc, n, workspace, workspace_bytes);
     if (rc) return rc;
     if (n == 0) return LLMS_OK;
     if (!buf || !meta || !kv_out) return LLMS_ERR_INVALID_ARG;
     if (!aligned(kv_out, 16) || !aligned(buf, 256)) return LLMS_ERR_MISALIGNED;
+    const llms_chunk_meta *live_meta = nullptr;
+    if (live_checksums) {  // only page-locked host memory is visible to the device
+        cudaPointerAttributes attr;
+        if (cudaPointerGetAttributes(&attr, meta) != cudaSuccess || attr.type != cudaMemoryTypeHost || !attr.devicePointer) {
+            cudaGetLastError();
+            return LLMS_ERR_INVALID_ARG;
+        }
+        live_meta = static_cast<const llms_chunk_meta *>(attr.devicePointer);
+    }
     const uint32_t nc = (uint32_t)n_chunks(*desc);
     std::vector<uint8_t> seen(nc, 0);
     std::vector<llms_chunk_meta> staged(meta, meta + n);
@@ -1233,18 +1243,23 @@ extern "C" int llms_decompress_chunks(const llms_kv_desc *desc, const void *buf,
         if (rc) return rc;
         LLMS_CUDA_TRY(cudaGetLastError());
     }
-    // expected sums in stream order when the device can read the caller's meta (see llms.h)
-    const llms_chunk_meta *live_meta = nullptr;
-    {
-        cudaPointerAttributes attr;
-        if (cudaPointerGetAttributes(&attr, meta) == cudaSuccess && attr.type == cudaMemoryTypeHost && attr.devicePointer)
-            live_meta = static_cast<const llms_chunk_meta *>(attr.devicePointer);
-        else
-            cudaGetLastError();
-    }
     verify_kernel<<<1, 256, 0, st>>>(a.entries, a.sums, n, status, live_meta);
     LLMS_CUDA_TRY(cudaGetLastError());
     return LLMS_OK;
+}
+
+extern "C" int llms_decompress_chunks(const llms_kv_desc *desc, const void *buf, const llms_chunk_meta *meta,
+                                      const uint32_t *dst_chunk_ids, int n, void *kv_out,
+                                      void *workspace, uint64_t workspace_bytes, void *stream)
+{
+    return decompress_chunks(desc, buf, meta, dst_chunk_ids, n, kv_out, workspace, workspace_bytes, stream, false);
+}
+
+extern "C" int llms_decompress_chunks_ordered(const llms_kv_desc *desc, const void *buf, const llms_chunk_meta *meta,
+                                              const uint32_t *dst_chunk_ids, int n, void *kv_out,
+                                              void *workspace, uint64_t workspace_bytes, void *stream)
+{
+    return decompress_chunks(desc, buf, meta, dst_chunk_ids, n, kv_out, workspace, workspace_bytes, stream, true);
 }
 
 extern "C" int llms_codec_corrupt_count(const void *workspace, uint32_t *n_corrupt, void *stream)

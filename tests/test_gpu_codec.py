@@ -235,8 +235,8 @@ def test_corrupted_record_is_reported():
 
 
 def test_pinned_meta_gives_stream_ordered_checksums():
-    """With meta in pinned host memory the expected checksums are read by the device when the check runs: the decode
-    call may follow the encode call on the same stream with no synchronisation in between."""
+    """llms_decompress_chunks_ordered: the expected checksums are read from the pinned meta by the device when the
+    check runs, so the decode call may follow the encode call on the same stream with no synchronisation in between."""
     sh = synth.CONFIGS["gemma2b"].with_(n_layers=4)
     kv = synth.kv_tensor(sh)
     kv_dev = kv.cuda()
@@ -252,7 +252,7 @@ def test_pinned_meta_gives_stream_ordered_checksums():
     for _ in range(3):                                   # checksums of the call before never stand in: meta is zeroed
         meta["checksum"] = 0
         B.compress_chunks(d, kv_dev, ids, bits, buf, meta, ws_c)
-        B.decompress_chunks(d, buf, meta, None, out, ws_d)     # no synchronisation: the checksums are still on their way
+        B.decompress_chunks_ordered(d, buf, meta, None, out, ws_d)     # no synchronisation: the checksums are still on their way
         assert B.codec_corrupt_count(ws_d) == 0
     want_buf, want_meta = oracle.compress_chunks(odesc(sh), bits_view(kv), ids, bits)
     assert_meta_equal(meta, want_meta)
@@ -261,12 +261,15 @@ def test_pinned_meta_gives_stream_ordered_checksums():
     assert first_mismatch(bits_view(out).reshape(-1), want.reshape(-1)) is None
     # a wrong expectation in the pinned array is reported, and so is a damaged record
     meta["checksum"][5] ^= 1
-    B.decompress_chunks(d, buf, meta, None, out, ws_d)
+    B.decompress_chunks_ordered(d, buf, meta, None, out, ws_d)
     assert B.codec_corrupt_count(ws_d) == 1
     meta["checksum"][5] ^= 1
     buf[int(meta[7]["offset"]) + 1000] ^= 0x04
-    B.decompress_chunks(d, buf, meta, None, out, ws_d)
+    B.decompress_chunks_ordered(d, buf, meta, None, out, ws_d)
     assert B.codec_corrupt_count(ws_d) == 1
+    with pytest.raises(B.LlmsError) as e:                # pageable meta is refused: the device could not read it
+        B.decompress_chunks_ordered(d, buf, meta.copy(), None, out, ws_d)
+    assert e.value.status == B.ERR_INVALID_ARG
 
 
 def test_recompression_is_stable():
