@@ -511,7 +511,8 @@ def run_multiapp(args):
     sampler.begin()
     t0 = time.perf_counter()
     for _ in range(steps):
-        app.step(per_step)              # ends with a device synchronisation
+        app.step(per_step)              # ends with a device synchronisation (an ahead-of-time write-back runs on)
+    app.finish()
     dt = time.perf_counter() - t0
     sampler.end()
     clocks = sampler.finish()

@@ -123,9 +123,10 @@ int llms_codec_workspace_bytes(int n, uint64_t *nbytes);
  *   out_buf    device, 256-byte aligned, out_bytes >= llms_compressed_size(...); every byte of
  *              every record, padding included, is written
  *   meta       host, n entries, filled before return except `checksum`, which the device
- *              computes: it is copied back into meta[] in stream order, so it is valid once the
- *              stream has been synchronised (pass pinned memory to keep that copy asynchronous;
- *              with pageable memory the call may block until the kernel is done)
+ *              computes: it reaches meta[] in stream order, so it is valid once the stream has
+ *              been synchronised.  Into pinned (page-locked) memory a kernel stores it, which
+ *              neither blocks the call nor waits for copies other streams have in flight; into
+ *              pageable memory it is copied, and the call may block until the kernel is done
  *   workspace  device, 16-byte aligned, llms_codec_workspace_bytes(n); may be reused by the
  *              next call on the same stream
  * n == 0 is valid and does nothing. */

@@ -870,6 +870,25 @@ __global__ void verify_kernel(const ChunkEntry *entries, const uint32_t *sums, i
     if ((threadIdx.x & 31) == 0 && bad) atomicAdd(status, bad);
 }
 
+// The finished checksums, stored by the device into the caller's page-locked meta array.  A device-to-host copy
+// would do the same, but it queues on the copy engine behind whatever bulk copies other streams have in flight
+// (measured in the multi-app driver: the encoder's stream then advances at the pace of the swap-out copies).
+__global__ void publish_checksums_kernel(const ChunkEntry *entries, llms_chunk_meta *live_meta, int n)
+{
+    for (int i = blockIdx.x * blockDim.x + threadIdx.x; i < n; i += gridDim.x * blockDim.x)
+        live_meta[i].checksum = entries[i].checksum;
+}
+
+// The device's view of a host pointer if it is page-locked memory the device can access, else NULL.
+static void *device_view_of_pinned(const void *host_ptr)
+{
+    cudaPointerAttributes attr;
+    if (cudaPointerGetAttributes(&attr, host_ptr) == cudaSuccess && attr.type == cudaMemoryTypeHost && attr.devicePointer)
+        return attr.devicePointer;
+    cudaGetLastError();
+    return nullptr;
+}
+
 // ---------------------------------------------------------------------------------------------- host side
 
 static int fill_args(const llms_kv_desc &d, CodecArgs &a, int n, void *workspace, bool wide)
@@ -1168,7 +1187,13 @@ extern "C" int llms_compress_chunks(const llms_kv_desc *desc, const void *kv, co
         LLMS_CUDA_TRY(attr_err);
         LLMS_CUDA_TRY(cudaGetLastError());
     }
-    LLMS_CUDA_TRY(cudaMemcpyAsync(meta, a.entries, (size_t)n * sizeof(ChunkEntry), cudaMemcpyDeviceToHost, st));
+    // checksums back to the caller's meta (every other field is already there)
+    if (void *live = device_view_of_pinned(meta)) {
+        publish_checksums_kernel<<<(n + 255) / 256, 256, 0, st>>>(a.entries, static_cast<llms_chunk_meta *>(live), n);
+        LLMS_CUDA_TRY(cudaGetLastError());
+    } else {
+        LLMS_CUDA_TRY(cudaMemcpyAsync(meta, a.entries, (size_t)n * sizeof(ChunkEntry), cudaMemcpyDeviceToHost, st));
+    }
     return LLMS_OK;
 }
 
@@ -1184,12 +1209,8 @@ static int decompress_chunks(const llms_kv_desc *desc, const void *buf, const ll
     if (!aligned(kv_out, 16) || !aligned(buf, 256)) return LLMS_ERR_MISALIGNED;
     const llms_chunk_meta *live_meta = nullptr;
     if (live_checksums) {  // only page-locked host memory is visible to the device
-        cudaPointerAttributes attr;
-        if (cudaPointerGetAttributes(&attr, meta) != cudaSuccess || attr.type != cudaMemoryTypeHost || !attr.devicePointer) {
-            cudaGetLastError();
-            return LLMS_ERR_INVALID_ARG;
-        }
-        live_meta = static_cast<const llms_chunk_meta *>(attr.devicePointer);
+        live_meta = static_cast<const llms_chunk_meta *>(device_view_of_pinned(meta));
+        if (!live_meta) return LLMS_ERR_INVALID_ARG;
     }
     const uint32_t nc = (uint32_t)n_chunks(*desc);
     std::vector<uint8_t> seen(nc, 0);

@@ -46,6 +46,8 @@ class MultiApp:
         self.orders = [] if log_ops else None     # (table copy, order) of every LCTRU query
         self._pending = []                        # (meta, rows) of compress calls whose checksums are not read yet
         self._draw = 0
+        self._aot_rows = None                     # rows whose ahead-of-time write-back may still be in flight
+        self._ev_aot = None                       # recorded on the copy-out stream behind that write-back
         self.bytes_out = self.bytes_in = 0
         self.kernel_launches = 0                  # codec kernels launched (one per bit-width present, plus the checksum check)
 
@@ -91,15 +93,18 @@ class MultiApp:
         if hasattr(self, "arena"):
             return
         worst = self.cpc * self.rec_bytes[8]
-        self.stage_out = [torch.empty(worst, dtype=torch.uint8, device="cuda") for _ in range(2)]
+        # staging buffers on the way out: two take turns; with ahead-of-time swap-out one per context of a step, so
+        # that all of a step's write-back kernels run at once and only their copies stay behind
+        n_out = 8 if self.aot else 2
+        self.stage_out = [torch.empty(worst, dtype=torch.uint8, device="cuda") for _ in range(n_out)]
         self.stage_in = [torch.empty(worst, dtype=torch.uint8, device="cuda") for _ in range(2)]
-        self.ws = [torch.empty(B.codec_workspace_bytes(self.cpc), dtype=torch.uint8, device="cuda") for _ in range(32)]
-        self.metas = [B.new_meta(self.cpc, pinned=True) for _ in range(32)]
+        self.ws = [torch.empty(B.codec_workspace_bytes(self.cpc), dtype=torch.uint8, device="cuda") for _ in range(64)]
+        self.metas = [B.new_meta(self.cpc, pinned=True) for _ in range(64)]
         self._ws_next = 0
         self._used_ws = []
-        self.ev_stage_out_free = [B.new_event() for _ in range(2)]
+        self.ev_stage_out_free = [B.new_event() for _ in range(n_out)]
         self.ev_stage_in_free = [B.new_event() for _ in range(2)]
-        self.ev_compressed = [B.new_event() for _ in range(2)]
+        self.ev_compressed = [B.new_event() for _ in range(n_out)]
         self.ev_landed = [B.new_event() for _ in range(2)]
         self._out_k = self._in_k = 0
         # the arena: every (context, chunk) record at its own offset, bit-widths fixed at set-up by the tertiles
@@ -122,7 +127,7 @@ class MultiApp:
         self._alloc_buffers()
         rows = np.arange(c * self.cpc, (c + 1) * self.cpc)
         ws, meta = self._next_ws()
-        k = self._out_k % 2
+        k = self._out_k % len(self.stage_out)
         self._out_k += 1
         self.main.wait_event(self.ev_stage_out_free[k])
         B.compress_chunks(self.desc_ctx, kv, np.arange(self.cpc, dtype=np.uint32), bits, self.stage_out[k], meta, ws)
@@ -161,7 +166,7 @@ class MultiApp:
             slots = self.slot[part].astype(np.uint32)
             bits = self.table["bits"][part].astype(np.uint8)
             ws, meta = self._next_ws()
-            k = self._out_k % 2
+            k = self._out_k % len(self.stage_out)
             self._out_k += 1
             self.main.wait_event(self.ev_stage_out_free[k])
             B.compress_chunks(self.desc_pool, self.pool, slots, bits, self.stage_out[k], meta, ws)
@@ -182,9 +187,24 @@ class MultiApp:
             else:
                 self.clean[part] = True
 
+    def _settle_write_back(self):
+        """Wait for the ahead-of-time write-back that was left running and take its checksums."""
+        if self._aot_rows is not None:
+            self._ev_aot.synchronize()
+            self._collect_checksums()
+            self._aot_rows = None
+
+    def finish(self):
+        """Everything queued has completed and every checksum is known on the host."""
+        torch.cuda.synchronize()
+        self._collect_checksums()
+        self._aot_rows = None
+
     def _load(self, rows):
         """Load: copy the records of the chunks in `rows` from the arena, unpack + dequantize into free slots."""
         rows = np.asarray(rows)
+        if self._aot_rows is not None and np.isin(rows, self._aot_rows).any():
+            self._settle_write_back()             # a record still on its way out must land before it is read back
         for r0 in range(0, len(rows), self.cpc):
             part = rows[r0:r0 + self.cpc]
             slots = np.array([self.free.pop() for _ in part], dtype=np.uint32)
@@ -265,10 +285,17 @@ class MultiApp:
             self.table["last_access_step"][rows] = self.step_no
         self._ev_ready.record(self.main)                 # the working sets are resident: inference could start
         self.clean[locked_rows] = False                  # a served context counts as modified by its call
-        if self.aot:
-            self._write_back(locked_rows, release=False)
         self.table["locked"][locked_rows] = 0
-        self._end_of_step()
+        self._end_of_step()                              # also settles the write-back left running by the step before
+        self._aot_rows = None
+        if self.aot:
+            # ahead-of-time swap-out when the call returns (Sec. 3.4 i): queued now, left running, so that its
+            # copies out share the link with the next step's copies in
+            self._write_back(locked_rows, release=False)
+            if self._ev_aot is None:
+                self._ev_aot = B.new_event(self.side_out)
+            self._ev_aot.record(self.side_out)
+            self._aot_rows = locked_rows
         self.ready_ms.append(self._ev_t0.elapsed_time(self._ev_ready))
         return ctxs
 
