@@ -473,7 +473,7 @@ def run_ours(args):
                 "serial_ms_per_step": e2e_serial_ms, "batch_chunks": e2e_batch,
                 "what": "compress -> swap-out to pinned host -> swap-in -> decompress, pipelined in batches of chunks",
                 "layerwise_load": layerwise},
-        "gpu_launches": args.steps * 11,   # 4 score kernels, compress and decompress once per bit-width, 1 verify
+        "gpu_launches": args.steps * 12,   # 4 score kernels, compress and decompress once per bit-width, 1 checksum store, 1 verify
         "roofline": roofline, "clocks": clocks,
         "wall_ms_per_step": t_wall * 1e3 / args.steps,
         "step_ms_median_best": [statistics.median(step_ms), step_ms[0]],

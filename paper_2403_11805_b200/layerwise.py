@@ -56,7 +56,7 @@ class LayerwiseContext:
             self.ev_packed[k].record(self.main)
             B.swap_out(self.stage_out[k], self.meta[l], self.layer_arena(l), side_stream=self.side_out,
                        after=self.ev_packed[k], done=self.ev_out_free[k], n=self.n)
-            self.kernel_launches += self._widths
+            self.kernel_launches += self._widths + 1
 
     def swap_in(self, kv_out):
         """Load layer after layer; self.ready[l] is recorded on the main stream when layer l of kv_out is complete.
