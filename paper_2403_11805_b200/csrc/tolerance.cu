@@ -226,7 +226,9 @@ __device__ __forceinline__ void tile_statistics(const TolArgs &a, const float (&
     }
 }
 
-template <int SEG, int D>
+// NBG: n-tiles (8 flattened window rows each) that share one pass over a tile's A fragments - 4 for grouped-query
+// shapes whose rows come in multiples of 32 per KV head, else 1.
+template <int SEG, int D, int NBG>
 __global__ void __launch_bounds__(kTileWarps * 32) logits_mma_kernel(const TolArgs a)
 {
     constexpr int kRowBytes = D * 2, kChunks = D / 8, kTileBytes = kTileTokens * kRowBytes;
@@ -305,28 +307,37 @@ __global__ void __launch_bounds__(kTileWarps * 32) logits_mma_kernel(const TolAr
                 opens[mb][h] = t_tok[mb][h] < a.T && t_tok[mb][h] % SEG == 0;
             }
         const bool tail_tile = tile * kTileTokens + kTileTokens > a.T - a.W + 1;
-        for (int nb = 0; nb < n_blocks; ++nb) {
-            float acc[2][4];
+        for (int nb0 = 0; nb0 < n_blocks; nb0 += NBG) {
+            float acc[NBG][2][4];
 #pragma unroll
-            for (int mb = 0; mb < 2; ++mb)
+            for (int j = 0; j < NBG; ++j)
 #pragma unroll
-                for (int i = 0; i < 4; ++i) acc[mb][i] = 0.0f;
-            const unsigned char *q_row = q_s + (nb * 8 + g) * kQRowBytes + q4 * 4;
+                for (int mb = 0; mb < 2; ++mb)
+#pragma unroll
+                    for (int i = 0; i < 4; ++i) acc[j][mb][i] = 0.0f;
+            const unsigned char *q_row = q_s + (nb0 * 8 + g) * kQRowBytes + q4 * 4;
 #pragma unroll
             for (int ks = 0; ks < D / 16; ++ks) {
-                const uint32_t b0 = *reinterpret_cast<const uint32_t *>(q_row + ks * 32);
-                const uint32_t b1 = *reinterpret_cast<const uint32_t *>(q_row + ks * 32 + 16);
+                uint32_t af[2][4];
 #pragma unroll
                 for (int mb = 0; mb < 2; ++mb) {
                     const int row = mb * 16 + a_row;
-                    uint32_t af[4];
-                    ldmatrix_x4(tile_s + row * kRowBytes + (((2 * ks + a_chunk) ^ (row & 7)) << 4), af);
-                    mma_16816(acc[mb], af, b0, b1);
+                    ldmatrix_x4(tile_s + row * kRowBytes + (((2 * ks + a_chunk) ^ (row & 7)) << 4), af[mb]);
+                }
+#pragma unroll
+                for (int j = 0; j < NBG; ++j) {
+                    const uint32_t b0 = *reinterpret_cast<const uint32_t *>(q_row + j * 8 * kQRowBytes + ks * 32);
+                    const uint32_t b1 = *reinterpret_cast<const uint32_t *>(q_row + j * 8 * kQRowBytes + ks * 32 + 16);
+#pragma unroll
+                    for (int mb = 0; mb < 2; ++mb) mma_16816(acc[j][mb], af[mb], b0, b1);
                 }
             }
-            // acc[mb][0..1]: token mb*16 + g, window rows 2*q4, 2*q4+1;  acc[mb][2..3]: token mb*16 + 8 + g
-            if (tail_tile) tile_statistics<SEG, true>(a, acc, nb, q4, last_col_s, t_tok, w_tok, opens, row0);
-            else tile_statistics<SEG, false>(a, acc, nb, q4, last_col_s, t_tok, w_tok, opens, row0);
+            // acc[j][mb][0..1]: token mb*16 + g, window rows 2*q4, 2*q4+1 of n-tile nb0 + j;  [2..3]: token mb*16 + 8 + g
+#pragma unroll
+            for (int j = 0; j < NBG; ++j) {
+                if (tail_tile) tile_statistics<SEG, true>(a, acc[j], nb0 + j, q4, last_col_s, t_tok, w_tok, opens, row0);
+                else tile_statistics<SEG, false>(a, acc[j], nb0 + j, q4, last_col_s, t_tok, w_tok, opens, row0);
+            }
         }
         __syncwarp();  // the buffer is free for the copy issued two tiles from now
     }
@@ -540,10 +551,15 @@ extern "C" int llms_chunk_tolerance(const llms_kv_desc *desc, const void *kv, co
         int splits = (sm_count() * 6 + pairs - 1) / pairs;
         splits = std::max(1, std::min(splits, (n_tiles + kTileWarps - 1) / kTileWarps));
         const dim3 grid(splits, pairs);
-#define LLMS_LAUNCH_MMA(S, DD)                                                                                                    \
-    do {                                                                                                                          \
-        LLMS_CUDA_TRY(cudaFuncSetAttribute(logits_mma_kernel<S, DD>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)mma_smem)); \
-        logits_mma_kernel<S, DD><<<grid, kTileWarps * 32, mma_smem, st>>>(a);                                                     \
+#define LLMS_LAUNCH_MMA_G(S, DD, G)                                                                                                  \
+    do {                                                                                                                             \
+        LLMS_CUDA_TRY(cudaFuncSetAttribute(logits_mma_kernel<S, DD, G>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)mma_smem)); \
+        logits_mma_kernel<S, DD, G><<<grid, kTileWarps * 32, mma_smem, st>>>(a);                                                     \
+    } while (0)
+#define LLMS_LAUNCH_MMA(S, DD)                                      \
+    do {                                                            \
+        if (((a.NR + 7) / 8) % 4 == 0) LLMS_LAUNCH_MMA_G(S, DD, 4); \
+        else LLMS_LAUNCH_MMA_G(S, DD, 1);                           \
     } while (0)
 #define LLMS_LAUNCH_MMA_SEG(S)                                                      \
     case S:                                                                         \
@@ -562,6 +578,7 @@ extern "C" int llms_chunk_tolerance(const llms_kv_desc *desc, const void *kv, co
         }
 #undef LLMS_LAUNCH_MMA_SEG
 #undef LLMS_LAUNCH_MMA
+#undef LLMS_LAUNCH_MMA_G
     } else {
         const size_t q_bytes = (size_t)a.NR * a.d * sizeof(float);
         if (q_bytes > 200 * 1024) return LLMS_ERR_UNSUPPORTED;
