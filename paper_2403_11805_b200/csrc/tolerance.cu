@@ -229,7 +229,7 @@ __device__ __forceinline__ void tile_statistics(const TolArgs &a, const float (&
 // NBG: n-tiles (8 flattened window rows each) that share one pass over a tile's A fragments - 4 for grouped-query
 // shapes whose rows come in multiples of 32 per KV head, else 1.
 template <int SEG, int D, int NBG>
-__global__ void __launch_bounds__(kTileWarps * 32) logits_mma_kernel(const TolArgs a)
+__global__ void __launch_bounds__(kTileWarps * 32, 3) logits_mma_kernel(const TolArgs a)
 {
     constexpr int kRowBytes = D * 2, kChunks = D / 8, kTileBytes = kTileTokens * kRowBytes;
     constexpr int kQRowBytes = kRowBytes + 16;                               // padded: B fragments read conflict-free
