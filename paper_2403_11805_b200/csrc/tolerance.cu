@@ -378,7 +378,23 @@ __global__ void __launch_bounds__(256) column_sum_kernel(const TolArgs a)
     const int r_end = min(a.rows, r_begin + rows_per_slice);
     float acc = 0.0f;
     if (seg < a.n_seg) {
-        for (int row = r_begin + threadIdx.y; row < r_end; row += 8) {
+        // four rows per trip, their loads issued together; the terms are still added in row order
+        int row = r_begin + threadIdx.y;
+        for (; row + 24 < r_end; row += 32) {
+            float ms[4], pp[4], rm[4], ri[4];
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                const int64_t o = (int64_t)(row + 8 * u) * a.n_seg + seg;
+                ms[u] = a.pm[o];
+                pp[u] = a.pp[o];
+                rm[u] = a.row_max[row + 8 * u];
+                ri[u] = a.row_inv[row + 8 * u];
+            }
+#pragma unroll
+            for (int u = 0; u < 4; ++u)
+                if (ms[u] != -INFINITY) acc += pp[u] * expf(ms[u] - rm[u]) * ri[u];
+        }
+        for (; row < r_end; row += 8) {
             const int64_t o = (int64_t)row * a.n_seg + seg;
             const float ms = a.pm[o];
             if (ms != -INFINITY) acc += a.pp[o] * expf(ms - a.row_max[row]) * a.row_inv[row];
@@ -394,18 +410,19 @@ __global__ void __launch_bounds__(256) column_sum_kernel(const TolArgs a)
     }
 }
 
-// thread per chunk: sum the row slices and the chunk's segments, scale to the mean
+// warp per chunk: lane y takes row slices y, y+32, ... of every segment of the chunk; the lanes' sums are then
+// added pairwise in a fixed tree, so a score does not depend on the launch
 __global__ void chunk_mean_kernel(const TolArgs a)
 {
-    const int c = blockIdx.x * blockDim.x + threadIdx.x;
+    const int c = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
     if (c >= a.n_chunks) return;
+    const int lane = threadIdx.x & 31;
     float tot = 0.0f;
-    for (int s = c * a.seg_per_chunk; s < (c + 1) * a.seg_per_chunk; ++s) {
-        float col = 0.0f;
-        for (int y = 0; y < a.Y; ++y) col += a.part[(int64_t)y * a.n_seg + s];
-        tot += col;
-    }
-    a.scores[c] = tot / ((float)a.CL * (float)a.L * (float)a.Hq);
+    for (int y = lane; y < a.Y; y += 32)
+        for (int s = c * a.seg_per_chunk; s < (c + 1) * a.seg_per_chunk; ++s) tot += a.part[(int64_t)y * a.n_seg + s];
+#pragma unroll
+    for (int m = 16; m > 0; m >>= 1) tot += __shfl_xor_sync(0xffffffffu, tot, m);
+    if (lane == 0) a.scores[c] = tot / ((float)a.CL * (float)a.L * (float)a.Hq);
 }
 
 // ------------------------------------------------------------------ probabilities -> scores
@@ -604,7 +621,7 @@ extern "C" int llms_chunk_tolerance(const llms_kv_desc *desc, const void *kv, co
     LLMS_CUDA_TRY(cudaGetLastError());
     column_sum_kernel<<<dim3((a.n_seg + 31) / 32, a.Y), dim3(32, 8), 0, st>>>(a);
     LLMS_CUDA_TRY(cudaGetLastError());
-    chunk_mean_kernel<<<(a.n_chunks + 127) / 128, 128, 0, st>>>(a);
+    chunk_mean_kernel<<<(a.n_chunks + 7) / 8, 256, 0, st>>>(a);
     LLMS_CUDA_TRY(cudaGetLastError());
     return LLMS_OK;
 }
