@@ -124,7 +124,8 @@ __global__ void __launch_bounds__(kTokThreads) logits_kernel(const TolArgs a)
 // The window's query rows sit in shared memory (rows padded by 16 bytes against conflicts) and are read as B
 // fragments.  The softmax statistics are then taken straight from the accumulator fragments.
 constexpr int kTileTokens = 32;
-constexpr int kTileWarps = 8;
+constexpr int kTileWarps = 12;     // most warps a CTA is launched with; 8 when twelve tiles do not fit twice into an SM
+constexpr int kTileWarpsSmall = 8;  // (measured on the 7B shape: 12 warps x 2 CTAs 0.2175 ms, 8 x 3 0.227, 4 x 6 0.269)
 constexpr int kTileBuffers = 1;   // per warp; with 1 the other warps of the SM cover a warp's copy latency
 
 // 16-byte asynchronous copy global -> shared, bypassing L1; src_bytes = 0 fills zeros instead
@@ -229,7 +230,7 @@ __device__ __forceinline__ void tile_statistics(const TolArgs &a, const float (&
 // NBG: n-tiles (8 flattened window rows each) that share one pass over a tile's A fragments - 4 for grouped-query
 // shapes whose rows come in multiples of 32 per KV head, else 1.
 template <int SEG, int D, int NBG>
-__global__ void __launch_bounds__(kTileWarps * 32, 3) logits_mma_kernel(const TolArgs a)
+__global__ void __launch_bounds__(kTileWarps * 32, 2) logits_mma_kernel(const TolArgs a)
 {
     constexpr int kRowBytes = D * 2, kChunks = D / 8, kTileBytes = kTileTokens * kRowBytes;
     constexpr int kQRowBytes = kRowBytes + 16;                               // padded: B fragments read conflict-free
@@ -282,12 +283,13 @@ __global__ void __launch_bounds__(kTileWarps * 32, 3) logits_mma_kernel(const To
 
     int buf = 0;
     if (kTileBuffers == 2 && tile_begin < tile_end) issue_tile(tile_begin, 0);
-    for (int tile = tile_begin; tile < tile_end; tile += kTileWarps, buf ^= (kTileBuffers - 1)) {
+    const int cta_warps = blockDim.x >> 5;
+    for (int tile = tile_begin; tile < tile_end; tile += cta_warps, buf ^= (kTileBuffers - 1)) {
         if (kTileBuffers == 1) {
             issue_tile(tile, 0);
             cp_async_wait<0>();
-        } else if (tile + kTileWarps < tile_end) {
-            issue_tile(tile + kTileWarps, buf ^ 1);
+        } else if (tile + cta_warps < tile_end) {
+            issue_tile(tile + cta_warps, buf ^ 1);
             cp_async_wait<1>();
         } else {
             cp_async_wait<0>();
@@ -560,18 +562,21 @@ extern "C" int llms_chunk_tolerance(const llms_kv_desc *desc, const void *kv, co
     if ((unsigned)(a.L * a.Hkv) > 65535u) return LLMS_ERR_UNSUPPORTED;
     const size_t mma_q_bytes = ((size_t)((a.NR + 7) / 8 * 8) * (a.d * 2 + 16) + 127) / 128 * 128 +
                                ((size_t)((a.NR + 7) / 8 * 8) * 4 + 127) / 128 * 128;   // query rows + each row's last visible token
-    const size_t mma_smem = mma_q_bytes + (size_t)kTileWarps * kTileBuffers * kTileTokens * a.d * 2;
+    const size_t tile_bytes = (size_t)kTileBuffers * kTileTokens * a.d * 2;
+    // twelve warps per CTA when two such CTAs fit into an SM's shared memory, else eight
+    const int cta_warps = 2 * (mma_q_bytes + kTileWarps * tile_bytes + 1024) <= 227 * 1024 ? kTileWarps : kTileWarpsSmall;
+    const size_t mma_smem = mma_q_bytes + (size_t)cta_warps * tile_bytes;
     if ((a.d == 64 || a.d == 128 || a.d == 256) && mma_smem <= 200 * 1024) {
         // enough blocks per (layer, KV head) to fill the GPU a few times over
         const int n_tiles = (a.T + kTileTokens - 1) / kTileTokens;
         const int pairs = a.L * a.Hkv;
         int splits = (sm_count() * 6 + pairs - 1) / pairs;
-        splits = std::max(1, std::min(splits, (n_tiles + kTileWarps - 1) / kTileWarps));
+        splits = std::max(1, std::min(splits, (n_tiles + cta_warps - 1) / cta_warps));
         const dim3 grid(splits, pairs);
 #define LLMS_LAUNCH_MMA_G(S, DD, G)                                                                                                  \
     do {                                                                                                                             \
         LLMS_CUDA_TRY(cudaFuncSetAttribute(logits_mma_kernel<S, DD, G>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)mma_smem)); \
-        logits_mma_kernel<S, DD, G><<<grid, kTileWarps * 32, mma_smem, st>>>(a);                                                     \
+        logits_mma_kernel<S, DD, G><<<grid, cta_warps * 32, mma_smem, st>>>(a);                                                     \
     } while (0)
 #define LLMS_LAUNCH_MMA(S, DD)                                      \
     do {                                                            \
