@@ -272,6 +272,23 @@ def test_pinned_meta_gives_stream_ordered_checksums():
     assert e.value.status == B.ERR_INVALID_ARG
 
 
+def test_pageable_meta_takes_the_copy_path():
+    """Checksums reach a pageable meta array by a device-to-host copy (into pinned memory a kernel stores them)."""
+    sh = synth.CONFIGS["tiny"]
+    kv = synth.kv_tensor(sh)
+    d = B.desc_of(sh)
+    ids = np.arange(sh.n_chunks, dtype=np.uint32)
+    bits = synth.random_bits(sh.n_chunks, 4).numpy()
+    buf = torch.empty(B.compressed_size(d, bits), dtype=torch.uint8, device="cuda")
+    ws = torch.empty(B.codec_workspace_bytes(len(ids)), dtype=torch.uint8, device="cuda")
+    meta = B.new_meta(len(ids), pinned=False)
+    B.compress_chunks(d, kv.cuda(), ids, bits, buf, meta, ws)
+    torch.cuda.synchronize()
+    want_buf, want_meta = oracle.compress_chunks(odesc(sh), bits_view(kv), ids, bits)
+    assert first_mismatch(buf.cpu().numpy(), want_buf) is None
+    assert_meta_equal(meta, want_meta)
+
+
 def test_recompression_is_stable():
     # decode(encode(x)) encoded again at the same width gives the same codes whenever the scale is unchanged
     sh = synth.CONFIGS["tiny"]
