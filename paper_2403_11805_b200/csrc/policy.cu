@@ -1,4 +1,5 @@
-// Host-side policies: rank -> bit-width (Eq. 2) and the LCTRU eviction order (Sec. 3.4 ii).
+// Host-side policies: rank -> bit-width (Eq. 2), the thresholds of Eq. 3 and the LCTRU eviction order (Sec. 3.4 ii);
+// and the call that strings score, ranking and compression of a whole context together.
 #include <algorithm>
 #include <cmath>
 #include <numeric>
