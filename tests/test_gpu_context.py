@@ -68,3 +68,44 @@ def test_compress_context_argument_errors():
     rc = B.lib().llms_compress_context(None, None, None, 8, None, None, None, None, None, None, 0, None, None, 0, None, 0,
                                        None, None)
     assert rc == B.ERR_INVALID_ARG
+
+
+def test_full_size_step_as_the_benchmark_runs_it():
+    """The 7B-shaped context through llms_compress_context and llms_decompress_chunks_ordered, back to back without a
+    synchronisation in between: levels against the oracle's rule on the GPU's scores, sampled records and their decoded
+    chunks against the oracle, every record through its checksum."""
+    sh = synth.CONFIGS["llama7b"]
+    W, n, CL = sh.window, sh.n_chunks, sh.chunk_len
+    kv_dev = synth.kv_tensor(sh, device="cuda")
+    q_dev = synth.q_window(sh, W, device="cuda")
+    d = B.desc_of(sh)
+    frac, levels = np.asarray(sh.frac, dtype=np.float32), np.asarray((8, 4, 2), dtype=np.uint8)
+    scores_dev = torch.empty(n, dtype=torch.float32, device="cuda")
+    scores_host = torch.empty(n, dtype=torch.float32).pin_memory()
+    bits = np.zeros(n, dtype=np.uint8)
+    buf = torch.empty(B.compressed_size(d, np.full(n, 8, np.uint8)), dtype=torch.uint8, device="cuda")
+    meta = B.new_meta(n, pinned=True)
+    ws_t = torch.empty(B.tolerance_workspace_bytes(d, W), dtype=torch.uint8, device="cuda")
+    ws_c = torch.empty(B.codec_workspace_bytes(n), dtype=torch.uint8, device="cuda")
+    ws_d = torch.empty(B.codec_workspace_bytes(n), dtype=torch.uint8, device="cuda")
+    out = torch.empty_like(kv_dev)
+    for _ in range(2):
+        B.compress_context(d, kv_dev, q_dev, W, frac, levels, scores_dev, scores_host, bits, buf, meta, ws_t, ws_c)
+        B.decompress_chunks_ordered(d, buf, meta, None, out, ws_d)
+        assert B.codec_corrupt_count(ws_d) == 0
+    obits, _ = oracle.assign_levels(scores_host.numpy(), sh.frac, (8, 4, 2))
+    assert np.array_equal(bits, obits)
+    assert tuple(int((bits == b).sum()) for b in (8, 4, 2)) == (85, 86, 85)
+    one = sh.with_(n_tokens=CL)
+    picks = {0, n - 1} | {int(np.flatnonzero(bits == b)[40]) for b in (8, 4, 2)}
+    for cid in sorted(picks):
+        chunk = kv_dev[..., cid * CL:(cid + 1) * CL, :].contiguous().cpu()
+        want_buf, want_meta = oracle.compress_chunks(odesc(one), bits_view(chunk), [0], [bits[cid]])
+        m = meta[cid]
+        got = buf[int(m["offset"]):int(m["offset"] + m["nbytes"])].cpu().numpy()
+        assert first_mismatch(got, want_buf) is None, cid
+        assert m["checksum"] == want_meta[0]["checksum"]
+        want = np.zeros(chunk.numel(), dtype=np.uint16).reshape(chunk.shape)
+        oracle.decompress_chunks(odesc(one), want_buf, want_meta, want)
+        got_chunk = out[..., cid * CL:(cid + 1) * CL, :].contiguous().cpu()
+        assert first_mismatch(bits_view(got_chunk).reshape(-1), want.reshape(-1)) is None, cid
