@@ -117,7 +117,16 @@ struct UnitPos {
     uint64_t rec_off;
     int e0;                // first element of this lane, counted from the start of slab s_idx
     int limit;             // elements of this unit that exist, counted from the unit's first element
+    int64_t kv_off;        // element offset of the unit's first element in the KV tensor (not packed)
 };
+
+__device__ __forceinline__ int64_t slab_offset(const CodecArgs &a, uint32_t s_idx, uint32_t chunk)
+{
+    uint32_t ls, h;
+    a.div_heads.divmod(s_idx, ls, h);
+    return (int64_t)(ls >> 1) * a.stride_l + (int64_t)(ls & 1) * a.stride_s + (int64_t)h * a.stride_h +
+           (int64_t)chunk * a.chunk_stride;
+}
 
 template <bool PACKED>
 __device__ __forceinline__ void decode_unit(const CodecArgs &a, uint32_t unit, int lane, UnitPos &u)
@@ -140,15 +149,8 @@ __device__ __forceinline__ void decode_unit(const CodecArgs &a, uint32_t unit, i
         u.s_idx = row;
         u.e0 = (int)pass * kPassElems + lane * kLaneElems;
         u.limit = min(kPassElems, a.slab_elems - (int)pass * kPassElems);
+        u.kv_off = slab_offset(a, row, head.x) + (int)pass * kPassElems;
     }
-}
-
-__device__ __forceinline__ int64_t slab_offset(const CodecArgs &a, uint32_t s_idx, uint32_t chunk)
-{
-    uint32_t ls, h;
-    a.div_heads.divmod(s_idx, ls, h);
-    return (int64_t)(ls >> 1) * a.stride_l + (int64_t)(ls & 1) * a.stride_s + (int64_t)h * a.stride_h +
-           (int64_t)chunk * a.chunk_stride;
 }
 
 // KV offset of element v of a unit (v counted from the unit's first element)
@@ -514,7 +516,7 @@ template <bool WIDE, bool PACKED>
 __device__ __forceinline__ void load_unit(const CodecArgs &a, const UnitPos &u, int lane, uint32_t (&w)[kPieces][8])
 {
     const __half *src0 = nullptr;  // piece 0 when the unit lies inside one slab
-    if constexpr (!PACKED) src0 = a.kv_in + slab_offset(a, u.s_idx, u.chunk_id) + (u.e0 - lane * kLaneElems) + lane * kPieceElems;
+    if constexpr (!PACKED) src0 = a.kv_in + u.kv_off + lane * kPieceElems;
 #pragma unroll
     for (int j = 0; j < kPieces; ++j) {
         const int v = j * (32 * kPieceElems) + lane * kPieceElems;
@@ -558,18 +560,15 @@ __device__ __forceinline__ void to_lane_contiguous(uint32_t (&w)[kPieces][8], un
 // Ask for a unit's KV bytes to be brought into L2 (one bulk prefetch by one lane): the register loads of that
 // unit, issued one unit later, then find them there instead of waiting for DRAM.
 template <bool PACKED>
-__device__ __forceinline__ void prefetch_unit_l2(const CodecArgs &a, uint32_t unit, int lane)
+__device__ __forceinline__ void prefetch_unit_l2(const CodecArgs &a, const UnitPos &u, int lane)
 {
-    UnitPos u;
-    decode_unit<PACKED>(a, unit, 0, u);
     if constexpr (PACKED) {  // one prefetch per slab of the unit
         if (lane < a.slabs_per_unit && lane * a.slab_elems < u.limit) {
             const __half *src = a.kv_in + slab_offset(a, u.s_idx + lane, u.chunk_id);
             asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" :: "l"(src), "r"((uint32_t)a.slab_elems * 2) : "memory");
         }
     } else if (lane == 0) {
-        const __half *src = a.kv_in + slab_offset(a, u.s_idx, u.chunk_id) + u.e0;
-        asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" :: "l"(src), "r"((uint32_t)u.limit * 2) : "memory");
+        asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" :: "l"(a.kv_in + u.kv_off), "r"((uint32_t)u.limit * 2) : "memory");
     }
 }
 
@@ -596,27 +595,40 @@ __global__ void __launch_bounds__(kThreads, 2) compress_kernel(const CodecArgs a
     cta_sums_clear(sum_slots, a.n);
     if (unit < a.total_units) {
         unsigned char *patch = patches[threadIdx.x >> 5];
-        UnitPos pa, pb;
+        // A unit is decoded once, two strides ahead of its turn: then its bytes are asked into L2, one trip later
+        // its loads are issued (pn -> pa / pb), another trip later it is computed.
+        static_assert(kPrefetchAhead == 2, "the loop below looks exactly two units ahead");
+        UnitPos pa, pb, pn;
         uint32_t wa[kPieces][8], wb[kPieces][8];
         decode_unit<PACKED>(a, unit, lane, pa);
         load_unit<WIDE, PACKED>(a, pa, lane, wa);
-        for (;;) {  // two units per trip, so that the buffers swap roles without register copies
-            bool more = a.total_units - unit > n_warps;
+        bool has_next = a.total_units - unit > n_warps;
+        if (has_next) decode_unit<PACKED>(a, unit + n_warps, lane, pn);
+        for (;;) {  // two units per trip, so that the data buffers swap roles without register copies
+            bool more = has_next;
             if (more) {
-                decode_unit<PACKED>(a, unit + n_warps, lane, pb);
+                pb = pn;
                 load_unit<WIDE, PACKED>(a, pb, lane, wb);
             }
-            if (a.total_units - unit > kPrefetchAhead * n_warps) prefetch_unit_l2<PACKED>(a, unit + kPrefetchAhead * n_warps, lane);
+            has_next = a.total_units - unit > 2 * n_warps;
+            if (has_next) {
+                decode_unit<PACKED>(a, unit + 2 * n_warps, lane, pn);
+                prefetch_unit_l2<PACKED>(a, pn, lane);
+            }
             to_lane_contiguous(wa, patch, lane);
             compress_unit<BITS, G, WIDE>(a, pa, wa, lane, sum_slots);
             if (!more) break;
             unit += n_warps;
-            more = a.total_units - unit > n_warps;
+            more = has_next;
             if (more) {
-                decode_unit<PACKED>(a, unit + n_warps, lane, pa);
+                pa = pn;
                 load_unit<WIDE, PACKED>(a, pa, lane, wa);
             }
-            if (a.total_units - unit > kPrefetchAhead * n_warps) prefetch_unit_l2<PACKED>(a, unit + kPrefetchAhead * n_warps, lane);
+            has_next = a.total_units - unit > 2 * n_warps;
+            if (has_next) {
+                decode_unit<PACKED>(a, unit + 2 * n_warps, lane, pn);
+                prefetch_unit_l2<PACKED>(a, pn, lane);
+            }
             to_lane_contiguous(wb, patch, lane);
             compress_unit<BITS, G, WIDE>(a, pb, wb, lane, sum_slots);
             if (!more) break;
