@@ -332,6 +332,34 @@ def run_ours(args):
     kv_bytes = shape.n_elements * 2
     value = world * 2 * kv_bytes / (ms_per_step * 1e-3) / 1e9
 
+    # ---- every codec launch by itself: the chunks of one level go through one compress call and one decompress call
+    # (one codec kernel each, plus the few-microsecond checksum kernel), bracketed by events on the launching stream.
+    # Each launch reads or writes its level's share of the fp16 KV (a third of 2 GiB on the metric's workload: larger than L2).
+    per_launch = []
+    reps = max(3, min(20, args.steps))
+    for b in LEVELS:
+        sel = ids[bits == b]
+        if len(sel) == 0:
+            continue
+        sel_bits = np.full(len(sel), b, dtype=np.uint8)
+        sel_meta = B.new_meta(len(sel), pinned=True)
+        launch_bytes = len(sel) * shape.n_slabs * shape.chunk_len * shape.head_dim * 2 + B.compressed_size(d, sel_bits)
+        for which in ("compress_kernel", "decompress_kernel"):
+            evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(reps + 3)]
+            for e0, e1 in evs:
+                e0.record(stream)
+                if which == "compress_kernel":
+                    B.compress_chunks(d, kv, sel, sel_bits, buf, sel_meta, ws)
+                else:
+                    B.decompress_chunks_ordered(d, buf, sel_meta, None, kv_out, ws_dec)
+                e1.record(stream)
+            torch.cuda.synchronize()
+            ms = sum(e0.elapsed_time(e1) for e0, e1 in evs[3:]) / reps
+            ms = sharding.max_over_ranks([ms], dist, "cuda")[0]
+            per_launch.append({"kernel": which, "bits": int(b), "chunks": int(len(sel)), "ms": ms,
+                               "algorithmic_bytes": int(launch_bytes), "gbs": launch_bytes / (ms * 1e-3) / 1e9})
+        assert B.codec_corrupt_count(ws_dec) == 0
+
     # ---- end to end: compress -> swap-out -> swap-in -> decompress with the pinned arena in the loop.
     # The chunks go in batches: while batch j travels to the host, batch j-1 is already on its way back and batch
     # j-2 is being decoded (the two copy directions and the kernels overlap); "serial" does one batch of everything.
@@ -448,6 +476,8 @@ def run_ours(args):
                     if args.quant_mode == 0 and LEVELS == (8, 4, 2) and not args.chunk_len else None),
         "algorithmic_bytes_per_launch": algo_bytes,
         "frac_of_nominal_8000": achieved / 8000.0,
+        # each codec launch timed alone (events around one call = one codec kernel + its checksum kernel)
+        "per_launch": [dict(pl, frac=pl["gbs"] / peak) for pl in per_launch],
         "per_stage": {
             "tolerance_ms": tol_ms, "compress_ms": comp_ms, "decompress_ms": decomp_ms,
             "tolerance_gbs_of_K_read": (kv_bytes / 2) / (tol_ms * 1e-3) / 1e9,

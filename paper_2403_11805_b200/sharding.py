@@ -1,5 +1,7 @@
-"""How the path spreads over several GPUs: contexts are independent (Sec. 3.1), so each rank owns whole contexts and
-nothing of the data path crosses ranks.  Only the timing is reduced (maximum over ranks)."""
+"""How the path spreads over several GPUs.  Contexts are independent (Sec. 3.1), so by default each rank owns whole
+contexts and nothing of the data path crosses ranks; only the timing is reduced (maximum over ranks).  Where a
+context's KV heads are split over the ranks instead (tensor-parallel serving), the codec still works per rank on its
+own heads and only the per-chunk scores of Eq. 1 are exchanged."""
 import torch
 
 
@@ -16,3 +18,27 @@ def max_over_ranks(values, dist=None, device="cpu"):
     if dist is not None and dist.is_initialized() and dist.get_world_size() > 1:
         dist.all_reduce(t, op=dist.ReduceOp.MAX)
     return t.tolist()
+
+
+def heads_of_rank(n_kv_heads: int, n_q_heads: int, rank: int, world: int):
+    """Tensor-parallel serving: a rank holds a contiguous block of KV heads and the query heads that read them.
+    Returns ((kv_first, kv_end), (q_first, q_end)).  Every rank holds the same number of heads."""
+    if not (0 <= rank < world):
+        raise ValueError("rank out of range")
+    if n_kv_heads % world or n_q_heads % n_kv_heads:
+        raise ValueError("heads must split evenly over the ranks")
+    per = n_kv_heads // world
+    rep = n_q_heads // n_kv_heads
+    return (rank * per, (rank + 1) * per), (rank * per * rep, (rank + 1) * per * rep)
+
+
+def combine_head_sharded_scores(local_scores: torch.Tensor, dist=None):
+    """Eq. 1 is a mean over layers, heads and a chunk's tokens.  When every rank scored the chunks from its own,
+    equally many heads, the information density of the whole model is the mean of the ranks' results: one sum
+    all-reduce of n_chunks fp32 values (the only exchange on the path), then a division by the number of ranks.
+    Every rank receives the same bits, so the rank -> bits rule and the eviction order come out the same everywhere."""
+    t = local_scores.to(torch.float32).clone()
+    if dist is not None and dist.is_initialized() and dist.get_world_size() > 1:
+        dist.all_reduce(t, op=dist.ReduceOp.SUM)
+        t /= dist.get_world_size()
+    return t

@@ -52,3 +52,59 @@ def test_two_ranks_partition_contexts_and_reduce_times():
 def test_single_rank_is_the_identity():
     assert sharding.contexts_of_rank(5, 0, 1) == [0, 1, 2, 3, 4]
     assert sharding.max_over_ranks([3.5]) == [3.5]
+
+
+def _head_worker(rank, world, port, out):
+    import numpy as np
+    import oracle
+    os.environ.update(MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port), RANK=str(rank), WORLD_SIZE=str(world))
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    sh = synth.KVShape("tp", 2, 4, 8, 32, 96, 16, 32, seed=3)     # 2 layers, 4 KV heads read by 8 query heads
+    W = 8
+    kv, q = synth.kv_tensor(sh), synth.q_window(sh, W)
+    (k0, k1), (q0, q1) = sharding.heads_of_rank(sh.n_kv_heads, sh.n_q_heads, rank, world)
+    kv_mine = kv[:, :, k0:k1].contiguous().view(torch.int16).numpy().view(np.uint16)
+    q_mine = q[:, q0:q1].contiguous().view(torch.int16).numpy().view(np.uint16)
+    od = oracle.make_desc(sh.n_layers, k1 - k0, q1 - q0, sh.head_dim, sh.n_tokens, sh.chunk_len, sh.group_size)
+    local = torch.from_numpy(oracle.chunk_tolerance(od, kv_mine, q_mine, W).astype(np.float32))
+    combined = sharding.combine_head_sharded_scores(local, dist)
+    bits, order = oracle.assign_bits(combined.numpy(), (1 / 3, 1 / 3, 1 / 3))
+    gathered = [None] * world
+    dist.all_gather_object(gathered, (combined.numpy().tobytes(), bits.tobytes(), order.tobytes()))
+    if rank == 0:
+        out.put(gathered)
+    dist.barrier()
+    dist.destroy_process_group()
+
+
+def test_head_sharded_scores_combine_to_the_whole_model_score():
+    import numpy as np
+    import oracle
+    ctx = mp.get_context("spawn")
+    out = ctx.Queue()
+    port = _free_port()
+    procs = [ctx.Process(target=_head_worker, args=(r, 2, port, out)) for r in range(2)]
+    for p in procs:
+        p.start()
+    gathered = out.get(timeout=120)
+    for p in procs:
+        p.join(timeout=60)
+        assert p.exitcode == 0
+    assert gathered[0] == gathered[1]                      # same score bits, same levels, same order on both ranks
+    combined = np.frombuffer(gathered[0][0], dtype=np.float32)
+    sh = synth.KVShape("tp", 2, 4, 8, 32, 96, 16, 32, seed=3)
+    kv = synth.kv_tensor(sh).view(torch.int16).numpy().view(np.uint16)
+    q = synth.q_window(sh, 8).view(torch.int16).numpy().view(np.uint16)
+    od = oracle.make_desc(sh.n_layers, sh.n_kv_heads, sh.n_q_heads, sh.head_dim, sh.n_tokens, sh.chunk_len, sh.group_size)
+    whole = oracle.chunk_tolerance(od, kv, q, 8)
+    assert np.allclose(combined, whole, rtol=1e-6, atol=0)
+
+
+def test_heads_of_rank_blocks():
+    assert sharding.heads_of_rank(8, 32, 1, 4) == ((2, 4), (8, 16))
+    assert sharding.heads_of_rank(1, 8, 0, 1) == ((0, 1), (0, 8))
+    import pytest
+    with pytest.raises(ValueError):
+        sharding.heads_of_rank(1, 8, 0, 2)                 # one KV head cannot be split
+    t = torch.tensor([0.25, 0.5])
+    assert torch.equal(sharding.combine_head_sharded_scores(t), t)
