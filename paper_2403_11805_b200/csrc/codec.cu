@@ -1143,14 +1143,18 @@ extern "C" int llms_compress_chunks(const llms_kv_desc *desc, const void *kv, co
     }
     if (off > out_bytes) return LLMS_ERR_BUF_TOO_SMALL;
     const uint32_t n_groups = (uint32_t)groups_per_chunk(*desc);
+    // The device's table is built from a private copy: `meta` may be page-locked memory into which an earlier
+    // call's kernel is still storing checksums, and the accumulators uploaded below have to start at zero.
+    std::vector<llms_chunk_meta> staged(n);
     off = 0;
     for (int i = 0; i < n; ++i) {
-        meta[i].chunk_id = chunk_ids[i];
-        meta[i].bits = bits[i];
-        meta[i].offset = off;
-        meta[i].nbytes = bytes_at[bits[i]];
-        meta[i].n_groups = n_groups;
-        meta[i].checksum = 0;  // the kernel accumulates into the device copy
+        staged[i].chunk_id = chunk_ids[i];
+        staged[i].bits = bits[i];
+        staged[i].offset = off;
+        staged[i].nbytes = bytes_at[bits[i]];
+        staged[i].n_groups = n_groups;
+        staged[i].checksum = 0;  // the kernel accumulates into the device copy
+        meta[i] = staged[i];
         off += bytes_at[bits[i]];
     }
     CodecArgs a{};
@@ -1159,8 +1163,8 @@ extern "C" int llms_compress_chunks(const llms_kv_desc *desc, const void *kv, co
     a.kv_in = static_cast<const __half *>(kv);
     a.buf = static_cast<uint8_t *>(out_buf);
     cudaStream_t st = static_cast<cudaStream_t>(stream);
-    const BitGroups groups = group_by_bits(n, meta, [&](int i) { return (uint32_t)bits[i]; });
-    rc = upload_tables(workspace, meta, groups, n, false, st);
+    const BitGroups groups = group_by_bits(n, staged.data(), [&](int i) { return (uint32_t)bits[i]; });
+    rc = upload_tables(workspace, staged.data(), groups, n, false, st);
     if (rc) return rc;
     for (int k = 0; k < kNumWidths; ++k) {
         if (groups.count[k] == 0) continue;
