@@ -272,30 +272,33 @@ def test_pinned_meta_gives_stream_ordered_checksums():
     assert e.value.status == B.ERR_INVALID_ARG
 
 
-def test_back_to_back_encode_calls_share_one_pinned_meta():
+@pytest.mark.parametrize("layers", [1, 2])
+def test_back_to_back_encode_calls_share_one_pinned_meta(layers):
     """Encode calls that follow each other on a stream with no synchronisation may all name the same pinned meta
     array: while the host prepares call k+1 the device is still storing call k's checksums into it.  Every call's
-    sums must start from zero all the same (short launches, so that the device keeps pace with the host)."""
-    sh = synth.CONFIGS["tiny"]
+    sums must start from zero all the same.  (Launches about as long as the host's part of a call, so that the
+    device's stores fall into the host's preparation of the next call.)"""
+    sh = synth.CONFIGS["llama7b"].with_(n_layers=layers)
     kv = synth.kv_tensor(sh)
     kv_dev = kv.cuda()
     d = B.desc_of(sh)
-    n = sh.n_chunks
-    ids = np.arange(n, dtype=np.uint32)
-    bits = synth.random_bits(n, 5).numpy()
-    buf = torch.empty(B.compressed_size(d, bits), dtype=torch.uint8, device="cuda")
-    ws_c = torch.empty(B.codec_workspace_bytes(n), dtype=torch.uint8, device="cuda")
-    ws_d = torch.empty(B.codec_workspace_bytes(n), dtype=torch.uint8, device="cuda")
+    ids = np.arange(0, sh.n_chunks, 3, dtype=np.uint32)
+    n = len(ids)
     out = torch.empty(kv.shape, dtype=torch.float16, device="cuda")
-    meta = B.new_meta(n, pinned=True)
-    want_buf, want_meta = oracle.compress_chunks(odesc(sh), bits_view(kv), ids, bits)
-    for _ in range(20):
-        for _ in range(25):
-            B.compress_chunks(d, kv_dev, ids, bits, buf, meta, ws_c)
-        B.decompress_chunks_ordered(d, buf, meta, None, out, ws_d)
-        assert B.codec_corrupt_count(ws_d) == 0          # synchronises
-        assert_meta_equal(meta, want_meta)
-    assert first_mismatch(buf.cpu().numpy(), want_buf) is None
+    for b in (8, 2):
+        bits = np.full(n, b, dtype=np.uint8)
+        buf = torch.empty(B.compressed_size(d, bits), dtype=torch.uint8, device="cuda")
+        ws_c = torch.empty(B.codec_workspace_bytes(n), dtype=torch.uint8, device="cuda")
+        ws_d = torch.empty(B.codec_workspace_bytes(n), dtype=torch.uint8, device="cuda")
+        meta = B.new_meta(n, pinned=True)
+        want_buf, want_meta = oracle.compress_chunks(odesc(sh), bits_view(kv), ids, bits)
+        for _ in range(10):
+            for _ in range(20):
+                B.compress_chunks(d, kv_dev, ids, bits, buf, meta, ws_c)
+            B.decompress_chunks_ordered(d, buf, meta, None, out, ws_d)
+            assert B.codec_corrupt_count(ws_d) == 0      # synchronises
+            assert_meta_equal(meta, want_meta)
+        assert first_mismatch(buf.cpu().numpy(), want_buf) is None
 
 
 def test_pageable_meta_takes_the_copy_path():
