@@ -36,7 +36,7 @@ def parse_args():
     p.add_argument("--chunk-len", type=int, default=0, help="override the workload's tokens per chunk (chunk-size sweep, Sec. 5.4)")
     p.add_argument("--levels", default="8,4,2", help="bit-widths of the three levels, top first (Sec. 3.2: 8,4,2 or 4,2,1)")
     p.add_argument("--e2e-steps", type=int, default=10)
-    p.add_argument("--e2e-batches", type=int, default=8, help="batches of chunks the pipelined round trip is cut into")
+    p.add_argument("--e2e-batches", type=int, default=16, help="batches of chunks the pipelined round trip is cut into")
     p.add_argument("--no-cpu-baseline", action="store_true")
     p.add_argument("--no-layerwise", dest="layerwise", action="store_false",
                    help="skip the layer-wise swap timing (records split per layer, Sec. 4: first layer ready / all layers ready)")
