@@ -247,10 +247,11 @@ int llms_lctru_order(const llms_chunk_state *table, int n, uint32_t *order_out);
  * window, the scores copied to the host, llms_assign_levels, then llms_compress_chunks over all chunks
  * in index order (chunk_ids 0 .. n-1).  Results are those of the three calls made one after the other;
  * what this call saves is the host time between them, during which the stream would sit empty.
- * The ranking is a host step: the call synchronises `stream` once, after the scores' copy.
- *   scores_dev   device fp32 [n_chunks];  scores_host  host fp32 [n_chunks] (pinned for a truly asynchronous copy)
+ * The ranking is a host step: the call synchronises `stream` once, when the scores have reached the host.
+ *   scores_dev   device fp32 [n_chunks];  scores_host  host fp32 [n_chunks]: into page-locked memory the
+ *                last score kernel stores the scores itself, pageable memory receives them by a copy
  *   bits_out     host, n_chunks bytes: the level each chunk got
- *   after_scores optional cudaEvent_t, recorded on `stream` behind the score kernels and the scores' copy
+ *   after_scores optional cudaEvent_t, recorded on `stream` behind the score kernels (and the scores' copy)
  *   everything else as in the three calls. */
 int llms_compress_context(const llms_kv_desc *desc, const void *kv, const void *q_win, int W,
                           const float frac[3], const uint8_t levels[3],

@@ -891,16 +891,6 @@ __global__ void publish_checksums_kernel(const ChunkEntry *entries, llms_chunk_m
         live_meta[i].checksum = entries[i].checksum;
 }
 
-// The device's view of a host pointer if it is page-locked memory the device can access, else NULL.
-static void *device_view_of_pinned(const void *host_ptr)
-{
-    cudaPointerAttributes attr;
-    if (cudaPointerGetAttributes(&attr, host_ptr) == cudaSuccess && attr.type == cudaMemoryTypeHost && attr.devicePointer)
-        return attr.devicePointer;
-    cudaGetLastError();
-    return nullptr;
-}
-
 // ---------------------------------------------------------------------------------------------- host side
 
 static int fill_args(const llms_kv_desc &d, CodecArgs &a, int n, void *workspace, bool wide)

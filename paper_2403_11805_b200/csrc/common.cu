@@ -27,6 +27,15 @@ int sm_count()
     return cached[dev];
 }
 
+void *device_view_of_pinned(const void *host_ptr)
+{
+    cudaPointerAttributes attr;
+    if (cudaPointerGetAttributes(&attr, host_ptr) == cudaSuccess && attr.type == cudaMemoryTypeHost && attr.devicePointer)
+        return attr.devicePointer;
+    cudaGetLastError();
+    return nullptr;
+}
+
 int check_desc(const llms_kv_desc *d)
 {
     if (!d) return LLMS_ERR_INVALID_ARG;

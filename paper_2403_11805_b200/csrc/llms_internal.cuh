@@ -42,6 +42,14 @@ inline int check_bits(int b) { return (b == 1 || b == 2 || b == 4 || b == 8) ? L
 // Number of SMs of the current device (cached per device).
 int sm_count();
 
+// The device's view of a host pointer if it is page-locked memory the device can access, else NULL.
+void *device_view_of_pinned(const void *host_ptr);
+
+// llms_chunk_tolerance with a second destination: scores_live, when not NULL, is a device-visible address (page-locked
+// host memory) into which the last kernel also stores the scores, so that no copy has to follow the kernels.
+int chunk_tolerance_impl(const llms_kv_desc *desc, const void *kv, const void *q_win, int W, float *scores,
+                         float *scores_live, void *workspace, uint64_t workspace_bytes, void *stream);
+
 // Device-side copy of the per-chunk table, kept in the workspace.
 struct ChunkEntry {          // same bytes as llms_chunk_meta
     uint32_t chunk_id, bits;

@@ -113,11 +113,16 @@ extern "C" int llms_compress_context(const llms_kv_desc *desc, const void *kv, c
                                      void *after_scores, void *stream)
 {
     if (!desc || !scores_dev || !scores_host || !bits_out) return LLMS_ERR_INVALID_ARG;
-    int rc = llms_chunk_tolerance(desc, kv, q_win, W, scores_dev, tolerance_workspace, tolerance_workspace_bytes, stream);
+    // Into page-locked memory the last score kernel stores the scores itself (a copy after the kernels costs a switch to
+    // the copy engine and back: about 15 us per context); pageable memory gets them by a copy.
+    float *scores_live = static_cast<float *>(llms::device_view_of_pinned(scores_host));
+    int rc = llms::chunk_tolerance_impl(desc, kv, q_win, W, scores_dev, scores_live, tolerance_workspace,
+                                        tolerance_workspace_bytes, stream);
     if (rc) return rc;
     const int n = (int)llms::n_chunks(*desc);
     cudaStream_t st = static_cast<cudaStream_t>(stream);
-    LLMS_CUDA_TRY(cudaMemcpyAsync(scores_host, scores_dev, (size_t)n * sizeof(float), cudaMemcpyDeviceToHost, st));
+    if (!scores_live)
+        LLMS_CUDA_TRY(cudaMemcpyAsync(scores_host, scores_dev, (size_t)n * sizeof(float), cudaMemcpyDeviceToHost, st));
     if (after_scores) LLMS_CUDA_TRY(cudaEventRecord(static_cast<cudaEvent_t>(after_scores), st));
     LLMS_CUDA_TRY(cudaStreamSynchronize(st));
     rc = llms_assign_levels(scores_host, n, frac, levels, bits_out, nullptr);

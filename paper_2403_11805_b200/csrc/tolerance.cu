@@ -34,6 +34,7 @@ struct TolArgs {
     float *row_max, *row_inv; // [rows]
     float *part;              // [Y][n_seg]
     float *scores;
+    float *scores_live;       // optional second destination of the scores (page-locked host memory), or NULL
     int Y, rows;
 };
 
@@ -424,7 +425,11 @@ __global__ void chunk_mean_kernel(const TolArgs a)
         for (int s = c * a.seg_per_chunk; s < (c + 1) * a.seg_per_chunk; ++s) tot += a.part[(int64_t)y * a.n_seg + s];
 #pragma unroll
     for (int m = 16; m > 0; m >>= 1) tot += __shfl_xor_sync(0xffffffffu, tot, m);
-    if (lane == 0) a.scores[c] = tot / ((float)a.CL * (float)a.L * (float)a.Hq);
+    if (lane == 0) {
+        const float score = tot / ((float)a.CL * (float)a.L * (float)a.Hq);
+        a.scores[c] = score;
+        if (a.scores_live) a.scores_live[c] = score;
+    }
 }
 
 // ------------------------------------------------------------------ probabilities -> scores
@@ -529,6 +534,12 @@ extern "C" int llms_tolerance_workspace_bytes(const llms_kv_desc *desc, int W, u
 extern "C" int llms_chunk_tolerance(const llms_kv_desc *desc, const void *kv, const void *q_win, int W,
                                     float *scores, void *workspace, uint64_t workspace_bytes, void *stream)
 {
+    return llms::chunk_tolerance_impl(desc, kv, q_win, W, scores, nullptr, workspace, workspace_bytes, stream);
+}
+
+int llms::chunk_tolerance_impl(const llms_kv_desc *desc, const void *kv, const void *q_win, int W, float *scores,
+                               float *scores_live, void *workspace, uint64_t workspace_bytes, void *stream)
+{
     int rc = check_tol(desc, W);
     if (rc) return rc;
     if (!kv || !q_win || !scores || !workspace) return LLMS_ERR_INVALID_ARG;
@@ -557,6 +568,7 @@ extern "C" int llms_chunk_tolerance(const llms_kv_desc *desc, const void *kv, co
     a.row_inv = reinterpret_cast<float *>(ws + t.off_rinv);
     a.part = reinterpret_cast<float *>(ws + t.off_part);
     a.scores = scores;
+    a.scores_live = scores_live;
     a.Y = t.Y; a.rows = t.rows;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     if ((unsigned)(a.L * a.Hkv) > 65535u) return LLMS_ERR_UNSUPPORTED;

@@ -11,8 +11,9 @@ from gpu_helpers import assert_meta_equal, bits_view, first_mismatch, odesc
 pytestmark = pytest.mark.gpu
 
 
+@pytest.mark.parametrize("pinned_scores", [True, False], ids=["pinned", "pageable"])
 @pytest.mark.parametrize("levels,frac", [((8, 4, 2), (1 / 3, 1 / 3, 1 / 3)), ((4, 2, 1), (0.2, 0.5, 0.3))])
-def test_compress_context_equals_the_separate_calls_and_the_oracle(levels, frac):
+def test_compress_context_equals_the_separate_calls_and_the_oracle(levels, frac, pinned_scores):
     sh = synth.KVShape("ctx", 3, 2, 4, 64, 208, 16, 64, seed=13)          # 13 chunks, GQA
     W = sh.window
     kv, q = synth.kv_tensor(sh), synth.q_window(sh, W)
@@ -23,7 +24,10 @@ def test_compress_context_equals_the_separate_calls_and_the_oracle(levels, frac)
 
     # one call
     scores_dev = torch.empty(n, dtype=torch.float32, device="cuda")
-    scores_host = torch.empty(n, dtype=torch.float32).pin_memory()
+    # into pinned memory the score kernel stores the scores itself, pageable memory gets them by a copy
+    scores_host = torch.full((n,), -1.0, dtype=torch.float32)
+    if pinned_scores:
+        scores_host = scores_host.pin_memory()
     bits = np.zeros(n, dtype=np.uint8)
     total = B.compressed_size(d, np.full(n, levels[0], np.uint8))
     buf = torch.zeros(total, dtype=torch.uint8, device="cuda")
