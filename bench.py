@@ -55,7 +55,7 @@ def measured_peaks():
     return 6650.0, "fallback"
 
 
-# dram__bytes_read.sum + dram__bytes_write.sum of one stage (its three launches, one per bit-width) on the full
+# dram__bytes_read.sum + dram__bytes_write.sum of one stage (one launch, the bit-widths as phases) on the full
 # llama7b workload, from one ncu capture of the kernels as they are now (profiles/codec_and_score_kernels_llama7b.md).
 # Set an entry to None when its kernel changes.
 NCU_DRAM_TRAFFIC = {
@@ -471,7 +471,7 @@ def run_ours(args):
     achieved = algo_bytes / (k_ms[dominant] * 1e-3) / 1e9
     roofline = {
         "kernel": dominant, "bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
-        "peak_source": f"{peak_kind} copy bandwidth", "launches_per_stage": 3,
+        "peak_source": f"{peak_kind} copy bandwidth", "launches_per_stage": B.codec_launches(d, bits) - 1,
         "traffic": (NCU_DRAM_TRAFFIC.get((shape.name, shape.n_layers, dominant))
                     if args.quant_mode == 0 and LEVELS == (8, 4, 2) and not args.chunk_len else None),
         "algorithmic_bytes_per_launch": algo_bytes,
@@ -504,7 +504,9 @@ def run_ours(args):
                 "serial_ms_per_step": e2e_serial_ms, "batch_chunks": e2e_batch,
                 "what": "compress -> swap-out to pinned host -> swap-in -> decompress, pipelined in batches of chunks",
                 "layerwise_load": layerwise},
-        "gpu_launches": args.steps * 12,   # 4 score kernels, compress and decompress once per bit-width, 1 checksum store, 1 verify
+        # 4 score kernels, then per codec call one codec kernel (one per bit-width in channel-wise mode) and the kernel
+        # that stores or checks the sums
+        "gpu_launches": args.steps * (4 + 2 * B.codec_launches(d, bits)),
         "roofline": roofline, "clocks": clocks,
         "wall_ms_per_step": t_wall * 1e3 / args.steps,
         "step_ms_median_best": [statistics.median(step_ms), step_ms[0]],

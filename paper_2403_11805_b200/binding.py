@@ -204,6 +204,12 @@ def tolerance_workspace_bytes(desc, W):
 
 # ----------------------------------------------------------------------------- codec
 
+def codec_launches(desc, bits):
+    """Kernels one compress or decompress call launches: one codec kernel for the whole call (the bit-widths are phases
+    of it; channel-wise mode launches one per bit-width present) and one small kernel that stores or checks the sums."""
+    return (len(set(int(b) for b in bits)) if desc.quant_mode == 1 else 1) + 1
+
+
 def compress_chunks(desc, kv, chunk_ids, bits, out_buf, meta, workspace, stream=None, out_bytes=None, workspace_bytes=None):
     chunk_ids = np.ascontiguousarray(chunk_ids, dtype=np.uint32)
     bits = np.ascontiguousarray(bits, dtype=np.uint8)

@@ -19,6 +19,7 @@
 // nothing is contracted or approximated.
 #include <string.h>
 
+#include <algorithm>
 #include <map>
 #include <mutex>
 #include <utility>
@@ -582,16 +583,13 @@ __device__ __forceinline__ void compress_unit(const CodecArgs &a, const UnitPos 
     unit_sum_add(sum_slots, a.n, u.k, &a.entries[u.i].checksum, sum, lane);
 }
 
-// One launch per bit-width present in the call: a single code path per kernel keeps the instruction
-// working set small (with all three widths in one kernel the warps stalled on instruction fetch).
+// The chunks of one bit-width, start to finish: one phase of the kernel below.
 template <int BITS, int G, bool WIDE, bool PACKED>
-__global__ void __launch_bounds__(kThreads, 2) compress_kernel(const CodecArgs a)
+__device__ __forceinline__ void compress_phase(const CodecArgs &a, unsigned char (*patches)[kTransposeBytes], uint32_t *sum_slots)
 {
     const int lane = threadIdx.x & 31;
     const uint32_t n_warps = gridDim.x * kWarpsPerBlock;
     uint32_t unit = blockIdx.x * kWarpsPerBlock + (threadIdx.x >> 5);
-    __shared__ __align__(16) unsigned char patches[kWarpsPerBlock][kTransposeBytes];
-    __shared__ uint32_t sum_slots[kSumSlots];
     cta_sums_clear(sum_slots, a.n);
     if (unit < a.total_units) {
         unsigned char *patch = patches[threadIdx.x >> 5];
@@ -639,6 +637,27 @@ __global__ void __launch_bounds__(kThreads, 2) compress_kernel(const CodecArgs a
     if (a.n <= kSumSlots)
         for (int k = threadIdx.x; k < a.n; k += kThreads)
             if (sum_slots[k]) atomicAdd(&a.entries[a.order[k]].checksum, sum_slots[k]);
+}
+
+// The launch arguments of a call, one set per bit-width (8, 4, 2, 1; n == 0: that width is absent).
+struct CodecArgsByWidth {
+    CodecArgs w[4];
+};
+
+// One launch per call.  The bit-widths are phases in time, not branches per unit: every warp first works through
+// its share of the 8-bit chunks, then of the 4-bit ones, and so on, so the SM runs one code path at a time (with
+// the widths mixed unit by unit the warps stalled on instruction fetch), no launch boundary separates the widths
+// (one launch per width cost a drained GPU and a few microseconds between each pair), and a warp that is done
+// with one width starts on the next while others finish.
+template <int G, bool WIDE, bool PACKED>
+__global__ void __launch_bounds__(kThreads, 2) compress_kernel(const __grid_constant__ CodecArgsByWidth all)
+{
+    __shared__ __align__(16) unsigned char patches[kWarpsPerBlock][kTransposeBytes];
+    __shared__ uint32_t sum_slots[kSumSlots];
+    if (all.w[0].n) compress_phase<8, G, WIDE, PACKED>(all.w[0], patches, sum_slots);
+    if (all.w[1].n) compress_phase<4, G, WIDE, PACKED>(all.w[1], patches, sum_slots);
+    if (all.w[2].n) compress_phase<2, G, WIDE, PACKED>(all.w[2], patches, sum_slots);
+    if (all.w[3].n) compress_phase<1, G, WIDE, PACKED>(all.w[3], patches, sum_slots);
 }
 
 // ---------------------------------------------------------------------------------------------- dequantize
@@ -848,18 +867,28 @@ __device__ __forceinline__ void decompress_warp(const CodecArgs &a, uint32_t uni
 }
 
 template <int BITS, int G, bool WIDE, bool PACKED>
-__global__ void __launch_bounds__(kThreads, kDecodeBlocksPerSm) decompress_kernel(const CodecArgs a)
+__device__ __forceinline__ void decompress_phase(const CodecArgs &a, uint32_t *sum_slots)
 {
     const int lane = threadIdx.x & 31;
     const uint32_t n_warps = gridDim.x * kWarpsPerBlock;
     const uint32_t unit = blockIdx.x * kWarpsPerBlock + (threadIdx.x >> 5);
-    __shared__ uint32_t sum_slots[kSumSlots];
     cta_sums_clear(sum_slots, a.n);
     if (unit < a.total_units) decompress_warp<BITS, G, WIDE, PACKED>(a, unit, n_warps, lane, sum_slots);
     __syncthreads();
     if (a.n <= kSumSlots)
         for (int k = threadIdx.x; k < a.n; k += kThreads)
             if (sum_slots[k]) atomicAdd(&a.sums[a.table[k].entry], sum_slots[k]);
+}
+
+// One launch per call, the bit-widths as phases in time (see compress_kernel).
+template <int G, bool WIDE, bool PACKED>
+__global__ void __launch_bounds__(kThreads, kDecodeBlocksPerSm) decompress_kernel(const __grid_constant__ CodecArgsByWidth all)
+{
+    __shared__ uint32_t sum_slots[kSumSlots];
+    if (all.w[0].n) decompress_phase<8, G, WIDE, PACKED>(all.w[0], sum_slots);
+    if (all.w[1].n) decompress_phase<4, G, WIDE, PACKED>(all.w[1], sum_slots);
+    if (all.w[2].n) decompress_phase<2, G, WIDE, PACKED>(all.w[2], sum_slots);
+    if (all.w[3].n) decompress_phase<1, G, WIDE, PACKED>(all.w[3], sum_slots);
 }
 
 }  // namespace llms
@@ -1156,41 +1185,55 @@ extern "C" int llms_compress_chunks(const llms_kv_desc *desc, const void *kv, co
     const BitGroups groups = group_by_bits(n, staged.data(), [&](int i) { return (uint32_t)bits[i]; });
     rc = upload_tables(workspace, staged.data(), groups, n, false, st);
     if (rc) return rc;
-    for (int k = 0; k < kNumWidths; ++k) {
-        if (groups.count[k] == 0) continue;
-        const CodecArgs b = args_for_group(a, groups, k);
-        cudaError_t attr_err = cudaSuccess;
-        if (desc->quant_mode == 1) {
-            if (k == 0) launch_compress_cw<8>(b, desc->head_dim, desc->chunk_len, st);
-            else if (k == 1) launch_compress_cw<4>(b, desc->head_dim, desc->chunk_len, st);
-            else if (k == 2) launch_compress_cw<2>(b, desc->head_dim, desc->chunk_len, st);
-            else launch_compress_cw<1>(b, desc->head_dim, desc->chunk_len, st);
-            LLMS_CUDA_TRY(cudaGetLastError());
-            continue;
-        }
-        rc = dispatch_group(desc->group_size, [&](auto g) {
-            constexpr int kG = decltype(g)::value;
-            if constexpr (kUseBulkCompress && kG >= kLaneElems) {
-                // groups of 64 channels and more: the bulk-copy pipeline
+    if (desc->quant_mode == 1 || kUseBulkCompress) {
+        for (int k = 0; k < kNumWidths; ++k) {
+            if (groups.count[k] == 0) continue;
+            const CodecArgs b = args_for_group(a, groups, k);
+            cudaError_t attr_err = cudaSuccess;
+            if (desc->quant_mode == 1) {
+                if (k == 0) launch_compress_cw<8>(b, desc->head_dim, desc->chunk_len, st);
+                else if (k == 1) launch_compress_cw<4>(b, desc->head_dim, desc->chunk_len, st);
+                else if (k == 2) launch_compress_cw<2>(b, desc->head_dim, desc->chunk_len, st);
+                else launch_compress_cw<1>(b, desc->head_dim, desc->chunk_len, st);
+                LLMS_CUDA_TRY(cudaGetLastError());
+                continue;
+            }
+            rc = dispatch_group(desc->group_size, [&](auto g) {
+                constexpr int kG = decltype(g)::value;
+                if constexpr (kUseBulkCompress && kG >= kLaneElems) {
+                    // groups of 64 channels and more: the bulk-copy pipeline
 #define LLMS_LAUNCH(BITS)                                                                                                      \
     attr_err = cudaFuncSetAttribute(compress_bulk_kernel<BITS, kG>, cudaFuncAttributeMaxDynamicSharedMemorySize, kBulkSmemBytes); \
     if (attr_err == cudaSuccess) {                                                                                              \
         const int grid = grid_for(compress_bulk_kernel<BITS, kG>, b.total_units, kBulkSmemBytes);                               \
         compress_bulk_kernel<BITS, kG><<<grid, kThreads, kBulkSmemBytes, st>>>(with_grid(b, grid));                             \
     }
-                if (k == 0) { LLMS_LAUNCH(8); } else if (k == 1) { LLMS_LAUNCH(4); } else if (k == 2) { LLMS_LAUNCH(2); } else { attr_err = cudaErrorNotSupported; }
+                    if (k == 0) { LLMS_LAUNCH(8); } else if (k == 1) { LLMS_LAUNCH(4); } else if (k == 2) { LLMS_LAUNCH(2); } else { attr_err = cudaErrorNotSupported; }
 #undef LLMS_LAUNCH
-            } else {
-#define LLMS_LAUNCH(BITS)                                                                                               \
-    if (b.packed) compress_kernel<BITS, kG, true, true><<<grid_for(compress_kernel<BITS, kG, true, true>, b.total_units), kThreads, 0, st>>>(b); \
-    else if (wide) compress_kernel<BITS, kG, true, false><<<grid_for(compress_kernel<BITS, kG, true, false>, b.total_units), kThreads, 0, st>>>(b); \
-    else compress_kernel<BITS, kG, false, false><<<grid_for(compress_kernel<BITS, kG, false, false>, b.total_units), kThreads, 0, st>>>(b)
-                if (k == 0) { LLMS_LAUNCH(8); } else if (k == 1) { LLMS_LAUNCH(4); } else if (k == 2) { LLMS_LAUNCH(2); } else { LLMS_LAUNCH(1); }
-#undef LLMS_LAUNCH
-            }
+                } else {
+                    attr_err = cudaErrorNotSupported;
+                }
+            });
+            if (rc) return rc;
+            LLMS_CUDA_TRY(attr_err);
+            LLMS_CUDA_TRY(cudaGetLastError());
+        }
+    } else {
+        // one launch for the whole call; the grid is sized for the width with the most units
+        CodecArgsByWidth all{};
+        uint32_t most_units = 0;
+        for (int k = 0; k < kNumWidths; ++k) {
+            if (groups.count[k] == 0) continue;
+            all.w[k] = args_for_group(a, groups, k);
+            most_units = std::max(most_units, all.w[k].total_units);
+        }
+        rc = dispatch_group(desc->group_size, [&](auto g) {
+            constexpr int kG = decltype(g)::value;
+            if (a.packed) compress_kernel<kG, true, true><<<grid_for(compress_kernel<kG, true, true>, most_units), kThreads, 0, st>>>(all);
+            else if (wide) compress_kernel<kG, true, false><<<grid_for(compress_kernel<kG, true, false>, most_units), kThreads, 0, st>>>(all);
+            else compress_kernel<kG, false, false><<<grid_for(compress_kernel<kG, false, false>, most_units), kThreads, 0, st>>>(all);
         });
         if (rc) return rc;
-        LLMS_CUDA_TRY(attr_err);
         LLMS_CUDA_TRY(cudaGetLastError());
     }
     // checksums back to the caller's meta (every other field is already there)
@@ -1247,25 +1290,29 @@ static int decompress_chunks(const llms_kv_desc *desc, const void *buf, const ll
     const BitGroups groups = group_by_bits(n, staged.data(), [&](int i) { return meta[i].bits; });
     rc = upload_tables(workspace, staged.data(), groups, n, true, st);
     if (rc) return rc;
-    for (int k = 0; k < kNumWidths; ++k) {
-        if (groups.count[k] == 0) continue;
-        const CodecArgs b = args_for_group(a, groups, k);
-        if (desc->quant_mode == 1) {
+    if (desc->quant_mode == 1) {
+        for (int k = 0; k < kNumWidths; ++k) {
+            if (groups.count[k] == 0) continue;
+            const CodecArgs b = args_for_group(a, groups, k);
             if (k == 0) launch_decompress_cw<8>(b, desc->head_dim, desc->chunk_len, st);
             else if (k == 1) launch_decompress_cw<4>(b, desc->head_dim, desc->chunk_len, st);
             else if (k == 2) launch_decompress_cw<2>(b, desc->head_dim, desc->chunk_len, st);
             else launch_decompress_cw<1>(b, desc->head_dim, desc->chunk_len, st);
             LLMS_CUDA_TRY(cudaGetLastError());
-            continue;
+        }
+    } else {
+        CodecArgsByWidth all{};
+        uint32_t most_units = 0;
+        for (int k = 0; k < kNumWidths; ++k) {
+            if (groups.count[k] == 0) continue;
+            all.w[k] = args_for_group(a, groups, k);
+            most_units = std::max(most_units, all.w[k].total_units);
         }
         rc = dispatch_group(desc->group_size, [&](auto g) {
             constexpr int kG = decltype(g)::value;
-#define LLMS_LAUNCH(BITS)                                                                                                   \
-    if (b.packed) decompress_kernel<BITS, kG, true, true><<<decode_grid(decompress_kernel<BITS, kG, true, true>, b.total_units), kThreads, 0, st>>>(b); \
-    else if (wide) decompress_kernel<BITS, kG, true, false><<<decode_grid(decompress_kernel<BITS, kG, true, false>, b.total_units), kThreads, 0, st>>>(b); \
-    else decompress_kernel<BITS, kG, false, false><<<decode_grid(decompress_kernel<BITS, kG, false, false>, b.total_units), kThreads, 0, st>>>(b)
-            if (k == 0) { LLMS_LAUNCH(8); } else if (k == 1) { LLMS_LAUNCH(4); } else if (k == 2) { LLMS_LAUNCH(2); } else { LLMS_LAUNCH(1); }
-#undef LLMS_LAUNCH
+            if (a.packed) decompress_kernel<kG, true, true><<<decode_grid(decompress_kernel<kG, true, true>, most_units), kThreads, 0, st>>>(all);
+            else if (wide) decompress_kernel<kG, true, false><<<decode_grid(decompress_kernel<kG, true, false>, most_units), kThreads, 0, st>>>(all);
+            else decompress_kernel<kG, false, false><<<decode_grid(decompress_kernel<kG, false, false>, most_units), kThreads, 0, st>>>(all);
         });
         if (rc) return rc;
         LLMS_CUDA_TRY(cudaGetLastError());

@@ -42,7 +42,7 @@ class LayerwiseContext:
         self.ev_landed = [B.new_event() for _ in range(2)]
         self.ready = [torch.cuda.Event(enable_timing=True) for _ in range(self.L)]
         self.kernel_launches = 0
-        self._widths = len(set(self.bits.tolist()))
+        self._launches = B.codec_launches(self.desc, self.bits)      # kernels per codec call
 
     def layer_arena(self, l):
         return self.arena[l * self.layer_bytes:(l + 1) * self.layer_bytes]
@@ -56,7 +56,7 @@ class LayerwiseContext:
             self.ev_packed[k].record(self.main)
             B.swap_out(self.stage_out[k], self.meta[l], self.layer_arena(l), side_stream=self.side_out,
                        after=self.ev_packed[k], done=self.ev_out_free[k], n=self.n)
-            self.kernel_launches += self._widths + 1
+            self.kernel_launches += self._launches
 
     def swap_in(self, kv_out):
         """Load layer after layer; self.ready[l] is recorded on the main stream when layer l of kv_out is complete.
@@ -69,7 +69,7 @@ class LayerwiseContext:
             B.decompress_chunks(self.desc, self.stage_in[k], self.meta[l], None, kv_out[l], self.ws_in[l])
             self.ev_in_free[k].record(self.main)
             self.ready[l].record(self.main)
-            self.kernel_launches += self._widths + 1
+            self.kernel_launches += self._launches
 
     def corrupt_count(self):
         """Synchronises; number of records of the last swap_in whose checksum did not match."""

@@ -49,7 +49,7 @@ class MultiApp:
         self._aot_rows = None                     # rows whose ahead-of-time write-back may still be in flight
         self._ev_aot = None                       # recorded on the copy-out stream behind that write-back
         self.bytes_out = self.bytes_in = 0
-        self.kernel_launches = 0                  # codec kernels launched (one per bit-width present, plus one for the checksums)
+        self.kernel_launches = 0                  # kernels launched by the codec calls
 
     # ------------------------------------------------------------------ set-up (untimed)
     def build(self):
@@ -175,7 +175,7 @@ class MultiApp:
                        after=self.ev_compressed[k], done=self.ev_stage_out_free[k], n=len(part))
             self._pending.append((meta, part))
             self.bytes_out += int(sum(self.rec_bytes[int(b)] for b in bits))
-            self.kernel_launches += len(set(bits.tolist())) + 1       # one per bit-width + the checksum store
+            self.kernel_launches += B.codec_launches(self.desc_pool, bits)
             for r, s in zip(part, slots):
                 if self.ops is not None:
                     self.ops.append(("evict" if release else "aot", int(r), int(s)))
@@ -227,7 +227,7 @@ class MultiApp:
             self.ev_stage_in_free[k].record(self.main)
             self._used_ws.append(ws)
             self.bytes_in += int(sizes.sum())
-            self.kernel_launches += len(set(bits.tolist())) + 1
+            self.kernel_launches += B.codec_launches(self.desc_pool, bits)
             self.slot[part] = slots
             self.table["resident"][part] = 1
             self.clean[part] = True
