@@ -471,7 +471,7 @@ def run_ours(args):
     achieved = algo_bytes / (k_ms[dominant] * 1e-3) / 1e9
     roofline = {
         "kernel": dominant, "bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
-        "peak_source": f"{peak_kind} copy bandwidth", "launches_per_stage": B.codec_launches(d, bits) - 1,
+        "peak_source": f"{peak_kind} copy bandwidth", "launches_per_stage": B.codec_launches(d, bits) - (1 if args.quant_mode == 1 else 0),
         "traffic": (NCU_DRAM_TRAFFIC.get((shape.name, shape.n_layers, dominant))
                     if args.quant_mode == 0 and LEVELS == (8, 4, 2) and not args.chunk_len else None),
         "algorithmic_bytes_per_launch": algo_bytes,
@@ -504,8 +504,7 @@ def run_ours(args):
                 "serial_ms_per_step": e2e_serial_ms, "batch_chunks": e2e_batch,
                 "what": "compress -> swap-out to pinned host -> swap-in -> decompress, pipelined in batches of chunks",
                 "layerwise_load": layerwise},
-        # 4 score kernels, then per codec call one codec kernel (one per bit-width in channel-wise mode) and the kernel
-        # that stores or checks the sums
+        # 4 score kernels, then one codec kernel per call (channel-wise mode: one per bit-width and one for the sums)
         "gpu_launches": args.steps * (4 + 2 * B.codec_launches(d, bits)),
         "roofline": roofline, "clocks": clocks,
         "wall_ms_per_step": t_wall * 1e3 / args.steps,

@@ -205,9 +205,10 @@ def tolerance_workspace_bytes(desc, W):
 # ----------------------------------------------------------------------------- codec
 
 def codec_launches(desc, bits):
-    """Kernels one compress or decompress call launches: one codec kernel for the whole call (the bit-widths are phases
-    of it; channel-wise mode launches one per bit-width present) and one small kernel that stores or checks the sums."""
-    return (len(set(int(b) for b in bits)) if desc.quant_mode == 1 else 1) + 1
+    """Kernels one compress or decompress call launches.  Groups of channels of a token: one codec kernel for the whole
+    call (the bit-widths are phases of it, and its last CTA stores or checks the sums; a pageable meta array gets the
+    sums by a copy).  Channel-wise mode: one kernel per bit-width present and one small kernel for the sums."""
+    return len(set(int(b) for b in bits)) + 1 if desc.quant_mode == 1 else 1
 
 
 def compress_chunks(desc, kv, chunk_ids, bits, out_buf, meta, workspace, stream=None, out_bytes=None, workspace_bytes=None):

@@ -642,7 +642,29 @@ __device__ __forceinline__ void compress_phase(const CodecArgs &a, unsigned char
 // The launch arguments of a call, one set per bit-width (8, 4, 2, 1; n == 0: that width is absent).
 struct CodecArgsByWidth {
     CodecArgs w[4];
+    // what the CTA that finishes last does with the sums of the whole call
+    uint32_t *done;                   // third word of the workspace header: CTAs that have finished (starts at 0)
+    const ChunkEntry *entries;        // all n_total entries of the call
+    const uint32_t *sums;             // decoder: recomputed sums
+    uint32_t *status;                 // decoder: first word of the header, records whose sum is wrong
+    llms_chunk_meta *live_meta;       // the caller's meta array if the device can reach it (page-locked), else NULL
+    int n_total;
+    int expect_live;                  // decoder: 1 = the expected sums are read from live_meta now, 0 = from entries
 };
+
+// True in every thread of exactly one CTA of the grid: the one that comes here last.  Each thread's earlier atomics
+// on global memory are visible to that CTA's loads that bypass L1 (__ldcg).  Nobody waits for anybody.
+__device__ __forceinline__ bool cta_is_last(uint32_t *done)
+{
+    __shared__ uint32_t ticket;
+    __threadfence();
+    __syncthreads();
+    if (threadIdx.x == 0) ticket = atomicAdd(done, 1u);
+    __syncthreads();
+    const bool last = ticket == gridDim.x - 1;
+    if (last) __threadfence();
+    return last;
+}
 
 // One launch per call.  The bit-widths are phases in time, not branches per unit: every warp first works through
 // its share of the 8-bit chunks, then of the 4-bit ones, and so on, so the SM runs one code path at a time (with
@@ -658,6 +680,11 @@ __global__ void __launch_bounds__(kThreads, 2) compress_kernel(const __grid_cons
     if (all.w[1].n) compress_phase<4, G, WIDE, PACKED>(all.w[1], patches, sum_slots);
     if (all.w[2].n) compress_phase<2, G, WIDE, PACKED>(all.w[2], patches, sum_slots);
     if (all.w[3].n) compress_phase<1, G, WIDE, PACKED>(all.w[3], patches, sum_slots);
+    // The finished checksums go to the caller's page-locked meta array from the CTA that ends last (a kernel of its
+    // own for these few stores cost a launch boundary; a device-to-host copy would also queue on the copy engine
+    // behind whatever bulk copies other streams have in flight).
+    if (all.live_meta && cta_is_last(all.done))
+        for (int i = threadIdx.x; i < all.n_total; i += kThreads) all.live_meta[i].checksum = __ldcg(&all.entries[i].checksum);
 }
 
 // ---------------------------------------------------------------------------------------------- dequantize
@@ -889,6 +916,17 @@ __global__ void __launch_bounds__(kThreads, kDecodeBlocksPerSm) decompress_kerne
     if (all.w[1].n) decompress_phase<4, G, WIDE, PACKED>(all.w[1], sum_slots);
     if (all.w[2].n) decompress_phase<2, G, WIDE, PACKED>(all.w[2], sum_slots);
     if (all.w[3].n) decompress_phase<1, G, WIDE, PACKED>(all.w[3], sum_slots);
+    // the CTA that ends last compares every record's recomputed sum with the expected one
+    if (cta_is_last(all.done)) {
+        uint32_t bad = 0;
+        for (int i = threadIdx.x; i < all.n_total; i += kThreads) {
+            const uint32_t want = all.expect_live ? *reinterpret_cast<const volatile uint32_t *>(&all.live_meta[i].checksum)
+                                                  : __ldcg(&all.entries[i].checksum);
+            bad += __ldcg(&all.sums[i]) != want;
+        }
+        bad = __reduce_add_sync(0xffffffffu, bad);
+        if ((threadIdx.x & 31) == 0 && bad) atomicAdd(all.status, bad);
+    }
 }
 
 }  // namespace llms
@@ -1185,6 +1223,7 @@ extern "C" int llms_compress_chunks(const llms_kv_desc *desc, const void *kv, co
     const BitGroups groups = group_by_bits(n, staged.data(), [&](int i) { return (uint32_t)bits[i]; });
     rc = upload_tables(workspace, staged.data(), groups, n, false, st);
     if (rc) return rc;
+    bool published = false;  // the codec kernel itself stores the checksums into a page-locked meta array
     if (desc->quant_mode == 1 || kUseBulkCompress) {
         for (int k = 0; k < kNumWidths; ++k) {
             if (groups.count[k] == 0) continue;
@@ -1227,6 +1266,11 @@ extern "C" int llms_compress_chunks(const llms_kv_desc *desc, const void *kv, co
             all.w[k] = args_for_group(a, groups, k);
             most_units = std::max(most_units, all.w[k].total_units);
         }
+        all.done = static_cast<uint32_t *>(workspace) + 2;
+        all.entries = a.entries;
+        all.n_total = n;
+        all.live_meta = static_cast<llms_chunk_meta *>(device_view_of_pinned(meta));
+        published = all.live_meta != nullptr;
         rc = dispatch_group(desc->group_size, [&](auto g) {
             constexpr int kG = decltype(g)::value;
             if (a.packed) compress_kernel<kG, true, true><<<grid_for(compress_kernel<kG, true, true>, most_units), kThreads, 0, st>>>(all);
@@ -1237,7 +1281,9 @@ extern "C" int llms_compress_chunks(const llms_kv_desc *desc, const void *kv, co
         LLMS_CUDA_TRY(cudaGetLastError());
     }
     // checksums back to the caller's meta (every other field is already there)
-    if (void *live = device_view_of_pinned(meta)) {
+    if (published) {
+        // nothing left to do
+    } else if (void *live = device_view_of_pinned(meta)) {
         publish_checksums_kernel<<<(n + 255) / 256, 256, 0, st>>>(a.entries, static_cast<llms_chunk_meta *>(live), n);
         LLMS_CUDA_TRY(cudaGetLastError());
     } else {
@@ -1290,6 +1336,7 @@ static int decompress_chunks(const llms_kv_desc *desc, const void *buf, const ll
     const BitGroups groups = group_by_bits(n, staged.data(), [&](int i) { return meta[i].bits; });
     rc = upload_tables(workspace, staged.data(), groups, n, true, st);
     if (rc) return rc;
+    bool verified = false;  // the codec kernel itself checks the sums
     if (desc->quant_mode == 1) {
         for (int k = 0; k < kNumWidths; ++k) {
             if (groups.count[k] == 0) continue;
@@ -1308,6 +1355,14 @@ static int decompress_chunks(const llms_kv_desc *desc, const void *buf, const ll
             all.w[k] = args_for_group(a, groups, k);
             most_units = std::max(most_units, all.w[k].total_units);
         }
+        all.done = static_cast<uint32_t *>(workspace) + 2;
+        all.entries = a.entries;
+        all.sums = a.sums;
+        all.status = status;
+        all.n_total = n;
+        all.live_meta = const_cast<llms_chunk_meta *>(live_meta);
+        all.expect_live = live_meta != nullptr;
+        verified = true;
         rc = dispatch_group(desc->group_size, [&](auto g) {
             constexpr int kG = decltype(g)::value;
             if (a.packed) decompress_kernel<kG, true, true><<<decode_grid(decompress_kernel<kG, true, true>, most_units), kThreads, 0, st>>>(all);
@@ -1317,8 +1372,10 @@ static int decompress_chunks(const llms_kv_desc *desc, const void *buf, const ll
         if (rc) return rc;
         LLMS_CUDA_TRY(cudaGetLastError());
     }
-    verify_kernel<<<1, 256, 0, st>>>(a.entries, a.sums, n, status, live_meta);
-    LLMS_CUDA_TRY(cudaGetLastError());
+    if (!verified) {  // channel-wise launches: the check is a kernel of its own
+        verify_kernel<<<1, 256, 0, st>>>(a.entries, a.sums, n, status, live_meta);
+        LLMS_CUDA_TRY(cudaGetLastError());
+    }
     return LLMS_OK;
 }
 

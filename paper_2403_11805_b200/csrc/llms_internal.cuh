@@ -59,7 +59,7 @@ struct ChunkEntry {          // same bytes as llms_chunk_meta
 static_assert(sizeof(ChunkEntry) == sizeof(llms_chunk_meta) && sizeof(ChunkEntry) == 32, "meta layout");
 
 // Workspace of the codec calls:
-// [two status words, padded to 16 bytes][n entries][n 16-byte unit-table rows][n entry indices grouped by
+// [two status words and a count of finished CTAs, padded to 16 bytes][n entries][n 16-byte unit-table rows][n entry indices grouped by
 // bit-width][n recomputed sums].  Everything up to the sums is written by one host-to-device copy per call.
 constexpr uint64_t kWsEntriesOffset = 16;
 constexpr uint64_t kWsBytesPerChunk = sizeof(ChunkEntry) + 16 + 4 + 4;
