@@ -239,6 +239,8 @@ def run_ours(args):
     world = int(os.environ.get("WORLD_SIZE", "1"))
     rank = int(os.environ.get("RANK", "0"))
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    if world != args.gpus:
+        raise SystemExit(f"bench.py --gpus {args.gpus} was started with WORLD_SIZE={world}: one rank per GPU is expected")
     if not torch.cuda.is_available():
         raise SystemExit("bench.py needs a CUDA device: the hot path has no CPU fallback")
     torch.cuda.set_device(local_rank)
@@ -576,6 +578,13 @@ def main():
     assert len(LEVELS) == 3
     if args.impl == "reference":
         run_reference(args)
+    elif args.gpus > 1 and "WORLD_SIZE" not in os.environ:
+        # started as one plain process: become the launcher of args.gpus ranks, one per GPU, and relay their exit code
+        import torch
+        from paper_2403_11805_b200 import sharding
+        if torch.cuda.device_count() < args.gpus:
+            raise SystemExit(f"bench.py --gpus {args.gpus}: only {torch.cuda.device_count()} CUDA devices are visible")
+        sys.exit(sharding.launch_ranks(os.path.abspath(__file__), sys.argv[1:], args.gpus))
     elif args.workload == "multiapp":
         run_multiapp(args)
     else:

@@ -159,9 +159,12 @@ int llms_compress_chunks_static(const llms_kv_desc *desc, const void *kv, const 
  * are not touched.  While decoding, each record's checksum is recomputed; the number of
  * records whose sum differs from meta[i].checksum is left in the workspace and can be read
  * with llms_codec_corrupt_count (decoded values of such a record are still written).
- *   buf        device, 256-byte aligned;  meta, dst_chunk_ids  host;  kv_out  device fp16
+ *   buf        device, 256-byte aligned, buf_bytes long: a record that does not lie inside it
+ *              (meta[i].offset + meta[i].nbytes > buf_bytes) is refused with LLMS_ERR_BUF_TOO_SMALL
+ *              before anything is launched, so a stale or damaged meta table cannot turn into a read
+ *              outside the buffer;  meta, dst_chunk_ids  host;  kv_out  device fp16
  * Everything in meta, the expected checksums included, is read when the call is made. */
-int llms_decompress_chunks(const llms_kv_desc *desc, const void *buf, const llms_chunk_meta *meta,
+int llms_decompress_chunks(const llms_kv_desc *desc, const void *buf, uint64_t buf_bytes, const llms_chunk_meta *meta,
                            const uint32_t *dst_chunk_ids, int n, void *kv_out,
                            void *workspace, uint64_t workspace_bytes, void *stream);
 
@@ -171,7 +174,7 @@ int llms_decompress_chunks(const llms_kv_desc *desc, const void *buf, const llms
  * on the same stream and without a synchronisation in between, the llms_compress_chunks call that is still
  * producing those checksums into the same array.  The host must neither free nor change the array (a new
  * llms_compress_chunks into it changes it) until the stream has passed this call. */
-int llms_decompress_chunks_ordered(const llms_kv_desc *desc, const void *buf, const llms_chunk_meta *meta,
+int llms_decompress_chunks_ordered(const llms_kv_desc *desc, const void *buf, uint64_t buf_bytes, const llms_chunk_meta *meta,
                                    const uint32_t *dst_chunk_ids, int n, void *kv_out,
                                    void *workspace, uint64_t workspace_bytes, void *stream);
 
@@ -270,11 +273,12 @@ int llms_compress_context(const llms_kv_desc *desc, const void *kv, const void *
  * adjacent on both sides travel as one copy.  If `after` (a cudaEvent_t) is not NULL the side
  * stream first waits for it - record it on the stream that produced (swap-out) or last used
  * (swap-in) the device buffer.  If `done` is not NULL it is recorded on the side stream after
- * the last copy. */
-int llms_swap_out(const void *dev_buf, const llms_chunk_meta *meta, int n, void *pinned_dst,
-                  const uint64_t *host_offsets, void *side_stream, void *after, void *done);
-int llms_swap_in(const void *pinned_src, const uint64_t *host_offsets, const llms_chunk_meta *meta, int n,
-                 void *dev_buf, void *side_stream, void *after, void *done);
+ * the last copy.  dev_bytes and host_bytes are the sizes of the device buffer and of the arena: a
+ * record that ends beyond either is refused with LLMS_ERR_BUF_TOO_SMALL before any copy is queued. */
+int llms_swap_out(const void *dev_buf, uint64_t dev_bytes, const llms_chunk_meta *meta, int n, void *pinned_dst,
+                  uint64_t host_bytes, const uint64_t *host_offsets, void *side_stream, void *after, void *done);
+int llms_swap_in(const void *pinned_src, uint64_t host_bytes, const uint64_t *host_offsets, const llms_chunk_meta *meta,
+                 int n, void *dev_buf, uint64_t dev_bytes, void *side_stream, void *after, void *done);
 /* Poll a cudaEvent_t until it has completed or timeout_ms has passed (LLMS_ERR_TIMEOUT). */
 int llms_wait(void *event, uint32_t timeout_ms);
 

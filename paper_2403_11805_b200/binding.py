@@ -50,10 +50,10 @@ _SIGNATURES = {
                                        C.c_uint64, C.c_void_p, C.c_void_p, C.c_uint64, C.c_void_p]),
     "llms_compress_chunks_static": (C.c_int, [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_int, C.c_void_p,
                                               C.c_uint64, C.c_void_p, C.c_void_p]),
-    "llms_decompress_chunks": (C.c_int, [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_int, C.c_void_p,
+    "llms_decompress_chunks": (C.c_int, [C.c_void_p, C.c_void_p, C.c_uint64, C.c_void_p, C.c_void_p, C.c_int, C.c_void_p,
                                          C.c_void_p, C.c_uint64, C.c_void_p]),
-    "llms_decompress_chunks_ordered": (C.c_int, [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_int, C.c_void_p,
-                                         C.c_void_p, C.c_uint64, C.c_void_p]),
+    "llms_decompress_chunks_ordered": (C.c_int, [C.c_void_p, C.c_void_p, C.c_uint64, C.c_void_p, C.c_void_p, C.c_int,
+                                                 C.c_void_p, C.c_void_p, C.c_uint64, C.c_void_p]),
     "llms_codec_corrupt_count": (C.c_int, [C.c_void_p, C.c_void_p, C.c_void_p]),
     "llms_tolerance_workspace_bytes": (C.c_int, [C.c_void_p, C.c_int, C.c_void_p]),
     "llms_chunk_tolerance": (C.c_int, [C.c_void_p, C.c_void_p, C.c_void_p, C.c_int, C.c_void_p, C.c_void_p,
@@ -68,10 +68,10 @@ _SIGNATURES = {
                                         C.c_void_p, C.c_void_p, C.c_void_p, C.c_uint64, C.c_void_p, C.c_void_p, C.c_uint64,
                                         C.c_void_p, C.c_uint64, C.c_void_p, C.c_void_p]),
     "llms_lctru_order": (C.c_int, [C.c_void_p, C.c_int, C.c_void_p]),
-    "llms_swap_out": (C.c_int, [C.c_void_p, C.c_void_p, C.c_int, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p,
-                                C.c_void_p]),
-    "llms_swap_in": (C.c_int, [C.c_void_p, C.c_void_p, C.c_void_p, C.c_int, C.c_void_p, C.c_void_p, C.c_void_p,
-                               C.c_void_p]),
+    "llms_swap_out": (C.c_int, [C.c_void_p, C.c_uint64, C.c_void_p, C.c_int, C.c_void_p, C.c_uint64, C.c_void_p,
+                                C.c_void_p, C.c_void_p, C.c_void_p]),
+    "llms_swap_in": (C.c_int, [C.c_void_p, C.c_uint64, C.c_void_p, C.c_void_p, C.c_int, C.c_void_p, C.c_uint64,
+                               C.c_void_p, C.c_void_p, C.c_void_p]),
     "llms_wait": (C.c_int, [C.c_void_p, C.c_uint32]),
 }
 
@@ -234,20 +234,22 @@ def compress_chunks_static(desc, kv, chunk_ids, bits, out_buf, meta, stream=None
         _nbytes(out_buf) if out_bytes is None else out_bytes, _ptr(meta), _stream(stream)), "llms_compress_chunks_static")
 
 
-def decompress_chunks(desc, buf, meta, dst_chunk_ids, kv_out, workspace, stream=None, n=None, workspace_bytes=None):
+def decompress_chunks(desc, buf, meta, dst_chunk_ids, kv_out, workspace, stream=None, n=None, workspace_bytes=None,
+                      buf_bytes=None):
     ids = None if dst_chunk_ids is None else np.ascontiguousarray(dst_chunk_ids, dtype=np.uint32)
     n = len(meta) if n is None else n
     _check(lib().llms_decompress_chunks(
-        C.addressof(desc), _ptr(buf), _ptr(meta), _ptr(ids), n, _ptr(kv_out), _ptr(workspace),
+        C.addressof(desc), _ptr(buf), _nbytes(buf) if buf_bytes is None else buf_bytes, _ptr(meta), _ptr(ids), n, _ptr(kv_out), _ptr(workspace),
         _nbytes(workspace) if workspace_bytes is None else workspace_bytes, _stream(stream)), "llms_decompress_chunks")
 
 
-def decompress_chunks_ordered(desc, buf, meta, dst_chunk_ids, kv_out, workspace, stream=None, n=None, workspace_bytes=None):
+def decompress_chunks_ordered(desc, buf, meta, dst_chunk_ids, kv_out, workspace, stream=None, n=None, workspace_bytes=None,
+                              buf_bytes=None):
     """llms_decompress_chunks_ordered: meta pinned; its checksums are read by the device in stream order."""
     ids = None if dst_chunk_ids is None else np.ascontiguousarray(dst_chunk_ids, dtype=np.uint32)
     n = len(meta) if n is None else n
     _check(lib().llms_decompress_chunks_ordered(
-        C.addressof(desc), _ptr(buf), _ptr(meta), _ptr(ids), n, _ptr(kv_out), _ptr(workspace),
+        C.addressof(desc), _ptr(buf), _nbytes(buf) if buf_bytes is None else buf_bytes, _ptr(meta), _ptr(ids), n, _ptr(kv_out), _ptr(workspace),
         _nbytes(workspace) if workspace_bytes is None else workspace_bytes, _stream(stream)), "llms_decompress_chunks_ordered")
 
 
@@ -334,15 +336,21 @@ def compress_context(desc, kv, q_win, W, frac, levels, scores_dev, scores_host, 
 
 # ----------------------------------------------------------------------------- swap
 
-def swap_out(dev_buf, meta, pinned_dst, host_offsets=None, side_stream=None, after=None, done=None, n=None):
+def swap_out(dev_buf, meta, pinned_dst, host_offsets=None, side_stream=None, after=None, done=None, n=None,
+             dev_bytes=None, host_bytes=None):
     ho = None if host_offsets is None else np.ascontiguousarray(host_offsets, dtype=np.uint64)
-    _check(lib().llms_swap_out(_ptr(dev_buf), _ptr(meta), len(meta) if n is None else n, _ptr(pinned_dst), _ptr(ho),
+    _check(lib().llms_swap_out(_ptr(dev_buf), _nbytes(dev_buf) if dev_bytes is None else dev_bytes, _ptr(meta),
+                               len(meta) if n is None else n, _ptr(pinned_dst),
+                               _nbytes(pinned_dst) if host_bytes is None else host_bytes, _ptr(ho),
                                _stream(side_stream), _event(after), _event(done)), "llms_swap_out")
 
 
-def swap_in(pinned_src, meta, dev_buf, host_offsets=None, side_stream=None, after=None, done=None, n=None):
+def swap_in(pinned_src, meta, dev_buf, host_offsets=None, side_stream=None, after=None, done=None, n=None,
+            dev_bytes=None, host_bytes=None):
     ho = None if host_offsets is None else np.ascontiguousarray(host_offsets, dtype=np.uint64)
-    _check(lib().llms_swap_in(_ptr(pinned_src), _ptr(ho), _ptr(meta), len(meta) if n is None else n, _ptr(dev_buf),
+    _check(lib().llms_swap_in(_ptr(pinned_src), _nbytes(pinned_src) if host_bytes is None else host_bytes, _ptr(ho),
+                              _ptr(meta), len(meta) if n is None else n, _ptr(dev_buf),
+                              _nbytes(dev_buf) if dev_bytes is None else dev_bytes,
                               _stream(side_stream), _event(after), _event(done)), "llms_swap_in")
 
 

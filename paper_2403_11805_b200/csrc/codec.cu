@@ -1293,7 +1293,7 @@ extern "C" int llms_compress_chunks(const llms_kv_desc *desc, const void *kv, co
 }
 
 // live_checksums: the expected sums are read from the caller's pinned meta array by the device, in stream order
-static int decompress_chunks(const llms_kv_desc *desc, const void *buf, const llms_chunk_meta *meta,
+static int decompress_chunks(const llms_kv_desc *desc, const void *buf, uint64_t buf_bytes, const llms_chunk_meta *meta,
                              const uint32_t *dst_chunk_ids, int n, void *kv_out, void *workspace,
                              uint64_t workspace_bytes, void *stream, bool live_checksums)
 {
@@ -1321,6 +1321,8 @@ static int decompress_chunks(const llms_kv_desc *desc, const void *buf, const ll
         }
         if (meta[i].nbytes != bytes_at[b] || meta[i].n_groups != n_groups) return LLMS_ERR_INVALID_ARG;
         if (meta[i].offset % 256) return LLMS_ERR_MISALIGNED;
+        // the record lies inside the buffer (nothing here can wrap around: nbytes is the size just checked)
+        if (meta[i].nbytes > buf_bytes || meta[i].offset > buf_bytes - meta[i].nbytes) return LLMS_ERR_BUF_TOO_SMALL;
         const uint32_t dst = dst_chunk_ids ? dst_chunk_ids[i] : meta[i].chunk_id;
         if (dst >= nc || seen[dst]) return LLMS_ERR_INVALID_ARG;
         seen[dst] = 1;
@@ -1379,18 +1381,18 @@ static int decompress_chunks(const llms_kv_desc *desc, const void *buf, const ll
     return LLMS_OK;
 }
 
-extern "C" int llms_decompress_chunks(const llms_kv_desc *desc, const void *buf, const llms_chunk_meta *meta,
-                                      const uint32_t *dst_chunk_ids, int n, void *kv_out,
+extern "C" int llms_decompress_chunks(const llms_kv_desc *desc, const void *buf, uint64_t buf_bytes,
+                                      const llms_chunk_meta *meta, const uint32_t *dst_chunk_ids, int n, void *kv_out,
                                       void *workspace, uint64_t workspace_bytes, void *stream)
 {
-    return decompress_chunks(desc, buf, meta, dst_chunk_ids, n, kv_out, workspace, workspace_bytes, stream, false);
+    return decompress_chunks(desc, buf, buf_bytes, meta, dst_chunk_ids, n, kv_out, workspace, workspace_bytes, stream, false);
 }
 
-extern "C" int llms_decompress_chunks_ordered(const llms_kv_desc *desc, const void *buf, const llms_chunk_meta *meta,
-                                              const uint32_t *dst_chunk_ids, int n, void *kv_out,
+extern "C" int llms_decompress_chunks_ordered(const llms_kv_desc *desc, const void *buf, uint64_t buf_bytes,
+                                              const llms_chunk_meta *meta, const uint32_t *dst_chunk_ids, int n, void *kv_out,
                                               void *workspace, uint64_t workspace_bytes, void *stream)
 {
-    return decompress_chunks(desc, buf, meta, dst_chunk_ids, n, kv_out, workspace, workspace_bytes, stream, true);
+    return decompress_chunks(desc, buf, buf_bytes, meta, dst_chunk_ids, n, kv_out, workspace, workspace_bytes, stream, true);
 }
 
 extern "C" int llms_codec_corrupt_count(const void *workspace, uint32_t *n_corrupt, void *stream)

@@ -29,7 +29,8 @@ static int copy_records(uint8_t *dst, const uint8_t *src, const llms_chunk_meta 
     return LLMS_OK;
 }
 
-static int check_swap(const void *a, const void *b, const llms_chunk_meta *meta, const uint64_t *host_offsets, int n)
+static int check_swap(const void *a, const void *b, const llms_chunk_meta *meta, const uint64_t *host_offsets, int n,
+                      uint64_t dev_bytes, uint64_t host_bytes)
 {
     if (n < 0) return LLMS_ERR_INVALID_ARG;
     if (n == 0) return LLMS_OK;
@@ -39,6 +40,12 @@ static int check_swap(const void *a, const void *b, const llms_chunk_meta *meta,
         if (meta[i].nbytes == 0 || meta[i].nbytes % 256 || meta[i].offset % 256) return LLMS_ERR_MISALIGNED;
         if (host_offsets && host_offsets[i] % 16) return LLMS_ERR_MISALIGNED;
     }
+    // every record inside both buffers (written so that nothing can wrap around)
+    for (int i = 0; i < n; ++i) {
+        const uint64_t host_off = host_offsets ? host_offsets[i] : meta[i].offset;
+        if (meta[i].nbytes > dev_bytes || meta[i].offset > dev_bytes - meta[i].nbytes) return LLMS_ERR_BUF_TOO_SMALL;
+        if (meta[i].nbytes > host_bytes || host_off > host_bytes - meta[i].nbytes) return LLMS_ERR_BUF_TOO_SMALL;
+    }
     return LLMS_OK;
 }
 
@@ -46,10 +53,10 @@ static int check_swap(const void *a, const void *b, const llms_chunk_meta *meta,
 
 using namespace llms;
 
-extern "C" int llms_swap_out(const void *dev_buf, const llms_chunk_meta *meta, int n, void *pinned_dst,
-                             const uint64_t *host_offsets, void *side_stream, void *after, void *done)
+extern "C" int llms_swap_out(const void *dev_buf, uint64_t dev_bytes, const llms_chunk_meta *meta, int n, void *pinned_dst,
+                             uint64_t host_bytes, const uint64_t *host_offsets, void *side_stream, void *after, void *done)
 {
-    int rc = check_swap(dev_buf, pinned_dst, meta, host_offsets, n);
+    int rc = check_swap(dev_buf, pinned_dst, meta, host_offsets, n, dev_bytes, host_bytes);
     if (rc) return rc;
     cudaStream_t st = static_cast<cudaStream_t>(side_stream);
     if (after) LLMS_CUDA_TRY(cudaStreamWaitEvent(st, static_cast<cudaEvent_t>(after), 0));
@@ -59,10 +66,11 @@ extern "C" int llms_swap_out(const void *dev_buf, const llms_chunk_meta *meta, i
     return LLMS_OK;
 }
 
-extern "C" int llms_swap_in(const void *pinned_src, const uint64_t *host_offsets, const llms_chunk_meta *meta, int n,
-                            void *dev_buf, void *side_stream, void *after, void *done)
+extern "C" int llms_swap_in(const void *pinned_src, uint64_t host_bytes, const uint64_t *host_offsets,
+                            const llms_chunk_meta *meta, int n, void *dev_buf, uint64_t dev_bytes, void *side_stream,
+                            void *after, void *done)
 {
-    int rc = check_swap(pinned_src, dev_buf, meta, host_offsets, n);
+    int rc = check_swap(pinned_src, dev_buf, meta, host_offsets, n, dev_bytes, host_bytes);
     if (rc) return rc;
     cudaStream_t st = static_cast<cudaStream_t>(side_stream);
     if (after) LLMS_CUDA_TRY(cudaStreamWaitEvent(st, static_cast<cudaEvent_t>(after), 0));

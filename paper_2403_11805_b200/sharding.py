@@ -2,6 +2,11 @@
 contexts and nothing of the data path crosses ranks; only the timing is reduced (maximum over ranks).  Where a
 context's KV heads are split over the ranks instead (tensor-parallel serving), the codec still works per rank on its
 own heads and only the per-chunk scores of Eq. 1 are exchanged."""
+import os
+import socket
+import subprocess
+import sys
+
 import torch
 
 
@@ -42,3 +47,22 @@ def combine_head_sharded_scores(local_scores: torch.Tensor, dist=None):
         dist.all_reduce(t, op=dist.ReduceOp.SUM)
         t /= dist.get_world_size()
     return t
+
+
+def launch_ranks(script: str, argv, n_ranks: int, env=None) -> int:
+    """Start `script argv...` as n_ranks processes of one node (one per GPU) under torch.distributed.run, with the
+    rendezvous on 127.0.0.1 and a free port, and wait for them.  Each process finds RANK, LOCAL_RANK and WORLD_SIZE
+    in its environment.  Output passes through; the return value is the launcher's exit code (non-zero if any rank
+    failed).  Unless the caller's environment says otherwise, NCCL's initialisation log is switched on and sent to
+    stderr, so that the communicator's rank count can be read from a run's log without touching stdout."""
+    if n_ranks < 1:
+        raise ValueError("need at least one rank")
+    with socket.socket(socket.AF_INET, socket.SOCK_STREAM) as s:
+        s.bind(("127.0.0.1", 0))
+        port = s.getsockname()[1]
+    child_env = dict(os.environ if env is None else env)
+    if "NCCL_DEBUG" not in child_env:
+        child_env.update(NCCL_DEBUG="INFO", NCCL_DEBUG_SUBSYS="INIT", NCCL_DEBUG_FILE="/dev/stderr")
+    cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", f"--nproc-per-node={n_ranks}",
+           "--master-addr", "127.0.0.1", "--master-port", str(port), script] + list(argv)
+    return subprocess.run(cmd, env=child_env).returncode

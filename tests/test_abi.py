@@ -161,3 +161,40 @@ def test_argument_errors_on_the_host():
     assert call(ids=ok_ids, desc=d2) == B.ERR_UNSUPPORTED
     assert B.lib().llms_wait(None, 1) == B.ERR_INVALID_ARG
     assert B.lib().llms_strerror(B.ERR_CORRUPT).decode() == "record checksum mismatch"
+
+
+def test_records_outside_their_buffers_are_refused_on_the_host():
+    """A meta table that points past the end of the swap buffer or of the arena (stale, damaged) is an error code,
+    found before anything is enqueued: the addresses here are dummies that no kernel or copy could survive."""
+    sh = synth.CONFIGS["tiny"]
+    d = B.desc_of(sh)
+    lib = B.lib()
+    nb8, nb4 = B.record_bytes(d, 8), B.record_bytes(d, 4)
+    meta = B.new_meta(2)
+    meta["chunk_id"] = [0, 1]
+    meta["bits"] = [8, 4]
+    meta["offset"] = [0, nb8]
+    meta["nbytes"] = [nb8, nb4]
+    meta["n_groups"] = sh.n_slabs * sh.chunk_len * (sh.head_dim // sh.group_size)
+    for fn in (lib.llms_decompress_chunks,):
+        dec = lambda buf_bytes, m=meta: fn(ctypes.addressof(d), 8192, buf_bytes, B._ptr(m), None, 2, 4096, 4096, 4096, None)
+        assert dec(nb8 + nb4 - 1) == B.ERR_BUF_TOO_SMALL
+        assert dec(nb8) == B.ERR_BUF_TOO_SMALL
+        assert dec(0) == B.ERR_BUF_TOO_SMALL
+        far = meta.copy()
+        far["offset"][1] = (1 << 64) - 256                               # offset + nbytes wraps around
+        assert dec(1 << 40, far) == B.ERR_BUF_TOO_SMALL
+        wrong = meta.copy()
+        wrong["nbytes"][1] = nb8                                         # not the size of a 4-bit record
+        assert dec(1 << 40, wrong) == B.ERR_INVALID_ARG
+    out = lambda dev_bytes, host_bytes, ho=None, m=meta: lib.llms_swap_out(
+        8192, dev_bytes, B._ptr(m), 2, 1 << 20, host_bytes, B._ptr(ho), None, None, None)
+    inn = lambda dev_bytes, host_bytes, ho=None, m=meta: lib.llms_swap_in(
+        1 << 20, host_bytes, B._ptr(ho), B._ptr(m), 2, 8192, dev_bytes, None, None, None)
+    for call in (out, inn):
+        assert call(nb8 + nb4 - 256, 1 << 30) == B.ERR_BUF_TOO_SMALL     # device buffer too short
+        assert call(1 << 30, nb8 + nb4 - 256) == B.ERR_BUF_TOO_SMALL     # arena too short at the same offsets
+        ho = np.array([0, 1 << 20], dtype=np.uint64)
+        assert call(1 << 30, (1 << 20) + nb4 - 16, ho) == B.ERR_BUF_TOO_SMALL   # arena too short at its own offsets
+        ho[1] = (1 << 64) - 16
+        assert call(1 << 30, 1 << 40, ho) == B.ERR_BUF_TOO_SMALL         # wraps around

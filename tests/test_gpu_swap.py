@@ -92,6 +92,6 @@ def test_wait_times_out_and_then_succeeds():
 def test_swap_argument_errors():
     meta = B.new_meta(1)
     meta[0]["nbytes"] = 100          # not a multiple of 256
-    assert B.lib().llms_swap_out(4096, meta.ctypes.data, 1, 8192, None, None, None, None) == B.ERR_MISALIGNED
-    assert B.lib().llms_swap_out(None, meta.ctypes.data, 1, 8192, None, None, None, None) == B.ERR_INVALID_ARG
-    assert B.lib().llms_swap_in(4096, None, meta.ctypes.data, 0, 8192, None, None, None) == B.OK
+    assert B.lib().llms_swap_out(4096, 1 << 20, meta.ctypes.data, 1, 8192, 1 << 20, None, None, None, None) == B.ERR_MISALIGNED
+    assert B.lib().llms_swap_out(None, 1 << 20, meta.ctypes.data, 1, 8192, 1 << 20, None, None, None, None) == B.ERR_INVALID_ARG
+    assert B.lib().llms_swap_in(4096, 0, None, meta.ctypes.data, 0, 8192, 0, None, None, None) == B.OK

@@ -108,3 +108,36 @@ def test_heads_of_rank_blocks():
         sharding.heads_of_rank(1, 8, 0, 2)                 # one KV head cannot be split
     t = torch.tensor([0.25, 0.5])
     assert torch.equal(sharding.combine_head_sharded_scores(t), t)
+
+
+def test_launcher_starts_one_process_per_rank():
+    """sharding.launch_ranks (what `bench.py --gpus N` becomes when it is started as one plain process): two ranks
+    come up with the rendezvous on 127.0.0.1, rank 0 prints one JSON line, a failing rank fails the launch."""
+    import json
+    import subprocess
+    import sys
+    here = os.path.dirname(os.path.abspath(__file__))
+    code = ("import sys; from paper_2403_11805_b200 import sharding; "
+            "sys.exit(sharding.launch_ranks(sys.argv[1], sys.argv[2:], 2))")
+    env = dict(os.environ, PYTHONPATH=os.path.dirname(here))
+    for k in ("RANK", "WORLD_SIZE", "LOCAL_RANK", "MASTER_ADDR", "MASTER_PORT"):
+        env.pop(k, None)
+    run = subprocess.run([sys.executable, "-c", code, os.path.join(here, "rank_stub.py"), "--steps", "3"],
+                         env=env, capture_output=True, text=True, timeout=300)
+    assert run.returncode == 0, run.stderr[-2000:]
+    lines = [json.loads(l) for l in run.stdout.splitlines() if l.startswith("{")]
+    assert lines == [{"n_gpus": 2, "ms_per_step": 11.0, "argv": ["--steps", "3"]}]
+    bad = subprocess.run([sys.executable, "-c", code, os.path.join(here, "rank_stub.py"), "--fail"],
+                         env=env, capture_output=True, text=True, timeout=300)
+    assert bad.returncode != 0
+
+
+def test_bench_refuses_a_rank_count_it_was_not_started_with():
+    """Under a launcher, bench.py's --gpus must equal WORLD_SIZE (checked before any CUDA call)."""
+    import subprocess
+    import sys
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    env = dict(os.environ, WORLD_SIZE="2", RANK="0", LOCAL_RANK="0")
+    run = subprocess.run([sys.executable, os.path.join(root, "bench.py"), "--gpus", "4"], env=env, capture_output=True,
+                         text=True, timeout=300)
+    assert run.returncode != 0 and "WORLD_SIZE=2" in run.stderr
