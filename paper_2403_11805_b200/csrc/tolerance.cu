@@ -4,8 +4,8 @@
 // From K and the last W queries: K is streamed once.  The logits S = K q^T are a dense contraction and run as
 // warp-level tensor-core MMAs (logits_mma_kernel; an fp32-FMA kernel with a thread per token remains for head
 // dimensions the MMA kernel does not take).  The rows' softmax statistics are kept per *segment* of SEG
-// neighbouring tokens (SEG = the largest power of two <= 32 that divides chunk_len), as (segment max, sum of exp,
-// 1/n_vis-weighted sum of exp).  Three small kernels then turn the per-segment statistics into row normalisers,
+// neighbouring tokens (SEG = the largest power of two <= 32 that divides chunk_len), as (segment max, sum of exp)
+// and, for the few segments that reach into the last W columns, the 1/n_vis-weighted sum of exp.  Three small kernels then turn the per-segment statistics into row normalisers,
 // column means and chunk means.  All sums run in a fixed order, so the scores - and the ranking made from them -
 // are reproducible bit for bit.
 #include <math.h>
@@ -26,11 +26,13 @@ struct TolArgs {
     int rep;          // query heads per KV head
     int NR;           // rep * W query rows per KV head
     int n_seg;        // ceil(T / SEG)
+    int seg_tail0;    // first segment that holds a token of the last W - 1 columns (where rows stop seeing tokens)
     int seg_per_chunk;
     int n_chunks;
     int64_t stride_l, stride_h;
     float inv_sqrt_d;
-    float *pm, *ps, *pp;      // [rows][n_seg]: segment max, sum exp, weighted sum exp
+    float *pm, *ps, *pp;      // [rows][n_seg]: segment max, sum of exp, 1/n_vis-weighted sum of exp (pp: only the
+                              // segments from seg_tail0 on are read; before them it is ps / W)
     float *row_max, *row_inv; // [rows]
     float *part;              // [Y][n_seg]
     float *scores;
@@ -115,15 +117,20 @@ __global__ void __launch_bounds__(kTokThreads) logits_kernel(const TolArgs a)
 
 // ------------------------------------------------------------------ the same on the tensor cores
 //
-// S = K q^T is a dense contraction (tokens x head_dim times head_dim x window rows): with plain fp32 fma the
-// kernel is bound by instruction issue (measured 0.56 ms for the 7B shape against 0.17 ms for reading K once),
-// so for head_dim 64, 128 and 256 it runs as warp-level matrix multiply-accumulate, m16n8k16 with fp16 inputs
-// and fp32 accumulators: 8 window rows are exactly one n-tile.  A warp owns tiles of 32 consecutive tokens of one
-// (layer, KV head).  It copies a tile (32 x head_dim fp16, contiguous in memory) into shared memory with
-// coalesced 16-byte asynchronous copies (cp.async, two buffers: the next tile lands while this one is used),
+// S = q K^T is a dense contraction (window rows x head_dim times head_dim x tokens): with plain fp32 fma the kernel
+// is bound by instruction issue (measured 0.56 ms for the 7B shape against 0.17 ms for reading K once), so for
+// head_dim 64, 128 and 256 it runs as warp-level matrix multiply-accumulate, m16n8k16 with fp16 inputs and fp32
+// accumulators.  A warp owns tiles of 32 consecutive tokens of one (layer, KV head).  It copies a tile
+// (32 x head_dim fp16, contiguous in memory) into shared memory with coalesced 16-byte asynchronous copies,
 // swizzled by XOR-ing the 16-byte chunk index with the row index so that ldmatrix reads without bank conflicts.
-// The window's query rows sit in shared memory (rows padded by 16 bytes against conflicts) and are read as B
-// fragments.  The softmax statistics are then taken straight from the accumulator fragments.
+//
+// The window's query rows are the M side of the product (A operand, 16 rows per m-tile, rows of shared memory padded
+// by 16 bytes against conflicts) and the tile's tokens the N side (B operand, four n-tiles of 8 tokens).  An
+// accumulator fragment then holds, per lane, two window rows (g and g + 8) and for each of them eight tokens of the
+// tile (2*q4, 2*q4 + 1 of every n-tile): the softmax statistics of a row over a segment of tokens are mostly sums
+// inside a lane, finished by at most two shuffle steps.  (With the tokens on the M side, as this kernel first had
+// them, every statistic took three shuffle steps per pair of values and the kernel spent two thirds of its 1180
+// instructions per tile there: 0.52 ms for the 32K grouped-query shape, whose K streams past in 0.33 ms.)
 constexpr int kTileTokens = 32;
 constexpr int kTileWarps = 12;     // most warps a CTA is launched with; 8 when twelve tiles do not fit twice into an SM
 constexpr int kTileWarpsSmall = 8;  // (measured on the 7B shape: 12 warps x 2 CTAs 0.2175 ms, 8 x 3 0.227, 4 x 6 0.269)
@@ -148,112 +155,130 @@ __device__ __forceinline__ void mma_16816(float (&c)[4], const uint32_t (&a)[4],
     asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
                  : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3]) : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
 }
+// 2^x, one instruction (relative error about 2^-22; results below the normal range become 0)
+__device__ __forceinline__ float ex2_approx(float x)
+{
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
 
-// Reduce the four values a lane holds for one window row (tokens mb*16 + half*8 + g, g = lane/4) over the
-// tokens of each SEG-token segment; afterwards every slot holds its segment's result.
+// x[nt][e] belongs to token nt*8 + 2*q4 + e of the tile (q4 = lane & 3).  Reduce over the tokens of each SEG-token
+// segment; afterwards every slot holds its segment's result.  The order of the operations is fixed by SEG alone.
 template <int SEG, typename Op>
-__device__ __forceinline__ void segment_reduce(float (&x)[2][2], Op op)
+__device__ __forceinline__ void segment_reduce(float (&x)[4][2], Op op)
 {
-    if constexpr (SEG == 32) x[0][0] = op(op(x[0][0], x[0][1]), op(x[1][0], x[1][1]));
-    if constexpr (SEG == 16) {
-        x[0][0] = op(x[0][0], x[0][1]);
-        x[1][0] = op(x[1][0], x[1][1]);
-    }
+    if constexpr (SEG >= 2) {
+        float r[4];
 #pragma unroll
-    for (int mb = 0; mb < 2; ++mb)
-#pragma unroll
-        for (int h = 0; h < 2; ++h) {
-            if ((SEG == 32 && (mb || h)) || (SEG == 16 && h)) continue;  // folded into another slot above
-            float v = x[mb][h];
-            if constexpr (SEG >= 2) v = op(v, __shfl_xor_sync(0xffffffffu, v, 4));
-            if constexpr (SEG >= 4) v = op(v, __shfl_xor_sync(0xffffffffu, v, 8));
-            if constexpr (SEG >= 8) v = op(v, __shfl_xor_sync(0xffffffffu, v, 16));
-            x[mb][h] = v;
+        for (int nt = 0; nt < 4; ++nt) r[nt] = op(x[nt][0], x[nt][1]);
+        if constexpr (SEG == 32) r[0] = op(op(r[0], r[1]), op(r[2], r[3]));
+        if constexpr (SEG == 16) {
+            r[0] = op(r[0], r[1]);
+            r[2] = op(r[2], r[3]);
         }
-    if constexpr (SEG == 32) x[0][1] = x[1][0] = x[1][1] = x[0][0];
-    if constexpr (SEG == 16) {
-        x[0][1] = x[0][0];
-        x[1][1] = x[1][0];
+#pragma unroll
+        for (int nt = 0; nt < 4; ++nt) {
+            if ((SEG == 32 && nt) || (SEG == 16 && (nt & 1))) continue;  // folded into another slot above
+            if constexpr (SEG >= 4) r[nt] = op(r[nt], __shfl_xor_sync(0xffffffffu, r[nt], 1));
+            if constexpr (SEG >= 8) r[nt] = op(r[nt], __shfl_xor_sync(0xffffffffu, r[nt], 2));
+        }
+        if constexpr (SEG == 32) r[1] = r[2] = r[3] = r[0];
+        if constexpr (SEG == 16) {
+            r[1] = r[0];
+            r[3] = r[2];
+        }
+#pragma unroll
+        for (int nt = 0; nt < 4; ++nt) x[nt][0] = x[nt][1] = r[nt];
     }
 }
 
-// Softmax statistics of one n-tile (8 flattened window rows) from the accumulator fragments of a 32-token tile.
-// TAIL: the tile reaches into the last W columns, where rows stop seeing tokens and 1/n_vis varies; everywhere
-// else every row sees every token of the tile and the column weight is 1/W, so masks and weighted sums drop out.
+// Softmax statistics of one window row over the 32 tokens of a tile, from the eight dot products this lane holds
+// for it.  TAIL: the tile reaches into the last W columns, where rows stop seeing tokens and 1/n_vis varies;
+// everywhere else every row sees every token of the tile, and the 1/n_vis-weighted sum is the plain sum over W
+// (the column kernel applies that factor), so masks and weights drop out.
+//   dot[nt][e]  raw q.k of token tile*32 + nt*8 + 2*q4 + e;  j  the row's index among the KV head's rows;
+//   valid  false for the zero rows that pad the last m-tile (they take part in the shuffles and store nothing);
+//   last_col  (TAIL) the last token the row sees
 template <int SEG, bool TAIL>
-__device__ __forceinline__ void tile_statistics(const TolArgs &a, const float (&acc)[2][4], int nb, int q4, const int *last_col_s,
-                                                const int (&t_tok)[2][2], const float (&w_tok)[2][2], const bool (&opens)[2][2],
-                                                int64_t row0)
+__device__ __forceinline__ void row_statistics(const TolArgs &a, const float (&dot)[4][2], int tile, int q4, int j, bool valid,
+                                               int last_col, int64_t row0)
 {
-    const float inv_w = 1.0f / (float)a.W;
+    constexpr float kLog2e = 1.4426950408889634f;
+    const float c1 = a.inv_sqrt_d * kLog2e;                 // logit in units of log 2
+    const int t0 = tile * kTileTokens + 2 * q4;             // this lane's first token of the tile
+    float v[4][2], mx[4][2];
 #pragma unroll
-    for (int col = 0; col < 2; ++col) {
-        const int j = nb * 8 + 2 * q4 + col;       // flattened (head, window row)
-        const int last_col = last_col_s[j];        // last token this row sees; -1 for the zero padding rows
-        float lg[2][2], mx[2][2], se[2][2], sp[2][2];
+    for (int nt = 0; nt < 4; ++nt)
 #pragma unroll
-        for (int mb = 0; mb < 2; ++mb)
-#pragma unroll
-            for (int h = 0; h < 2; ++h) {
-                lg[mb][h] = acc[mb][2 * h + col] * a.inv_sqrt_d;
-                if constexpr (TAIL) lg[mb][h] = t_tok[mb][h] <= last_col ? lg[mb][h] : -INFINITY;
-                mx[mb][h] = lg[mb][h];
-            }
-        segment_reduce<SEG>(mx, [](float x, float y) { return fmaxf(x, y); });
-#pragma unroll
-        for (int mb = 0; mb < 2; ++mb)
-#pragma unroll
-            for (int h = 0; h < 2; ++h) {
-                // exp2-based exponential: relative error of a few 1e-6 for the arguments met here
-                float e = __expf(lg[mb][h] - mx[mb][h]);
-                if constexpr (TAIL) e = lg[mb][h] == -INFINITY ? 0.0f : e;
-                se[mb][h] = e;
-                if constexpr (TAIL) sp[mb][h] = e * w_tok[mb][h];
-            }
-        segment_reduce<SEG>(se, [](float x, float y) { return x + y; });
-        if constexpr (TAIL) segment_reduce<SEG>(sp, [](float x, float y) { return x + y; });
-        if (last_col >= 0) {
-#pragma unroll
-            for (int mb = 0; mb < 2; ++mb)
-#pragma unroll
-                for (int h = 0; h < 2; ++h) {
-                    if (opens[mb][h]) {   // the segment's first token writes
-                        const int64_t o = (row0 + j) * a.n_seg + t_tok[mb][h] / SEG;
-                        a.pm[o] = mx[mb][h];
-                        a.ps[o] = se[mb][h];
-                        a.pp[o] = TAIL ? sp[mb][h] : se[mb][h] * inv_w;
-                    }
-                }
+        for (int e = 0; e < 2; ++e) {
+            v[nt][e] = dot[nt][e];
+            if constexpr (TAIL) v[nt][e] = t0 + nt * 8 + e <= last_col ? v[nt][e] : -INFINITY;
+            mx[nt][e] = v[nt][e];
         }
-    }
+    segment_reduce<SEG>(mx, [](float x, float y) { return fmaxf(x, y); });
+    float se[4][2], sp[4][2];
+#pragma unroll
+    for (int nt = 0; nt < 4; ++nt)
+#pragma unroll
+        for (int e = 0; e < 2; ++e) {
+            // exp((v - max)/sqrt(d)) as 2^(v*c1 - max*c1): one fused multiply-add and one ex2
+            float p = ex2_approx(__fmaf_rn(v[nt][e], c1, -(mx[nt][e] * c1)));
+            if constexpr (TAIL) {
+                p = v[nt][e] == -INFINITY ? 0.0f : p;       // also the segments no token of which is visible (max = -inf)
+                const int n_vis = min(a.W, max(1, a.T - (t0 + nt * 8 + e)));
+                sp[nt][e] = p * (1.0f / (float)n_vis);
+            }
+            se[nt][e] = p;
+        }
+    segment_reduce<SEG>(se, [](float x, float y) { return x + y; });
+    if constexpr (TAIL) segment_reduce<SEG>(sp, [](float x, float y) { return x + y; });
+#pragma unroll
+    for (int nt = 0; nt < 4; ++nt)
+#pragma unroll
+        for (int e = 0; e < 2; ++e) {
+            if ((SEG >= 2 && e == 1) || (SEG >= 16 && (nt * 8) % SEG != 0)) continue;  // never a segment's first token
+            const int t = t0 + nt * 8 + e;
+            if (valid && t % SEG == 0 && t < a.T) {           // the segment's first token writes
+                const int seg = t / SEG;
+                const int64_t o = (row0 + j) * a.n_seg + seg;
+                a.pm[o] = mx[nt][e] * a.inv_sqrt_d;
+                a.ps[o] = se[nt][e];
+                if constexpr (TAIL)
+                    if (seg >= a.seg_tail0) a.pp[o] = sp[nt][e];
+            }
+        }
 }
 
-// NBG: n-tiles (8 flattened window rows each) that share one pass over a tile's A fragments - 4 for grouped-query
-// shapes whose rows come in multiples of 32 per KV head, else 1.
-template <int SEG, int D, int NBG>
+// MTG: m-tiles (16 flattened window rows each) that share one pass over a tile's B fragments - 2 where a KV head
+// has more than 16 rows (grouped-query shapes), else 1.
+template <int SEG, int D, int MTG>
 __global__ void __launch_bounds__(kTileWarps * 32, 2) logits_mma_kernel(const TolArgs a)
 {
     constexpr int kRowBytes = D * 2, kChunks = D / 8, kTileBytes = kTileTokens * kRowBytes;
-    constexpr int kQRowBytes = kRowBytes + 16;                               // padded: B fragments read conflict-free
-    extern __shared__ __align__(128) unsigned char smem_raw[];
+    constexpr int kQRowBytes = kRowBytes + 16;                               // padded: A fragments read conflict-free
+    static_assert(kTileBytes % 1024 == 0 && kRowBytes <= 1024, "tile buffers keep the alignment the swizzle relies on");
+    extern __shared__ __align__(256) unsigned char smem_raw[];
     const int lane = threadIdx.x & 31, wib = threadIdx.x >> 5;
     const int g = lane >> 2, q4 = lane & 3;
-    const int n_blocks = (a.NR + 7) / 8;                                     // window rows in n-tiles of 8, zero padded
-    unsigned char *q_s = smem_raw;                                           // [n_blocks*8][kQRowBytes]
-    const int q_total = (n_blocks * 8 * kQRowBytes + 127) / 128 * 128;
-    int *last_col_s = reinterpret_cast<int *>(smem_raw + q_total);           // [n_blocks*8]: last token a row sees
-    const int lc_total = (n_blocks * 8 * 4 + 127) / 128 * 128;
-    unsigned char *tiles = smem_raw + q_total + lc_total + wib * kTileBuffers * kTileBytes;   // this warp's buffers
-    const uint32_t tiles_s = (uint32_t)__cvta_generic_to_shared(tiles);
+    const int n_mt = (a.NR + 15) / 16;                                       // window rows in m-tiles of 16, zero padded
+    unsigned char *q_s = smem_raw;                                           // [n_mt*16][kQRowBytes]
+    const int q_total = (n_mt * 16 * kQRowBytes + 255) / 256 * 256;
+    int *last_col_s = reinterpret_cast<int *>(smem_raw + q_total);           // [n_mt*16]: last token a row sees
+    const int lc_total = (n_mt * 16 * 4 + 255) / 256 * 256;
+    // this warp's tile buffers, aligned to a 1 KiB boundary whatever the base of the dynamic shared memory: every bit
+    // of a chunk index then sits below the buffer's address bits and a chunk's swizzle is an XOR on the whole address
+    const uint32_t tiles_s = (((uint32_t)__cvta_generic_to_shared(smem_raw) + q_total + lc_total + 1023u) & ~1023u) +
+                             wib * kTileBuffers * kTileBytes;
 
     const int l = blockIdx.y / a.Hkv, kvh = blockIdx.y % a.Hkv;
     const __half *q_src = a.q_win + ((int64_t)(l * a.Hq + kvh * a.rep) * a.W) * D;
-    for (int i = threadIdx.x; i < n_blocks * 8 * kChunks; i += blockDim.x) {
+    for (int i = threadIdx.x; i < n_mt * 16 * kChunks; i += blockDim.x) {
         const int row = i / kChunks, c = i % kChunks;
         *reinterpret_cast<uint4 *>(q_s + row * kQRowBytes + c * 16) =
             row < a.NR ? __ldg(reinterpret_cast<const uint4 *>(q_src) + i) : make_uint4(0, 0, 0, 0);
     }
-    for (int j = threadIdx.x; j < n_blocks * 8; j += blockDim.x) last_col_s[j] = j < a.NR ? a.T - a.W + j % a.W : -1;
+    for (int j = threadIdx.x; j < n_mt * 16; j += blockDim.x) last_col_s[j] = j < a.NR ? a.T - a.W + j % a.W : -1;
     __syncthreads();
 
     const __half *k_plane = a.kv + (int64_t)l * a.stride_l + (int64_t)kvh * a.stride_h;
@@ -279,8 +304,12 @@ __global__ void __launch_bounds__(kTileWarps * 32, 2) logits_mma_kernel(const To
         cp_async_commit();
     };
 
-    // ldmatrix x4 of a 16 x 16 block: lanes 0-15 give the rows at column chunk 2*ks, lanes 16-31 at 2*ks + 1
-    const int a_row = lane & 15, a_chunk = lane >> 4;
+    // B fragments (tokens x channels as the "column" operand): one ldmatrix x4 covers 16 tokens and 16 channels.
+    // Lane L addresses token (L/16)*8 + L%8 of the 16 at channel chunk 2*ks + (L/8)%2; its row's swizzle (token & 7
+    // = L & 7) and the chunk's low bit fold into a per-lane base, the rest of the chunk index is an XOR of ks << 5.
+    const uint32_t b_lane = (uint32_t)((((lane >> 4) << 3) + (lane & 7)) * kRowBytes + ((((lane >> 3) & 1) ^ (lane & 7)) << 4));
+    // A fragments (window rows x channels): lanes 0-15 give rows 0-15 at chunk 2*ks, lanes 16-31 at chunk 2*ks + 1
+    const uint32_t a_lane = (uint32_t)__cvta_generic_to_shared(q_s) + (lane & 15) * kQRowBytes + ((lane >> 4) << 4);
 
     int buf = 0;
     if (kTileBuffers == 2 && tile_begin < tile_end) issue_tile(tile_begin, 0);
@@ -296,50 +325,49 @@ __global__ void __launch_bounds__(kTileWarps * 32, 2) logits_mma_kernel(const To
             cp_async_wait<0>();
         }
         __syncwarp();
-        const uint32_t tile_s = tiles_s + buf * kTileBytes;
-        // this lane's four tokens of the tile, their column weights 1/n_vis, and whether they open a segment
-        int t_tok[2][2];
-        float w_tok[2][2];
-        bool opens[2][2];
-#pragma unroll
-        for (int mb = 0; mb < 2; ++mb)
-#pragma unroll
-            for (int h = 0; h < 2; ++h) {
-                t_tok[mb][h] = tile * kTileTokens + mb * 16 + h * 8 + g;
-                w_tok[mb][h] = 1.0f / (float)min(a.W, max(1, a.T - t_tok[mb][h]));
-                opens[mb][h] = t_tok[mb][h] < a.T && t_tok[mb][h] % SEG == 0;
-            }
+        const uint32_t tile_s = tiles_s + buf * kTileBytes + b_lane;
         const bool tail_tile = tile * kTileTokens + kTileTokens > a.T - a.W + 1;
-        for (int nb0 = 0; nb0 < n_blocks; nb0 += NBG) {
-            float acc[NBG][2][4];
+        for (int mt0 = 0; mt0 < n_mt; mt0 += MTG) {
+            float acc[MTG][4][4];
 #pragma unroll
-            for (int j = 0; j < NBG; ++j)
+            for (int m = 0; m < MTG; ++m)
 #pragma unroll
-                for (int mb = 0; mb < 2; ++mb)
+                for (int nt = 0; nt < 4; ++nt)
 #pragma unroll
-                    for (int i = 0; i < 4; ++i) acc[j][mb][i] = 0.0f;
-            const unsigned char *q_row = q_s + (nb0 * 8 + g) * kQRowBytes + q4 * 4;
+                    for (int i = 0; i < 4; ++i) acc[m][nt][i] = 0.0f;
+            const bool second = MTG == 2 && mt0 + 1 < n_mt;
 #pragma unroll
             for (int ks = 0; ks < D / 16; ++ks) {
-                uint32_t af[2][4];
+                uint32_t bf[2][4];      // [tokens 0-15 | 16-31]: b0, b1 of the even n-tile, b0, b1 of the odd one
+                ldmatrix_x4((tile_s) ^ (ks << 5), bf[0]);
+                ldmatrix_x4((tile_s + 16 * kRowBytes) ^ (ks << 5), bf[1]);
 #pragma unroll
-                for (int mb = 0; mb < 2; ++mb) {
-                    const int row = mb * 16 + a_row;
-                    ldmatrix_x4(tile_s + row * kRowBytes + (((2 * ks + a_chunk) ^ (row & 7)) << 4), af[mb]);
-                }
+                for (int m = 0; m < MTG; ++m) {
+                    if (m == 1 && !second) break;
+                    uint32_t af[4];
+                    ldmatrix_x4(a_lane + (mt0 + m) * 16 * kQRowBytes + ks * 32, af);
 #pragma unroll
-                for (int j = 0; j < NBG; ++j) {
-                    const uint32_t b0 = *reinterpret_cast<const uint32_t *>(q_row + j * 8 * kQRowBytes + ks * 32);
-                    const uint32_t b1 = *reinterpret_cast<const uint32_t *>(q_row + j * 8 * kQRowBytes + ks * 32 + 16);
-#pragma unroll
-                    for (int mb = 0; mb < 2; ++mb) mma_16816(acc[j][mb], af[mb], b0, b1);
+                    for (int nt = 0; nt < 4; ++nt) mma_16816(acc[m][nt], af, bf[nt >> 1][(nt & 1) * 2], bf[nt >> 1][(nt & 1) * 2 + 1]);
                 }
             }
-            // acc[j][mb][0..1]: token mb*16 + g, window rows 2*q4, 2*q4+1 of n-tile nb0 + j;  [2..3]: token mb*16 + 8 + g
+            // acc[m][nt][0..1]: window row (mt0+m)*16 + g, tokens nt*8 + 2*q4, + 1;  [2..3]: row + 8, the same tokens
 #pragma unroll
-            for (int j = 0; j < NBG; ++j) {
-                if (tail_tile) tile_statistics<SEG, true>(a, acc[j], nb0 + j, q4, last_col_s, t_tok, w_tok, opens, row0);
-                else tile_statistics<SEG, false>(a, acc[j], nb0 + j, q4, last_col_s, t_tok, w_tok, opens, row0);
+            for (int m = 0; m < MTG; ++m) {
+                if (m == 1 && !second) break;
+#pragma unroll
+                for (int half = 0; half < 2; ++half) {
+                    const int j0 = (mt0 + m) * 16 + half * 8;
+                    if (j0 >= a.NR) break;                     // only zero padding from here on (the same for every lane)
+                    const int j = j0 + g;
+                    float dot[4][2];
+#pragma unroll
+                    for (int nt = 0; nt < 4; ++nt) {
+                        dot[nt][0] = acc[m][nt][2 * half];
+                        dot[nt][1] = acc[m][nt][2 * half + 1];
+                    }
+                    if (tail_tile) row_statistics<SEG, true>(a, dot, tile, q4, j, j < a.NR, last_col_s[j], row0);
+                    else row_statistics<SEG, false>(a, dot, tile, q4, j, j < a.NR, 0, row0);
+                }
             }
         }
         __syncwarp();  // the buffer is free for the copy issued two tiles from now
@@ -379,6 +407,9 @@ __global__ void __launch_bounds__(256) column_sum_kernel(const TolArgs a)
     const int rows_per_slice = (a.rows + a.Y - 1) / a.Y;
     const int r_begin = blockIdx.y * rows_per_slice;
     const int r_end = min(a.rows, r_begin + rows_per_slice);
+    // before the last W columns every row sees every token: the column weight 1/W is applied to the finished sum
+    const bool tail = seg >= a.seg_tail0;
+    const float *wsum = tail ? a.pp : a.ps;
     float acc = 0.0f;
     if (seg < a.n_seg) {
         // four rows per trip, their loads issued together; the terms are still added in row order
@@ -389,7 +420,7 @@ __global__ void __launch_bounds__(256) column_sum_kernel(const TolArgs a)
             for (int u = 0; u < 4; ++u) {
                 const int64_t o = (int64_t)(row + 8 * u) * a.n_seg + seg;
                 ms[u] = a.pm[o];
-                pp[u] = a.pp[o];
+                pp[u] = wsum[o];
                 rm[u] = a.row_max[row + 8 * u];
                 ri[u] = a.row_inv[row + 8 * u];
             }
@@ -400,7 +431,7 @@ __global__ void __launch_bounds__(256) column_sum_kernel(const TolArgs a)
         for (; row < r_end; row += 8) {
             const int64_t o = (int64_t)row * a.n_seg + seg;
             const float ms = a.pm[o];
-            if (ms != -INFINITY) acc += a.pp[o] * expf(ms - a.row_max[row]) * a.row_inv[row];
+            if (ms != -INFINITY) acc += wsum[o] * expf(ms - a.row_max[row]) * a.row_inv[row];
         }
     }
     red[threadIdx.y][threadIdx.x] = acc;
@@ -409,7 +440,7 @@ __global__ void __launch_bounds__(256) column_sum_kernel(const TolArgs a)
         float s = 0.0f;
 #pragma unroll
         for (int y = 0; y < 8; ++y) s += red[y][threadIdx.x];
-        a.part[(int64_t)blockIdx.y * a.n_seg + seg] = s;
+        a.part[(int64_t)blockIdx.y * a.n_seg + seg] = tail ? s : s * (1.0f / (float)a.W);
     }
 }
 
@@ -556,6 +587,7 @@ int llms::chunk_tolerance_impl(const llms_kv_desc *desc, const void *kv, const v
     a.rep = a.Hq / a.Hkv;
     a.NR = a.rep * W;
     a.n_seg = t.n_seg;
+    a.seg_tail0 = std::min(t.n_seg, (a.T - W + 1) / t.SEG);
     a.seg_per_chunk = a.CL / t.SEG;
     a.n_chunks = n_chunks(*desc);
     a.stride_l = desc->stride_l; a.stride_h = desc->stride_h;
@@ -572,8 +604,10 @@ int llms::chunk_tolerance_impl(const llms_kv_desc *desc, const void *kv, const v
     a.Y = t.Y; a.rows = t.rows;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     if ((unsigned)(a.L * a.Hkv) > 65535u) return LLMS_ERR_UNSUPPORTED;
-    const size_t mma_q_bytes = ((size_t)((a.NR + 7) / 8 * 8) * (a.d * 2 + 16) + 127) / 128 * 128 +
-                               ((size_t)((a.NR + 7) / 8 * 8) * 4 + 127) / 128 * 128;   // query rows + each row's last visible token
+    const size_t padded_rows = (size_t)(a.NR + 15) / 16 * 16;                            // whole m-tiles
+    const size_t mma_q_bytes = (padded_rows * (a.d * 2 + 16) + 255) / 256 * 256 +
+                               (padded_rows * 4 + 255) / 256 * 256 + 1024;               // query rows, each row's last visible
+                                                                                         // token, room to align the tiles
     const size_t tile_bytes = (size_t)kTileBuffers * kTileTokens * a.d * 2;
     // twelve warps per CTA when two such CTAs fit into an SM's shared memory, else eight
     const int cta_warps = 2 * (mma_q_bytes + kTileWarps * tile_bytes + 1024) <= 227 * 1024 ? kTileWarps : kTileWarpsSmall;
@@ -590,10 +624,10 @@ int llms::chunk_tolerance_impl(const llms_kv_desc *desc, const void *kv, const v
         LLMS_CUDA_TRY(cudaFuncSetAttribute(logits_mma_kernel<S, DD, G>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)mma_smem)); \
         logits_mma_kernel<S, DD, G><<<grid, cta_warps * 32, mma_smem, st>>>(a);                                                     \
     } while (0)
-#define LLMS_LAUNCH_MMA(S, DD)                                      \
-    do {                                                            \
-        if (((a.NR + 7) / 8) % 4 == 0) LLMS_LAUNCH_MMA_G(S, DD, 4); \
-        else LLMS_LAUNCH_MMA_G(S, DD, 1);                           \
+#define LLMS_LAUNCH_MMA(S, DD)                        \
+    do {                                              \
+        if (a.NR > 16) LLMS_LAUNCH_MMA_G(S, DD, 2);   \
+        else LLMS_LAUNCH_MMA_G(S, DD, 1);             \
     } while (0)
 #define LLMS_LAUNCH_MMA_SEG(S)                                                      \
     case S:                                                                         \
