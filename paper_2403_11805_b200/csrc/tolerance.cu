@@ -33,8 +33,14 @@ struct TolArgs {
     float inv_sqrt_d;
     float *pm, *ps, *pp;      // [rows][n_seg]: segment max, sum of exp, 1/n_vis-weighted sum of exp (pp: only the
                               // segments from seg_tail0 on are read; before them it is ps / W)
-    float *row_max, *row_inv; // [rows]
+    float *row_max, *row_inv; // [rows]: filled by row_stats_kernel (only the fp32 logits kernel's path uses them)
+    float2 *row_part;         // [rows][n_slots]: (max, sum of exp) of a row over the tiles of one CTA of the MMA kernel
+    int n_slots;              // CTAs per (layer, KV head) pair; 0: the row normalisers are in row_max / row_inv
     float *part;              // [Y][n_seg]
+    float *colsum;            // [n_seg]: column sums over all rows
+    uint32_t *tickets;        // [n_x + 1]: finished row slices per group of 32 segments, finished groups; the logits
+                              // kernel of the same call clears them
+    int n_x;                  // groups of 32 segments
     float *scores;
     float *scores_live;       // optional second destination of the scores (page-locked host memory), or NULL
     int Y, rows;
@@ -51,6 +57,8 @@ __global__ void __launch_bounds__(kTokThreads) logits_kernel(const TolArgs a)
     for (int i = threadIdx.x; i < a.NR * a.d; i += blockDim.x) q_s[i] = __half2float(q_src[i]);
     __syncthreads();
 
+    if (blockIdx.x == 0 && blockIdx.y == 0)
+        for (int i = threadIdx.x; i <= a.n_x; i += blockDim.x) a.tickets[i] = 0;   // for the column kernel of this call
     const int t = blockIdx.x * kTokThreads + threadIdx.x;
     const bool valid = t < a.T;
     const int lane = threadIdx.x & 31;
@@ -199,10 +207,12 @@ __device__ __forceinline__ void segment_reduce(float (&x)[4][2], Op op)
 // (the column kernel applies that factor), so masks and weights drop out.
 //   dot[nt][e]  raw q.k of token tile*32 + nt*8 + 2*q4 + e;  j  the row's index among the KV head's rows;
 //   valid  false for the zero rows that pad the last m-tile (they take part in the shuffles and store nothing);
-//   last_col  (TAIL) the last token the row sees
+//   last_col  (TAIL) the last token the row sees;
+//   run  this warp's running (max of q.k, sum of exp relative to it) of the row over the tiles it has seen, or NULL
+//        (kept for segments of 16 and 32 tokens, where one lane per row holds a tile's statistics)
 template <int SEG, bool TAIL>
 __device__ __forceinline__ void row_statistics(const TolArgs &a, const float (&dot)[4][2], int tile, int q4, int j, bool valid,
-                                               int last_col, int64_t row0)
+                                               int last_col, int64_t row0, float2 *run)
 {
     constexpr float kLog2e = 1.4426950408889634f;
     const float c1 = a.inv_sqrt_d * kLog2e;                 // logit in units of log 2
@@ -248,6 +258,19 @@ __device__ __forceinline__ void row_statistics(const TolArgs &a, const float (&d
                     if (seg >= a.seg_tail0) a.pp[o] = sp[nt][e];
             }
         }
+    if constexpr (SEG >= 16) {
+        if (run != nullptr && valid && q4 == 0) {
+            float2 r = *run;
+#pragma unroll
+            for (int nt = 0; nt < 4; nt += SEG / 8) {
+                if (TAIL && mx[nt][0] == -INFINITY) continue;                  // a segment the row does not see
+                const float m_new = fmaxf(r.x, mx[nt][0]);
+                r.y = r.y * ex2_approx((r.x - m_new) * c1) + se[nt][0] * ex2_approx((mx[nt][0] - m_new) * c1);
+                r.x = m_new;
+            }
+            *run = r;
+        }
+    }
 }
 
 // MTG: m-tiles (16 flattened window rows each) that share one pass over a tile's B fragments - 2 where a KV head
@@ -266,9 +289,12 @@ __global__ void __launch_bounds__(kTileWarps * 32, 2) logits_mma_kernel(const To
     const int q_total = (n_mt * 16 * kQRowBytes + 255) / 256 * 256;
     int *last_col_s = reinterpret_cast<int *>(smem_raw + q_total);           // [n_mt*16]: last token a row sees
     const int lc_total = (n_mt * 16 * 4 + 255) / 256 * 256;
+    // [n_mt*16][warps of the CTA]: each warp's running (max of q.k, sum of exp relative to it) of a row over its tiles
+    float2 *run_s = reinterpret_cast<float2 *>(smem_raw + q_total + lc_total);
+    const int run_total = (n_mt * 16 * (int)(blockDim.x >> 5) * 8 + 255) / 256 * 256;
     // this warp's tile buffers, aligned to a 1 KiB boundary whatever the base of the dynamic shared memory: every bit
     // of a chunk index then sits below the buffer's address bits and a chunk's swizzle is an XOR on the whole address
-    const uint32_t tiles_s = (((uint32_t)__cvta_generic_to_shared(smem_raw) + q_total + lc_total + 1023u) & ~1023u) +
+    const uint32_t tiles_s = (((uint32_t)__cvta_generic_to_shared(smem_raw) + q_total + lc_total + run_total + 1023u) & ~1023u) +
                              wib * kTileBuffers * kTileBytes;
 
     const int l = blockIdx.y / a.Hkv, kvh = blockIdx.y % a.Hkv;
@@ -279,6 +305,7 @@ __global__ void __launch_bounds__(kTileWarps * 32, 2) logits_mma_kernel(const To
             row < a.NR ? __ldg(reinterpret_cast<const uint4 *>(q_src) + i) : make_uint4(0, 0, 0, 0);
     }
     for (int j = threadIdx.x; j < n_mt * 16; j += blockDim.x) last_col_s[j] = j < a.NR ? a.T - a.W + j % a.W : -1;
+    for (int i = threadIdx.x; i < n_mt * 16 * (int)(blockDim.x >> 5); i += blockDim.x) run_s[i] = make_float2(-INFINITY, 0.0f);
     __syncthreads();
 
     const __half *k_plane = a.kv + (int64_t)l * a.stride_l + (int64_t)kvh * a.stride_h;
@@ -365,12 +392,34 @@ __global__ void __launch_bounds__(kTileWarps * 32, 2) logits_mma_kernel(const To
                         dot[nt][0] = acc[m][nt][2 * half];
                         dot[nt][1] = acc[m][nt][2 * half + 1];
                     }
-                    if (tail_tile) row_statistics<SEG, true>(a, dot, tile, q4, j, j < a.NR, last_col_s[j], row0);
-                    else row_statistics<SEG, false>(a, dot, tile, q4, j, j < a.NR, 0, row0);
+                    float2 *run = a.n_slots > 0 ? run_s + j * cta_warps + wib : nullptr;
+                    if (tail_tile) row_statistics<SEG, true>(a, dot, tile, q4, j, j < a.NR, last_col_s[j], row0, run);
+                    else row_statistics<SEG, false>(a, dot, tile, q4, j, j < a.NR, 0, row0, run);
                 }
             }
         }
         __syncwarp();  // the buffer is free for the copy issued two tiles from now
+    }
+
+    // ---- what the column kernel that follows needs from this CTA
+    if (blockIdx.x == 0 && blockIdx.y == 0)
+        for (int i = threadIdx.x; i <= a.n_x; i += blockDim.x) a.tickets[i] = 0;
+    // Every row's (max, sum of exp) over this CTA's tiles: the warps' running pairs, combined in warp order.  The
+    // column kernel combines a row's n_slots such pairs into the row's softmax normaliser.
+    __syncthreads();
+    if (a.n_slots > 0) {
+        constexpr float kLog2e = 1.4426950408889634f;
+        const float c1 = a.inv_sqrt_d * kLog2e;
+        for (int j = threadIdx.x; j < a.NR; j += blockDim.x) {
+            float m_all = -INFINITY;
+            for (int k = 0; k < cta_warps; ++k) m_all = fmaxf(m_all, run_s[j * cta_warps + k].x);
+            float s_all = 0.0f;
+            for (int k = 0; k < cta_warps; ++k) {
+                const float2 c = run_s[j * cta_warps + k];
+                if (c.x != -INFINITY) s_all += c.y * ex2_approx((c.x - m_all) * c1);
+            }
+            a.row_part[(row0 + j) * a.n_slots + blockIdx.x] = make_float2(m_all * a.inv_sqrt_d, s_all);
+        }
     }
 }
 
@@ -399,14 +448,53 @@ __global__ void row_stats_kernel(const TolArgs a)
     }
 }
 
-// block (32 segments x 8 row lanes); blockIdx.y picks a slice of rows
-__global__ void __launch_bounds__(256) column_sum_kernel(const TolArgs a)
+// True in every thread of exactly one of the `expected` blocks that pass through with this counter: the one that comes
+// last.  What the others wrote to global memory before is then visible to loads that bypass L1.  Nobody waits.
+__device__ __forceinline__ bool arrives_last(uint32_t *counter, uint32_t expected)
+{
+    __shared__ uint32_t ticket;
+    __threadfence();
+    __syncthreads();
+    if (threadIdx.x == 0 && threadIdx.y == 0) ticket = atomicAdd(counter, 1u);
+    __syncthreads();
+    const bool last = ticket == expected - 1;
+    if (last) __threadfence();
+    return last;
+}
+
+constexpr int kMaxSliceRows = 1024;   // rows of one slice of the column kernel (their normalisers sit in shared memory)
+
+// Column sums, then chunk means, in one launch.  Block (32 segments x 8 row lanes); blockIdx.y picks a slice of rows.
+// A block first makes its rows' softmax normalisers (from the per-CTA pairs the MMA kernel left, or copies them
+// where row_stats_kernel made them), then adds up its rows' normalised, 1/n_vis-weighted probabilities per segment.
+// The last slice to finish a group of 32 segments adds the slices in index order; the last group to finish adds
+// every chunk's segments.  All sums run in a fixed order: the scores do not depend on which block came last.
+__global__ void __launch_bounds__(256) column_chunk_kernel(const TolArgs a)
 {
     __shared__ float red[8][33];
+    __shared__ float rm_s[kMaxSliceRows], ri_s[kMaxSliceRows];
+    const int tid = threadIdx.y * 32 + threadIdx.x;
     const int seg = blockIdx.x * 32 + threadIdx.x;
     const int rows_per_slice = (a.rows + a.Y - 1) / a.Y;
     const int r_begin = blockIdx.y * rows_per_slice;
     const int r_end = min(a.rows, r_begin + rows_per_slice);
+    for (int r = r_begin + tid; r < r_end; r += 256) {
+        float m = -INFINITY, sum = 0.0f;
+        if (a.n_slots > 0) {
+            const float2 *rp = a.row_part + (int64_t)r * a.n_slots;
+            for (int k = 0; k < a.n_slots; ++k) m = fmaxf(m, rp[k].x);
+            for (int k = 0; k < a.n_slots; ++k) {
+                const float2 c = rp[k];
+                if (c.x != -INFINITY) sum += c.y * expf(c.x - m);
+            }
+            rm_s[r - r_begin] = m;
+            ri_s[r - r_begin] = 1.0f / sum;
+        } else {
+            rm_s[r - r_begin] = a.row_max[r];
+            ri_s[r - r_begin] = a.row_inv[r];
+        }
+    }
+    __syncthreads();
     // before the last W columns every row sees every token: the column weight 1/W is applied to the finished sum
     const bool tail = seg >= a.seg_tail0;
     const float *wsum = tail ? a.pp : a.ps;
@@ -415,23 +503,21 @@ __global__ void __launch_bounds__(256) column_sum_kernel(const TolArgs a)
         // four rows per trip, their loads issued together; the terms are still added in row order
         int row = r_begin + threadIdx.y;
         for (; row + 24 < r_end; row += 32) {
-            float ms[4], pp[4], rm[4], ri[4];
+            float ms[4], pp[4];
 #pragma unroll
             for (int u = 0; u < 4; ++u) {
                 const int64_t o = (int64_t)(row + 8 * u) * a.n_seg + seg;
                 ms[u] = a.pm[o];
                 pp[u] = wsum[o];
-                rm[u] = a.row_max[row + 8 * u];
-                ri[u] = a.row_inv[row + 8 * u];
             }
 #pragma unroll
             for (int u = 0; u < 4; ++u)
-                if (ms[u] != -INFINITY) acc += pp[u] * expf(ms[u] - rm[u]) * ri[u];
+                if (ms[u] != -INFINITY) acc += pp[u] * expf(ms[u] - rm_s[row + 8 * u - r_begin]) * ri_s[row + 8 * u - r_begin];
         }
         for (; row < r_end; row += 8) {
             const int64_t o = (int64_t)row * a.n_seg + seg;
             const float ms = a.pm[o];
-            if (ms != -INFINITY) acc += wsum[o] * expf(ms - a.row_max[row]) * a.row_inv[row];
+            if (ms != -INFINITY) acc += wsum[o] * expf(ms - rm_s[row - r_begin]) * ri_s[row - r_begin];
         }
     }
     red[threadIdx.y][threadIdx.x] = acc;
@@ -442,22 +528,29 @@ __global__ void __launch_bounds__(256) column_sum_kernel(const TolArgs a)
         for (int y = 0; y < 8; ++y) s += red[y][threadIdx.x];
         a.part[(int64_t)blockIdx.y * a.n_seg + seg] = tail ? s : s * (1.0f / (float)a.W);
     }
-}
+    if (!arrives_last(a.tickets + blockIdx.x, gridDim.y)) return;
 
-// warp per chunk: lane y takes row slices y, y+32, ... of every segment of the chunk; the lanes' sums are then
-// added pairwise in a fixed tree, so a score does not depend on the launch
-__global__ void chunk_mean_kernel(const TolArgs a)
-{
-    const int c = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
-    if (c >= a.n_chunks) return;
-    const int lane = threadIdx.x & 31;
-    float tot = 0.0f;
-    for (int y = lane; y < a.Y; y += 32)
-        for (int s = c * a.seg_per_chunk; s < (c + 1) * a.seg_per_chunk; ++s) tot += a.part[(int64_t)y * a.n_seg + s];
+    // ---- this group's column sums: row lane y adds slices y, y + 8, ... in order, then the eight lanes are added in order
+    acc = 0.0f;
+    if (seg < a.n_seg)
+        for (int y = threadIdx.y; y < a.Y; y += 8) acc += __ldcg(a.part + (int64_t)y * a.n_seg + seg);
+    __syncthreads();
+    red[threadIdx.y][threadIdx.x] = acc;
+    __syncthreads();
+    if (threadIdx.y == 0 && seg < a.n_seg) {
+        float s = 0.0f;
 #pragma unroll
-    for (int m = 16; m > 0; m >>= 1) tot += __shfl_xor_sync(0xffffffffu, tot, m);
-    if (lane == 0) {
-        const float score = tot / ((float)a.CL * (float)a.L * (float)a.Hq);
+        for (int y = 0; y < 8; ++y) s += red[y][threadIdx.x];
+        a.colsum[seg] = s;
+    }
+    if (!arrives_last(a.tickets + a.n_x, gridDim.x)) return;
+
+    // ---- every chunk's mean over its tokens, layers and heads
+    const float norm = (float)a.CL * (float)a.L * (float)a.Hq;
+    for (int c = tid; c < a.n_chunks; c += 256) {
+        float tot = 0.0f;
+        for (int sg = c * a.seg_per_chunk; sg < (c + 1) * a.seg_per_chunk; ++sg) tot += __ldcg(a.colsum + sg);
+        const float score = tot / norm;
         a.scores[c] = score;
         if (a.scores_live) a.scores_live[c] = score;
     }
@@ -513,11 +606,18 @@ static int seg_len(int chunk_len)
     return s;
 }
 
-static int row_slices(int rows) { return rows >= 4096 ? 64 : (rows >= 512 ? 16 : (rows >= 64 ? 4 : 1)); }
+// slices of rows in the column kernel: enough blocks to fill the GPU, and no slice longer than the kernel's arrays
+static int row_slices(int rows)
+{
+    const int y = rows >= 4096 ? 64 : (rows >= 512 ? 16 : (rows >= 64 ? 4 : 1));
+    return std::max(y, (rows + kMaxSliceRows - 1) / kMaxSliceRows);
+}
+
+constexpr int kMaxRowSlots = 32;   // most CTAs of the MMA kernel per (layer, KV head) pair
 
 struct TolLayout {
-    int SEG, n_seg, rows, Y;
-    uint64_t off_pm, off_ps, off_pp, off_rmax, off_rinv, off_part, total;
+    int SEG, n_seg, rows, Y, n_x;
+    uint64_t off_pm, off_ps, off_pp, off_rmax, off_rinv, off_part, off_rpart, off_colsum, off_tickets, total;
 };
 
 static TolLayout tol_layout(const llms_kv_desc &d, int W)
@@ -534,7 +634,11 @@ static TolLayout tol_layout(const llms_kv_desc &d, int W)
     t.off_rmax = 3 * stat;
     t.off_rinv = t.off_rmax + round_up((uint64_t)t.rows * 4, 256);
     t.off_part = t.off_rinv + round_up((uint64_t)t.rows * 4, 256);
-    t.total = t.off_part + round_up((uint64_t)t.Y * t.n_seg * 4, 256);
+    t.n_x = (t.n_seg + 31) / 32;
+    t.off_rpart = t.off_part + round_up((uint64_t)t.Y * t.n_seg * 4, 256);
+    t.off_colsum = t.off_rpart + round_up((uint64_t)t.rows * kMaxRowSlots * sizeof(float2), 256);
+    t.off_tickets = t.off_colsum + round_up((uint64_t)t.n_seg * 4, 256);
+    t.total = t.off_tickets + round_up((uint64_t)(t.n_x + 1) * 4, 256);
     return t;
 }
 
@@ -599,15 +703,20 @@ int llms::chunk_tolerance_impl(const llms_kv_desc *desc, const void *kv, const v
     a.row_max = reinterpret_cast<float *>(ws + t.off_rmax);
     a.row_inv = reinterpret_cast<float *>(ws + t.off_rinv);
     a.part = reinterpret_cast<float *>(ws + t.off_part);
+    a.row_part = reinterpret_cast<float2 *>(ws + t.off_rpart);
+    a.colsum = reinterpret_cast<float *>(ws + t.off_colsum);
+    a.tickets = reinterpret_cast<uint32_t *>(ws + t.off_tickets);
+    a.n_x = t.n_x;
     a.scores = scores;
     a.scores_live = scores_live;
     a.Y = t.Y; a.rows = t.rows;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
-    if ((unsigned)(a.L * a.Hkv) > 65535u) return LLMS_ERR_UNSUPPORTED;
+    if ((unsigned)(a.L * a.Hkv) > 65535u || a.Y > 65535) return LLMS_ERR_UNSUPPORTED;
     const size_t padded_rows = (size_t)(a.NR + 15) / 16 * 16;                            // whole m-tiles
     const size_t mma_q_bytes = (padded_rows * (a.d * 2 + 16) + 255) / 256 * 256 +
-                               (padded_rows * 4 + 255) / 256 * 256 + 1024;               // query rows, each row's last visible
-                                                                                         // token, room to align the tiles
+                               (padded_rows * 4 + 255) / 256 * 256 +                     // query rows, each row's last visible
+                               (padded_rows * kTileWarps * 8 + 255) / 256 * 256 + 1024;  // token, the warps' running row sums,
+                                                                                         // room to align the tiles
     const size_t tile_bytes = (size_t)kTileBuffers * kTileTokens * a.d * 2;
     // twelve warps per CTA when two such CTAs fit into an SM's shared memory, else eight
     const int cta_warps = 2 * (mma_q_bytes + kTileWarps * tile_bytes + 1024) <= 227 * 1024 ? kTileWarps : kTileWarpsSmall;
@@ -617,7 +726,12 @@ int llms::chunk_tolerance_impl(const llms_kv_desc *desc, const void *kv, const v
         const int n_tiles = (a.T + kTileTokens - 1) / kTileTokens;
         const int pairs = a.L * a.Hkv;
         int splits = (sm_count() * 6 + pairs - 1) / pairs;
-        splits = std::max(1, std::min(splits, (n_tiles + cta_warps - 1) / cta_warps));
+        splits = std::max(1, std::min({splits, (n_tiles + cta_warps - 1) / cta_warps, kMaxRowSlots}));
+        // With up to 16 rows per KV head and segments of 16 or 32 tokens every CTA leaves its rows' (max, sum of exp)
+        // for the column kernel (7B shape: 2 us more in this kernel, 6 us of row_stats_kernel and a launch less).
+        // Elsewhere the normalisers come from a pass of row_stats_kernel over all statistics: with 32 rows per KV
+        // head the running sums made this kernel 24 us slower (32K grouped-query shape), more than that pass costs.
+        a.n_slots = t.SEG >= 16 && a.NR <= 16 ? splits : 0;
         const dim3 grid(splits, pairs);
 #define LLMS_LAUNCH_MMA_G(S, DD, G)                                                                                                  \
     do {                                                                                                                             \
@@ -668,11 +782,11 @@ int llms::chunk_tolerance_impl(const llms_kv_desc *desc, const void *kv, const v
 #undef LLMS_LAUNCH_LOGITS
     }
     LLMS_CUDA_TRY(cudaGetLastError());
-    row_stats_kernel<<<(a.rows + 7) / 8, 256, 0, st>>>(a);
-    LLMS_CUDA_TRY(cudaGetLastError());
-    column_sum_kernel<<<dim3((a.n_seg + 31) / 32, a.Y), dim3(32, 8), 0, st>>>(a);
-    LLMS_CUDA_TRY(cudaGetLastError());
-    chunk_mean_kernel<<<(a.n_chunks + 7) / 8, 256, 0, st>>>(a);
+    if (a.n_slots == 0) {  // the fp32 kernel leaves no per-CTA row sums: a pass over all statistics makes the normalisers
+        row_stats_kernel<<<(a.rows + 7) / 8, 256, 0, st>>>(a);
+        LLMS_CUDA_TRY(cudaGetLastError());
+    }
+    column_chunk_kernel<<<dim3(a.n_x, a.Y), dim3(32, 8), 0, st>>>(a);
     LLMS_CUDA_TRY(cudaGetLastError());
     return LLMS_OK;
 }
