@@ -280,18 +280,22 @@ def run_ours(args):
 
     frac_a = np.asarray(frac, dtype=np.float32)
     levels_a = np.asarray(LEVELS, dtype=np.uint8)
-    bits = np.zeros(n, dtype=np.uint8)
+    bits = B.new_pinned(n)
+    planned = B.new_event()
 
     def step(ev=None):
         if ev:
             ev[0].record(stream)
-        # score -> (scores to the host, ranking: a host step) -> levels -> records, as one library call;
-        # the event sits behind the score kernels and the copy of the scores
+        # score -> rank -> levels -> chunk table -> records, as one library call; scores, levels and meta are
+        # page-locked, so a kernel does the ranking and nothing synchronises.  The event sits behind that kernel.
+        after = ev[1] if ev else planned
         B.compress_context(d, kv, q_win, W, frac_a, levels_a, scores, scores_host, bits, buf, meta, ws_tol, ws,
-                           after_scores=ev[1] if ev else None)
+                           after_scores=after)
         if ev:
             ev[2].record(stream)
-        # meta is pinned: the expected checksums are read by the device in stream order, no synchronisation here
+        # the decode call reads sizes and offsets from meta on the host: wait for the ranking (the encoder runs on);
+        # the expected checksums are read by the device in stream order
+        B.wait(after)
         B.decompress_chunks_ordered(d, buf, meta, None, kv_out, ws_dec)
         if ev:
             ev[3].record(stream)
@@ -506,8 +510,10 @@ def run_ours(args):
                 "serial_ms_per_step": e2e_serial_ms, "batch_chunks": e2e_batch,
                 "what": "compress -> swap-out to pinned host -> swap-in -> decompress, pipelined in batches of chunks",
                 "layerwise_load": layerwise},
-        # 4 score kernels, then one codec kernel per call (channel-wise mode: one per bit-width and one for the sums)
-        "gpu_launches": args.steps * (4 + 2 * B.codec_launches(d, bits)),
+        # score kernels (logits, column sums + chunk means; a row pass in between for more than 16 rows per KV head),
+        # the ranking kernel, then one codec kernel per call (channel-wise mode: one per bit-width and one for the sums)
+        "gpu_launches": args.steps * ((2 if shape.n_q_heads // shape.n_kv_heads * W <= 16 and shape.chunk_len % 16 == 0 else 3)
+                                      + 1 + 2 * B.codec_launches(d, bits)),
         "roofline": roofline, "clocks": clocks,
         "wall_ms_per_step": t_wall * 1e3 / args.steps,
         "step_ms_median_best": [statistics.median(step_ms), step_ms[0]],

@@ -178,10 +178,9 @@ int llms_decompress_chunks_ordered(const llms_kv_desc *desc, const void *buf, ui
                                    const uint32_t *dst_chunk_ids, int n, void *kv_out,
                                    void *workspace, uint64_t workspace_bytes, void *stream);
 
-/* Synchronises `stream`, then reports on the last llms_compress_chunks or llms_decompress_chunks
- * that used this workspace: LLMS_ERR_TIMEOUT if one of its kernels abandoned a bounded wait for a
- * copy (its output is then incomplete), else LLMS_ERR_CORRUPT if a decoded record's checksum did
- * not match, else LLMS_OK; *n_corrupt (host, may be NULL) receives the number of such records. */
+/* Synchronises `stream`, then reports on the last llms_decompress_chunks that used this workspace:
+ * LLMS_ERR_CORRUPT if a decoded record's checksum did not match, else LLMS_OK; *n_corrupt (host, may
+ * be NULL) receives the number of such records. */
 int llms_codec_corrupt_count(const void *workspace, uint32_t *n_corrupt, void *stream);
 
 /* ------------------------------------------------------------------ tolerance score (Eq. 1) */
@@ -221,7 +220,8 @@ int llms_assign_levels(const float *scores, int n, const float frac[3], const ui
 
 /* Eq. 3: the shares of chunks per level that maximise the context's information under a global average
  * ratio, for the levels {8/8, 4/8, 2/8} (Sec. 3.2: one free variable is left).  A chunk at level w keeps
- * weight ratio_w of its density (reading of the garbled 1/ratio_w; see the format notes of the build).
+ * weight ratio_w of its density (the printed weight 1/ratio_w would reward compressing the densest chunks most and
+ * is read as a misprint).
  * ratio_global in [0.25, 1] is relative to 8 bits: f8 + f4/2 + f2/4 = ratio_global, hence
  * f2 = 2*f8 + 2 - 4*ratio_global.  Every count n8 of 8-bit chunks is tried on the density-ordered list
  * (n2 = floor(2*n8 + (2 - 4*ratio_global)*n + 1/2), n4 the rest); the best wins, the smaller n8 on a tie.
@@ -247,15 +247,24 @@ int llms_lctru_order(const llms_chunk_state *table, int n, uint32_t *order_out);
 
 /* The compression half of swapping a context out (Sec. 3.2, "Compressing chunks": density of every
  * chunk, its rank, its level, then quantization) as one call: llms_chunk_tolerance on K and the query
- * window, the scores copied to the host, llms_assign_levels, then llms_compress_chunks over all chunks
- * in index order (chunk_ids 0 .. n-1).  Results are those of the three calls made one after the other;
- * what this call saves is the host time between them, during which the stream would sit empty.
- * The ranking is a host step: the call synchronises `stream` once, when the scores have reached the host.
- *   scores_dev   device fp32 [n_chunks];  scores_host  host fp32 [n_chunks]: into page-locked memory the
- *                last score kernel stores the scores itself, pageable memory receives them by a copy
+ * window, llms_assign_levels on the scores, then llms_compress_chunks over all chunks in index order
+ * (chunk_ids 0 .. n-1).  Results are those of the three calls made one after the other.
+ *   scores_dev   device fp32 [n_chunks];  scores_host  host fp32 [n_chunks]
  *   bits_out     host, n_chunks bytes: the level each chunk got
- *   after_scores optional cudaEvent_t, recorded on `stream` behind the score kernels (and the scores' copy)
- *   everything else as in the three calls. */
+ *   after_scores optional cudaEvent_t, recorded on `stream` behind the score kernels and whatever
+ *                brings scores, levels and meta to the host
+ *   everything else as in the three calls.
+ * Stream-ordered form: when scores_host, bits_out and meta all lie in page-locked memory (and the
+ * context has at most 4096 chunks), a kernel ranks the chunks, assigns the levels and lays the
+ * encoder's chunk table down on the device, and stores scores, levels and meta (sizes, offsets)
+ * into the three host arrays itself: the call returns without synchronising, and the three arrays
+ * are valid once after_scores has completed (meta[].checksum once the whole call has).  A call that
+ * needs meta on the host - llms_decompress_chunks, llms_swap_out - waits for that event first
+ * (llms_wait), while the encoder is still running.
+ * Otherwise the ranking is a host step: the call synchronises `stream` once, when the scores have
+ * reached the host, and the arrays are filled when it returns (checksums as in llms_compress_chunks).
+ * All arguments, the room in out_buf included (the number of chunks per level follows from frac and
+ * n_chunks alone), are checked before the first launch. */
 int llms_compress_context(const llms_kv_desc *desc, const void *kv, const void *q_win, int W,
                           const float frac[3], const uint8_t levels[3],
                           float *scores_dev, float *scores_host, uint8_t *bits_out,

@@ -161,6 +161,14 @@ def new_meta(n, pinned=False):
     return t.numpy()[:n * META_DTYPE.itemsize].view(META_DTYPE)   # the view keeps the pinned storage alive
 
 
+def new_pinned(n, dtype=np.uint8):
+    """n zeroed elements as a numpy array over page-locked memory (e.g. the level array of compress_context)."""
+    import torch
+    dt = np.dtype(dtype)
+    t = torch.zeros(max(n, 1) * dt.itemsize, dtype=torch.uint8).pin_memory()
+    return t.numpy()[:n * dt.itemsize].view(dt)                  # the view keeps the pinned storage alive
+
+
 def new_event(stream=None):
     """A created cudaEvent_t wrapped by torch (recorded once so that the handle exists)."""
     import torch
@@ -325,8 +333,10 @@ def lctru_order(table):
 
 def compress_context(desc, kv, q_win, W, frac, levels, scores_dev, scores_host, bits_out, out_buf, meta,
                      tolerance_workspace, codec_workspace, after_scores=None, stream=None):
-    """llms_compress_context: scores, levels and records of every chunk in one call (synchronises the stream once).
-    frac: float32[3], levels: uint8[3], bits_out: uint8[n_chunks] numpy arrays; scores_host: pinned fp32 tensor."""
+    """llms_compress_context: scores, levels and records of every chunk in one call.
+    frac: float32[3], levels: uint8[3], bits_out: uint8[n_chunks] numpy arrays; scores_host: fp32 tensor.
+    With scores_host, bits_out and meta all in page-locked memory nothing synchronises: the three arrays are valid
+    once after_scores has completed.  Otherwise the stream is synchronised once inside the call."""
     assert frac.dtype == np.float32 and levels.dtype == np.uint8 and bits_out.dtype == np.uint8
     _check(lib().llms_compress_context(
         C.addressof(desc), _ptr(kv), _ptr(q_win), int(W), _ptr(frac), _ptr(levels), _ptr(scores_dev), _ptr(scores_host),

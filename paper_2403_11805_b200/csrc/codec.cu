@@ -40,11 +40,6 @@ __host__ __device__ constexpr int piece_words(int bits) { return bits >= 2 ? bit
 constexpr uint32_t kPrefetchAhead = 2;          // compress: units ahead that are pulled into L2 (measured: 2 -> 0.521 ms,
                                                 // 3 -> 0.535, 5 -> 0.59, 8 -> 0.79 for compress on the 7B shape)
 
-// Measured on the 7B-shaped context (same box, same run): register-prefetch kernel 0.561 ms, bulk-copy pipeline
-// 0.579-0.591 ms.  Both are bound by instruction issue, not by the memory path, and the pipeline spends more
-// instructions (shared-memory traffic, barrier polling, single-lane sections), so the direct kernel is used.
-constexpr bool kUseBulkCompress = false;
-
 // Division by a launch-time constant as multiply-high and shift: exact for numerators below 2^31.
 struct FastDiv {
     uint32_t d, mul, shr;
@@ -68,21 +63,12 @@ struct FastDiv {
     }
 };
 
-// One chunk of a launch, in the order the launch walks them.
-struct UnitEntry {
-    uint32_t chunk_id;  // source / destination chunk (slot) in the KV tensor
-    uint32_t entry;     // index into the caller-ordered entry table (checksums)
-    uint64_t rec_off;   // byte offset of the record in the swap buffer
-};
-static_assert(sizeof(UnitEntry) == 16, "table layout");
-
 struct CodecArgs {
     const __half *kv_in;   // compress: source
     __half *kv_out;        // decompress: destination
     uint8_t *buf;          // swap buffer (written by compress, read by decompress)
     ChunkEntry *entries;   // n entries in the workspace (caller's order)
     uint32_t *sums;        // decompress: recomputed checksums
-    uint32_t *gave_up;     // second status word: warps that abandoned a bounded wait
     const uint32_t *order; // entry indices grouped by bit-width; this launch covers order[0 .. n)
     const UnitEntry *table; // the same chunks with what a unit needs to know, one 16-byte load
     int n;                 // chunks of this launch (all of one bit-width)
@@ -97,7 +83,6 @@ struct CodecArgs {
     int slabs_per_unit;    // packed: kPassElems / slab_elems
     uint32_t chunk_elems;  // n_slabs * slab_elems
     FastDiv div_passes, div_n, div_heads;
-    uint32_t step_units, step_pass, step_k, step_s;  // stride between a warp's units (= warps of the grid), split by radix
     uint32_t total_units;  // n * n_slabs * passes
     uint32_t codes_off;    // byte offset of the code stream in a record
     uint32_t params_bytes; // 4 * n_groups
@@ -931,7 +916,6 @@ __global__ void __launch_bounds__(kThreads, kDecodeBlocksPerSm) decompress_kerne
 
 }  // namespace llms
 
-#include "codec_bulk.cuh"
 #include "codec_cw.cuh"
 
 namespace llms {
@@ -974,9 +958,9 @@ static int fill_args(const llms_kv_desc &d, CodecArgs &a, int n, void *workspace
     a.stride_h = d.stride_h;
     a.chunk_stride = (int64_t)d.chunk_len * d.head_dim;
     a.chunk_elems = (uint32_t)a.n_slabs * (uint32_t)a.slab_elems;
-    // slabs shorter than a pass: whole slabs are packed into a unit (only with 256-bit accesses; the bulk-copy
-    // and channel-wise kernels keep their own walk over slabs)
-    a.packed = wide && d.quant_mode == 0 && !kUseBulkCompress && a.slab_elems < kPassElems && kPassElems % a.slab_elems == 0 &&
+    // slabs shorter than a pass: whole slabs are packed into a unit (only with 256-bit accesses; the channel-wise
+    // kernels keep their own walk over slabs)
+    a.packed = wide && d.quant_mode == 0 && a.slab_elems < kPassElems && kPassElems % a.slab_elems == 0 &&
                a.slab_elems % kLaneElems == 0;
     if (a.packed) {
         a.passes = 1;
@@ -996,7 +980,6 @@ static int fill_args(const llms_kv_desc &d, CodecArgs &a, int n, void *workspace
     a.sums = reinterpret_cast<uint32_t *>(static_cast<uint8_t *>(workspace) + ws_sums_offset(n));
     a.order = reinterpret_cast<const uint32_t *>(static_cast<uint8_t *>(workspace) + ws_order_offset(n));
     a.table = reinterpret_cast<const UnitEntry *>(static_cast<uint8_t *>(workspace) + ws_table_offset(n));
-    a.gave_up = static_cast<uint32_t *>(workspace) + 1;
     return LLMS_OK;
 }
 
@@ -1121,17 +1104,6 @@ static int decode_grid(K kernel, int64_t items)
 }
 
 
-// The stride between a warp's units, split into (passes, chunks, slab indices).
-static CodecArgs with_grid(CodecArgs a, int grid)
-{
-    a.step_units = (uint32_t)grid * kWarpsPerBlock;
-    a.step_pass = a.step_units % (uint32_t)a.passes;
-    const uint32_t items = a.step_units / (uint32_t)a.passes;
-    a.step_k = items % (uint32_t)a.n;
-    a.step_s = items / (uint32_t)a.n;
-    return a;
-}
-
 // 256-bit accesses need every slab to start on a 32-byte boundary
 static bool wide_ok(const llms_kv_desc &d, const void *kv)
 {
@@ -1167,6 +1139,69 @@ static int check_common(const llms_kv_desc *desc, int n, const void *workspace, 
     if (slab_elems(*desc) > 0x7fffffff / 8) return LLMS_ERR_UNSUPPORTED;
     const uint64_t passes = ((uint64_t)slab_elems(*desc) + kPassElems - 1) / kPassElems;
     if ((uint64_t)n * (uint64_t)slabs_per_chunk(*desc) * passes > 0x7fffffffull) return LLMS_ERR_UNSUPPORTED;
+    return LLMS_OK;
+}
+
+// Launch the encoder over the chunk tables that sit in the workspace (entries, unit table, order grouped by bit-width;
+// first[k] / count[k]: where the chunks of width 8, 4, 2, 1 start in the grouped order and how many there are), and see
+// to it that the checksums reach `meta` (host) in stream order.
+static int launch_compress(const llms_kv_desc &desc, const void *kv, void *out_buf, void *workspace, int n,
+                           const int (&first)[kNumWidths], const int (&count)[kNumWidths], llms_chunk_meta *meta, cudaStream_t st)
+{
+    CodecArgs a{};
+    const bool wide = wide_ok(desc, kv);
+    fill_args(desc, a, n, workspace, wide);
+    a.kv_in = static_cast<const __half *>(kv);
+    a.buf = static_cast<uint8_t *>(out_buf);
+    BitGroups groups;
+    for (int k = 0; k < kNumWidths; ++k) {
+        groups.first[k] = first[k];
+        groups.count[k] = count[k];
+    }
+    int rc = LLMS_OK;
+    bool published = false;  // the codec kernel itself stores the checksums into a page-locked meta array
+    if (desc.quant_mode == 1) {
+        for (int k = 0; k < kNumWidths; ++k) {
+            if (groups.count[k] == 0) continue;
+            const CodecArgs b = args_for_group(a, groups, k);
+            if (k == 0) launch_compress_cw<8>(b, desc.head_dim, desc.chunk_len, st);
+            else if (k == 1) launch_compress_cw<4>(b, desc.head_dim, desc.chunk_len, st);
+            else if (k == 2) launch_compress_cw<2>(b, desc.head_dim, desc.chunk_len, st);
+            else launch_compress_cw<1>(b, desc.head_dim, desc.chunk_len, st);
+            LLMS_CUDA_TRY(cudaGetLastError());
+        }
+    } else {
+        // one launch for the whole call; the grid is sized for the width with the most units
+        CodecArgsByWidth all{};
+        uint32_t most_units = 0;
+        for (int k = 0; k < kNumWidths; ++k) {
+            if (groups.count[k] == 0) continue;
+            all.w[k] = args_for_group(a, groups, k);
+            most_units = std::max(most_units, all.w[k].total_units);
+        }
+        all.done = static_cast<uint32_t *>(workspace) + 2;
+        all.entries = a.entries;
+        all.n_total = n;
+        all.live_meta = static_cast<llms_chunk_meta *>(device_view_of_pinned(meta));
+        published = all.live_meta != nullptr;
+        rc = dispatch_group(desc.group_size, [&](auto g) {
+            constexpr int kG = decltype(g)::value;
+            if (a.packed) compress_kernel<kG, true, true><<<grid_for(compress_kernel<kG, true, true>, most_units), kThreads, 0, st>>>(all);
+            else if (wide) compress_kernel<kG, true, false><<<grid_for(compress_kernel<kG, true, false>, most_units), kThreads, 0, st>>>(all);
+            else compress_kernel<kG, false, false><<<grid_for(compress_kernel<kG, false, false>, most_units), kThreads, 0, st>>>(all);
+        });
+        if (rc) return rc;
+        LLMS_CUDA_TRY(cudaGetLastError());
+    }
+    // checksums back to the caller's meta (every other field is already there)
+    if (published) {
+        // nothing left to do
+    } else if (void *live = device_view_of_pinned(meta)) {
+        publish_checksums_kernel<<<(n + 255) / 256, 256, 0, st>>>(a.entries, static_cast<llms_chunk_meta *>(live), n);
+        LLMS_CUDA_TRY(cudaGetLastError());
+    } else {
+        LLMS_CUDA_TRY(cudaMemcpyAsync(meta, a.entries, (size_t)n * sizeof(ChunkEntry), cudaMemcpyDeviceToHost, st));
+    }
     return LLMS_OK;
 }
 
@@ -1214,81 +1249,35 @@ extern "C" int llms_compress_chunks(const llms_kv_desc *desc, const void *kv, co
         meta[i] = staged[i];
         off += bytes_at[bits[i]];
     }
-    CodecArgs a{};
-    const bool wide = wide_ok(*desc, kv);
-    fill_args(*desc, a, n, workspace, wide);
-    a.kv_in = static_cast<const __half *>(kv);
-    a.buf = static_cast<uint8_t *>(out_buf);
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     const BitGroups groups = group_by_bits(n, staged.data(), [&](int i) { return (uint32_t)bits[i]; });
     rc = upload_tables(workspace, staged.data(), groups, n, false, st);
     if (rc) return rc;
-    bool published = false;  // the codec kernel itself stores the checksums into a page-locked meta array
-    if (desc->quant_mode == 1 || kUseBulkCompress) {
-        for (int k = 0; k < kNumWidths; ++k) {
-            if (groups.count[k] == 0) continue;
-            const CodecArgs b = args_for_group(a, groups, k);
-            cudaError_t attr_err = cudaSuccess;
-            if (desc->quant_mode == 1) {
-                if (k == 0) launch_compress_cw<8>(b, desc->head_dim, desc->chunk_len, st);
-                else if (k == 1) launch_compress_cw<4>(b, desc->head_dim, desc->chunk_len, st);
-                else if (k == 2) launch_compress_cw<2>(b, desc->head_dim, desc->chunk_len, st);
-                else launch_compress_cw<1>(b, desc->head_dim, desc->chunk_len, st);
-                LLMS_CUDA_TRY(cudaGetLastError());
-                continue;
-            }
-            rc = dispatch_group(desc->group_size, [&](auto g) {
-                constexpr int kG = decltype(g)::value;
-                if constexpr (kUseBulkCompress && kG >= kLaneElems) {
-                    // groups of 64 channels and more: the bulk-copy pipeline
-#define LLMS_LAUNCH(BITS)                                                                                                      \
-    attr_err = cudaFuncSetAttribute(compress_bulk_kernel<BITS, kG>, cudaFuncAttributeMaxDynamicSharedMemorySize, kBulkSmemBytes); \
-    if (attr_err == cudaSuccess) {                                                                                              \
-        const int grid = grid_for(compress_bulk_kernel<BITS, kG>, b.total_units, kBulkSmemBytes);                               \
-        compress_bulk_kernel<BITS, kG><<<grid, kThreads, kBulkSmemBytes, st>>>(with_grid(b, grid));                             \
+    return launch_compress(*desc, kv, out_buf, workspace, n, groups.first, groups.count, meta, st);
+}
+
+// The encoder over chunk tables that a kernel has already put into the workspace (llms_compress_context's stream-ordered
+// path): chunks 0 .. n-1 in index order, count[k] of them at width 8, 4, 2, 1.
+int llms::compress_planned(const llms_kv_desc *desc, const void *kv, int n, const int count[4], void *out_buf,
+                           llms_chunk_meta *meta, void *workspace, void *stream)
+{
+    int first[kNumWidths], cnt[kNumWidths], at = 0;
+    for (int k = 0; k < kNumWidths; ++k) {
+        first[k] = at;
+        cnt[k] = count[k];
+        at += count[k];
     }
-                    if (k == 0) { LLMS_LAUNCH(8); } else if (k == 1) { LLMS_LAUNCH(4); } else if (k == 2) { LLMS_LAUNCH(2); } else { attr_err = cudaErrorNotSupported; }
-#undef LLMS_LAUNCH
-                } else {
-                    attr_err = cudaErrorNotSupported;
-                }
-            });
-            if (rc) return rc;
-            LLMS_CUDA_TRY(attr_err);
-            LLMS_CUDA_TRY(cudaGetLastError());
-        }
-    } else {
-        // one launch for the whole call; the grid is sized for the width with the most units
-        CodecArgsByWidth all{};
-        uint32_t most_units = 0;
-        for (int k = 0; k < kNumWidths; ++k) {
-            if (groups.count[k] == 0) continue;
-            all.w[k] = args_for_group(a, groups, k);
-            most_units = std::max(most_units, all.w[k].total_units);
-        }
-        all.done = static_cast<uint32_t *>(workspace) + 2;
-        all.entries = a.entries;
-        all.n_total = n;
-        all.live_meta = static_cast<llms_chunk_meta *>(device_view_of_pinned(meta));
-        published = all.live_meta != nullptr;
-        rc = dispatch_group(desc->group_size, [&](auto g) {
-            constexpr int kG = decltype(g)::value;
-            if (a.packed) compress_kernel<kG, true, true><<<grid_for(compress_kernel<kG, true, true>, most_units), kThreads, 0, st>>>(all);
-            else if (wide) compress_kernel<kG, true, false><<<grid_for(compress_kernel<kG, true, false>, most_units), kThreads, 0, st>>>(all);
-            else compress_kernel<kG, false, false><<<grid_for(compress_kernel<kG, false, false>, most_units), kThreads, 0, st>>>(all);
-        });
-        if (rc) return rc;
-        LLMS_CUDA_TRY(cudaGetLastError());
-    }
-    // checksums back to the caller's meta (every other field is already there)
-    if (published) {
-        // nothing left to do
-    } else if (void *live = device_view_of_pinned(meta)) {
-        publish_checksums_kernel<<<(n + 255) / 256, 256, 0, st>>>(a.entries, static_cast<llms_chunk_meta *>(live), n);
-        LLMS_CUDA_TRY(cudaGetLastError());
-    } else {
-        LLMS_CUDA_TRY(cudaMemcpyAsync(meta, a.entries, (size_t)n * sizeof(ChunkEntry), cudaMemcpyDeviceToHost, st));
-    }
+    if (at != n) return LLMS_ERR_INVALID_ARG;
+    return launch_compress(*desc, kv, out_buf, workspace, n, first, cnt, meta, static_cast<cudaStream_t>(stream));
+}
+
+int llms::check_compress_args(const llms_kv_desc *desc, int n, const void *kv, const void *out_buf, const void *workspace,
+                              uint64_t workspace_bytes)
+{
+    int rc = check_common(desc, n, workspace, workspace_bytes);
+    if (rc) return rc;
+    if (n > 0 && (!kv || !out_buf)) return LLMS_ERR_INVALID_ARG;
+    if (!aligned(kv, 16) || !aligned(out_buf, 256)) return LLMS_ERR_MISALIGNED;
     return LLMS_OK;
 }
 
@@ -1398,13 +1387,12 @@ extern "C" int llms_decompress_chunks_ordered(const llms_kv_desc *desc, const vo
 extern "C" int llms_codec_corrupt_count(const void *workspace, uint32_t *n_corrupt, void *stream)
 {
     if (!workspace) return LLMS_ERR_INVALID_ARG;
-    uint32_t status[2] = {0, 0};  // {records with a wrong checksum, warps that gave up a bounded wait}
+    uint32_t status = 0;  // records with a wrong checksum
     cudaStream_t st = static_cast<cudaStream_t>(stream);
-    LLMS_CUDA_TRY(cudaMemcpyAsync(status, workspace, 8, cudaMemcpyDeviceToHost, st));
+    LLMS_CUDA_TRY(cudaMemcpyAsync(&status, workspace, 4, cudaMemcpyDeviceToHost, st));
     LLMS_CUDA_TRY(cudaStreamSynchronize(st));
-    if (n_corrupt) *n_corrupt = status[0];
-    if (status[1]) return LLMS_ERR_TIMEOUT;
-    return status[0] ? LLMS_ERR_CORRUPT : LLMS_OK;
+    if (n_corrupt) *n_corrupt = status;
+    return status ? LLMS_ERR_CORRUPT : LLMS_OK;
 }
 
 // ---------------------------------------------------------------------------------------------- no-allocation variant

@@ -50,6 +50,13 @@ void *device_view_of_pinned(const void *host_ptr);
 int chunk_tolerance_impl(const llms_kv_desc *desc, const void *kv, const void *q_win, int W, float *scores,
                          float *scores_live, void *workspace, uint64_t workspace_bytes, void *stream);
 
+// The encoder over chunk tables already present in the workspace (see codec.cu), and the argument checks of the
+// compress call that do not depend on the chunk list.
+int compress_planned(const llms_kv_desc *desc, const void *kv, int n, const int count[4], void *out_buf,
+                     llms_chunk_meta *meta, void *workspace, void *stream);
+int check_compress_args(const llms_kv_desc *desc, int n, const void *kv, const void *out_buf, const void *workspace,
+                        uint64_t workspace_bytes);
+
 // Device-side copy of the per-chunk table, kept in the workspace.
 struct ChunkEntry {          // same bytes as llms_chunk_meta
     uint32_t chunk_id, bits;
@@ -58,14 +65,22 @@ struct ChunkEntry {          // same bytes as llms_chunk_meta
 };
 static_assert(sizeof(ChunkEntry) == sizeof(llms_chunk_meta) && sizeof(ChunkEntry) == 32, "meta layout");
 
+// One chunk of a codec launch, in the order the launch walks them (chunks grouped by bit-width).
+struct UnitEntry {
+    uint32_t chunk_id;  // source / destination chunk (slot) in the KV tensor
+    uint32_t entry;     // index into the caller-ordered entry table (checksums)
+    uint64_t rec_off;   // byte offset of the record in the swap buffer
+};
+static_assert(sizeof(UnitEntry) == 16, "table layout");
+
 // Workspace of the codec calls:
-// [two status words and a count of finished CTAs, padded to 16 bytes][n entries][n 16-byte unit-table rows][n entry indices grouped by
+// [a status word, a spare word and a count of finished CTAs, padded to 16 bytes][n entries][n 16-byte unit-table rows][n entry indices grouped by
 // bit-width][n recomputed sums].  Everything up to the sums is written by one host-to-device copy per call.
 constexpr uint64_t kWsEntriesOffset = 16;
 constexpr uint64_t kWsBytesPerChunk = sizeof(ChunkEntry) + 16 + 4 + 4;
-inline uint64_t ws_table_offset(int n) { return kWsEntriesOffset + (uint64_t)n * sizeof(ChunkEntry); }
-inline uint64_t ws_order_offset(int n) { return ws_table_offset(n) + (uint64_t)n * 16; }
-inline uint64_t ws_sums_offset(int n) { return ws_order_offset(n) + (uint64_t)n * 4; }
+__host__ __device__ inline uint64_t ws_table_offset(int n) { return kWsEntriesOffset + (uint64_t)n * sizeof(ChunkEntry); }
+__host__ __device__ inline uint64_t ws_order_offset(int n) { return ws_table_offset(n) + (uint64_t)n * 16; }
+__host__ __device__ inline uint64_t ws_sums_offset(int n) { return ws_order_offset(n) + (uint64_t)n * 4; }
 inline uint64_t ws_total(int n) { return round_up(kWsEntriesOffset + (uint64_t)n * kWsBytesPerChunk, 16); }
 
 }  // namespace llms

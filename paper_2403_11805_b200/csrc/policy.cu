@@ -102,6 +102,131 @@ extern "C" int llms_lctru_order(const llms_chunk_state *table, int n, uint32_t *
     return m;
 }
 
+namespace llms {
+
+// Eq. 2 and the chunk tables of the encoder on the device, for a context whose scores have just been computed on the
+// same stream (one CTA; n <= kPlanMaxChunks).  Chunk i's rank is the number of chunks that come before it in the
+// order "denser first, equal densities by index" - exactly the order the host's stable sort produces - so levels and
+// record offsets equal those of llms_assign_levels followed by llms_compress_chunks on the same score bits.
+constexpr int kPlanMaxChunks = 4096;
+constexpr int kPlanThreads = 1024;
+
+struct PlanArgs {
+    const float *scores;       // device, n
+    int n, n_top, n_top_mid;   // ranks below n_top keep levels[0], below n_top_mid levels[1], the rest levels[2]
+    uint32_t levels[3];
+    uint64_t rec_bytes[3];     // record size per level
+    uint32_t n_groups;
+    int first[4];              // where the chunks of width 8, 4, 2, 1 start in the grouped order
+    uint8_t *workspace;        // codec workspace: header, entries, unit table, grouped order
+    llms_chunk_meta *meta;     // the caller's page-locked meta array (device view)
+    uint8_t *bits_out;         // the caller's page-locked level array (device view)
+};
+
+__device__ __forceinline__ int width_class(uint32_t bits) { return bits == 8 ? 0 : (bits == 4 ? 1 : (bits == 2 ? 2 : 3)); }
+
+// inclusive scan of one value per thread over the CTA (kPlanThreads threads), fixed order
+template <typename T>
+__device__ __forceinline__ T block_inclusive_scan(T v, T *warp_totals)
+{
+    const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
+#pragma unroll
+    for (int d = 1; d < 32; d <<= 1) {
+        const T up = __shfl_up_sync(0xffffffffu, v, d);
+        if (lane >= d) v += up;
+    }
+    if (lane == 31) warp_totals[w] = v;
+    __syncthreads();
+    if (w == 0) {
+        T t = warp_totals[lane];
+#pragma unroll
+        for (int d = 1; d < 32; d <<= 1) {
+            const T up = __shfl_up_sync(0xffffffffu, t, d);
+            if (lane >= d) t += up;
+        }
+        warp_totals[lane] = t;
+    }
+    __syncthreads();
+    const T before = w > 0 ? warp_totals[w - 1] : T(0);
+    __syncthreads();
+    return v + before;
+}
+
+__global__ void __launch_bounds__(kPlanThreads) plan_context_kernel(const PlanArgs a)
+{
+    __shared__ float s_scores[kPlanMaxChunks];
+    __shared__ uint8_t s_level[kPlanMaxChunks];                // index into levels[]
+    __shared__ unsigned long long s_scan[32];
+    const int n = a.n;
+    for (int i = threadIdx.x; i < n; i += kPlanThreads) s_scores[i] = a.scores[i];
+    if (threadIdx.x < 4) reinterpret_cast<uint32_t *>(a.workspace)[threadIdx.x] = 0;   // status word, spare, finished-CTA count
+    __syncthreads();
+    for (int i = threadIdx.x; i < n; i += kPlanThreads) {
+        const float mine = s_scores[i];
+        int rank = 0;
+        for (int j = 0; j < n; ++j) {
+            const float other = s_scores[j];
+            rank += (other > mine) || (other == mine && j < i);
+        }
+        s_level[i] = rank < a.n_top ? 0 : (rank < a.n_top_mid ? 1 : 2);
+    }
+    __syncthreads();
+    // every thread owns a run of consecutive chunks: record bytes and per-width counts before each chunk by two scans
+    const int per = (n + kPlanThreads - 1) / kPlanThreads;
+    const int begin = min(n, (int)threadIdx.x * per), end = min(n, begin + per);
+    unsigned long long bytes = 0, counts = 0;                  // counts: four 16-bit fields, one per width class
+    for (int i = begin; i < end; ++i) {
+        bytes += a.rec_bytes[s_level[i]];
+        counts += 1ull << (16 * width_class(a.levels[s_level[i]]));
+    }
+    unsigned long long off = block_inclusive_scan(bytes, s_scan) - bytes;
+    unsigned long long seen = block_inclusive_scan(counts, s_scan) - counts;
+    ChunkEntry *entries = reinterpret_cast<ChunkEntry *>(a.workspace + kWsEntriesOffset);
+    UnitEntry *table = reinterpret_cast<UnitEntry *>(a.workspace + ws_table_offset(n));
+    uint32_t *order = reinterpret_cast<uint32_t *>(a.workspace + ws_order_offset(n));
+    for (int i = begin; i < end; ++i) {
+        const int lv = s_level[i];
+        const uint32_t bits = a.levels[lv];
+        const int k = width_class(bits);
+        ChunkEntry e;
+        e.chunk_id = (uint32_t)i;
+        e.bits = bits;
+        e.offset = off;
+        e.nbytes = a.rec_bytes[lv];
+        e.n_groups = a.n_groups;
+        e.checksum = 0;                                        // the encoder accumulates into the device copy
+        entries[i] = e;
+        const int at = a.first[k] + (int)((seen >> (16 * k)) & 0xffffu);
+        order[at] = (uint32_t)i;
+        UnitEntry u;
+        u.chunk_id = (uint32_t)i;
+        u.entry = (uint32_t)i;
+        u.rec_off = off;
+        table[at] = u;
+        llms_chunk_meta m;
+        m.chunk_id = (uint32_t)i;
+        m.bits = bits;
+        m.offset = off;
+        m.nbytes = a.rec_bytes[lv];
+        m.n_groups = a.n_groups;
+        m.checksum = 0;
+        a.meta[i] = m;
+        a.bits_out[i] = (uint8_t)bits;
+        off += a.rec_bytes[lv];
+        seen += 1ull << (16 * k);
+    }
+}
+
+// The counts of Eq. 2's three levels for n chunks: the first n_top ranks, then up to n_top_mid.
+static void level_counts(int n, const float frac[3], long &n_top, long &n_top_mid)
+{
+    const double f_top = frac[0], f_mid = frac[1];
+    n_top = std::min<long>((long)std::floor(f_top * n + 0.5), n);
+    n_top_mid = std::max(std::min<long>((long)std::floor((f_top + f_mid) * n + 0.5), n), n_top);
+}
+
+}  // namespace llms
+
 // Score -> levels -> records for all chunks of a context: the three calls a swap-out makes, without the host
 // round trips between them.
 extern "C" int llms_compress_context(const llms_kv_desc *desc, const void *kv, const void *q_win, int W,
@@ -112,15 +237,68 @@ extern "C" int llms_compress_context(const llms_kv_desc *desc, const void *kv, c
                                      void *codec_workspace, uint64_t codec_workspace_bytes,
                                      void *after_scores, void *stream)
 {
-    if (!desc || !scores_dev || !scores_host || !bits_out) return LLMS_ERR_INVALID_ARG;
+    using namespace llms;
+    if (!desc || !scores_dev || !scores_host || !bits_out || !frac || !levels || !meta) return LLMS_ERR_INVALID_ARG;
+    // ---- everything that can be wrong is found before the first launch
+    int rc = check_desc(desc);
+    if (rc) return rc;
+    const int n = (int)n_chunks(*desc);
+    for (int w = 0; w < 3; ++w)
+        if (check_bits(levels[w])) return LLMS_ERR_BAD_BITS;
+    if (!(levels[0] > levels[1] && levels[1] > levels[2])) return LLMS_ERR_INVALID_ARG;
+    if (!(frac[0] >= 0) || !(frac[1] >= 0) || !(frac[2] >= 0) || std::fabs((double)frac[0] + frac[1] + frac[2] - 1.0) > 1e-3)
+        return LLMS_ERR_INVALID_ARG;
+    rc = check_compress_args(desc, n, kv, out_buf, codec_workspace, codec_workspace_bytes);
+    if (rc) return rc;
+    long n_top, n_top_mid;
+    level_counts(n, frac, n_top, n_top_mid);
+    uint64_t rec_bytes[3], need = 0;
+    for (int w = 0; w < 3; ++w) {
+        rc = llms_record_bytes(desc, levels[w], &rec_bytes[w]);
+        if (rc) return rc;
+    }
+    need = (uint64_t)n_top * rec_bytes[0] + (uint64_t)(n_top_mid - n_top) * rec_bytes[1] + (uint64_t)(n - n_top_mid) * rec_bytes[2];
+    if (need > out_bytes) return LLMS_ERR_BUF_TOO_SMALL;      // the levels' counts follow from frac and n alone
+
     // Into page-locked memory the last score kernel stores the scores itself (a copy after the kernels costs a switch to
     // the copy engine and back: about 15 us per context); pageable memory gets them by a copy.
-    float *scores_live = static_cast<float *>(llms::device_view_of_pinned(scores_host));
-    int rc = llms::chunk_tolerance_impl(desc, kv, q_win, W, scores_dev, scores_live, tolerance_workspace,
-                                        tolerance_workspace_bytes, stream);
+    float *scores_live = static_cast<float *>(device_view_of_pinned(scores_host));
+    uint8_t *bits_live = static_cast<uint8_t *>(device_view_of_pinned(bits_out));
+    llms_chunk_meta *meta_live = static_cast<llms_chunk_meta *>(device_view_of_pinned(meta));
+    rc = chunk_tolerance_impl(desc, kv, q_win, W, scores_dev, scores_live, tolerance_workspace, tolerance_workspace_bytes, stream);
     if (rc) return rc;
-    const int n = (int)llms::n_chunks(*desc);
     cudaStream_t st = static_cast<cudaStream_t>(stream);
+    if (n == 0) return LLMS_OK;
+
+    if (scores_live && bits_live && meta_live && n <= kPlanMaxChunks) {
+        // ---- stream-ordered: a kernel ranks the chunks and lays the encoder's tables down; nothing waits for the host
+        PlanArgs p{};
+        p.scores = scores_dev;
+        p.n = n;
+        p.n_top = (int)n_top;
+        p.n_top_mid = (int)n_top_mid;
+        int count[4] = {0, 0, 0, 0};
+        const long level_n[3] = {n_top, n_top_mid - n_top, n - n_top_mid};
+        for (int w = 0; w < 3; ++w) {
+            p.levels[w] = levels[w];
+            p.rec_bytes[w] = rec_bytes[w];
+            count[levels[w] == 8 ? 0 : (levels[w] == 4 ? 1 : (levels[w] == 2 ? 2 : 3))] = (int)level_n[w];
+        }
+        for (int k = 0, at = 0; k < 4; ++k) {
+            p.first[k] = at;
+            at += count[k];
+        }
+        p.n_groups = (uint32_t)groups_per_chunk(*desc);
+        p.workspace = static_cast<uint8_t *>(codec_workspace);
+        p.meta = meta_live;
+        p.bits_out = bits_live;
+        plan_context_kernel<<<1, kPlanThreads, 0, st>>>(p);
+        LLMS_CUDA_TRY(cudaGetLastError());
+        if (after_scores) LLMS_CUDA_TRY(cudaEventRecord(static_cast<cudaEvent_t>(after_scores), st));
+        return compress_planned(desc, kv, n, count, out_buf, meta, codec_workspace, stream);
+    }
+
+    // ---- the ranking as a host step: one synchronisation, when the scores have reached the host
     if (!scores_live)
         LLMS_CUDA_TRY(cudaMemcpyAsync(scores_host, scores_dev, (size_t)n * sizeof(float), cudaMemcpyDeviceToHost, st));
     if (after_scores) LLMS_CUDA_TRY(cudaEventRecord(static_cast<cudaEvent_t>(after_scores), st));

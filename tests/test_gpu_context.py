@@ -11,9 +11,12 @@ from gpu_helpers import assert_meta_equal, bits_view, first_mismatch, odesc
 pytestmark = pytest.mark.gpu
 
 
-@pytest.mark.parametrize("pinned_scores", [True, False], ids=["pinned", "pageable"])
+@pytest.mark.parametrize("pinned_scores,pinned_bits", [(True, True), (True, False), (False, False)],
+                         ids=["stream_ordered", "pinned_scores", "pageable"])
 @pytest.mark.parametrize("levels,frac", [((8, 4, 2), (1 / 3, 1 / 3, 1 / 3)), ((4, 2, 1), (0.2, 0.5, 0.3))])
-def test_compress_context_equals_the_separate_calls_and_the_oracle(levels, frac, pinned_scores):
+def test_compress_context_equals_the_separate_calls_and_the_oracle(levels, frac, pinned_scores, pinned_bits):
+    """With scores, levels and meta all in page-locked memory the ranking and the chunk table are made by a kernel and
+    the call does not synchronise; with any of them pageable the ranking is a host step.  Same bytes either way."""
     sh = synth.KVShape("ctx", 3, 2, 4, 64, 208, 16, 64, seed=13)          # 13 chunks, GQA
     W = sh.window
     kv, q = synth.kv_tensor(sh), synth.q_window(sh, W)
@@ -28,20 +31,25 @@ def test_compress_context_equals_the_separate_calls_and_the_oracle(levels, frac,
     scores_host = torch.full((n,), -1.0, dtype=torch.float32)
     if pinned_scores:
         scores_host = scores_host.pin_memory()
-    bits = np.zeros(n, dtype=np.uint8)
+    bits = B.new_pinned(n) if pinned_bits else np.zeros(n, dtype=np.uint8)
     total = B.compressed_size(d, np.full(n, levels[0], np.uint8))
     buf = torch.zeros(total, dtype=torch.uint8, device="cuda")
     meta = B.new_meta(n, pinned=True)
     ws_t = torch.empty(B.tolerance_workspace_bytes(d, W), dtype=torch.uint8, device="cuda")
-    ws_c = torch.empty(B.codec_workspace_bytes(n), dtype=torch.uint8, device="cuda")
+    ws_c = torch.full((B.codec_workspace_bytes(n),), 0xA5, dtype=torch.uint8, device="cuda")   # nothing relies on zeros
     before, after = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     after.record()                                                        # creates the handle the library records
     torch.cuda.synchronize()
     before.record()
     B.compress_context(d, kv_dev, q_dev, W, frac_a, levels_a, scores_dev, scores_host, bits, buf, meta, ws_t, ws_c,
                        after_scores=after)
+    B.wait(after)                                                         # scores, levels and meta are on the host now
+    early_bits, early_meta = bits.copy(), meta.copy()
     torch.cuda.synchronize()
     assert before.elapsed_time(after) > 0                                 # recorded behind the score kernels
+    assert np.array_equal(early_bits, bits)
+    for f in ("chunk_id", "bits", "offset", "nbytes", "n_groups"):
+        assert np.array_equal(early_meta[f], meta[f]), f
 
     # the three calls
     scores2 = torch.empty(n, dtype=torch.float32, device="cuda")
@@ -72,6 +80,32 @@ def test_compress_context_argument_errors():
     rc = B.lib().llms_compress_context(None, None, None, 8, None, None, None, None, None, None, 0, None, None, 0, None, 0,
                                        None, None)
     assert rc == B.ERR_INVALID_ARG
+    # everything is checked before the first launch: nothing of the outputs is touched on an error
+    W, n = sh.window, sh.n_chunks
+    kv_dev, q_dev = synth.kv_tensor(sh).cuda(), synth.q_window(sh, W).cuda()
+    scores_dev = torch.full((n,), -7.0, dtype=torch.float32, device="cuda")
+    scores_host = torch.full((n,), -7.0, dtype=torch.float32).pin_memory()
+    bits = B.new_pinned(n)
+    meta = B.new_meta(n, pinned=True)
+    buf = torch.zeros(B.compressed_size(d, np.full(n, 8, np.uint8)), dtype=torch.uint8, device="cuda")
+    ws_t = torch.empty(B.tolerance_workspace_bytes(d, W), dtype=torch.uint8, device="cuda")
+    ws_c = torch.empty(B.codec_workspace_bytes(n), dtype=torch.uint8, device="cuda")
+    good = dict(frac=np.asarray((1 / 3, 1 / 3, 1 / 3), np.float32), levels=np.asarray((8, 4, 2), np.uint8), out=buf, ws_c=ws_c)
+
+    def call(**kw):
+        a = dict(good, **kw)
+        with pytest.raises(B.LlmsError) as e:
+            B.compress_context(d, kv_dev, q_dev, W, a["frac"], a["levels"], scores_dev, scores_host, bits, a["out"], meta, ws_t,
+                               a["ws_c"])
+        return e.value.status
+
+    assert call(frac=np.asarray((0.5, 0.6, 0.2), np.float32)) == B.ERR_INVALID_ARG
+    assert call(levels=np.asarray((8, 3, 2), np.uint8)) == B.ERR_BAD_BITS
+    assert call(levels=np.asarray((2, 4, 8), np.uint8)) == B.ERR_INVALID_ARG
+    assert call(out=buf[:B.compressed_size(d, np.full(n, 4, np.uint8))]) == B.ERR_BUF_TOO_SMALL   # 5 or 6 of 16 chunks keep 8 bits
+    assert call(ws_c=ws_c[:64]) == B.ERR_BUF_TOO_SMALL
+    torch.cuda.synchronize()
+    assert (scores_dev.cpu() == -7.0).all() and (scores_host == -7.0).all() and not bits.any() and not meta["nbytes"].any()
 
 
 def test_full_size_step_as_the_benchmark_runs_it():
@@ -86,15 +120,18 @@ def test_full_size_step_as_the_benchmark_runs_it():
     frac, levels = np.asarray(sh.frac, dtype=np.float32), np.asarray((8, 4, 2), dtype=np.uint8)
     scores_dev = torch.empty(n, dtype=torch.float32, device="cuda")
     scores_host = torch.empty(n, dtype=torch.float32).pin_memory()
-    bits = np.zeros(n, dtype=np.uint8)
+    bits = B.new_pinned(n)
     buf = torch.empty(B.compressed_size(d, np.full(n, 8, np.uint8)), dtype=torch.uint8, device="cuda")
     meta = B.new_meta(n, pinned=True)
     ws_t = torch.empty(B.tolerance_workspace_bytes(d, W), dtype=torch.uint8, device="cuda")
     ws_c = torch.empty(B.codec_workspace_bytes(n), dtype=torch.uint8, device="cuda")
     ws_d = torch.empty(B.codec_workspace_bytes(n), dtype=torch.uint8, device="cuda")
     out = torch.empty_like(kv_dev)
+    planned = B.new_event()
     for _ in range(2):
-        B.compress_context(d, kv_dev, q_dev, W, frac, levels, scores_dev, scores_host, bits, buf, meta, ws_t, ws_c)
+        B.compress_context(d, kv_dev, q_dev, W, frac, levels, scores_dev, scores_host, bits, buf, meta, ws_t, ws_c,
+                           after_scores=planned)
+        B.wait(planned)                                   # levels and record offsets are on the host; the encoder still runs
         B.decompress_chunks_ordered(d, buf, meta, None, out, ws_d)
         assert B.codec_corrupt_count(ws_d) == 0
     obits, _ = oracle.assign_levels(scores_host.numpy(), sh.frac, (8, 4, 2))
