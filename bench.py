@@ -55,26 +55,36 @@ def measured_peaks():
     return 6650.0, "fallback"
 
 
-# dram__bytes_read.sum + dram__bytes_write.sum of one stage (one launch, the bit-widths as phases) on the full
-# llama7b workload, from one ncu capture of the kernels as they are now (profiles/codec_and_score_kernels_llama7b.md).
-# Set an entry to None when its kernel changes.
+# dram__bytes_read.sum + dram__bytes_write.sum of one codec launch on the full llama7b workload, from one ncu capture.
+# Each figure is tied to the codec source it was taken with: when that source has changed since, the line reports null
+# instead of a number that may no longer hold.
+CODEC_SOURCES = ("paper_2403_11805_b200/csrc/codec.cu", "paper_2403_11805_b200/csrc/codec_cw.cuh",
+                 "paper_2403_11805_b200/csrc/llms_internal.cuh")
 NCU_DRAM_TRAFFIC = {
-    ("llama7b", 32, "compress_kernel"): 2148047616 + 646768384,
-    ("llama7b", 32, "decompress_kernel"): 670340096 + 2084697088,
+    "codec_sha256_16": "",                      # hash of CODEC_SOURCES at the capture
+    "source": "",                               # what was captured, with which command
+    ("llama7b", 32, "compress_kernel"): None,
+    ("llama7b", 32, "decompress_kernel"): None,
 }
 
 
+def codec_source_hash():
+    import hashlib
+    h = hashlib.sha256()
+    for rel in CODEC_SOURCES:
+        with open(os.path.join(ROOT, rel), "rb") as f:
+            h.update(f.read())
+    return h.hexdigest()[:16]
+
+
+def measured_traffic(key):
+    """The captured DRAM bytes of a launch, or None when there is no capture for it or the codec has changed since."""
+    if codec_source_hash() != NCU_DRAM_TRAFFIC["codec_sha256_16"]:
+        return None, "no capture for the codec source as it is now"
+    return NCU_DRAM_TRAFFIC.get(key), NCU_DRAM_TRAFFIC["source"]
+
+
 LEVELS = (8, 4, 2)      # set from --levels
-
-
-def target_bits(shape):
-    """Bit mix of the workload by chunk rank: counts as the rank -> bits rule gives them."""
-    import numpy as np
-    n = shape.n_chunks
-    f8, f4, _ = shape.frac if shape.frac is not None else (1 / 3, 1 / 3, 1 / 3)
-    n8 = int(np.floor(f8 * n + 0.5))
-    n84 = int(np.floor((f8 + f4) * n + 0.5))
-    return n8, n84 - n8, n - n84
 
 
 class ClockSampler:
@@ -265,7 +275,7 @@ def run_ours(args):
     d = B.desc_of(shape, quant_mode=args.quant_mode)
     n = shape.n_chunks
     ids = np.arange(n, dtype=np.uint32)
-    n8, n4, n2 = target_bits(shape)
+    n8, n4, n2 = B.level_counts(n, frac, LEVELS)          # what the rank -> bits rule gives each level
     worst_bits = np.full(n, 8, dtype=np.uint8)
     buf = torch.empty(B.compressed_size(d, worst_bits), dtype=torch.uint8, device="cuda")
     kv_out = torch.empty_like(kv)
@@ -414,6 +424,36 @@ def run_ours(args):
         barrier()
         return sharding.max_over_ranks([e0.elapsed_time(e1) / args.e2e_steps], dist, "cuda")[0]
 
+    # ---- what the host link gives a bare copy of the same bytes: one way each, then both ways at once
+    def time_copies(pairs):
+        streams = [side_out, side_in][:len(pairs)]
+        best = None
+        for it in range(6):
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            torch.cuda.synchronize()
+            e0.record(stream)
+            for st, (dst, src) in zip(streams, pairs):
+                st.wait_event(e0)
+                with torch.cuda.stream(st):
+                    dst.copy_(src, non_blocking=True)
+                ev = torch.cuda.Event()
+                ev.record(st)
+                stream.wait_event(ev)
+            e1.record(stream)
+            torch.cuda.synchronize()
+            ms = e0.elapsed_time(e1)
+            if it >= 2:
+                best = ms if best is None else min(best, ms)
+        return record_bytes / (best * 1e-3) / 1e9
+
+    arena2 = torch.empty(record_bytes, dtype=torch.uint8).pin_memory()
+    link = {"d2h_gbs": time_copies([(arena, buf[:record_bytes])]), "h2d_gbs": time_copies([(back, arena2)]),
+            "both_at_once_gbs_each_way": time_copies([(arena, buf[:record_bytes]), (back, arena2)]),
+            "what": "bare cudaMemcpyAsync of the records' bytes between device and pinned host memory, best of 4"}
+    del arena2
+    # the slowest rank's link counts
+    link = {k: (-sharding.max_over_ranks([-v], dist, "cuda")[0] if isinstance(v, float) else v) for k, v in link.items()}
+
     e2e_batch = max(1, n // max(1, args.e2e_batches))
     e2e_serial_ms = time_e2e(make_plan(n))
     e2e_ms = time_e2e(make_plan(e2e_batch))
@@ -475,15 +515,31 @@ def run_ours(args):
     k_ms = {"compress_kernel": comp_ms, "decompress_kernel": decomp_ms}
     dominant = max(k_ms, key=k_ms.get)
     achieved = algo_bytes / (k_ms[dominant] * 1e-3) / 1e9
+    if args.quant_mode == 0 and LEVELS == (8, 4, 2) and not args.chunk_len:
+        traffic, traffic_source = measured_traffic((shape.name, shape.n_layers, dominant))
+    else:
+        traffic, traffic_source = None, "no capture for this workload"
+    # the score stage: K read once, the per-segment softmax statistics written by the logits kernel and read back by
+    # the kernels behind it (twice where a pass over all statistics makes the row normalisers)
+    rows = shape.n_layers * shape.n_q_heads * W
+    seg = 1
+    while seg < 32 and shape.chunk_len % (seg * 2) == 0:
+        seg *= 2
+    stat_bytes = 2 * rows * ((shape.n_tokens + seg - 1) // seg) * 4
+    row_pass = not (shape.n_q_heads // shape.n_kv_heads * W <= 16 and seg >= 16)
+    score_bytes = kv_bytes // 2 + stat_bytes * (3 if row_pass else 2)
     roofline = {
         "kernel": dominant, "bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
         "peak_source": f"{peak_kind} copy bandwidth", "launches_per_stage": B.codec_launches(d, bits) - (1 if args.quant_mode == 1 else 0),
-        "traffic": (NCU_DRAM_TRAFFIC.get((shape.name, shape.n_layers, dominant))
-                    if args.quant_mode == 0 and LEVELS == (8, 4, 2) and not args.chunk_len else None),
+        "traffic": traffic, "traffic_source": traffic_source,
         "algorithmic_bytes_per_launch": algo_bytes,
         "frac_of_nominal_8000": achieved / 8000.0,
         # each codec launch timed alone (events around one call = one codec kernel + its checksum kernel)
         "per_launch": [dict(pl, frac=pl["gbs"] / peak) for pl in per_launch],
+        "score": {"what": "score stage: K read once + softmax statistics written and read back; stage time includes the ranking kernel",
+                  "bytes": score_bytes, "k_bytes": kv_bytes // 2, "ms": tol_ms,
+                  "achieved": score_bytes / (tol_ms * 1e-3) / 1e9, "frac": score_bytes / (tol_ms * 1e-3) / 1e9 / peak,
+                  "frac_k_only": (kv_bytes // 2) / (tol_ms * 1e-3) / 1e9 / peak},
         "per_stage": {
             "tolerance_ms": tol_ms, "compress_ms": comp_ms, "decompress_ms": decomp_ms,
             "tolerance_gbs_of_K_read": (kv_bytes / 2) / (tol_ms * 1e-3) / 1e9,
@@ -507,6 +563,8 @@ def run_ours(args):
         "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": record_bytes, "d2h_bytes_per_step": record_bytes,
                 "ms_per_step": e2e_ms, "context_switches_per_s": world / (e2e_ms * 1e-3),
                 "host_copy_gbs_each_way": record_bytes / (e2e_ms * 1e-3) / 1e9,
+                "link_gbs": link,
+                "frac_of_link": record_bytes / (e2e_ms * 1e-3) / 1e9 / link["both_at_once_gbs_each_way"],
                 "serial_ms_per_step": e2e_serial_ms, "batch_chunks": e2e_batch,
                 "what": "compress -> swap-out to pinned host -> swap-in -> decompress, pipelined in batches of chunks",
                 "layerwise_load": layerwise},

@@ -305,6 +305,13 @@ def assign_levels(scores, frac, levels):
     return bits, order
 
 
+def level_counts(n, frac, levels=(8, 4, 2)):
+    """How many of n chunks each level gets under llms_assign_levels (the counts depend on n and frac alone):
+    asked of the library itself, on n distinct scores."""
+    bits, _ = assign_levels(np.arange(n, 0, -1, dtype=np.float32), frac, levels)
+    return tuple(int((bits == b).sum()) for b in levels)
+
+
 def optimize_thresholds(scores, ratio_global):
     s = np.ascontiguousarray(scores, dtype=np.float32)
     frac = np.zeros(3, dtype=np.float32)

@@ -108,15 +108,9 @@ class MultiApp:
         self.ev_landed = [B.new_event() for _ in range(2)]
         self._out_k = self._in_k = 0
         # the arena: every (context, chunk) record at its own offset, bit-widths fixed at set-up by the tertiles
-        n8, n4, n2 = self._tertile_counts()
+        n8, n4, n2 = B.level_counts(self.cpc, self.frac)
         total = self.n_ctx * (n8 * self.rec_bytes[8] + n4 * self.rec_bytes[4] + n2 * self.rec_bytes[2])
         self.arena = torch.empty(total, dtype=torch.uint8).pin_memory()
-
-    def _tertile_counts(self):
-        n = self.cpc
-        n8 = int(np.floor(np.float32(self.frac[0]).astype(np.float64) * n + 0.5))
-        n84 = int(np.floor((np.float64(np.float32(self.frac[0])) + np.float64(np.float32(self.frac[1]))) * n + 0.5))
-        return n8, n84 - n8, n - n84
 
     def _next_ws(self):
         i = self._ws_next % len(self.ws)

@@ -168,9 +168,10 @@ def random_bits(n: int, seed: int = 0) -> torch.Tensor:
     return levels[(_lsr(z, 33) % 3)]
 
 
-def attention_probs(shape: KVShape, W: int = None, device="cpu", sharpness: float = 2.0) -> torch.Tensor:
+def attention_probs(shape: KVShape, W: int = None, device="cpu", sharpness: float = 8.0) -> torch.Tensor:
     """fp32 [L, Hq, W, T]: a valid causal attention window (row r sits at position T-W+r, sees columns
-    0..T-W+r, sums to 1, masked entries are 0) built from random logits."""
+    0..T-W+r, sums to 1, masked entries are 0).  Rows are heavy-tailed positive draws (a uniform number raised to
+    the power `sharpness`: a few columns carry most of a row) divided by their sum over the visible columns."""
     W = shape.window if W is None else W
     L, H, T = shape.n_layers, shape.n_q_heads, shape.n_tokens
     out = torch.empty(L, H, W, T, dtype=torch.float32, device=device)
@@ -178,7 +179,7 @@ def attention_probs(shape: KVShape, W: int = None, device="cpu", sharpness: floa
     col = torch.arange(T, device=device).view(1, 1, T)
     pos = (T - W + torch.arange(W, device=device)).view(1, W, 1)
     for l in range(L):
-        logits = sharpness * normal(key, l * H * W * T, H * W * T, device).view(H, W, T)
-        logits = logits.masked_fill(col > pos, float("-inf"))
-        out[l] = torch.softmax(logits, dim=-1).to(torch.float32)
+        weights = _uniform(_draw_u64(key, l * H * W * T, H * W * T, device)).view(H, W, T) ** sharpness
+        weights = weights.masked_fill(col > pos, 0.0)
+        out[l] = (weights / weights.sum(dim=-1, keepdim=True)).to(torch.float32)
     return out

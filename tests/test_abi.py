@@ -113,6 +113,47 @@ def test_optimize_thresholds_levels_matches_oracle_bit_for_bit():
         B.optimize_thresholds_levels([0.1, 0.2, 0.3], 0.1, (8, 4, 2))       # below the low level's ratio
 
 
+def test_optimize_thresholds_against_an_exhaustive_search():
+    """Eq. 3 by search, in exact rational arithmetic, sharing no formula with the library or the oracle: for every count
+    of top-level chunks the count of low-level chunks is the one whose achieved ratio comes closest to the wanted one
+    (searched, not solved for; a tie goes to more compression), the objective is the plain weighted sum over the
+    density-ordered chunks, the best triple wins, the smaller top count on a tie."""
+    from fractions import Fraction as F
+    rng = np.random.default_rng(11)
+    for levels in ((8, 4, 2), (4, 2, 1), (8, 2, 1), (8, 4, 1)):
+        r1, r2 = F(levels[1], levels[0]), F(levels[2], levels[0])
+        for n in (1, 2, 3, 5, 8, 12):
+            for R in (F(1, 2), F(3, 8), F(3, 4), F(5, 16), F(1), r2):
+                if R < r2:
+                    continue
+                # dyadic scores: every sum below is exact in binary64 too, so ties are ties on both sides
+                scores = (rng.integers(1, 64, n) / 64.0).astype(np.float32)
+                dens = sorted((F(float(x)) for x in scores), reverse=True)
+                best = None
+                step = (r1 - r2) / n                       # what one more low-level chunk takes off the achieved ratio
+                for n_top in range(n + 1):
+                    cands = []
+                    for n_low in range(n + 1):
+                        achieved = (n_top + r1 * (n - n_top - n_low) + r2 * n_low) / n
+                        cands.append((abs(achieved - R), -n_low, achieved))
+                    _, neg_low, achieved = min(cands)
+                    n_low = -neg_low
+                    if not (-step / 2 <= achieved - R < step / 2):    # even the nearest count is more than half a step off
+                        continue
+                    if n_top + n_low > n:                             # more chunks than there are
+                        continue
+                    info = sum(dens[:n_top]) + r1 * sum(dens[n_top:n - n_low]) + r2 * sum(dens[n - n_low:])
+                    if best is None or info > best[0]:
+                        best = (info, n_top, n_low)
+                if best is None:
+                    with pytest.raises(B.LlmsError):
+                        B.optimize_thresholds_levels(scores, float(R), levels)
+                    continue
+                got = B.optimize_thresholds_levels(scores, float(R), levels)
+                want = np.array([best[1], n - best[1] - best[2], best[2]], dtype=np.float64) / n
+                assert np.array_equal(got, want.astype(np.float32)), (levels, n, R, scores, got, want)
+
+
 def test_lctru_order_matches_oracle_bit_for_bit():
     rng = np.random.default_rng(1)
     for n in (0, 1, 5, 64, 2048):

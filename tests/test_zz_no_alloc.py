@@ -11,7 +11,9 @@ import numpy as np
 import pytest
 import torch
 
+import oracle
 from paper_2403_11805_b200 import binding as B, synth
+from gpu_helpers import assert_meta_equal, bits_view, odesc
 
 pytestmark = pytest.mark.gpu
 
@@ -45,6 +47,32 @@ def test_static_entry_matches_workspace_entry_twice_in_a_row():
     big_kv = synth.kv_tensor(big, device="cuda")
     bits = np.array([(8, 4, 2)[i % 3] for i in range(big.n_chunks)], dtype=np.uint8)
     run_both(big, big_kv, np.arange(big.n_chunks, dtype=np.uint32), bits)
+
+
+def test_static_entry_against_the_oracle_without_taking_device_memory():
+    """The records and meta of the no-scratch entry point equal the CPU oracle's, call after call, and the device's
+    free memory does not move across the calls: whoever could not allocate before the call still has not had to."""
+    sh = synth.CONFIGS["tiny"]
+    kv = synth.kv_tensor(sh)
+    kv_dev = kv.cuda()
+    d = B.desc_of(sh)
+    cases = [(np.arange(sh.n_chunks, dtype=np.uint32), synth.random_bits(sh.n_chunks, 5).numpy()),
+             (np.array([3, 12, 0, 7], dtype=np.uint32), np.array([4, 4, 8, 2], dtype=np.uint8)),
+             (np.arange(sh.n_chunks, dtype=np.uint32)[::-1].copy(), np.full(sh.n_chunks, 2, dtype=np.uint8))]
+    # every buffer exists before the first measured call; the calls themselves get raw pointers only
+    outs = [torch.zeros(B.compressed_size(d, bits), dtype=torch.uint8, device="cuda") for _, bits in cases]
+    metas = [B.new_meta(len(ids), pinned=True) for ids, _ in cases]
+    B.compress_chunks_static(d, kv_dev, cases[0][0], cases[0][1], outs[0], metas[0])   # first call: looks the array's address up
+    torch.cuda.synchronize()
+    free_before = torch.cuda.mem_get_info()[0]
+    for (ids, bits), out, meta in zip(cases[1:], outs[1:], metas[1:]):
+        B.compress_chunks_static(d, kv_dev, ids, bits, out, meta)
+        torch.cuda.synchronize()
+        assert torch.cuda.mem_get_info()[0] == free_before
+    for (ids, bits), out, meta in zip(cases, outs, metas):
+        want_buf, want_meta = oracle.compress_chunks(odesc(sh), bits_view(kv), ids, bits)
+        assert np.array_equal(out.cpu().numpy(), want_buf)
+        assert_meta_equal(meta, want_meta)
 
 
 def test_static_entry_rejects_more_chunks_than_its_table_holds():
