@@ -40,6 +40,9 @@ def parse_args():
     p.add_argument("--no-cpu-baseline", action="store_true")
     p.add_argument("--no-layerwise", dest="layerwise", action="store_false",
                    help="skip the layer-wise swap timing (records split per layer, Sec. 4: first layer ready / all layers ready)")
+    p.add_argument("--fused-swap", action="store_true",
+                   help="also time swap-out and swap-in without a staging buffer: the encoder writes into, the decoder reads "
+                        "from page-locked host memory directly (e2e.fused_swap)")
     p.add_argument("--aot", action="store_true", help="multiapp: swap served contexts out ahead of time (Sec. 3.4 i)")
     p.add_argument("--quant-mode", type=int, default=0, choices=[0, 1],
                    help="0: groups of group_size channels of one token (the metric's setting); 1: one group per channel "
@@ -376,6 +379,27 @@ def run_ours(args):
                                "algorithmic_bytes": int(launch_bytes), "gbs": launch_bytes / (ms * 1e-3) / 1e9})
         assert B.codec_corrupt_count(ws_dec) == 0
 
+    # ---- what a plain stream of the codec's access shape reaches on this GPU, per read:write mix (the encoder reads
+    # about four bytes per byte written, the decoder the reverse): context for the roofline fractions
+    def stream_ceiling(read_kib, write_kib, reps=6):
+        per_iter = (read_kib + write_kib) * 1024
+        iters = min(kv.numel() * 2 // (max(read_kib, 1) * 1024), kv_out.numel() * 2 // (max(write_kib, 1) * 1024))
+        best = None
+        for it in range(reps):
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record(stream)
+            B.stream_probe(kv, kv_out, iters, read_kib, write_kib)
+            e1.record(stream)
+            torch.cuda.synchronize()
+            if it >= 2:
+                ms = e0.elapsed_time(e1)
+                best = ms if best is None else min(best, ms)
+        return iters * per_iter / (best * 1e-3) / 1e9
+
+    mix = {"read_only": stream_ceiling(4, 0), "write_only": stream_ceiling(0, 4), "read4_write1": stream_ceiling(4, 1),
+           "read1_write4": stream_ceiling(1, 4), "read1_write1": stream_ceiling(2, 2)}
+    mix = {k: -sharding.max_over_ranks([-v], dist, "cuda")[0] for k, v in mix.items()}
+
     # ---- end to end: compress -> swap-out -> swap-in -> decompress with the pinned arena in the loop.
     # The chunks go in batches: while batch j travels to the host, batch j-1 is already on its way back and batch
     # j-2 is being decoded (the two copy directions and the kernels overlap); "serial" does one batch of everything.
@@ -459,6 +483,44 @@ def run_ours(args):
     e2e_ms = time_e2e(make_plan(e2e_batch))
     e2e_value = world * 2 * kv_bytes / (e2e_ms * 1e-3) / 1e9
 
+    # ---- swap without a staging buffer: the kernels work straight on the page-locked arena, against kernel + copy engine
+    fused_swap = None
+    if args.fused_swap:
+        p_ = make_plan(n)[0]
+        def timed(fn, reps=5):
+            ts = []
+            for it in range(reps + 2):
+                e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                torch.cuda.synchronize()
+                e0.record(stream)
+                fn()
+                e1.record(stream)
+                torch.cuda.synchronize()
+                if it >= 2:
+                    ts.append(e0.elapsed_time(e1))
+            return statistics.median(ts)
+
+        def staged_out():
+            B.compress_chunks(d, kv, p_["ids"], p_["bits"], buf, p_["meta"], p_["ws"])
+            p_["ev_c"].record(stream)
+            B.swap_out(buf[:record_bytes], p_["meta"], arena, side_stream=side_out, after=p_["ev_c"], done=p_["ev_out"], n=n)
+            stream.wait_event(p_["ev_out"])
+
+        def staged_in():
+            p_["ev_out"].record(stream)
+            B.swap_in(arena, p_["meta"], back, side_stream=side_in, after=p_["ev_out"], done=p_["ev_in"], n=n)
+            stream.wait_event(p_["ev_in"])
+            B.decompress_chunks(d, back, p_["meta"], None, kv_out, p_["ws"])
+
+        fused_swap = {
+            "swap_out_staged_ms": timed(staged_out),
+            "swap_out_fused_ms": timed(lambda: B.compress_chunks(d, kv, p_["ids"], p_["bits"], arena, p_["meta"], p_["ws"])),
+            "swap_in_staged_ms": timed(staged_in),
+            "swap_in_fused_ms": timed(lambda: B.decompress_chunks(d, arena, p_["meta"], None, kv_out, p_["ws"])),
+            "what": "whole context in one call; staged = codec kernel on a device buffer + copy engine, fused = the codec "
+                    "kernel reads or writes the page-locked arena itself"}
+        assert B.codec_corrupt_count(p_["ws"]) == 0
+
     # ---- layer-wise load (Sec. 4): records split per layer; how soon is the first layer usable, when the last
     layerwise = None
     if args.e2e_steps > 0 and args.layerwise:
@@ -533,6 +595,10 @@ def run_ours(args):
         "peak_source": f"{peak_kind} copy bandwidth", "launches_per_stage": B.codec_launches(d, bits) - (1 if args.quant_mode == 1 else 0),
         "traffic": traffic, "traffic_source": traffic_source,
         "algorithmic_bytes_per_launch": algo_bytes,
+        # plain streams with the codec's access shape, GB/s of bytes read + written, best of 4 launches over this
+        # workload's buffers; the dominant kernel's own mix beside it
+        "stream_ceilings_gbs": mix,
+        "frac_of_stream_with_its_mix": achieved / mix["read4_write1" if dominant == "compress_kernel" else "read1_write4"],
         "frac_of_nominal_8000": achieved / 8000.0,
         # each codec launch timed alone (events around one call = one codec kernel + its checksum kernel)
         "per_launch": [dict(pl, frac=pl["gbs"] / peak) for pl in per_launch],
@@ -567,7 +633,7 @@ def run_ours(args):
                 "frac_of_link": record_bytes / (e2e_ms * 1e-3) / 1e9 / link["both_at_once_gbs_each_way"],
                 "serial_ms_per_step": e2e_serial_ms, "batch_chunks": e2e_batch,
                 "what": "compress -> swap-out to pinned host -> swap-in -> decompress, pipelined in batches of chunks",
-                "layerwise_load": layerwise},
+                "layerwise_load": layerwise, "fused_swap": fused_swap},
         # score kernels (logits, column sums + chunk means; a row pass in between for more than 16 rows per KV head),
         # the ranking kernel, then one codec kernel per call (channel-wise mode: one per bit-width and one for the sums)
         "gpu_launches": args.steps * ((2 if shape.n_q_heads // shape.n_kv_heads * W <= 16 and shape.chunk_len % 16 == 0 else 3)

@@ -291,6 +291,18 @@ int llms_swap_in(const void *pinned_src, uint64_t host_bytes, const uint64_t *ho
 /* Poll a cudaEvent_t until it has completed or timeout_ms has passed (LLMS_ERR_TIMEOUT). */
 int llms_wait(void *event, uint32_t timeout_ms);
 
+/* ------------------------------------------------------------------ measurement aid */
+
+/* Not a step of the method (the paper has no counterpart): a plain streaming kernel with the codec kernels' access
+ * shape - every load or store instruction of a warp covers 1 KiB of consecutive bytes in 256-bit accesses - that reads
+ * read_kib KiB from src and writes write_kib KiB to dst per warp iteration, `iters` iterations in all.  Timing it
+ * tells what the memory system gives a stream of that read:write mix, the yardstick for the encoder (about 4:1) and
+ * the decoder (about 1:4).  Mixes: (4,0) read only, (0,4) write only, (4,1), (1,4), (2,2); others return
+ * LLMS_ERR_UNSUPPORTED.  src and dst are device pointers, 32-byte aligned, of at least iters*read_kib KiB and
+ * iters*write_kib KiB (LLMS_ERR_BUF_TOO_SMALL otherwise, before any launch); dst is overwritten with arbitrary bytes. */
+int llms_stream_probe(const void *src, uint64_t src_bytes, void *dst, uint64_t dst_bytes, uint64_t iters,
+                      int read_kib, int write_kib, void *stream);
+
 #ifdef __cplusplus
 }
 #endif

@@ -73,6 +73,7 @@ _SIGNATURES = {
     "llms_swap_in": (C.c_int, [C.c_void_p, C.c_uint64, C.c_void_p, C.c_void_p, C.c_int, C.c_void_p, C.c_uint64,
                                C.c_void_p, C.c_void_p, C.c_void_p]),
     "llms_wait": (C.c_int, [C.c_void_p, C.c_uint32]),
+    "llms_stream_probe": (C.c_int, [C.c_void_p, C.c_uint64, C.c_void_p, C.c_uint64, C.c_uint64, C.c_int, C.c_int, C.c_void_p]),
 }
 
 
@@ -373,3 +374,11 @@ def swap_in(pinned_src, meta, dev_buf, host_offsets=None, side_stream=None, afte
 
 def wait(event, timeout_ms=10000):
     _check(lib().llms_wait(_event(event), int(timeout_ms)), "llms_wait")
+
+
+# ----------------------------------------------------------------------------- measurement aid
+
+def stream_probe(src, dst, iters, read_kib, write_kib, stream=None):
+    """llms_stream_probe: a plain stream of the given read:write mix (KiB per warp iteration) over src / dst."""
+    _check(lib().llms_stream_probe(_ptr(src), _nbytes(src), _ptr(dst), _nbytes(dst), int(iters), int(read_kib), int(write_kib),
+                                   _stream(stream)), "llms_stream_probe")

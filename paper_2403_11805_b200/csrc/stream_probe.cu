@@ -1,0 +1,75 @@
+// A plain streaming kernel with the codec's access shape (every load or store instruction of a warp covers 1 KiB of
+// consecutive bytes in 256-bit accesses) and a chosen mix of bytes read to bytes written.  It does nothing useful: it
+// measures what the memory system gives such a stream, which is the yardstick the codec kernels' throughput is read
+// against (the encoder reads about four bytes for each one it writes, the decoder the reverse).
+#include <algorithm>
+
+#include "llms_internal.cuh"
+
+namespace llms {
+
+constexpr int kProbeThreads = 256;
+
+template <int RK, int WK>
+__global__ void __launch_bounds__(kProbeThreads) stream_probe_kernel(const uint8_t *__restrict__ src, uint8_t *__restrict__ dst,
+                                                                     uint64_t iters, uint32_t *sink)
+{
+    const int lane = threadIdx.x & 31;
+    const uint64_t n_warps = (uint64_t)gridDim.x * (kProbeThreads / 32);
+    uint32_t acc = 0;
+    for (uint64_t i = (uint64_t)blockIdx.x * (kProbeThreads / 32) + (threadIdx.x >> 5); i < iters; i += n_warps) {
+        uint32_t w[RK > 0 ? RK : 1][8];
+#pragma unroll
+        for (int k = 0; k < RK; ++k) {
+            const uint8_t *p = src + (i * RK + k) * 1024 + lane * 32;
+            asm volatile("ld.global.nc.L1::no_allocate.v8.b32 {%0,%1,%2,%3,%4,%5,%6,%7}, [%8];"
+                         : "=r"(w[k][0]), "=r"(w[k][1]), "=r"(w[k][2]), "=r"(w[k][3]), "=r"(w[k][4]), "=r"(w[k][5]), "=r"(w[k][6]),
+                           "=r"(w[k][7])
+                         : "l"(p));
+        }
+#pragma unroll
+        for (int k = 0; k < RK; ++k)
+#pragma unroll
+            for (int j = 0; j < 8; ++j) acc ^= w[k][j];
+#pragma unroll
+        for (int k = 0; k < WK; ++k) {
+            uint8_t *p = dst + (i * WK + k) * 1024 + lane * 32;
+            const uint32_t v = (uint32_t)i;
+            asm volatile("st.global.L1::no_allocate.v8.b32 [%8], {%0,%1,%2,%3,%4,%5,%6,%7};"
+                         :: "r"(v), "r"(v), "r"(v), "r"(v), "r"(v), "r"(v), "r"(v), "r"(v), "l"(p) : "memory");
+        }
+    }
+    if (acc == 0x9E3779B9u && sink) *sink = acc;   // keeps the loads alive; practically never taken
+}
+
+}  // namespace llms
+
+using namespace llms;
+
+extern "C" int llms_stream_probe(const void *src, uint64_t src_bytes, void *dst, uint64_t dst_bytes, uint64_t iters,
+                                 int read_kib, int write_kib, void *stream)
+{
+    if (iters == 0 || read_kib < 0 || write_kib < 0 || read_kib + write_kib == 0) return LLMS_ERR_INVALID_ARG;
+    if ((read_kib > 0 && !src) || (write_kib > 0 && !dst)) return LLMS_ERR_INVALID_ARG;
+    if (!aligned(src, 32) || !aligned(dst, 32)) return LLMS_ERR_MISALIGNED;
+    if (iters > (1ull << 40) || iters * (uint64_t)read_kib * 1024 > src_bytes || iters * (uint64_t)write_kib * 1024 > dst_bytes)
+        return LLMS_ERR_BUF_TOO_SMALL;
+    const uint64_t want = (iters + kProbeThreads / 32 - 1) / (kProbeThreads / 32);
+    const int grid = (int)std::min<uint64_t>(want, (uint64_t)sm_count() * 8);
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const uint8_t *s = static_cast<const uint8_t *>(src);
+    uint8_t *d = static_cast<uint8_t *>(dst);
+#define LLMS_PROBE(R, W)                                                                        \
+    if (read_kib == R && write_kib == W) {                                                      \
+        stream_probe_kernel<R, W><<<grid, kProbeThreads, 0, st>>>(s, d, iters, nullptr);        \
+        LLMS_CUDA_TRY(cudaGetLastError());                                                      \
+        return LLMS_OK;                                                                         \
+    }
+    LLMS_PROBE(4, 0)
+    LLMS_PROBE(0, 4)
+    LLMS_PROBE(4, 1)
+    LLMS_PROBE(1, 4)
+    LLMS_PROBE(2, 2)
+#undef LLMS_PROBE
+    return LLMS_ERR_UNSUPPORTED;
+}

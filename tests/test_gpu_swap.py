@@ -89,9 +89,60 @@ def test_wait_times_out_and_then_succeeds():
     B.wait(ev, 20000)
 
 
+def test_codec_works_straight_on_mapped_pinned_memory():
+    """Swap-out and swap-in without a staging buffer: the encoder writes its records straight into page-locked host
+    memory (which the device reaches over the link) and the decoder reads them from there.  The ABI takes such
+    pointers as they are; bytes, checksums and decoded values are the oracle's."""
+    import oracle
+    from gpu_helpers import assert_meta_equal, bits_view, first_mismatch, odesc
+    sh = synth.CONFIGS["llama7b"].with_(n_layers=1, n_tokens=512)
+    kv = synth.kv_tensor(sh)
+    kv_dev = kv.cuda()
+    d = B.desc_of(sh)
+    n = sh.n_chunks
+    ids = np.arange(n, dtype=np.uint32)
+    bits = np.array([(8, 4, 2, 1)[i % 4] for i in range(n)], dtype=np.uint8)
+    total = B.compressed_size(d, bits)
+    arena = torch.full((total + 4096,), 0x5A, dtype=torch.uint8).pin_memory()
+    meta = B.new_meta(n, pinned=True)
+    ws = torch.empty(B.codec_workspace_bytes(n), dtype=torch.uint8, device="cuda")
+    B.compress_chunks(d, kv_dev, ids, bits, arena, meta, ws, out_bytes=total)
+    torch.cuda.synchronize()
+    want_buf, want_meta = oracle.compress_chunks(odesc(sh), bits_view(kv), ids, bits)
+    assert first_mismatch(arena.numpy()[:total], want_buf) is None
+    assert (arena.numpy()[total:] == 0x5A).all()
+    assert_meta_equal(meta, want_meta)
+    out = torch.zeros_like(kv_dev)
+    B.decompress_chunks(d, arena, meta, None, out, ws, buf_bytes=total)
+    assert B.codec_corrupt_count(ws) == 0
+    want = np.zeros(kv.numel(), dtype=np.uint16).reshape(kv.shape)
+    oracle.decompress_chunks(odesc(sh), want_buf, want_meta, want)
+    assert first_mismatch(bits_view(out).reshape(-1), want.reshape(-1)) is None
+
+
 def test_swap_argument_errors():
     meta = B.new_meta(1)
     meta[0]["nbytes"] = 100          # not a multiple of 256
     assert B.lib().llms_swap_out(4096, 1 << 20, meta.ctypes.data, 1, 8192, 1 << 20, None, None, None, None) == B.ERR_MISALIGNED
     assert B.lib().llms_swap_out(None, 1 << 20, meta.ctypes.data, 1, 8192, 1 << 20, None, None, None, None) == B.ERR_INVALID_ARG
     assert B.lib().llms_swap_in(4096, 0, None, meta.ctypes.data, 0, 8192, 0, None, None, None) == B.OK
+
+
+def test_stream_probe_stays_inside_its_buffers():
+    """The measurement aid: every supported mix runs, writes exactly iters * write_kib KiB and refuses buffers that
+    are too short or mixes it has no kernel for, before anything is launched."""
+    src = torch.arange(1 << 20, dtype=torch.int32, device="cuda")              # 4 MiB
+    for rk, wk in ((4, 0), (0, 4), (4, 1), (1, 4), (2, 2)):
+        iters = 300
+        dst = torch.full((iters * wk * 1024 + 4096,), 0x77, dtype=torch.uint8, device="cuda")
+        B.stream_probe(src, dst, iters, rk, wk)
+        torch.cuda.synchronize()
+        assert bool((dst[iters * wk * 1024:] == 0x77).all())
+        if wk:
+            assert not bool((dst[:iters * wk * 1024] == 0x77).all())
+    dst = torch.zeros(8192, dtype=torch.uint8, device="cuda")
+    for args, status in (((src, dst, 3, 1, 4), B.ERR_BUF_TOO_SMALL), ((src, dst, 2000, 4, 0), B.ERR_BUF_TOO_SMALL),
+                         ((src, dst, 2, 3, 1), B.ERR_UNSUPPORTED), ((src, dst, 0, 4, 1), B.ERR_INVALID_ARG)):
+        with pytest.raises(B.LlmsError) as e:
+            B.stream_probe(*args)
+        assert e.value.status == status
