@@ -661,6 +661,7 @@ __global__ void __launch_bounds__(kThreads, 2) compress_kernel(const __grid_cons
 {
     __shared__ __align__(16) unsigned char patches[kWarpsPerBlock][kTransposeBytes];
     __shared__ uint32_t sum_slots[kSumSlots];
+    grid_dependency_wait();   // the chunk tables may come from a kernel that is still finishing (a no-op otherwise)
     if (all.w[0].n) compress_phase<8, G, WIDE, PACKED>(all.w[0], patches, sum_slots);
     if (all.w[1].n) compress_phase<4, G, WIDE, PACKED>(all.w[1], patches, sum_slots);
     if (all.w[2].n) compress_phase<2, G, WIDE, PACKED>(all.w[2], patches, sum_slots);
@@ -1146,7 +1147,8 @@ static int check_common(const llms_kv_desc *desc, int n, const void *workspace, 
 // first[k] / count[k]: where the chunks of width 8, 4, 2, 1 start in the grouped order and how many there are), and see
 // to it that the checksums reach `meta` (host) in stream order.
 static int launch_compress(const llms_kv_desc &desc, const void *kv, void *out_buf, void *workspace, int n,
-                           const int (&first)[kNumWidths], const int (&count)[kNumWidths], llms_chunk_meta *meta, cudaStream_t st)
+                           const int (&first)[kNumWidths], const int (&count)[kNumWidths], llms_chunk_meta *meta, cudaStream_t st,
+                           bool after_kernel = false)
 {
     CodecArgs a{};
     const bool wide = wide_ok(desc, kv);
@@ -1159,6 +1161,7 @@ static int launch_compress(const llms_kv_desc &desc, const void *kv, void *out_b
         groups.count[k] = count[k];
     }
     int rc = LLMS_OK;
+    cudaError_t launch_err = cudaSuccess;
     bool published = false;  // the codec kernel itself stores the checksums into a page-locked meta array
     if (desc.quant_mode == 1) {
         for (int k = 0; k < kNumWidths; ++k) {
@@ -1186,11 +1189,18 @@ static int launch_compress(const llms_kv_desc &desc, const void *kv, void *out_b
         published = all.live_meta != nullptr;
         rc = dispatch_group(desc.group_size, [&](auto g) {
             constexpr int kG = decltype(g)::value;
-            if (a.packed) compress_kernel<kG, true, true><<<grid_for(compress_kernel<kG, true, true>, most_units), kThreads, 0, st>>>(all);
-            else if (wide) compress_kernel<kG, true, false><<<grid_for(compress_kernel<kG, true, false>, most_units), kThreads, 0, st>>>(all);
-            else compress_kernel<kG, false, false><<<grid_for(compress_kernel<kG, false, false>, most_units), kThreads, 0, st>>>(all);
+            // after_kernel: the tables come from a kernel just ahead on the stream; this one may be set up while that one ends
+            auto go = [&](auto kernel) {
+                const int grid = grid_for(kernel, most_units);
+                if (after_kernel) launch_err = launch_dependent(kernel, dim3(grid), dim3(kThreads), 0, st, all);
+                else kernel<<<grid, kThreads, 0, st>>>(all);
+            };
+            if (a.packed) go(compress_kernel<kG, true, true>);
+            else if (wide) go(compress_kernel<kG, true, false>);
+            else go(compress_kernel<kG, false, false>);
         });
         if (rc) return rc;
+        LLMS_CUDA_TRY(launch_err);
         LLMS_CUDA_TRY(cudaGetLastError());
     }
     // checksums back to the caller's meta (every other field is already there)
@@ -1268,7 +1278,7 @@ int llms::compress_planned(const llms_kv_desc *desc, const void *kv, int n, cons
         at += count[k];
     }
     if (at != n) return LLMS_ERR_INVALID_ARG;
-    return launch_compress(*desc, kv, out_buf, workspace, n, first, cnt, meta, static_cast<cudaStream_t>(stream));
+    return launch_compress(*desc, kv, out_buf, workspace, n, first, cnt, meta, static_cast<cudaStream_t>(stream), true);
 }
 
 int llms::check_compress_args(const llms_kv_desc *desc, int n, const void *kv, const void *out_buf, const void *workspace,

@@ -20,6 +20,30 @@ void set_cuda_error(cudaError_t e, const char *where);
         }                                                     \
     } while (0)
 
+// Programmatic dependent launch: `kernel` may be set up on the GPU while the kernel before it on the stream is still
+// finishing, once all CTAs of that kernel have called grid_launch_dependents() (or left).  The launched kernel must
+// call grid_dependency_wait() before it touches anything its predecessor wrote: that returns when the predecessor has
+// completed and its writes are visible.  Both calls do nothing in a kernel that was launched the ordinary way.
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_dependent(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st, Args &&...args)
+{
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid;
+    cfg.blockDim = block;
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
+}
+#ifdef __CUDACC__
+__device__ __forceinline__ void grid_dependency_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void grid_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+#endif
+
 inline uint64_t round_up(uint64_t x, uint64_t a) { return (x + a - 1) / a * a; }
 inline bool aligned(const void *p, uintptr_t a) { return (reinterpret_cast<uintptr_t>(p) & (a - 1)) == 0; }
 inline bool is_pow2(int x) { return x > 0 && (x & (x - 1)) == 0; }

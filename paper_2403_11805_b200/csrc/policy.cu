@@ -157,18 +157,27 @@ __global__ void __launch_bounds__(kPlanThreads) plan_context_kernel(const PlanAr
     __shared__ float s_scores[kPlanMaxChunks];
     __shared__ uint8_t s_level[kPlanMaxChunks];                // index into levels[]
     __shared__ unsigned long long s_scan[32];
+    grid_dependency_wait();
     const int n = a.n;
     for (int i = threadIdx.x; i < n; i += kPlanThreads) s_scores[i] = a.scores[i];
     if (threadIdx.x < 4) reinterpret_cast<uint32_t *>(a.workspace)[threadIdx.x] = 0;   // status word, spare, finished-CTA count
     __syncthreads();
-    for (int i = threadIdx.x; i < n; i += kPlanThreads) {
-        const float mine = s_scores[i];
+    // rank of chunk i = chunks that come before it; `parts` neighbouring lanes share a chunk and split the others
+    // among them (a power of two, at most 32, so that they sit in one warp)
+    int parts = 1;
+    while (parts < 32 && n * parts * 2 <= kPlanThreads) parts *= 2;
+    for (int base = 0; base < n; base += kPlanThreads / parts) {
+        const int i = base + (int)threadIdx.x / parts, p = threadIdx.x % parts;
         int rank = 0;
-        for (int j = 0; j < n; ++j) {
-            const float other = s_scores[j];
-            rank += (other > mine) || (other == mine && j < i);
+        if (i < n) {
+            const float mine = s_scores[i];
+            for (int j = p; j < n; j += parts) {
+                const float other = s_scores[j];
+                rank += (other > mine) || (other == mine && j < i);
+            }
         }
-        s_level[i] = rank < a.n_top ? 0 : (rank < a.n_top_mid ? 1 : 2);
+        for (int d = 1; d < parts; d <<= 1) rank += __shfl_xor_sync(0xffffffffu, rank, d);
+        if (i < n && p == 0) s_level[i] = rank < a.n_top ? 0 : (rank < a.n_top_mid ? 1 : 2);
     }
     __syncthreads();
     // every thread owns a run of consecutive chunks: record bytes and per-width counts before each chunk by two scans
@@ -203,17 +212,29 @@ __global__ void __launch_bounds__(kPlanThreads) plan_context_kernel(const PlanAr
         u.entry = (uint32_t)i;
         u.rec_off = off;
         table[at] = u;
-        llms_chunk_meta m;
-        m.chunk_id = (uint32_t)i;
-        m.bits = bits;
-        m.offset = off;
-        m.nbytes = a.rec_bytes[lv];
-        m.n_groups = a.n_groups;
-        m.checksum = 0;
-        a.meta[i] = m;
-        a.bits_out[i] = (uint8_t)bits;
         off += a.rec_bytes[lv];
         seen += 1ull << (16 * k);
+    }
+    grid_launch_dependents();   // the encoder may be set up now; it waits for this kernel to complete before it reads the tables
+    // The caller's meta and level arrays lie across the host link, where every store instruction of a lane is a
+    // transaction of its own: they are written as whole warps of neighbouring 16-byte pieces (the meta entries are the
+    // bytes of the entries just laid down, read back through L2).
+    __syncthreads();
+    const uint4 *from = reinterpret_cast<const uint4 *>(entries);
+    uint4 *to = reinterpret_cast<uint4 *>(a.meta);
+    for (int i = threadIdx.x; i < 2 * n; i += kPlanThreads) to[i] = __ldcg(from + i);
+    if ((reinterpret_cast<uintptr_t>(a.bits_out) & 15) == 0) {
+        for (int i0 = threadIdx.x * 16; i0 < n; i0 += kPlanThreads * 16) {
+            uint32_t w[4] = {0, 0, 0, 0};
+            for (int k = 0; k < 16 && i0 + k < n; ++k) w[k >> 2] |= a.levels[s_level[i0 + k]] << (8 * (k & 3));
+            if (i0 + 16 <= n) {
+                *reinterpret_cast<uint4 *>(a.bits_out + i0) = make_uint4(w[0], w[1], w[2], w[3]);
+            } else {
+                for (int k = 0; i0 + k < n; ++k) a.bits_out[i0 + k] = (uint8_t)(w[k >> 2] >> (8 * (k & 3)));
+            }
+        }
+    } else {
+        for (int i = threadIdx.x; i < n; i += kPlanThreads) a.bits_out[i] = (uint8_t)a.levels[s_level[i]];
     }
 }
 
@@ -292,8 +313,7 @@ extern "C" int llms_compress_context(const llms_kv_desc *desc, const void *kv, c
         p.workspace = static_cast<uint8_t *>(codec_workspace);
         p.meta = meta_live;
         p.bits_out = bits_live;
-        plan_context_kernel<<<1, kPlanThreads, 0, st>>>(p);
-        LLMS_CUDA_TRY(cudaGetLastError());
+        LLMS_CUDA_TRY(launch_dependent(plan_context_kernel, dim3(1), dim3(kPlanThreads), 0, st, p));
         if (after_scores) LLMS_CUDA_TRY(cudaEventRecord(static_cast<cudaEvent_t>(after_scores), st));
         return compress_planned(desc, kv, n, count, out_buf, meta, codec_workspace, stream);
     }

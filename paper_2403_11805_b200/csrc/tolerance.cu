@@ -31,9 +31,12 @@ struct TolArgs {
     int n_chunks;
     int64_t stride_l, stride_h;
     float inv_sqrt_d;
-    float *pm, *ps, *pp;      // [rows][n_seg]: segment max, sum of exp, 1/n_vis-weighted sum of exp (pp: only the
-                              // segments from seg_tail0 on are read; before them it is ps / W)
-    float *row_max, *row_inv; // [rows]: filled by row_stats_kernel (only the fp32 logits kernel's path uses them)
+    float *pm, *ps, *pp;      // [n_seg][rows]: segment max, sum of exp, 1/n_vis-weighted sum of exp (pp: only the
+                              // segments from seg_tail0 on are read; before them it is ps / W).  Rows are the fast
+                              // index: the rows of a (layer, KV head) pair that a warp holds for one segment are then
+                              // neighbours in memory (with segments as the fast index every store touched a sector
+                              // per row, as many requests to L2 as the kernel's loads of K)
+    float *row_max, *row_inv; // [rows]: filled by row_stats_kernel where the logits kernel leaves no per-CTA row sums
     float2 *row_part;         // [rows][n_slots]: (max, sum of exp) of a row over the tiles of one CTA of the MMA kernel
     int n_slots;              // CTAs per (layer, KV head) pair; 0: the row normalisers are in row_max / row_inv
     float *part;              // [Y][n_seg]
@@ -41,6 +44,8 @@ struct TolArgs {
     uint32_t *tickets;        // [n_x + 1]: finished row slices per group of 32 segments, finished groups; the logits
                               // kernel of the same call clears them
     int n_x;                  // groups of 32 segments
+    uint32_t *status;         // set to a magic value by a logits kernel that gave a bounded wait up: the scores of the
+                              // call then come out as NaN (and the word is cleared)
     float *scores;
     float *scores_live;       // optional second destination of the scores (page-locked host memory), or NULL
     int Y, rows;
@@ -114,7 +119,7 @@ __global__ void __launch_bounds__(kTokThreads) logits_kernel(const TolArgs a)
                 sp += __shfl_xor_sync(0xffffffffu, sp, s);
             }
             if (valid && (lane & (SEG - 1)) == 0) {
-                const int64_t o = (row0 + j0 + j) * a.n_seg + seg;
+                const int64_t o = (int64_t)seg * a.rows + row0 + j0 + j;
                 a.pm[o] = m;
                 a.ps[o] = se;
                 a.pp[o] = sp;
@@ -251,7 +256,7 @@ __device__ __forceinline__ void row_statistics(const TolArgs &a, const float (&d
             const int t = t0 + nt * 8 + e;
             if (valid && t % SEG == 0 && t < a.T) {           // the segment's first token writes
                 const int seg = t / SEG;
-                const int64_t o = (row0 + j) * a.n_seg + seg;
+                const int64_t o = (int64_t)seg * a.rows + row0 + j;
                 a.pm[o] = mx[nt][e] * a.inv_sqrt_d;
                 a.ps[o] = se[nt][e];
                 if constexpr (TAIL)
@@ -401,6 +406,7 @@ __global__ void __launch_bounds__(kTileWarps * 32, 2) logits_mma_kernel(const To
         __syncwarp();  // the buffer is free for the copy issued two tiles from now
     }
 
+    grid_launch_dependents();   // the kernel behind this one may be set up now (it waits for this one to complete)
     // ---- what the column kernel that follows needs from this CTA
     if (blockIdx.x == 0 && blockIdx.y == 0)
         for (int i = threadIdx.x; i <= a.n_x; i += blockDim.x) a.tickets[i] = 0;
@@ -423,28 +429,65 @@ __global__ void __launch_bounds__(kTileWarps * 32, 2) logits_mma_kernel(const To
     }
 }
 
-// one warp per row: global max and 1 / sum of exp
-__global__ void row_stats_kernel(const TolArgs a)
+}  // namespace llms
+
+#include "tolerance_tc.cuh"
+
+namespace llms {
+
+// block = 32 neighbouring rows x 32 segment lanes: global max and 1 / sum of exp of every row.  A warp reads 32
+// neighbouring rows of one segment (128 consecutive bytes); four segments per trip are in flight.
+__global__ void __launch_bounds__(1024) row_stats_kernel(const TolArgs a)
 {
-    const int row = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
-    if (row >= a.rows) return;
-    const int lane = threadIdx.x & 31;
-    const float *pm = a.pm + (int64_t)row * a.n_seg;
-    const float *ps = a.ps + (int64_t)row * a.n_seg;
+    __shared__ float red[32][33];
+    grid_dependency_wait();
+    const int row = blockIdx.x * 32 + threadIdx.x;
+    const bool in = row < a.rows;
+    const float *pm = a.pm + row, *ps = a.ps + row;
     float m = -INFINITY;
-    for (int s = lane; s < a.n_seg; s += 32) m = fmaxf(m, pm[s]);
+    if (in) {
+        int s = threadIdx.y;
+        for (; s + 96 < a.n_seg; s += 128) {
+            float v[4];
 #pragma unroll
-    for (int s = 16; s > 0; s >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, s));
-    float sum = 0.0f;
-    for (int s = lane; s < a.n_seg; s += 32) {
-        const float ms = pm[s];
-        if (ms != -INFINITY) sum += ps[s] * expf(ms - m);
+            for (int u = 0; u < 4; ++u) v[u] = pm[(int64_t)(s + 32 * u) * a.rows];
+            m = fmaxf(fmaxf(m, fmaxf(v[0], v[1])), fmaxf(v[2], v[3]));
+        }
+        for (; s < a.n_seg; s += 32) m = fmaxf(m, pm[(int64_t)s * a.rows]);
     }
+    red[threadIdx.y][threadIdx.x] = m;
+    __syncthreads();
 #pragma unroll
-    for (int s = 16; s > 0; s >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, s);
-    if (lane == 0) {
+    for (int y = 0; y < 32; ++y) m = fmaxf(m, red[y][threadIdx.x]);
+    __syncthreads();
+    float sum = 0.0f;
+    if (in) {
+        int s = threadIdx.y;
+        for (; s + 96 < a.n_seg; s += 128) {   // the terms of a lane are added in segment order
+            float v[4], w[4];
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                v[u] = pm[(int64_t)(s + 32 * u) * a.rows];
+                w[u] = ps[(int64_t)(s + 32 * u) * a.rows];
+            }
+#pragma unroll
+            for (int u = 0; u < 4; ++u)
+                if (v[u] != -INFINITY) sum += w[u] * expf(v[u] - m);
+        }
+        for (; s < a.n_seg; s += 32) {
+            const float ms = pm[(int64_t)s * a.rows];
+            if (ms != -INFINITY) sum += ps[(int64_t)s * a.rows] * expf(ms - m);
+        }
+    }
+    red[threadIdx.y][threadIdx.x] = sum;
+    grid_launch_dependents();
+    __syncthreads();
+    if (threadIdx.y == 0 && in) {
+        float total = 0.0f;
+#pragma unroll
+        for (int y = 0; y < 32; ++y) total += red[y][threadIdx.x];
         a.row_max[row] = m;
-        a.row_inv[row] = 1.0f / sum;
+        a.row_inv[row] = 1.0f / total;
     }
 }
 
@@ -464,7 +507,8 @@ __device__ __forceinline__ bool arrives_last(uint32_t *counter, uint32_t expecte
 
 constexpr int kMaxSliceRows = 1024;   // rows of one slice of the column kernel (their normalisers sit in shared memory)
 
-// Column sums, then chunk means, in one launch.  Block (32 segments x 8 row lanes); blockIdx.y picks a slice of rows.
+// Column sums, then chunk means, in one launch.  Block (32 row lanes x 8 segment lanes) over 32 segments; blockIdx.y
+// picks a slice of rows.
 // A block first makes its rows' softmax normalisers (from the per-CTA pairs the MMA kernel left, or copies them
 // where row_stats_kernel made them), then adds up its rows' normalised, 1/n_vis-weighted probabilities per segment.
 // The last slice to finish a group of 32 segments adds the slices in index order; the last group to finish adds
@@ -473,6 +517,7 @@ __global__ void __launch_bounds__(256) column_chunk_kernel(const TolArgs a)
 {
     __shared__ float red[8][33];
     __shared__ float rm_s[kMaxSliceRows], ri_s[kMaxSliceRows];
+    grid_dependency_wait();
     const int tid = threadIdx.y * 32 + threadIdx.x;
     const int seg = blockIdx.x * 32 + threadIdx.x;
     const int rows_per_slice = (a.rows + a.Y - 1) / a.Y;
@@ -495,39 +540,39 @@ __global__ void __launch_bounds__(256) column_chunk_kernel(const TolArgs a)
         }
     }
     __syncthreads();
-    // before the last W columns every row sees every token: the column weight 1/W is applied to the finished sum
-    const bool tail = seg >= a.seg_tail0;
-    const float *wsum = tail ? a.pp : a.ps;
-    float acc = 0.0f;
-    if (seg < a.n_seg) {
-        // four rows per trip, their loads issued together; the terms are still added in row order
-        int row = r_begin + threadIdx.y;
-        for (; row + 24 < r_end; row += 32) {
-            float ms[4], pp[4];
+    // Row lane x takes rows r_begin + x, + 32, ...; segment lane y takes the block's segments y, y + 8, y + 16, y + 24.
+    // Before the last W columns every row sees every token: the column weight 1/W is applied to the finished sum.
+    float acc4[4] = {0.0f, 0.0f, 0.0f, 0.0f};
+    for (int row = r_begin + threadIdx.x; row < r_end; row += 32) {
+        const float rm = rm_s[row - r_begin], ri = ri_s[row - r_begin];
+        float ms[4], ws[4];
 #pragma unroll
-            for (int u = 0; u < 4; ++u) {
-                const int64_t o = (int64_t)(row + 8 * u) * a.n_seg + seg;
+        for (int u = 0; u < 4; ++u) {
+            const int sg = blockIdx.x * 32 + u * 8 + threadIdx.y;
+            if (sg < a.n_seg) {
+                const int64_t o = (int64_t)sg * a.rows + row;
                 ms[u] = a.pm[o];
-                pp[u] = wsum[o];
+                ws[u] = sg >= a.seg_tail0 ? a.pp[o] : a.ps[o];
+            } else {
+                ms[u] = -INFINITY;
+                ws[u] = 0.0f;
             }
-#pragma unroll
-            for (int u = 0; u < 4; ++u)
-                if (ms[u] != -INFINITY) acc += pp[u] * expf(ms[u] - rm_s[row + 8 * u - r_begin]) * ri_s[row + 8 * u - r_begin];
         }
-        for (; row < r_end; row += 8) {
-            const int64_t o = (int64_t)row * a.n_seg + seg;
-            const float ms = a.pm[o];
-            if (ms != -INFINITY) acc += wsum[o] * expf(ms - rm_s[row - r_begin]) * ri_s[row - r_begin];
-        }
-    }
-    red[threadIdx.y][threadIdx.x] = acc;
-    __syncthreads();
-    if (threadIdx.y == 0 && seg < a.n_seg) {
-        float s = 0.0f;
 #pragma unroll
-        for (int y = 0; y < 8; ++y) s += red[y][threadIdx.x];
-        a.part[(int64_t)blockIdx.y * a.n_seg + seg] = tail ? s : s * (1.0f / (float)a.W);
+        for (int u = 0; u < 4; ++u)
+            if (ms[u] != -INFINITY) acc4[u] += ws[u] * expf(ms[u] - rm) * ri;
     }
+    // the 32 row lanes of a segment, added in a fixed tree
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+#pragma unroll
+        for (int d = 16; d > 0; d >>= 1) acc4[u] += __shfl_xor_sync(0xffffffffu, acc4[u], d);
+        const int sg = blockIdx.x * 32 + u * 8 + threadIdx.y;
+        if (threadIdx.x == 0 && sg < a.n_seg)
+            a.part[(int64_t)blockIdx.y * a.n_seg + sg] = sg >= a.seg_tail0 ? acc4[u] : acc4[u] * (1.0f / (float)a.W);
+    }
+    float acc = 0.0f;
+    grid_launch_dependents();
     if (!arrives_last(a.tickets + blockIdx.x, gridDim.y)) return;
 
     // ---- this group's column sums: row lane y adds slices y, y + 8, ... in order, then the eight lanes are added in order
@@ -547,10 +592,13 @@ __global__ void __launch_bounds__(256) column_chunk_kernel(const TolArgs a)
 
     // ---- every chunk's mean over its tokens, layers and heads
     const float norm = (float)a.CL * (float)a.L * (float)a.Hq;
+    const bool gave_up = *reinterpret_cast<volatile uint32_t *>(a.status) == kTcGaveUp;   // the logits kernel did not finish
+    __syncthreads();
+    if (tid == 0 && gave_up) *a.status = 0;
     for (int c = tid; c < a.n_chunks; c += 256) {
         float tot = 0.0f;
         for (int sg = c * a.seg_per_chunk; sg < (c + 1) * a.seg_per_chunk; ++sg) tot += __ldcg(a.colsum + sg);
-        const float score = tot / norm;
+        const float score = gave_up ? __int_as_float(0x7fc00000) : tot / norm;
         a.scores[c] = score;
         if (a.scores_live) a.scores_live[c] = score;
     }
@@ -638,8 +686,98 @@ static TolLayout tol_layout(const llms_kv_desc &d, int W)
     t.off_rpart = t.off_part + round_up((uint64_t)t.Y * t.n_seg * 4, 256);
     t.off_colsum = t.off_rpart + round_up((uint64_t)t.rows * kMaxRowSlots * sizeof(float2), 256);
     t.off_tickets = t.off_colsum + round_up((uint64_t)t.n_seg * 4, 256);
-    t.total = t.off_tickets + round_up((uint64_t)(t.n_x + 1) * 4, 256);
+    t.total = t.off_tickets + round_up((uint64_t)(t.n_x + 2) * 4, 256);   // tickets, then the status word
     return t;
+}
+
+// ---- launching the tcgen05 kernel
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *, const cuuint64_t *,
+                                  const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                  CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+static EncodeTiledFn tensor_map_encoder()
+{
+    static EncodeTiledFn fn = [] {
+        void *p = nullptr;
+        cudaDriverEntryPointQueryResult found;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &found) != cudaSuccess ||
+            found != cudaDriverEntryPointSuccess)
+            p = nullptr;
+        return reinterpret_cast<EncodeTiledFn>(p);
+    }();
+    return fn;
+}
+
+static int tc_rows(const TolArgs &a)
+{
+    int r = 8;
+    while (r < a.NR) r *= 2;
+    return r;
+}
+
+// The tcgen05 kernel takes head_dim 64 or 128, up to 128 rows per KV head and segments of 16 or 32 tokens (chunk_len a
+// multiple of 16).  It is used from 32 rows per KV head on (grouped-query shapes), where it is the faster one.
+static bool tc_path_ok(const TolArgs &a, int SEG)
+{
+    return (a.d == 64 || a.d == 128) && a.NR >= 32 && a.NR <= 128 && SEG >= 16 && tensor_map_encoder() != nullptr;
+}
+
+template <int SEG, int D, int R>
+static int launch_logits_tc_inst(const TolArgs &a, const CUtensorMap &map_k, const CUtensorMap &map_q, cudaStream_t st)
+{
+    const size_t operand = (size_t)(D / 64) * kTcBlockBytes;
+    const int n_stages = (int)std::min<size_t>(8, (227 * 1024 - 2 * operand - sizeof(TcBarriers) - 1024) / operand);
+    const size_t smem = 1024 + (2 + (size_t)n_stages) * operand + sizeof(TcBarriers);
+    const int64_t total = (int64_t)a.L * a.Hkv * ((a.T + kTcTile - 1) / kTcTile);
+    const int grid = (int)std::min<int64_t>(total, sm_count());
+    LLMS_CUDA_TRY(cudaFuncSetAttribute(logits_tc_kernel<SEG, D, R>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    logits_tc_kernel<SEG, D, R><<<grid, kTcThreads, smem, st>>>(a, map_k, map_q, n_stages);
+    return LLMS_OK;
+}
+
+template <int SEG, int D>
+static int launch_logits_tc_rows(const TolArgs &a, int R, const CUtensorMap &map_k, const CUtensorMap &map_q, cudaStream_t st)
+{
+    switch (R) {
+    case 8: return launch_logits_tc_inst<SEG, D, 8>(a, map_k, map_q, st);
+    case 16: return launch_logits_tc_inst<SEG, D, 16>(a, map_k, map_q, st);
+    case 32: return launch_logits_tc_inst<SEG, D, 32>(a, map_k, map_q, st);
+    case 64: return launch_logits_tc_inst<SEG, D, 64>(a, map_k, map_q, st);
+    case 128: return launch_logits_tc_inst<SEG, D, 128>(a, map_k, map_q, st);
+    default: return LLMS_ERR_UNSUPPORTED;
+    }
+}
+
+static int launch_logits_tc(const TolArgs &a, int SEG, cudaStream_t st)
+{
+    EncodeTiledFn encode = tensor_map_encoder();
+    if (!encode) return LLMS_ERR_UNSUPPORTED;
+    const int R = tc_rows(a);
+    // K as a 4-D tensor (channel, token, KV head, layer), tiles of 64 channels x 128 tokens, 128-byte swizzle; tokens past
+    // the end of the context read as zeros
+    CUtensorMap map_k, map_q;
+    {
+        const cuuint64_t dims[4] = {(cuuint64_t)a.d, (cuuint64_t)a.T, (cuuint64_t)a.Hkv, (cuuint64_t)a.L};
+        const cuuint64_t strides[3] = {(cuuint64_t)a.d * 2, (cuuint64_t)a.stride_h * 2, (cuuint64_t)a.stride_l * 2};
+        const cuuint32_t box[4] = {64, (cuuint32_t)kTcTile, 1, 1}, elem[4] = {1, 1, 1, 1};
+        if (encode(&map_k, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 4, const_cast<__half *>(a.kv), dims, strides, box, elem,
+                   CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                   CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+            return LLMS_ERR_UNSUPPORTED;
+    }
+    {   // the query window as a matrix of (layer, head, row) x channel, R rows at a time
+        const cuuint64_t dims[2] = {(cuuint64_t)a.d, (cuuint64_t)a.L * a.Hq * a.W};
+        const cuuint64_t strides[1] = {(cuuint64_t)a.d * 2};
+        const cuuint32_t box[2] = {64, (cuuint32_t)R}, elem[2] = {1, 1};
+        if (encode(&map_q, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 2, const_cast<__half *>(a.q_win), dims, strides, box, elem,
+                   CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+                   CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+            return LLMS_ERR_UNSUPPORTED;
+    }
+    if (SEG == 16) return a.d == 64 ? launch_logits_tc_rows<16, 64>(a, R, map_k, map_q, st) : launch_logits_tc_rows<16, 128>(a, R, map_k, map_q, st);
+    if (SEG == 32) return a.d == 64 ? launch_logits_tc_rows<32, 64>(a, R, map_k, map_q, st) : launch_logits_tc_rows<32, 128>(a, R, map_k, map_q, st);
+    return LLMS_ERR_UNSUPPORTED;
 }
 
 static int check_tol(const llms_kv_desc *desc, int W)
@@ -707,11 +845,19 @@ int llms::chunk_tolerance_impl(const llms_kv_desc *desc, const void *kv, const v
     a.colsum = reinterpret_cast<float *>(ws + t.off_colsum);
     a.tickets = reinterpret_cast<uint32_t *>(ws + t.off_tickets);
     a.n_x = t.n_x;
+    a.status = a.tickets + t.n_x + 1;
     a.scores = scores;
     a.scores_live = scores_live;
     a.Y = t.Y; a.rows = t.rows;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     if ((unsigned)(a.L * a.Hkv) > 65535u || a.Y > 65535) return LLMS_ERR_UNSUPPORTED;
+    if (tc_path_ok(a, t.SEG)) {
+        rc = launch_logits_tc(a, t.SEG, st);
+        if (rc) return rc;
+        a.n_slots = 0;
+        goto tail;
+    }
+    {
     const size_t padded_rows = (size_t)(a.NR + 15) / 16 * 16;                            // whole m-tiles
     const size_t mma_q_bytes = (padded_rows * (a.d * 2 + 16) + 255) / 256 * 256 +
                                (padded_rows * 4 + 255) / 256 * 256 +                     // query rows, each row's last visible
@@ -781,13 +927,13 @@ int llms::chunk_tolerance_impl(const llms_kv_desc *desc, const void *kv, const v
         }
 #undef LLMS_LAUNCH_LOGITS
     }
-    LLMS_CUDA_TRY(cudaGetLastError());
-    if (a.n_slots == 0) {  // the fp32 kernel leaves no per-CTA row sums: a pass over all statistics makes the normalisers
-        row_stats_kernel<<<(a.rows + 7) / 8, 256, 0, st>>>(a);
-        LLMS_CUDA_TRY(cudaGetLastError());
     }
-    column_chunk_kernel<<<dim3(a.n_x, a.Y), dim3(32, 8), 0, st>>>(a);
+tail:
     LLMS_CUDA_TRY(cudaGetLastError());
+    if (a.n_slots == 0) {  // no per-CTA row sums were left: a pass over all statistics makes the normalisers
+        LLMS_CUDA_TRY(launch_dependent(row_stats_kernel, dim3((a.rows + 31) / 32), dim3(32, 32), 0, st, a));
+    }
+    LLMS_CUDA_TRY(launch_dependent(column_chunk_kernel, dim3(a.n_x, a.Y), dim3(32, 8), 0, st, a));
     return LLMS_OK;
 }
 
