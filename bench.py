@@ -64,10 +64,11 @@ def measured_peaks():
 CODEC_SOURCES = ("paper_2403_11805_b200/csrc/codec.cu", "paper_2403_11805_b200/csrc/codec_cw.cuh",
                  "paper_2403_11805_b200/csrc/llms_internal.cuh")
 NCU_DRAM_TRAFFIC = {
-    "codec_sha256_16": "",                      # hash of CODEC_SOURCES at the capture
-    "source": "",                               # what was captured, with which command
-    ("llama7b", 32, "compress_kernel"): None,
-    ("llama7b", 32, "decompress_kernel"): None,
+    "codec_sha256_16": "a98b85a4c628eec6",      # hash of CODEC_SOURCES at the capture
+    "source": "ncu dram__bytes_read.sum + dram__bytes_write.sum of one full-size launch, commit 3ed496a "
+              "(profiles/codec_and_score_kernels_llama7b.md)",
+    ("llama7b", 32, "compress_kernel"): 2148016640 + 647240192,
+    ("llama7b", 32, "decompress_kernel"): 671346432 + 2084710912,
 }
 
 

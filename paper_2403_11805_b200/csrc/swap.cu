@@ -83,7 +83,9 @@ extern "C" int llms_swap_in(const void *pinned_src, uint64_t host_bytes, const u
 extern "C" int llms_wait(void *event, uint32_t timeout_ms)
 {
     if (!event) return LLMS_ERR_INVALID_ARG;
-    const auto deadline = std::chrono::steady_clock::now() + std::chrono::milliseconds(timeout_ms);
+    const auto start = std::chrono::steady_clock::now();
+    const auto deadline = start + std::chrono::milliseconds(timeout_ms);
+    const auto spin_until = start + std::chrono::microseconds(200);   // short waits are polled without giving the core up
     for (;;) {
         const cudaError_t e = cudaEventQuery(static_cast<cudaEvent_t>(event));
         if (e == cudaSuccess) return LLMS_OK;
@@ -91,7 +93,8 @@ extern "C" int llms_wait(void *event, uint32_t timeout_ms)
             set_cuda_error(e, "cudaEventQuery");
             return LLMS_ERR_CUDA;
         }
-        if (std::chrono::steady_clock::now() >= deadline) return LLMS_ERR_TIMEOUT;
-        std::this_thread::sleep_for(std::chrono::microseconds(20));
+        const auto now = std::chrono::steady_clock::now();
+        if (now >= deadline) return LLMS_ERR_TIMEOUT;
+        if (now >= spin_until) std::this_thread::sleep_for(std::chrono::microseconds(20));
     }
 }

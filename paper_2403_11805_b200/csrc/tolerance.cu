@@ -1,13 +1,14 @@
 // Tolerance score (information density, Eq. 1) kernels for sm_100a.
 //
 // From probabilities: a column-mean reduction, one pass over the window.
-// From K and the last W queries: K is streamed once.  The logits S = K q^T are a dense contraction and run as
-// warp-level tensor-core MMAs (logits_mma_kernel; an fp32-FMA kernel with a thread per token remains for head
-// dimensions the MMA kernel does not take).  The rows' softmax statistics are kept per *segment* of SEG
-// neighbouring tokens (SEG = the largest power of two <= 32 that divides chunk_len), as (segment max, sum of exp)
-// and, for the few segments that reach into the last W columns, the 1/n_vis-weighted sum of exp.  Three small kernels then turn the per-segment statistics into row normalisers,
-// column means and chunk means.  All sums run in a fixed order, so the scores - and the ranking made from them -
-// are reproducible bit for bit.
+// From K and the last W queries: K is streamed once.  The logits S = q K^T are a dense contraction and run on the
+// tensor cores: warp-level MMAs (logits_mma_kernel) or, from 32 window rows per KV head on, tcgen05 MMAs fed by TMA
+// (logits_tc_kernel, tolerance_tc.cuh); an fp32-FMA kernel with a thread per token remains for head dimensions
+// neither takes.  The rows' softmax statistics are kept per *segment* of SEG neighbouring tokens (SEG = the largest
+// power of two <= 32 that divides chunk_len), as (segment max, sum of exp) and, for the few segments that reach into
+// the last W columns, the 1/n_vis-weighted sum of exp.  One kernel then turns the per-segment statistics into column
+// sums and chunk means (after a pass for the row normalisers where the logits kernel did not leave them).  All sums
+// run in a fixed order, so the scores - and the ranking made from them - are reproducible bit for bit.
 #include <math.h>
 
 #include <algorithm>
