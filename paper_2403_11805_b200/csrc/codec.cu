@@ -568,54 +568,103 @@ __device__ __forceinline__ void compress_unit(const CodecArgs &a, const UnitPos 
     unit_sum_add(sum_slots, a.n, u.k, &a.entries[u.i].checksum, sum, lane);
 }
 
+// ---------------------------------------------------------------------------------------------- work split
+// Which unit a warp takes next.  With a fixed split (warp w takes units w, w + W, w + 2W, ...) the kernel lasts as
+// long as its slowest warp, and the memory system does not serve all SMs at the same rate: in a plain stream with
+// the decoder's 1:4 read:write mix and a fixed split the CTAs ended between 305 and 454 us around a median of 378
+// (measured), a sixth of the time lost to waiting for the last ones.  Here only a warp's first batch of units is
+// fixed (batch number = warp number); every further batch number is drawn from a counter in the workspace header,
+// one draw ahead of need, so the round trip of the atomic hides behind a batch of work.  One counter would take a
+// draw every few nanoseconds, so the warps are spread over kFeedCounters of them, 128 bytes apart: counter j hands
+// out the batches W + j, W + j + C, W + j + 2C, ...  Consecutive draws get neighbouring units, so at any moment the
+// grid still works on one narrow band of addresses, as with the fixed split.
+constexpr int kFeedCounters = 16;
+constexpr int kFeedStrideWords = 32;
+
+struct UnitFeed {
+    uint32_t *ctr;
+    uint32_t slot, n_slots, n_warps, batch, cur, left, pending, total;
+
+    __device__ __forceinline__ void start(uint32_t *counters, uint32_t total_units, int lane)
+    {
+        const uint32_t gw = blockIdx.x * kWarpsPerBlock + (threadIdx.x >> 5);
+        n_warps = gridDim.x * kWarpsPerBlock;
+        n_slots = min((uint32_t)kFeedCounters, n_warps);  // every counter has warps that draw from it
+        slot = gw % n_slots;
+        ctr = counters + slot * kFeedStrideWords;
+        total = total_units;
+        batch = total_units >= 4 * n_warps ? 2u : 1u;     // little work: single units, so that every warp gets some
+        cur = gw * batch;
+        left = batch;
+        pending = 0;
+        if (cur < total && lane == 0) pending = atomicAdd(ctr, 1u);
+    }
+    // The next unit of this warp; total or more when there is none (and then on every later call too).  Called by
+    // all lanes of the warp together.
+    __device__ __forceinline__ uint32_t pop(int lane)
+    {
+        if (left == 0) {
+            const uint32_t drawn = __shfl_sync(0xffffffffu, pending, 0);
+            cur = (n_warps + drawn * n_slots + slot) * batch;
+            left = batch;
+            if (cur < total && lane == 0) pending = atomicAdd(ctr, 1u);
+        }
+        --left;
+        return cur++;
+    }
+};
+
 // The chunks of one bit-width, start to finish: one phase of the kernel below.
 template <int BITS, int G, bool WIDE, bool PACKED>
-__device__ __forceinline__ void compress_phase(const CodecArgs &a, unsigned char (*patches)[kTransposeBytes], uint32_t *sum_slots)
+__device__ __forceinline__ void compress_phase(const CodecArgs &a, uint32_t *counters, unsigned char (*patches)[kTransposeBytes],
+                                               uint32_t *sum_slots)
 {
     const int lane = threadIdx.x & 31;
-    const uint32_t n_warps = gridDim.x * kWarpsPerBlock;
-    uint32_t unit = blockIdx.x * kWarpsPerBlock + (threadIdx.x >> 5);
+    UnitFeed feed;
+    feed.start(counters, a.total_units, lane);
+    const uint32_t unit = feed.pop(lane);
     cta_sums_clear(sum_slots, a.n);
     if (unit < a.total_units) {
         unsigned char *patch = patches[threadIdx.x >> 5];
-        // A unit is decoded once, two strides ahead of its turn: then its bytes are asked into L2, one trip later
-        // its loads are issued (pn -> pa / pb), another trip later it is computed.
+        // A unit is decoded once, two turns ahead of its own: then its bytes are asked into L2, one trip later its
+        // loads are issued (pn -> pa / pb), another trip later it is computed.
         static_assert(kPrefetchAhead == 2, "the loop below looks exactly two units ahead");
         UnitPos pa, pb, pn;
         uint32_t wa[kPieces][8], wb[kPieces][8];
         decode_unit<PACKED>(a, unit, lane, pa);
         load_unit<WIDE, PACKED>(a, pa, lane, wa);
-        bool has_next = a.total_units - unit > n_warps;
-        if (has_next) decode_unit<PACKED>(a, unit + n_warps, lane, pn);
+        uint32_t ahead = feed.pop(lane);
+        bool has_next = ahead < a.total_units;
+        if (has_next) decode_unit<PACKED>(a, ahead, lane, pn);
         for (;;) {  // two units per trip, so that the data buffers swap roles without register copies
             bool more = has_next;
             if (more) {
                 pb = pn;
                 load_unit<WIDE, PACKED>(a, pb, lane, wb);
             }
-            has_next = a.total_units - unit > 2 * n_warps;
+            ahead = feed.pop(lane);
+            has_next = ahead < a.total_units;
             if (has_next) {
-                decode_unit<PACKED>(a, unit + 2 * n_warps, lane, pn);
+                decode_unit<PACKED>(a, ahead, lane, pn);
                 prefetch_unit_l2<PACKED>(a, pn, lane);
             }
             to_lane_contiguous(wa, patch, lane);
             compress_unit<BITS, G, WIDE>(a, pa, wa, lane, sum_slots);
             if (!more) break;
-            unit += n_warps;
             more = has_next;
             if (more) {
                 pa = pn;
                 load_unit<WIDE, PACKED>(a, pa, lane, wa);
             }
-            has_next = a.total_units - unit > 2 * n_warps;
+            ahead = feed.pop(lane);
+            has_next = ahead < a.total_units;
             if (has_next) {
-                decode_unit<PACKED>(a, unit + 2 * n_warps, lane, pn);
+                decode_unit<PACKED>(a, ahead, lane, pn);
                 prefetch_unit_l2<PACKED>(a, pn, lane);
             }
             to_lane_contiguous(wb, patch, lane);
             compress_unit<BITS, G, WIDE>(a, pb, wb, lane, sum_slots);
             if (!more) break;
-            unit += n_warps;
         }
     }
     __syncthreads();
@@ -629,6 +678,7 @@ struct CodecArgsByWidth {
     CodecArgs w[4];
     // what the CTA that finishes last does with the sums of the whole call
     uint32_t *done;                   // third word of the workspace header: CTAs that have finished (starts at 0)
+    uint32_t *feed;                   // the work-split counters of the header (all zero at the start), one set per width
     const ChunkEntry *entries;        // all n_total entries of the call
     const uint32_t *sums;             // decoder: recomputed sums
     uint32_t *status;                 // decoder: first word of the header, records whose sum is wrong
@@ -636,6 +686,11 @@ struct CodecArgsByWidth {
     int n_total;
     int expect_live;                  // decoder: 1 = the expected sums are read from live_meta now, 0 = from entries
 };
+
+__device__ __forceinline__ uint32_t *feed_counters(uint32_t *feed, int width_index)
+{
+    return feed + width_index * (kFeedCounters * kFeedStrideWords);
+}
 
 // True in every thread of exactly one CTA of the grid: the one that comes here last.  Each thread's earlier atomics
 // on global memory are visible to that CTA's loads that bypass L1 (__ldcg).  Nobody waits for anybody.
@@ -662,10 +717,10 @@ __global__ void __launch_bounds__(kThreads, 2) compress_kernel(const __grid_cons
     __shared__ __align__(16) unsigned char patches[kWarpsPerBlock][kTransposeBytes];
     __shared__ uint32_t sum_slots[kSumSlots];
     grid_dependency_wait();   // the chunk tables may come from a kernel that is still finishing (a no-op otherwise)
-    if (all.w[0].n) compress_phase<8, G, WIDE, PACKED>(all.w[0], patches, sum_slots);
-    if (all.w[1].n) compress_phase<4, G, WIDE, PACKED>(all.w[1], patches, sum_slots);
-    if (all.w[2].n) compress_phase<2, G, WIDE, PACKED>(all.w[2], patches, sum_slots);
-    if (all.w[3].n) compress_phase<1, G, WIDE, PACKED>(all.w[3], patches, sum_slots);
+    if (all.w[0].n) compress_phase<8, G, WIDE, PACKED>(all.w[0], feed_counters(all.feed, 0), patches, sum_slots);
+    if (all.w[1].n) compress_phase<4, G, WIDE, PACKED>(all.w[1], feed_counters(all.feed, 1), patches, sum_slots);
+    if (all.w[2].n) compress_phase<2, G, WIDE, PACKED>(all.w[2], feed_counters(all.feed, 2), patches, sum_slots);
+    if (all.w[3].n) compress_phase<1, G, WIDE, PACKED>(all.w[3], feed_counters(all.feed, 3), patches, sum_slots);
     // The finished checksums go to the caller's page-locked meta array from the CTA that ends last (a kernel of its
     // own for these few stores cost a launch boundary; a device-to-host copy would also queue on the copy engine
     // behind whatever bulk copies other streams have in flight).
@@ -841,52 +896,54 @@ __device__ __forceinline__ void decompress_unit(const CodecArgs &a, const Decode
 }
 
 // Units whose loads are in flight per warp, the one being decoded included, and resident CTAs per SM.  Measured
-// on the 7B shape (decompress stage, ms; depth x CTAs): 2x2 0.516-0.519, 4x1 0.513-0.514, 6x1 0.515, 2x3 0.535,
-// 3x2 0.534-0.537, 4x2 0.539, 2x4 0.539, 3x3 0.549, 2x1 0.583: the store-heavy stream runs best with 8 to 16
-// warps per SM as long as 32 or more units are in flight.
+// on the 7B shape (decompress call, ms; depth x CTAs): 2x2 0.448, 2x3 0.446, 3x2 0.448, 2x4 0.477, 4x1 0.495 (with
+// the fixed work split that preceded the drawn one: 2x2 0.481): the store-heavy stream runs best with 16 to 24 warps
+// per SM.
 constexpr int kDecodeDepth = 2;
 constexpr int kDecodeBlocksPerSm = 2;
 
 // The units of one warp, start to finish.
 template <int BITS, int G, bool WIDE, bool PACKED>
-__device__ __forceinline__ void decompress_warp(const CodecArgs &a, uint32_t unit, uint32_t n_warps, int lane, uint32_t *sum_slots)
+__device__ __forceinline__ void decompress_warp(const CodecArgs &a, UnitFeed &feed, int lane, uint32_t *sum_slots)
 {
     constexpr int D = kDecodeDepth;
+    static_assert(D >= 2, "the ring refills the slot freed one turn ago");
     DecodePos pos[D];
+    uint32_t id[D];
     uint32_t c[D][kPieces][piece_words(BITS)], p[D][kPieces];
 #pragma unroll
     for (int s = 0; s < D - 1; ++s) {
-        const uint32_t ahead = unit + s * n_warps;
-        if (ahead < a.total_units) {
-            decode_unit_for_decoder<BITS, G, PACKED>(a, ahead, lane, pos[s]);
+        id[s] = feed.pop(lane);
+        if (id[s] < a.total_units) {
+            decode_unit_for_decoder<BITS, G, PACKED>(a, id[s], lane, pos[s]);
             load_unit_codes<BITS, G>(pos[s], c[s], p[s]);
         }
     }
+    if (id[0] >= a.total_units) return;
     for (;;) {
 #pragma unroll
         for (int s = 0; s < D; ++s) {
-            // ring slot s holds the current unit; the slot freed last takes the unit D-1 strides ahead
+            // ring slot s holds the current unit; the slot freed last takes the unit D-1 turns ahead
             const int fill = (s + D - 1) % D;
-            const uint32_t ahead = unit + (D - 1) * n_warps;
-            if (ahead < a.total_units) {
-                decode_unit_for_decoder<BITS, G, PACKED>(a, ahead, lane, pos[fill]);
+            id[fill] = feed.pop(lane);
+            if (id[fill] < a.total_units) {
+                decode_unit_for_decoder<BITS, G, PACKED>(a, id[fill], lane, pos[fill]);
                 load_unit_codes<BITS, G>(pos[fill], c[fill], p[fill]);
             }
             decompress_unit<BITS, G, WIDE, PACKED>(a, pos[s], c[s], p[s], lane, sum_slots);
-            unit += n_warps;
-            if (unit >= a.total_units) return;
+            if (id[(s + 1) % D] >= a.total_units) return;
         }
     }
 }
 
 template <int BITS, int G, bool WIDE, bool PACKED>
-__device__ __forceinline__ void decompress_phase(const CodecArgs &a, uint32_t *sum_slots)
+__device__ __forceinline__ void decompress_phase(const CodecArgs &a, uint32_t *counters, uint32_t *sum_slots)
 {
     const int lane = threadIdx.x & 31;
-    const uint32_t n_warps = gridDim.x * kWarpsPerBlock;
-    const uint32_t unit = blockIdx.x * kWarpsPerBlock + (threadIdx.x >> 5);
+    UnitFeed feed;
+    feed.start(counters, a.total_units, lane);
     cta_sums_clear(sum_slots, a.n);
-    if (unit < a.total_units) decompress_warp<BITS, G, WIDE, PACKED>(a, unit, n_warps, lane, sum_slots);
+    decompress_warp<BITS, G, WIDE, PACKED>(a, feed, lane, sum_slots);
     __syncthreads();
     if (a.n <= kSumSlots)
         for (int k = threadIdx.x; k < a.n; k += kThreads)
@@ -898,10 +955,10 @@ template <int G, bool WIDE, bool PACKED>
 __global__ void __launch_bounds__(kThreads, kDecodeBlocksPerSm) decompress_kernel(const __grid_constant__ CodecArgsByWidth all)
 {
     __shared__ uint32_t sum_slots[kSumSlots];
-    if (all.w[0].n) decompress_phase<8, G, WIDE, PACKED>(all.w[0], sum_slots);
-    if (all.w[1].n) decompress_phase<4, G, WIDE, PACKED>(all.w[1], sum_slots);
-    if (all.w[2].n) decompress_phase<2, G, WIDE, PACKED>(all.w[2], sum_slots);
-    if (all.w[3].n) decompress_phase<1, G, WIDE, PACKED>(all.w[3], sum_slots);
+    if (all.w[0].n) decompress_phase<8, G, WIDE, PACKED>(all.w[0], feed_counters(all.feed, 0), sum_slots);
+    if (all.w[1].n) decompress_phase<4, G, WIDE, PACKED>(all.w[1], feed_counters(all.feed, 1), sum_slots);
+    if (all.w[2].n) decompress_phase<2, G, WIDE, PACKED>(all.w[2], feed_counters(all.feed, 2), sum_slots);
+    if (all.w[3].n) decompress_phase<1, G, WIDE, PACKED>(all.w[3], feed_counters(all.feed, 3), sum_slots);
     // the CTA that ends last compares every record's recomputed sum with the expected one
     if (cta_is_last(all.done)) {
         uint32_t bad = 0;
@@ -1183,6 +1240,7 @@ static int launch_compress(const llms_kv_desc &desc, const void *kv, void *out_b
             most_units = std::max(most_units, all.w[k].total_units);
         }
         all.done = static_cast<uint32_t *>(workspace) + 2;
+        all.feed = reinterpret_cast<uint32_t *>(static_cast<uint8_t *>(workspace) + kWsFeedOffset);
         all.entries = a.entries;
         all.n_total = n;
         all.live_meta = static_cast<llms_chunk_meta *>(device_view_of_pinned(meta));
@@ -1357,6 +1415,7 @@ static int decompress_chunks(const llms_kv_desc *desc, const void *buf, uint64_t
             most_units = std::max(most_units, all.w[k].total_units);
         }
         all.done = static_cast<uint32_t *>(workspace) + 2;
+        all.feed = reinterpret_cast<uint32_t *>(static_cast<uint8_t *>(workspace) + kWsFeedOffset);
         all.entries = a.entries;
         all.sums = a.sums;
         all.status = status;

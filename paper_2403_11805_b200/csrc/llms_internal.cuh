@@ -98,9 +98,13 @@ struct UnitEntry {
 static_assert(sizeof(UnitEntry) == 16, "table layout");
 
 // Workspace of the codec calls:
-// [a status word, a spare word and a count of finished CTAs, padded to 16 bytes][n entries][n 16-byte unit-table rows][n entry indices grouped by
-// bit-width][n recomputed sums].  Everything up to the sums is written by one host-to-device copy per call.
-constexpr uint64_t kWsEntriesOffset = 16;
+// [header][n entries][n 16-byte unit-table rows][n entry indices grouped by bit-width][n recomputed sums].  Header: a
+// status word, a spare word and a count of finished CTAs, then, from byte 128 on, the counters from which the codec
+// kernels' warps draw their work (four bit-widths x 16 counters, one per 128 bytes).  The header starts every call
+// as zeros; everything up to the sums is written by one host-to-device copy per call.
+constexpr uint64_t kWsFeedOffset = 128;
+constexpr uint64_t kWsFeedBytes = 4 * 16 * 128;
+constexpr uint64_t kWsEntriesOffset = kWsFeedOffset + kWsFeedBytes;
 constexpr uint64_t kWsBytesPerChunk = sizeof(ChunkEntry) + 16 + 4 + 4;
 __host__ __device__ inline uint64_t ws_table_offset(int n) { return kWsEntriesOffset + (uint64_t)n * sizeof(ChunkEntry); }
 __host__ __device__ inline uint64_t ws_order_offset(int n) { return ws_table_offset(n) + (uint64_t)n * 16; }

@@ -160,7 +160,8 @@ __global__ void __launch_bounds__(kPlanThreads) plan_context_kernel(const PlanAr
     grid_dependency_wait();
     const int n = a.n;
     for (int i = threadIdx.x; i < n; i += kPlanThreads) s_scores[i] = a.scores[i];
-    if (threadIdx.x < 4) reinterpret_cast<uint32_t *>(a.workspace)[threadIdx.x] = 0;   // status word, spare, finished-CTA count
+    // the header: status word, spare, finished-CTA count, work-split counters
+    for (int i = threadIdx.x; i < (int)(kWsEntriesOffset / 4); i += blockDim.x) reinterpret_cast<uint32_t *>(a.workspace)[i] = 0;
     __syncthreads();
     // rank of chunk i = chunks that come before it; `parts` neighbouring lanes share a chunk and split the others
     // among them (a power of two, at most 32, so that they sit in one warp)

@@ -2,6 +2,13 @@
 // consecutive bytes in 256-bit accesses) and a chosen mix of bytes read to bytes written.  It does nothing useful: it
 // measures what the memory system gives such a stream, which is the yardstick the codec kernels' throughput is read
 // against (the encoder reads about four bytes for each one it writes, the decoder the reverse).
+//
+// Work split: one warp per iteration and then the warp is done, eight consecutive iterations per CTA, CTAs handed to
+// the SMs in address order by the hardware as earlier ones leave.  Of the splits tried this one gives the most
+// (7B-sized buffers, GB/s, read:write 4:0 / 0:4 / 4:1 / 1:4 / 2:2): 7450 / 7460 / 7160 / 6570 / 6860, against
+// 6960 / 6250 / 6520 / 6200 / 6460 for resident CTAs whose warps stride through the buffer (the memory system does
+// not serve all SMs at the same rate, and a fixed split waits for the slowest), and 7290 / - / 7090 / 6560 / - for
+// resident CTAs whose warps draw their iterations from counters, which is what the codec kernels do.
 #include <algorithm>
 
 #include "llms_internal.cuh"
@@ -55,7 +62,7 @@ extern "C" int llms_stream_probe(const void *src, uint64_t src_bytes, void *dst,
     if (iters > (1ull << 40) || iters * (uint64_t)read_kib * 1024 > src_bytes || iters * (uint64_t)write_kib * 1024 > dst_bytes)
         return LLMS_ERR_BUF_TOO_SMALL;
     const uint64_t want = (iters + kProbeThreads / 32 - 1) / (kProbeThreads / 32);
-    const int grid = (int)std::min<uint64_t>(want, (uint64_t)sm_count() * 8);
+    const int grid = (int)std::min<uint64_t>(want, 0x7fffffffull);  // in practice one iteration per warp
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     const uint8_t *s = static_cast<const uint8_t *>(src);
     uint8_t *d = static_cast<uint8_t *>(dst);

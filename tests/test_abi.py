@@ -187,7 +187,7 @@ def test_argument_errors_on_the_host():
     bits = np.array([8, 4], dtype=np.uint8)
     call = lambda **kw: lib.llms_compress_chunks(
         ctypes.addressof(kw.get("desc", d)), kw.get("kv", 4096), B._ptr(kw.get("ids", ids)), B._ptr(kw.get("bits", bits)),
-        2, kw.get("out", 8192), kw.get("out_bytes", 1 << 20), B._ptr(meta), kw.get("ws", 4096), kw.get("ws_bytes", 4096), None)
+        2, kw.get("out", 8192), kw.get("out_bytes", 1 << 20), B._ptr(meta), kw.get("ws", 4096), kw.get("ws_bytes", B.codec_workspace_bytes(2)), None)
     assert call() == B.ERR_INVALID_ARG                                   # duplicate chunk id
     ok_ids = np.array([1, 2], dtype=np.uint32)
     assert call(ids=np.array([1, 16], dtype=np.uint32)) == B.ERR_INVALID_ARG   # id out of range
@@ -218,7 +218,7 @@ def test_records_outside_their_buffers_are_refused_on_the_host():
     meta["nbytes"] = [nb8, nb4]
     meta["n_groups"] = sh.n_slabs * sh.chunk_len * (sh.head_dim // sh.group_size)
     for fn in (lib.llms_decompress_chunks,):
-        dec = lambda buf_bytes, m=meta: fn(ctypes.addressof(d), 8192, buf_bytes, B._ptr(m), None, 2, 4096, 4096, 4096, None)
+        dec = lambda buf_bytes, m=meta: fn(ctypes.addressof(d), 8192, buf_bytes, B._ptr(m), None, 2, 4096, 4096, B.codec_workspace_bytes(2), None)
         assert dec(nb8 + nb4 - 1) == B.ERR_BUF_TOO_SMALL
         assert dec(nb8) == B.ERR_BUF_TOO_SMALL
         assert dec(0) == B.ERR_BUF_TOO_SMALL
