@@ -5,10 +5,12 @@
 // tensor cores: warp-level MMAs (logits_mma_kernel) or, from 32 window rows per KV head on, tcgen05 MMAs fed by TMA
 // (logits_tc_kernel, tolerance_tc.cuh); an fp32-FMA kernel with a thread per token remains for head dimensions
 // neither takes.  The rows' softmax statistics are kept per *segment* of SEG neighbouring tokens (SEG = the largest
-// power of two <= 32 that divides chunk_len), as (segment max, sum of exp) and, for the few segments that reach into
-// the last W columns, the 1/n_vis-weighted sum of exp.  One kernel then turns the per-segment statistics into column
-// sums and chunk means (after a pass for the row normalisers where the logits kernel did not leave them).  All sums
-// run in a fixed order, so the scores - and the ranking made from them - are reproducible bit for bit.
+// power of two <= 32 that divides chunk_len) as one number: the base-2 logarithm of the segment's sum of exp(logit),
+// its share of the row's softmax denominator (and, for the few segments that reach into the last W columns, the same
+// of the 1/n_vis-weighted sum).  One kernel then turns the per-segment statistics into column sums and chunk means,
+// once the rows' denominators are known: from partial sums the logits kernels keep while they run, or else from a
+// pass over the statistics.  All sums run in a fixed order, so the scores - and the ranking made from them - are
+// reproducible bit for bit.
 #include <math.h>
 
 #include <algorithm>
@@ -19,6 +21,8 @@ namespace llms {
 
 constexpr int kTokThreads = 256;   // tokens per block in the logits kernel
 constexpr int kRowTile = 8;        // query rows per pass over a key
+
+constexpr int kMaxRowSlots = 32;   // most partial sums a logits kernel leaves per row
 
 struct TolArgs {
     const __half *kv;
@@ -32,14 +36,19 @@ struct TolArgs {
     int n_chunks;
     int64_t stride_l, stride_h;
     float inv_sqrt_d;
-    float *pm, *ps, *pp;      // [n_seg][rows]: segment max, sum of exp, 1/n_vis-weighted sum of exp (pp: only the
-                              // segments from seg_tail0 on are read; before them it is ps / W).  Rows are the fast
-                              // index: the rows of a (layer, KV head) pair that a warp holds for one segment are then
-                              // neighbours in memory (with segments as the fast index every store touched a sector
-                              // per row, as many requests to L2 as the kernel's loads of K)
-    float *row_max, *row_inv; // [rows]: filled by row_stats_kernel where the logits kernel leaves no per-CTA row sums
-    float2 *row_part;         // [rows][n_slots]: (max, sum of exp) of a row over the tiles of one CTA of the MMA kernel
-    int n_slots;              // CTAs per (layer, KV head) pair; 0: the row normalisers are in row_max / row_inv
+    float *pl;                // [n_seg][rows]: log2 of the sum of exp(logit) over the segment's tokens that the row sees
+                              // (-inf where it sees none).  Rows are the fast index: the rows of a (layer, KV head)
+                              // pair that a warp holds for one segment are then neighbours in memory (with segments
+                              // as the fast index every store touched a sector per row, as many requests to L2 as
+                              // the kernel's loads of K)
+    float *pw;                // [n_seg - seg_tail0][rows]: the same of the 1/n_vis-weighted sum, for the segments from
+                              // seg_tail0 on (before them the weighted sum is the plain one over W)
+    float *row_lse;           // [rows]: log2 of a row's softmax denominator, where a kernel of its own makes it
+    float2 *row_part;         // [rows][n_slots]: (max, sum of 2^(l - max)) over the segment values l of a row that one
+                              // slot covers: a CTA of the MMA kernel, or a thread of a CTA of the tcgen05 kernel
+    int n_slots;              // slots per row; 0: the logits kernel keeps no partial sums (row_stats_kernel follows)
+    int lse_ready;            // column kernel: 1 = row_lse holds the denominators, 0 = combine the row's slots
+    int tc_grid, tc_spr;      // tcgen05 kernel: its CTAs, and its statistics threads per row
     float *part;              // [Y][n_seg]
     float *colsum;            // [n_seg]: column sums over all rows
     uint32_t *tickets;        // [n_x + 1]: finished row slices per group of 32 segments, finished groups; the logits
@@ -120,10 +129,11 @@ __global__ void __launch_bounds__(kTokThreads) logits_kernel(const TolArgs a)
                 sp += __shfl_xor_sync(0xffffffffu, sp, s);
             }
             if (valid && (lane & (SEG - 1)) == 0) {
-                const int64_t o = (int64_t)seg * a.rows + row0 + j0 + j;
-                a.pm[o] = m;
-                a.ps[o] = se;
-                a.pp[o] = sp;
+                constexpr float kLog2e = 1.4426950408889634f;
+                const int64_t row = row0 + j0 + j;
+                a.pl[(int64_t)seg * a.rows + row] = se > 0.0f ? fmaf(m, kLog2e, log2f(se)) : -INFINITY;
+                if (seg >= a.seg_tail0)
+                    a.pw[(int64_t)(seg - a.seg_tail0) * a.rows + row] = sp > 0.0f ? fmaf(m, kLog2e, log2f(sp)) : -INFINITY;
             }
         }
     }
@@ -175,6 +185,27 @@ __device__ __forceinline__ float ex2_approx(float x)
     float y;
     asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
     return y;
+}
+
+// log2(x), one instruction (absolute error about 2^-22; 0 gives -inf)
+__device__ __forceinline__ float lg2_approx(float x)
+{
+    float y;
+    asm("lg2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+
+// (M, Z) stands for M + log2(Z), the base-2 logarithm of a sum of powers of two; add 2^l to that sum.  l is finite.
+__device__ __forceinline__ void lse_accumulate(float &M, float &Z, float l)
+{
+    const float d = l - M;                      // +inf the first time (M = -inf, Z = 0)
+    const float e = ex2_approx(-fabsf(d));
+    if (d > 0.0f) {
+        Z = __fmaf_rn(Z, e, 1.0f);
+        M = l;
+    } else {
+        Z += e;
+    }
 }
 
 // x[nt][e] belongs to token nt*8 + 2*q4 + e of the tile (q4 = lane & 3).  Reduce over the tokens of each SEG-token
@@ -256,12 +287,12 @@ __device__ __forceinline__ void row_statistics(const TolArgs &a, const float (&d
             if ((SEG >= 2 && e == 1) || (SEG >= 16 && (nt * 8) % SEG != 0)) continue;  // never a segment's first token
             const int t = t0 + nt * 8 + e;
             if (valid && t % SEG == 0 && t < a.T) {           // the segment's first token writes
+                // -inf (no visible token: max = -inf, sum = 0) stays -inf
                 const int seg = t / SEG;
-                const int64_t o = (int64_t)seg * a.rows + row0 + j;
-                a.pm[o] = mx[nt][e] * a.inv_sqrt_d;
-                a.ps[o] = se[nt][e];
+                a.pl[(int64_t)seg * a.rows + row0 + j] = __fmaf_rn(mx[nt][e], c1, lg2_approx(se[nt][e]));
                 if constexpr (TAIL)
-                    if (seg >= a.seg_tail0) a.pp[o] = sp[nt][e];
+                    if (seg >= a.seg_tail0)
+                        a.pw[(int64_t)(seg - a.seg_tail0) * a.rows + row0 + j] = __fmaf_rn(mx[nt][e], c1, lg2_approx(sp[nt][e]));
             }
         }
     if constexpr (SEG >= 16) {
@@ -425,9 +456,16 @@ __global__ void __launch_bounds__(kTileWarps * 32, 2) logits_mma_kernel(const To
                 const float2 c = run_s[j * cta_warps + k];
                 if (c.x != -INFINITY) s_all += c.y * ex2_approx((c.x - m_all) * c1);
             }
-            a.row_part[(row0 + j) * a.n_slots + blockIdx.x] = make_float2(m_all * a.inv_sqrt_d, s_all);
+            a.row_part[(row0 + j) * a.n_slots + blockIdx.x] = make_float2(m_all * c1, s_all);
         }
     }
+}
+
+// Which CTA of the tcgen05 kernel has tile x of the sequence of all `total` tiles in its run (CTA c has the tiles
+// from total * c / grid up to, not including, total * (c + 1) / grid).
+__host__ __device__ inline int tc_cta_of_tile(int64_t x, int64_t total, int grid)
+{
+    return (int)(((x + 1) * grid - 1) / total);
 }
 
 }  // namespace llms
@@ -436,25 +474,25 @@ __global__ void __launch_bounds__(kTileWarps * 32, 2) logits_mma_kernel(const To
 
 namespace llms {
 
-// block = 32 neighbouring rows x 32 segment lanes: global max and 1 / sum of exp of every row.  A warp reads 32
-// neighbouring rows of one segment (128 consecutive bytes); four segments per trip are in flight.
+// block = 32 neighbouring rows x 32 segment lanes: log2 of every row's softmax denominator from its segment values.
+// A warp reads 32 neighbouring rows of one segment (128 consecutive bytes); four segments per trip are in flight.
 __global__ void __launch_bounds__(1024) row_stats_kernel(const TolArgs a)
 {
     __shared__ float red[32][33];
     grid_dependency_wait();
     const int row = blockIdx.x * 32 + threadIdx.x;
     const bool in = row < a.rows;
-    const float *pm = a.pm + row, *ps = a.ps + row;
+    const float *pl = a.pl + row;
     float m = -INFINITY;
     if (in) {
         int s = threadIdx.y;
         for (; s + 96 < a.n_seg; s += 128) {
             float v[4];
 #pragma unroll
-            for (int u = 0; u < 4; ++u) v[u] = pm[(int64_t)(s + 32 * u) * a.rows];
+            for (int u = 0; u < 4; ++u) v[u] = pl[(int64_t)(s + 32 * u) * a.rows];
             m = fmaxf(fmaxf(m, fmaxf(v[0], v[1])), fmaxf(v[2], v[3]));
         }
-        for (; s < a.n_seg; s += 32) m = fmaxf(m, pm[(int64_t)s * a.rows]);
+        for (; s < a.n_seg; s += 32) m = fmaxf(m, pl[(int64_t)s * a.rows]);
     }
     red[threadIdx.y][threadIdx.x] = m;
     __syncthreads();
@@ -465,20 +503,13 @@ __global__ void __launch_bounds__(1024) row_stats_kernel(const TolArgs a)
     if (in) {
         int s = threadIdx.y;
         for (; s + 96 < a.n_seg; s += 128) {   // the terms of a lane are added in segment order
-            float v[4], w[4];
+            float v[4];
 #pragma unroll
-            for (int u = 0; u < 4; ++u) {
-                v[u] = pm[(int64_t)(s + 32 * u) * a.rows];
-                w[u] = ps[(int64_t)(s + 32 * u) * a.rows];
-            }
+            for (int u = 0; u < 4; ++u) v[u] = pl[(int64_t)(s + 32 * u) * a.rows];
 #pragma unroll
-            for (int u = 0; u < 4; ++u)
-                if (v[u] != -INFINITY) sum += w[u] * expf(v[u] - m);
+            for (int u = 0; u < 4; ++u) sum += exp2f(v[u] - m);   // -inf (a segment the row does not see) adds 0
         }
-        for (; s < a.n_seg; s += 32) {
-            const float ms = pm[(int64_t)s * a.rows];
-            if (ms != -INFINITY) sum += ps[(int64_t)s * a.rows] * expf(ms - m);
-        }
+        for (; s < a.n_seg; s += 32) sum += exp2f(pl[(int64_t)s * a.rows] - m);
     }
     red[threadIdx.y][threadIdx.x] = sum;
     grid_launch_dependents();
@@ -487,9 +518,42 @@ __global__ void __launch_bounds__(1024) row_stats_kernel(const TolArgs a)
         float total = 0.0f;
 #pragma unroll
         for (int y = 0; y < 32; ++y) total += red[y][threadIdx.x];
-        a.row_max[row] = m;
-        a.row_inv[row] = 1.0f / total;
+        a.row_lse[row] = m + log2f(total);
     }
+}
+
+// log2 of a row's softmax denominator from its n <= 32 (max, sum) pairs, by a whole warp: lane k takes pair k, the
+// lanes are combined in a fixed tree.  Every lane returns the result.
+__device__ __forceinline__ float row_lse_from_pair(float2 c)   // c: this lane's pair, (-inf, 0) if it has none
+{
+    float m = c.x;
+#pragma unroll
+    for (int d = 16; d > 0; d >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, d));
+    float sum = c.x != -INFINITY ? c.y * exp2f(c.x - m) : 0.0f;
+#pragma unroll
+    for (int d = 16; d > 0; d >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, d);
+    return m + log2f(sum);
+}
+__device__ __forceinline__ float row_lse_from_slots(const float2 *rp, int n, int lane)
+{
+    return row_lse_from_pair(lane < n ? rp[lane] : make_float2(-INFINITY, 0.0f));
+}
+static_assert(kMaxRowSlots <= 32, "a lane per slot");
+
+// The tcgen05 kernel leaves, per row, one (max, sum) pair for every statistics thread of every CTA that had tiles of
+// the row's (layer, KV head) pair: a warp per row adds them up.
+__global__ void __launch_bounds__(256) row_combine_kernel(const TolArgs a)
+{
+    grid_dependency_wait();
+    grid_launch_dependents();
+    const int row = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5), lane = threadIdx.x & 31;
+    if (row >= a.rows) return;
+    const int tiles_per_pair = (a.T + 127) / 128;
+    const int64_t total = (int64_t)a.L * a.Hkv * tiles_per_pair;
+    const int64_t first = (int64_t)(row / a.NR) * tiles_per_pair;
+    const int n = (tc_cta_of_tile(first + tiles_per_pair - 1, total, a.tc_grid) - tc_cta_of_tile(first, total, a.tc_grid) + 1) * a.tc_spr;
+    const float lse = row_lse_from_slots(a.row_part + (int64_t)row * a.n_slots, n, lane);
+    if (lane == 0) a.row_lse[row] = lse;
 }
 
 // True in every thread of exactly one of the `expected` blocks that pass through with this counter: the one that comes
@@ -510,58 +574,62 @@ constexpr int kMaxSliceRows = 1024;   // rows of one slice of the column kernel 
 
 // Column sums, then chunk means, in one launch.  Block (32 row lanes x 8 segment lanes) over 32 segments; blockIdx.y
 // picks a slice of rows.
-// A block first makes its rows' softmax normalisers (from the per-CTA pairs the MMA kernel left, or copies them
-// where row_stats_kernel made them), then adds up its rows' normalised, 1/n_vis-weighted probabilities per segment.
+// A block first makes its rows' softmax denominators (from the per-CTA pairs the MMA kernel left, or copies them
+// where a kernel of its own made them), then adds up its rows' normalised, 1/n_vis-weighted probabilities per segment.
 // The last slice to finish a group of 32 segments adds the slices in index order; the last group to finish adds
 // every chunk's segments.  All sums run in a fixed order: the scores do not depend on which block came last.
 __global__ void __launch_bounds__(256) column_chunk_kernel(const TolArgs a)
 {
     __shared__ float red[8][33];
-    __shared__ float rm_s[kMaxSliceRows], ri_s[kMaxSliceRows];
+    __shared__ float rl_s[kMaxSliceRows];
     grid_dependency_wait();
     const int tid = threadIdx.y * 32 + threadIdx.x;
     const int seg = blockIdx.x * 32 + threadIdx.x;
     const int rows_per_slice = (a.rows + a.Y - 1) / a.Y;
     const int r_begin = blockIdx.y * rows_per_slice;
     const int r_end = min(a.rows, r_begin + rows_per_slice);
-    for (int r = r_begin + tid; r < r_end; r += 256) {
-        float m = -INFINITY, sum = 0.0f;
-        if (a.n_slots > 0) {
-            const float2 *rp = a.row_part + (int64_t)r * a.n_slots;
-            for (int k = 0; k < a.n_slots; ++k) m = fmaxf(m, rp[k].x);
-            for (int k = 0; k < a.n_slots; ++k) {
-                const float2 c = rp[k];
-                if (c.x != -INFINITY) sum += c.y * expf(c.x - m);
+    if (a.lse_ready) {
+        for (int r = r_begin + tid; r < r_end; r += 256) rl_s[r - r_begin] = a.row_lse[r];
+    } else {   // a warp per row, a lane per pair; eight rows per trip so that their loads are in flight together
+        for (int r0 = r_begin + threadIdx.y; r0 < r_end; r0 += 64) {
+            float2 c[8];
+#pragma unroll
+            for (int v = 0; v < 8; ++v) {
+                const int r = r0 + 8 * v;
+                c[v] = r < r_end && threadIdx.x < a.n_slots ? a.row_part[(int64_t)r * a.n_slots + threadIdx.x] : make_float2(-INFINITY, 0.0f);
             }
-            rm_s[r - r_begin] = m;
-            ri_s[r - r_begin] = 1.0f / sum;
-        } else {
-            rm_s[r - r_begin] = a.row_max[r];
-            ri_s[r - r_begin] = a.row_inv[r];
+#pragma unroll
+            for (int v = 0; v < 8; ++v) {
+                const float lse = row_lse_from_pair(c[v]);
+                if (threadIdx.x == 0 && r0 + 8 * v < r_end) rl_s[r0 + 8 * v - r_begin] = lse;
+            }
         }
     }
     __syncthreads();
     // Row lane x takes rows r_begin + x, + 32, ...; segment lane y takes the block's segments y, y + 8, y + 16, y + 24.
-    // Before the last W columns every row sees every token: the column weight 1/W is applied to the finished sum.
+    // A segment's probability mass in a row is 2^(its value - the row's log2 denominator).  Before the last W columns
+    // every row sees every token: the column weight 1/W is applied to the finished sum.  Four rows per trip: sixteen
+    // loads in flight per thread (with four the kernel waited on one round trip to memory after another).
     float acc4[4] = {0.0f, 0.0f, 0.0f, 0.0f};
-    for (int row = r_begin + threadIdx.x; row < r_end; row += 32) {
-        const float rm = rm_s[row - r_begin], ri = ri_s[row - r_begin];
-        float ms[4], ws[4];
+    for (int row0 = r_begin + threadIdx.x; row0 < r_end; row0 += 128) {
+        float rl[4], ls[4][4];
 #pragma unroll
-        for (int u = 0; u < 4; ++u) {
-            const int sg = blockIdx.x * 32 + u * 8 + threadIdx.y;
-            if (sg < a.n_seg) {
-                const int64_t o = (int64_t)sg * a.rows + row;
-                ms[u] = a.pm[o];
-                ws[u] = sg >= a.seg_tail0 ? a.pp[o] : a.ps[o];
-            } else {
-                ms[u] = -INFINITY;
-                ws[u] = 0.0f;
+        for (int v = 0; v < 4; ++v) {
+            const int row = row0 + 32 * v;
+            const bool in = row < r_end;
+            rl[v] = in ? rl_s[row - r_begin] : 0.0f;
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                const int sg = blockIdx.x * 32 + u * 8 + threadIdx.y;
+                if (!in || sg >= a.n_seg) ls[v][u] = -INFINITY;
+                else if (sg >= a.seg_tail0) ls[v][u] = a.pw[(int64_t)(sg - a.seg_tail0) * a.rows + row];
+                else ls[v][u] = a.pl[(int64_t)sg * a.rows + row];
             }
         }
 #pragma unroll
-        for (int u = 0; u < 4; ++u)
-            if (ms[u] != -INFINITY) acc4[u] += ws[u] * expf(ms[u] - rm) * ri;
+        for (int v = 0; v < 4; ++v)
+#pragma unroll
+            for (int u = 0; u < 4; ++u) acc4[u] += exp2f(ls[v][u] - rl[v]);   // rows in rising order; -inf adds 0
     }
     // the 32 row lanes of a segment, added in a fixed tree
 #pragma unroll
@@ -578,8 +646,15 @@ __global__ void __launch_bounds__(256) column_chunk_kernel(const TolArgs a)
 
     // ---- this group's column sums: row lane y adds slices y, y + 8, ... in order, then the eight lanes are added in order
     acc = 0.0f;
-    if (seg < a.n_seg)
-        for (int y = threadIdx.y; y < a.Y; y += 8) acc += __ldcg(a.part + (int64_t)y * a.n_seg + seg);
+    if (seg < a.n_seg) {
+        for (int y0 = threadIdx.y; y0 < a.Y; y0 += 64) {   // eight loads in flight, added in slice order
+            float v[8];
+#pragma unroll
+            for (int k = 0; k < 8; ++k) v[k] = y0 + 8 * k < a.Y ? __ldcg(a.part + (int64_t)(y0 + 8 * k) * a.n_seg + seg) : 0.0f;
+#pragma unroll
+            for (int k = 0; k < 8; ++k) acc += v[k];
+        }
+    }
     __syncthreads();
     red[threadIdx.y][threadIdx.x] = acc;
     __syncthreads();
@@ -662,11 +737,10 @@ static int row_slices(int rows)
     return std::max(y, (rows + kMaxSliceRows - 1) / kMaxSliceRows);
 }
 
-constexpr int kMaxRowSlots = 32;   // most CTAs of the MMA kernel per (layer, KV head) pair
 
 struct TolLayout {
-    int SEG, n_seg, rows, Y, n_x;
-    uint64_t off_pm, off_ps, off_pp, off_rmax, off_rinv, off_part, off_rpart, off_colsum, off_tickets, total;
+    int SEG, n_seg, seg_tail0, rows, Y, n_x;
+    uint64_t off_pl, off_pw, off_rlse, off_part, off_rpart, off_colsum, off_tickets, total;
 };
 
 static TolLayout tol_layout(const llms_kv_desc &d, int W)
@@ -674,15 +748,13 @@ static TolLayout tol_layout(const llms_kv_desc &d, int W)
     TolLayout t;
     t.SEG = seg_len(d.chunk_len);
     t.n_seg = (d.n_tokens + t.SEG - 1) / t.SEG;
+    t.seg_tail0 = std::min(t.n_seg, (d.n_tokens - W + 1) / t.SEG);
     t.rows = d.n_layers * d.n_q_heads * W;
     t.Y = row_slices(t.rows);
-    const uint64_t stat = round_up((uint64_t)t.rows * t.n_seg * 4, 256);
-    t.off_pm = 0;
-    t.off_ps = stat;
-    t.off_pp = 2 * stat;
-    t.off_rmax = 3 * stat;
-    t.off_rinv = t.off_rmax + round_up((uint64_t)t.rows * 4, 256);
-    t.off_part = t.off_rinv + round_up((uint64_t)t.rows * 4, 256);
+    t.off_pl = 0;
+    t.off_pw = round_up((uint64_t)t.rows * t.n_seg * 4, 256);
+    t.off_rlse = t.off_pw + round_up((uint64_t)t.rows * (t.n_seg - t.seg_tail0) * 4, 256);
+    t.off_part = t.off_rlse + round_up((uint64_t)t.rows * 4, 256);
     t.n_x = (t.n_seg + 31) / 32;
     t.off_rpart = t.off_part + round_up((uint64_t)t.Y * t.n_seg * 4, 256);
     t.off_colsum = t.off_rpart + round_up((uint64_t)t.rows * kMaxRowSlots * sizeof(float2), 256);
@@ -730,10 +802,8 @@ static int launch_logits_tc_inst(const TolArgs &a, const CUtensorMap &map_k, con
     const size_t operand = (size_t)(D / 64) * kTcBlockBytes;
     const int n_stages = (int)std::min<size_t>(8, (227 * 1024 - 2 * operand - sizeof(TcBarriers) - 1024) / operand);
     const size_t smem = 1024 + (2 + (size_t)n_stages) * operand + sizeof(TcBarriers);
-    const int64_t total = (int64_t)a.L * a.Hkv * ((a.T + kTcTile - 1) / kTcTile);
-    const int grid = (int)std::min<int64_t>(total, sm_count());
     LLMS_CUDA_TRY(cudaFuncSetAttribute(logits_tc_kernel<SEG, D, R>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-    logits_tc_kernel<SEG, D, R><<<grid, kTcThreads, smem, st>>>(a, map_k, map_q, n_stages);
+    logits_tc_kernel<SEG, D, R><<<a.tc_grid, kTcThreads, smem, st>>>(a, map_k, map_q, n_stages);
     return LLMS_OK;
 }
 
@@ -830,17 +900,15 @@ int llms::chunk_tolerance_impl(const llms_kv_desc *desc, const void *kv, const v
     a.rep = a.Hq / a.Hkv;
     a.NR = a.rep * W;
     a.n_seg = t.n_seg;
-    a.seg_tail0 = std::min(t.n_seg, (a.T - W + 1) / t.SEG);
+    a.seg_tail0 = t.seg_tail0;
     a.seg_per_chunk = a.CL / t.SEG;
     a.n_chunks = n_chunks(*desc);
     a.stride_l = desc->stride_l; a.stride_h = desc->stride_h;
     a.inv_sqrt_d = (float)(1.0 / sqrt((double)a.d));
     uint8_t *ws = static_cast<uint8_t *>(workspace);
-    a.pm = reinterpret_cast<float *>(ws + t.off_pm);
-    a.ps = reinterpret_cast<float *>(ws + t.off_ps);
-    a.pp = reinterpret_cast<float *>(ws + t.off_pp);
-    a.row_max = reinterpret_cast<float *>(ws + t.off_rmax);
-    a.row_inv = reinterpret_cast<float *>(ws + t.off_rinv);
+    a.pl = reinterpret_cast<float *>(ws + t.off_pl);
+    a.pw = reinterpret_cast<float *>(ws + t.off_pw);
+    a.row_lse = reinterpret_cast<float *>(ws + t.off_rlse);
     a.part = reinterpret_cast<float *>(ws + t.off_part);
     a.row_part = reinterpret_cast<float2 *>(ws + t.off_rpart);
     a.colsum = reinterpret_cast<float *>(ws + t.off_colsum);
@@ -853,9 +921,20 @@ int llms::chunk_tolerance_impl(const llms_kv_desc *desc, const void *kv, const v
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     if ((unsigned)(a.L * a.Hkv) > 65535u || a.Y > 65535) return LLMS_ERR_UNSUPPORTED;
     if (tc_path_ok(a, t.SEG)) {
+        // one CTA per SM, each with an equal run of the sequence of all 128-token tiles.  Every statistics thread
+        // keeps the partial sums of its row while it runs, if a row's slots - threads per row x the most CTAs that
+        // share a (layer, KV head) pair - fit; else a pass over the statistics follows.
+        const int tiles_per_pair = (a.T + kTcTile - 1) / kTcTile;
+        const int64_t total = (int64_t)a.L * a.Hkv * tiles_per_pair;
+        a.tc_grid = (int)std::min<int64_t>(total, sm_count());
+        a.tc_spr = kTcAcc * (kTcTile / tc_rows(a));
+        int most_ctas = 1;
+        for (int64_t pair = 0; pair < (int64_t)a.L * a.Hkv; ++pair)
+            most_ctas = std::max(most_ctas, tc_cta_of_tile((pair + 1) * tiles_per_pair - 1, total, a.tc_grid) -
+                                                tc_cta_of_tile(pair * tiles_per_pair, total, a.tc_grid) + 1);
+        a.n_slots = a.tc_spr * most_ctas <= kMaxRowSlots ? a.tc_spr * most_ctas : 0;
         rc = launch_logits_tc(a, t.SEG, st);
         if (rc) return rc;
-        a.n_slots = 0;
         goto tail;
     }
     {
@@ -931,8 +1010,12 @@ int llms::chunk_tolerance_impl(const llms_kv_desc *desc, const void *kv, const v
     }
 tail:
     LLMS_CUDA_TRY(cudaGetLastError());
-    if (a.n_slots == 0) {  // no per-CTA row sums were left: a pass over all statistics makes the normalisers
+    if (a.n_slots == 0) {  // no partial row sums were left: a pass over all statistics makes the denominators
         LLMS_CUDA_TRY(launch_dependent(row_stats_kernel, dim3((a.rows + 31) / 32), dim3(32, 32), 0, st, a));
+        a.lse_ready = 1;
+    } else if (a.tc_grid > 0) {  // one pair per statistics thread and CTA: added up per row first
+        LLMS_CUDA_TRY(launch_dependent(row_combine_kernel, dim3((a.rows + 7) / 8), dim3(256), 0, st, a));
+        a.lse_ready = 1;
     }
     LLMS_CUDA_TRY(launch_dependent(column_chunk_kernel, dim3(a.n_x, a.Y), dim3(32, 8), 0, st, a));
     return LLMS_OK;

@@ -150,9 +150,11 @@ __device__ __forceinline__ void tc_load(uint32_t taddr, float (&v)[N])
 // like the MMA kernel's (see row_statistics): segment max, sum of exp and, in the last W columns, the weighted sum.
 // N >= SEG: whole segments inside the thread.  N < SEG: the SEG/N threads that hold a segment's pieces are N lanes
 // apart (copies of the row); they combine by shuffles and the one with the first piece stores.
+// run_m, run_z: the thread's running (max, sum) pair over the segment values it has stored for its row (see
+// lse_accumulate).
 template <int SEG, int N, bool TAIL>
 __device__ __forceinline__ void tc_statistics(const TolArgs &a, const float (&dot)[N], int tok0, int last_col, bool valid, int64_t out,
-                                              int lane)
+                                              int lane, float &run_m, float &run_z)
 {
     constexpr float kLog2e = 1.4426950408889634f;
     constexpr int kPiece = SEG < N ? SEG : N;                    // tokens of one segment that this thread holds
@@ -189,11 +191,11 @@ __device__ __forceinline__ void tc_statistics(const TolArgs &a, const float (&do
         const bool first_piece = N >= SEG || (lane & (SEG - N)) == 0;   // lane bits N .. SEG/2 number the pieces
         if (valid && first_piece && (!TAIL || tok0 + s0 < a.T)) {
             const int seg = (tok0 + s0) / SEG;
-            const int64_t o = (int64_t)seg * a.rows + out;
-            a.pm[o] = m * a.inv_sqrt_d;
-            a.ps[o] = sum;
+            const float l = __fmaf_rn(m, c1, lg2_approx(sum));   // -inf where the row sees none of the segment's tokens
+            a.pl[(int64_t)seg * a.rows + out] = l;
             if constexpr (TAIL)
-                if (seg >= a.seg_tail0) a.pp[o] = wsum;
+                if (seg >= a.seg_tail0) a.pw[(int64_t)(seg - a.seg_tail0) * a.rows + out] = __fmaf_rn(m, c1, lg2_approx(wsum));
+            if (!TAIL || l != -INFINITY) lse_accumulate(run_m, run_z, l);
         }
     }
 }
@@ -345,40 +347,58 @@ __global__ void __launch_bounds__(kTcThreads, 1) logits_tc_kernel(const TolArgs 
         const int sub = R < 32 ? lane / kPiece : 0;              // with several copies in a warp: which piece of the 32 columns
         const bool valid = j < a.NR;
         const int row_in_window = j % a.W;
+        // this thread's place among the statistics threads of its row (the slot of its partial sums)
+        const int copy_index = g * (kTcTile / R) + m_index / R;
+        const bool keep = a.n_slots > 0;
         TcCursor at;
         at.start(run_begin + g, tiles_per_pair, a.Hkv);
-        for (int it = g; it < n_items; it += kTcAcc) {
-            const int tile = at.tile;
-            const int64_t row0 = (int64_t)(at.l * a.Hq + at.kvh * a.rep) * a.W;
-            const int64_t out = row0 + j;                        // this thread's row among all rows
-            const int last_col = valid ? a.T - a.W + row_in_window : -1;
+        int it = g;                                              // this thread's next tile, counted from the run's first
+        bool alive = true;
+        // pair by pair: every thread leaves a (max, sum) pair for every (layer, KV head) pair the run touches, also
+        // where none of the pair's tiles fell to its accumulator
+        for (int64_t pair = run_begin / tiles_per_pair; alive && pair * tiles_per_pair < run_end; ++pair) {
+            const int64_t next_pair = (pair + 1) * tiles_per_pair;
+            const int pair_end = (int)((run_end < next_pair ? run_end : next_pair) - run_begin);
+            float run_m = -INFINITY, run_z = 0.0f;
+            for (; it < pair_end; it += kTcAcc) {
+                const int tile = at.tile;
+                const int64_t out = pair * a.NR + j;             // this thread's row among all rows
+                const int last_col = valid ? a.T - a.W + row_in_window : -1;
 #pragma unroll
-            for (int k = 0; k < kTcAcc; ++k) at.next(tiles_per_pair, a.Hkv);   // where the next trip is
-            if (!mbar_wait(&bar->acc_full[g], (it / kTcAcc) & 1, gave_up)) break;
-            tc_fence_after();
-            const bool tail_tile = tile * kTcTile + kTcTile > a.T - a.W + 1;
-            // a load's column address is the same for the whole warp: with R < 32 the warp loads its quarter's 32 columns
-            // and every thread keeps the piece of its copy
-            const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + g * kTcTile + (R < 32 ? quarter * 32 : col0);
+                for (int k = 0; k < kTcAcc; ++k) at.next(tiles_per_pair, a.Hkv);   // where the next trip is
+                if (!mbar_wait(&bar->acc_full[g], (it / kTcAcc) & 1, gave_up)) {
+                    alive = false;
+                    break;
+                }
+                tc_fence_after();
+                const bool tail_tile = tile * kTcTile + kTcTile > a.T - a.W + 1;
+                // a load's column address is the same for the whole warp: with R < 32 the warp loads its quarter's 32
+                // columns and every thread keeps the piece of its copy
+                const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + g * kTcTile + (R < 32 ? quarter * 32 : col0);
 #pragma unroll
-            for (int c = 0; c < (R < 32 ? 1 : R / 32); ++c) {
-                float got[32], dot[kPiece];
-                tc_load<32>(taddr + c * 32, got);
+                for (int c = 0; c < (R < 32 ? 1 : R / 32); ++c) {
+                    float got[32], dot[kPiece];
+                    tc_load<32>(taddr + c * 32, got);
 #pragma unroll
-                for (int i = 0; i < kPiece; ++i) dot[i] = got[i];
+                    for (int i = 0; i < kPiece; ++i) dot[i] = got[i];
 #pragma unroll
-                for (int k = 1; k < 32 / kPiece; ++k)
-                    if (sub == k) {
+                    for (int k = 1; k < 32 / kPiece; ++k)
+                        if (sub == k) {
 #pragma unroll
-                        for (int i = 0; i < kPiece; ++i) dot[i] = got[k * kPiece + i];
-                    }
-                const int tok0 = tile * kTcTile + col0 + c * 32;
-                if (tail_tile) tc_statistics<SEG, kPiece, true>(a, dot, tok0, last_col, valid, out, lane);
-                else tc_statistics<SEG, kPiece, false>(a, dot, tok0, last_col, valid, out, lane);
+                            for (int i = 0; i < kPiece; ++i) dot[i] = got[k * kPiece + i];
+                        }
+                    const int tok0 = tile * kTcTile + col0 + c * 32;
+                    if (tail_tile) tc_statistics<SEG, kPiece, true>(a, dot, tok0, last_col, valid, out, lane, run_m, run_z);
+                    else tc_statistics<SEG, kPiece, false>(a, dot, tok0, last_col, valid, out, lane, run_m, run_z);
+                }
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(&bar->acc_empty[g]);
             }
-            tc_fence_before();
-            __syncwarp();
-            if (lane == 0) mbar_arrive(&bar->acc_empty[g]);
+            if (alive && keep && valid) {
+                const int first_cta = tc_cta_of_tile(pair * tiles_per_pair, total, (int)gridDim.x);
+                a.row_part[(pair * a.NR + j) * a.n_slots + ((int)blockIdx.x - first_cta) * a.tc_spr + copy_index] = make_float2(run_m, run_z);
+            }
         }
     }
 
