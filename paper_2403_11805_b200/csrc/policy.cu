@@ -105,11 +105,12 @@ extern "C" int llms_lctru_order(const llms_chunk_state *table, int n, uint32_t *
 namespace llms {
 
 // Eq. 2 and the chunk tables of the encoder on the device, for a context whose scores have just been computed on the
-// same stream (one CTA; n <= kPlanMaxChunks).  Chunk i's rank is the number of chunks that come before it in the
-// order "denser first, equal densities by index" - exactly the order the host's stable sort produces - so levels and
-// record offsets equal those of llms_assign_levels followed by llms_compress_chunks on the same score bits.
+// same stream (one CTA; n <= kPlanMaxChunks).  The chunks are ranked in the order "denser first, equal densities by
+// index" - exactly the order the host's stable sort produces - so levels and record offsets equal those of
+// llms_assign_levels followed by llms_compress_chunks on the same score bits.
 constexpr int kPlanMaxChunks = 4096;
 constexpr int kPlanThreads = 1024;
+constexpr int kPlanCountChunks = 256;   // up to here ranks are counted, above the keys are sorted
 
 struct PlanArgs {
     const float *scores;       // device, n
@@ -154,31 +155,66 @@ __device__ __forceinline__ T block_inclusive_scan(T v, T *warp_totals)
 
 __global__ void __launch_bounds__(kPlanThreads) plan_context_kernel(const PlanArgs a)
 {
-    __shared__ float s_scores[kPlanMaxChunks];
+    __shared__ unsigned long long s_key[kPlanMaxChunks];       // (descending score, ascending index) as one rising key
     __shared__ uint8_t s_level[kPlanMaxChunks];                // index into levels[]
     __shared__ unsigned long long s_scan[32];
     grid_dependency_wait();
     const int n = a.n;
-    for (int i = threadIdx.x; i < n; i += kPlanThreads) s_scores[i] = a.scores[i];
+    int n2 = 2;                                                // keys are sorted in a power-of-two array
+    while (n2 < n) n2 *= 2;
+    for (int i = threadIdx.x; i < n2; i += kPlanThreads) {
+        // the bits of a float as an unsigned number that rises with the float (for scores, which are not negative,
+        // this only sets the top bit), inverted so that the densest chunk gets the smallest key; padding sorts last
+        unsigned long long key = ~0ull;
+        if (i < n) {
+            uint32_t b = __float_as_uint(a.scores[i]);
+            if (b == 0x80000000u) b = 0;                       // -0 and +0 are one density
+            const uint32_t rising = b ^ ((b >> 31) ? 0xffffffffu : 0x80000000u);
+            key = ((unsigned long long)(~rising) << 32) | (uint32_t)i;
+        }
+        s_key[i] = key;
+    }
     // the header: status word, spare, finished-CTA count, work-split counters
     for (int i = threadIdx.x; i < (int)(kWsEntriesOffset / 4); i += blockDim.x) reinterpret_cast<uint32_t *>(a.workspace)[i] = 0;
     __syncthreads();
-    // rank of chunk i = chunks that come before it; `parts` neighbouring lanes share a chunk and split the others
-    // among them (a power of two, at most 32, so that they sit in one warp)
-    int parts = 1;
-    while (parts < 32 && n * parts * 2 <= kPlanThreads) parts *= 2;
-    for (int base = 0; base < n; base += kPlanThreads / parts) {
-        const int i = base + (int)threadIdx.x / parts, p = threadIdx.x % parts;
+    if (n <= kPlanCountChunks) {
+        // Few chunks: the rank of a chunk is the number of keys below its own, counted by `parts` neighbouring lanes
+        // that split the array among them (a power of two, at most 32, so that they sit in one warp).
+        int parts = 1;
+        while (parts < 32 && n * parts * 2 <= kPlanThreads) parts *= 2;
+        const int i = (int)threadIdx.x / parts, p = threadIdx.x % parts;
         int rank = 0;
         if (i < n) {
-            const float mine = s_scores[i];
-            for (int j = p; j < n; j += parts) {
-                const float other = s_scores[j];
-                rank += (other > mine) || (other == mine && j < i);
-            }
+            const unsigned long long mine = s_key[i];
+            for (int j = p; j < n; j += parts) rank += s_key[j] < mine;
         }
         for (int d = 1; d < parts; d <<= 1) rank += __shfl_xor_sync(0xffffffffu, rank, d);
         if (i < n && p == 0) s_level[i] = rank < a.n_top ? 0 : (rank < a.n_top_mid ? 1 : 2);
+    } else {
+        // Bitonic sort; a thread per comparator, and only the warps that have one take part in the barriers between
+        // the stages.  Position r of the sorted array then names the chunk of rank r.  (Counting takes n / 4 trips
+        // through the array per thread from 1024 chunks on: 6 us of this kernel's 20 at 512 chunks, growing with
+        // the square of n; the sort's 45 stages take 2 us there, but more than counting does up to 256 chunks.)
+        const int comparators = n2 / 2;
+        const int sort_threads = min(kPlanThreads, (comparators + 31) / 32 * 32);
+        if ((int)threadIdx.x < sort_threads) {
+            for (int k = 2; k <= n2; k <<= 1) {
+                for (int j = k >> 1; j > 0; j >>= 1) {
+                    for (int t = threadIdx.x; t < comparators; t += sort_threads) {
+                        const int lo = ((t & ~(j - 1)) << 1) | (t & (j - 1));   // comparator t: the positions lo and lo + j
+                        const int hi = lo | j;
+                        const unsigned long long x = s_key[lo], y = s_key[hi];
+                        if ((x > y) == ((lo & k) == 0)) {
+                            s_key[lo] = y;
+                            s_key[hi] = x;
+                        }
+                    }
+                    asm volatile("bar.sync 1, %0;" :: "r"(sort_threads) : "memory");
+                }
+            }
+            for (int r = threadIdx.x; r < n; r += sort_threads)
+                s_level[(uint32_t)s_key[r]] = r < a.n_top ? 0 : (r < a.n_top_mid ? 1 : 2);
+        }
     }
     __syncthreads();
     // every thread owns a run of consecutive chunks: record bytes and per-width counts before each chunk by two scans

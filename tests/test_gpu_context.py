@@ -108,6 +108,38 @@ def test_compress_context_argument_errors():
     assert (scores_dev.cpu() == -7.0).all() and (scores_host == -7.0).all() and not bits.any() and not meta["nbytes"].any()
 
 
+@pytest.mark.parametrize("n", [4096, 3001, 700, 200, 2])
+def test_device_ranking_with_equal_scores_and_many_chunks(n):
+    """The kernel that ranks the chunks (stream-ordered form) against the oracle's rule on the same scores: up to the
+    most chunks it takes, chunk counts that are no power of two, and contexts whose second half repeats the first,
+    so that whole runs of chunks have bit-equal scores and only their index orders them."""
+    sh = synth.KVShape("many", 1, 1, 1, 64, 4 * n, 4, 64, seed=21)
+    W = min(sh.window, sh.n_tokens)
+    kv = synth.kv_tensor(sh)
+    half = (n // 2) * sh.chunk_len
+    kv[..., half:2 * half, :] = kv[..., :half, :]
+    q = synth.q_window(sh, W)
+    d = B.desc_of(sh)
+    frac_a, levels_a = np.asarray((0.3, 0.4, 0.3), dtype=np.float32), np.asarray((8, 4, 2), dtype=np.uint8)
+    scores_dev = torch.empty(n, dtype=torch.float32, device="cuda")
+    scores_host = torch.empty(n, dtype=torch.float32).pin_memory()
+    bits = B.new_pinned(n)
+    buf = torch.zeros(B.compressed_size(d, np.full(n, 8, np.uint8)), dtype=torch.uint8, device="cuda")
+    meta = B.new_meta(n, pinned=True)
+    ws_t = torch.empty(B.tolerance_workspace_bytes(d, W), dtype=torch.uint8, device="cuda")
+    ws_c = torch.full((B.codec_workspace_bytes(n),), 0x5A, dtype=torch.uint8, device="cuda")
+    B.compress_context(d, kv.cuda(), q.cuda(), W, frac_a, levels_a, scores_dev, scores_host, bits, buf, meta, ws_t, ws_c)
+    torch.cuda.synchronize()
+    s = scores_host.numpy()
+    if n >= 200:
+        assert np.unique(s).size < n - n // 4                 # many chunks share their score with another one
+    obits, _ = oracle.assign_levels(s, (0.3, 0.4, 0.3), (8, 4, 2))
+    assert np.array_equal(bits, obits)
+    want_buf, want_meta = oracle.compress_chunks(odesc(sh), bits_view(kv), np.arange(n), obits)
+    assert_meta_equal(meta, want_meta)
+    assert first_mismatch(buf[:want_buf.size].cpu().numpy(), want_buf) is None
+
+
 def test_full_size_step_as_the_benchmark_runs_it():
     """The 7B-shaped context through llms_compress_context and llms_decompress_chunks_ordered, back to back without a
     synchronisation in between: levels against the oracle's rule on the GPU's scores, sampled records and their decoded
