@@ -64,11 +64,11 @@ def measured_peaks():
 CODEC_SOURCES = ("paper_2403_11805_b200/csrc/codec.cu", "paper_2403_11805_b200/csrc/codec_cw.cuh",
                  "paper_2403_11805_b200/csrc/llms_internal.cuh")
 NCU_DRAM_TRAFFIC = {
-    "codec_sha256_16": "a98b85a4c628eec6",      # hash of CODEC_SOURCES at the capture
-    "source": "ncu dram__bytes_read.sum + dram__bytes_write.sum of one full-size launch, commit 3ed496a "
+    "codec_sha256_16": "d370c1114a0552a6",      # hash of CODEC_SOURCES at the capture
+    "source": "ncu dram__bytes_read.sum + dram__bytes_write.sum of one full-size launch, commit b2f609c "
               "(profiles/codec_and_score_kernels_llama7b.md)",
-    ("llama7b", 32, "compress_kernel"): 2148016640 + 647240192,
-    ("llama7b", 32, "decompress_kernel"): 671346432 + 2084710912,
+    ("llama7b", 32, "compress_kernel"): 2148795648 + 646562816,
+    ("llama7b", 32, "decompress_kernel"): 659686912 + 2085607680,
 }
 
 
@@ -582,15 +582,14 @@ def run_ours(args):
         traffic, traffic_source = measured_traffic((shape.name, shape.n_layers, dominant))
     else:
         traffic, traffic_source = None, "no capture for this workload"
-    # the score stage: K read once, the per-segment softmax statistics written by the logits kernel and read back by
-    # the kernels behind it (twice where a pass over all statistics makes the row normalisers)
+    # the score stage: K read once, one float of softmax statistics per (segment, row) written by the logits kernel
+    # and read back once by the column kernel (a pass over them for the row sums, where one is needed, is not counted)
     rows = shape.n_layers * shape.n_q_heads * W
     seg = 1
     while seg < 32 and shape.chunk_len % (seg * 2) == 0:
         seg *= 2
-    stat_bytes = 2 * rows * ((shape.n_tokens + seg - 1) // seg) * 4
-    row_pass = not (shape.n_q_heads // shape.n_kv_heads * W <= 16 and seg >= 16)
-    score_bytes = kv_bytes // 2 + stat_bytes * (3 if row_pass else 2)
+    stat_bytes = rows * ((shape.n_tokens + seg - 1) // seg) * 4
+    score_bytes = kv_bytes // 2 + 2 * stat_bytes
     roofline = {
         "kernel": dominant, "bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
         "peak_source": f"{peak_kind} copy bandwidth", "launches_per_stage": B.codec_launches(d, bits) - (1 if args.quant_mode == 1 else 0),
