@@ -64,11 +64,11 @@ def measured_peaks():
 CODEC_SOURCES = ("paper_2403_11805_b200/csrc/codec.cu", "paper_2403_11805_b200/csrc/codec_cw.cuh",
                  "paper_2403_11805_b200/csrc/llms_internal.cuh")
 NCU_DRAM_TRAFFIC = {
-    "codec_sha256_16": "d370c1114a0552a6",      # hash of CODEC_SOURCES at the capture
-    "source": "ncu dram__bytes_read.sum + dram__bytes_write.sum of one full-size launch, commit b2f609c "
+    "codec_sha256_16": "08a5ec461fe40403",      # hash of CODEC_SOURCES at the capture
+    "source": "ncu dram__bytes_read.sum + dram__bytes_write.sum of one full-size launch, commit 4714444 "
               "(profiles/codec_and_score_kernels_llama7b.md)",
-    ("llama7b", 32, "compress_kernel"): 2148795648 + 646562816,
-    ("llama7b", 32, "decompress_kernel"): 659686912 + 2085607680,
+    ("llama7b", 32, "compress_kernel"): 2148881664 + 646544896,
+    ("llama7b", 32, "decompress_kernel"): 659666688 + 2085492736,
 }
 
 
@@ -382,14 +382,14 @@ def run_ours(args):
 
     # ---- what a plain stream of the codec's access shape reaches on this GPU, per read:write mix (the encoder reads
     # about four bytes per byte written, the decoder the reverse): context for the roofline fractions
-    def stream_ceiling(read_kib, write_kib, reps=6):
+    def stream_ceiling(read_kib, write_kib, reps=6, split=None):
         per_iter = (read_kib + write_kib) * 1024
         iters = min(kv.numel() * 2 // (max(read_kib, 1) * 1024), kv_out.numel() * 2 // (max(write_kib, 1) * 1024))
         best = None
         for it in range(reps):
             e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
             e0.record(stream)
-            B.stream_probe(kv, kv_out, iters, read_kib, write_kib)
+            B.stream_probe(kv, kv_out, iters, read_kib, write_kib, split=split)
             e1.record(stream)
             torch.cuda.synchronize()
             if it >= 2:
@@ -400,6 +400,12 @@ def run_ours(args):
     mix = {"read_only": stream_ceiling(4, 0), "write_only": stream_ceiling(0, 4), "read4_write1": stream_ceiling(4, 1),
            "read1_write4": stream_ceiling(1, 4), "read1_write1": stream_ceiling(2, 2)}
     mix = {k: -sharding.max_over_ranks([-v], dist, "cuda")[0] for k, v in mix.items()}
+    # the same two mixes under the work splits a persistent kernel can have: resident CTAs with a fixed split (what the
+    # codec kernels had at first) and resident CTAs whose warps draw their iterations from counters (what they have now)
+    by_split = {name: {"resident_ctas_fixed_split": stream_ceiling(r, w, split=1),
+                       "resident_ctas_drawn_split": stream_ceiling(r, w, split=2)}
+                for name, (r, w) in (("read4_write1", (4, 1)), ("read1_write4", (1, 4)))}
+    by_split = {m: {k: -sharding.max_over_ranks([-v], dist, "cuda")[0] for k, v in d.items()} for m, d in by_split.items()}
 
     # ---- end to end: compress -> swap-out -> swap-in -> decompress with the pinned arena in the loop.
     # The chunks go in batches: while batch j travels to the host, batch j-1 is already on its way back and batch
@@ -597,7 +603,7 @@ def run_ours(args):
         "algorithmic_bytes_per_launch": algo_bytes,
         # plain streams with the codec's access shape, GB/s of bytes read + written, best of 4 launches over this
         # workload's buffers; the dominant kernel's own mix beside it
-        "stream_ceilings_gbs": mix,
+        "stream_ceilings_gbs": mix, "stream_by_work_split_gbs": by_split,
         "frac_of_stream_with_its_mix": achieved / mix["read4_write1" if dominant == "compress_kernel" else "read1_write4"],
         "frac_of_nominal_8000": achieved / 8000.0,
         # each codec launch timed alone (events around one call = one codec kernel + its checksum kernel)

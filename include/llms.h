@@ -303,6 +303,15 @@ int llms_wait(void *event, uint32_t timeout_ms);
 int llms_stream_probe(const void *src, uint64_t src_bytes, void *dst, uint64_t dst_bytes, uint64_t iters,
                       int read_kib, int write_kib, void *stream);
 
+/* The same stream with a chosen work split (no counterpart in the paper either): 0 = a warp per iteration, CTAs handed
+ * out in address order as earlier ones leave (what llms_stream_probe runs, the fastest plain stream found); 1 = two
+ * resident CTAs per SM, warp w takes iterations w, w + W, ... (the split the codec kernels had at first); 2 = two
+ * resident CTAs per SM whose warps draw batches of two iterations from 16 counters (the codec kernels' split now; the
+ * counters live in the library, so calls with split 2 on one device must not overlap).  Other values:
+ * LLMS_ERR_INVALID_ARG.  Arguments and errors otherwise as llms_stream_probe. */
+int llms_stream_probe_split(const void *src, uint64_t src_bytes, void *dst, uint64_t dst_bytes, uint64_t iters,
+                            int read_kib, int write_kib, int split, void *stream);
+
 #ifdef __cplusplus
 }
 #endif

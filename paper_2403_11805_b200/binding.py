@@ -74,6 +74,8 @@ _SIGNATURES = {
                                C.c_void_p, C.c_void_p, C.c_void_p]),
     "llms_wait": (C.c_int, [C.c_void_p, C.c_uint32]),
     "llms_stream_probe": (C.c_int, [C.c_void_p, C.c_uint64, C.c_void_p, C.c_uint64, C.c_uint64, C.c_int, C.c_int, C.c_void_p]),
+    "llms_stream_probe_split": (C.c_int, [C.c_void_p, C.c_uint64, C.c_void_p, C.c_uint64, C.c_uint64, C.c_int, C.c_int, C.c_int,
+                                          C.c_void_p]),
 }
 
 
@@ -378,7 +380,13 @@ def wait(event, timeout_ms=10000):
 
 # ----------------------------------------------------------------------------- measurement aid
 
-def stream_probe(src, dst, iters, read_kib, write_kib, stream=None):
-    """llms_stream_probe: a plain stream of the given read:write mix (KiB per warp iteration) over src / dst."""
-    _check(lib().llms_stream_probe(_ptr(src), _nbytes(src), _ptr(dst), _nbytes(dst), int(iters), int(read_kib), int(write_kib),
-                                   _stream(stream)), "llms_stream_probe")
+def stream_probe(src, dst, iters, read_kib, write_kib, stream=None, split=None):
+    """llms_stream_probe: a plain stream of the given read:write mix (KiB per warp iteration) over src / dst.
+    split (llms_stream_probe_split): 0 a warp per iteration, 1 resident CTAs with a fixed split, 2 resident CTAs that
+    draw their iterations from counters."""
+    if split is None:
+        _check(lib().llms_stream_probe(_ptr(src), _nbytes(src), _ptr(dst), _nbytes(dst), int(iters), int(read_kib),
+                                       int(write_kib), _stream(stream)), "llms_stream_probe")
+    else:
+        _check(lib().llms_stream_probe_split(_ptr(src), _nbytes(src), _ptr(dst), _nbytes(dst), int(iters), int(read_kib),
+                                             int(write_kib), int(split), _stream(stream)), "llms_stream_probe_split")

@@ -129,20 +129,29 @@ def test_swap_argument_errors():
 
 
 def test_stream_probe_stays_inside_its_buffers():
-    """The measurement aid: every supported mix runs, writes exactly iters * write_kib KiB and refuses buffers that
-    are too short or mixes it has no kernel for, before anything is launched."""
+    """The measurement aid: every supported mix runs under every work split, writes every one of its iters * write_kib
+    KiB (each iteration stores its own number: a split that skipped an iteration would leave a hole) and nothing
+    behind them, and refuses buffers that are too short or mixes it has no kernel for, before anything is launched."""
     src = torch.arange(1 << 20, dtype=torch.int32, device="cuda")              # 4 MiB
-    for rk, wk in ((4, 0), (0, 4), (4, 1), (1, 4), (2, 2)):
-        iters = 300
-        dst = torch.full((iters * wk * 1024 + 4096,), 0x77, dtype=torch.uint8, device="cuda")
-        B.stream_probe(src, dst, iters, rk, wk)
-        torch.cuda.synchronize()
-        assert bool((dst[iters * wk * 1024:] == 0x77).all())
-        if wk:
-            assert not bool((dst[:iters * wk * 1024] == 0x77).all())
+    for split in (None, 0, 1, 2):
+        for rk, wk in ((4, 0), (0, 4), (4, 1), (1, 4), (2, 2)):
+            iters = 1000 if split in (None, 0) else 20011                      # resident CTAs: several draws per warp
+            if rk * iters * 1024 > src.numel() * 4:
+                iters = src.numel() * 4 // (rk * 1024)
+            dst = torch.full((iters * wk * 1024 + 4096,), 0x77, dtype=torch.uint8, device="cuda")
+            B.stream_probe(src, dst, iters, rk, wk, split=split)
+            torch.cuda.synchronize()
+            assert bool((dst[iters * wk * 1024:] == 0x77).all())
+            if wk:
+                words = dst[:iters * wk * 1024].view(torch.int32).view(iters, wk * 256)
+                want = torch.arange(iters, dtype=torch.int32, device="cuda")[:, None].expand(iters, wk * 256)
+                assert torch.equal(words, want)
     dst = torch.zeros(8192, dtype=torch.uint8, device="cuda")
     for args, status in (((src, dst, 3, 1, 4), B.ERR_BUF_TOO_SMALL), ((src, dst, 2000, 4, 0), B.ERR_BUF_TOO_SMALL),
                          ((src, dst, 2, 3, 1), B.ERR_UNSUPPORTED), ((src, dst, 0, 4, 1), B.ERR_INVALID_ARG)):
         with pytest.raises(B.LlmsError) as e:
             B.stream_probe(*args)
         assert e.value.status == status
+    with pytest.raises(B.LlmsError) as e:
+        B.stream_probe(src, dst, 1, 1, 4, split=3)
+    assert e.value.status == B.ERR_INVALID_ARG
