@@ -51,6 +51,12 @@ SHAPES = [
     ("odd_chunk", synth.KVShape("odd", 1, 1, 3, 16, 77, 7, 16, seed=7), 3),              # SEG 1
     ("one_row", synth.KVShape("w1", 1, 2, 2, 64, 300, 4, 64, seed=8), 1),
     ("window_longer_than_chunk", synth.KVShape("wl", 1, 1, 2, 32, 128, 8, 32, seed=9), 20),
+    # the tcgen05 kernel with its running row sums: at least as many (layer, KV head) pairs as SMs, so that a pair's
+    # tiles fall to one or two CTAs.  Pairs of three tiles (fewer than accumulators: some statistics threads see no tile
+    # of a pair), 40 rows per pair in a 64-row operand (padding rows), 128 rows per pair
+    ("tc_short_pairs", synth.KVShape("tcs", 20, 8, 32, 64, 272, 16, 64, seed=31), 8),
+    ("tc_padded_rows", synth.KVShape("tcp", 20, 8, 40, 128, 400, 32, 128, seed=32), 8),
+    ("tc_128_rows", synth.KVShape("tcr", 16, 10, 160, 64, 300, 16, 64, seed=33), 8),
 ]
 
 
