@@ -71,6 +71,7 @@ struct CodecArgs {
     uint32_t *sums;        // decompress: recomputed checksums
     const uint32_t *order; // entry indices grouped by bit-width; this launch covers order[0 .. n)
     const UnitEntry *table; // the same chunks with what a unit needs to know, one 16-byte load
+    uint32_t *feed;        // channel-wise launches: this launch's work-split counters (zero at the start)
     int n;                 // chunks of this launch (all of one bit-width)
     int n_slabs;           // slabs per chunk
     int slab_elems;        // chunk_len * head_dim
@@ -1038,6 +1039,7 @@ static int fill_args(const llms_kv_desc &d, CodecArgs &a, int n, void *workspace
     a.sums = reinterpret_cast<uint32_t *>(static_cast<uint8_t *>(workspace) + ws_sums_offset(n));
     a.order = reinterpret_cast<const uint32_t *>(static_cast<uint8_t *>(workspace) + ws_order_offset(n));
     a.table = reinterpret_cast<const UnitEntry *>(static_cast<uint8_t *>(workspace) + ws_table_offset(n));
+    a.feed = reinterpret_cast<uint32_t *>(static_cast<uint8_t *>(workspace) + kWsFeedOffset);
     return LLMS_OK;
 }
 
@@ -1092,6 +1094,7 @@ static CodecArgs args_for_group(const CodecArgs &a, const BitGroups &g, int k)
     b.order = a.order + g.first[k];
     b.table = a.table + g.first[k];
     b.n = g.count[k];
+    b.feed = a.feed + k * (kFeedCounters * kFeedStrideWords);
     b.total_units = (uint32_t)b.n * (uint32_t)b.unit_rows * (uint32_t)b.passes;
     b.div_n.set((uint32_t)b.n);
     return b;

@@ -37,9 +37,10 @@ __global__ void __launch_bounds__(kThreads) compress_cw_kernel(const CodecArgs a
 {
     const int lane = threadIdx.x & 31;
     const CwGeo geo(head_dim, lane);
-    const uint32_t n_warps = gridDim.x * kWarpsPerBlock;
     const uint32_t total = (uint32_t)a.n * (uint32_t)a.n_slabs;
-    for (uint32_t item = blockIdx.x * kWarpsPerBlock + (threadIdx.x >> 5); item < total; item += n_warps) {
+    UnitFeed feed;   // slabs are drawn like the units of the other kernels
+    feed.start(a.feed, total, lane);
+    for (uint32_t item = feed.pop(lane); item < total; item = feed.pop(lane)) {
         UnitEntry ent;
         uint32_t s_idx;
         cw_item(a, item, ent, s_idx);
@@ -146,9 +147,10 @@ __global__ void __launch_bounds__(kThreads, 3) compress_cw_reg_kernel(const Code
 {
     const int lane = threadIdx.x & 31;
     const CwGeo geo(head_dim, lane);
-    const uint32_t n_warps = gridDim.x * kWarpsPerBlock;
     const uint32_t total = (uint32_t)a.n * (uint32_t)a.n_slabs;
-    for (uint32_t item = blockIdx.x * kWarpsPerBlock + (threadIdx.x >> 5); item < total; item += n_warps) {
+    UnitFeed feed;   // slabs are drawn like the units of the other kernels
+    feed.start(a.feed, total, lane);
+    for (uint32_t item = feed.pop(lane); item < total; item = feed.pop(lane)) {
         UnitEntry ent;
         uint32_t s_idx;
         cw_item(a, item, ent, s_idx);
@@ -250,6 +252,7 @@ __global__ void __launch_bounds__(kThreads) decompress_cw_kernel(const CodecArgs
     const int lane = threadIdx.x & 31;
     const CwGeo geo(head_dim, lane);
     constexpr float kQmax = (float)((1 << BITS) - 1);
+    // fixed split: with drawn slabs this kernel, which keeps no load ahead of its stores, ran 5% slower (0.580 -> 0.611 ms)
     const uint32_t n_warps = gridDim.x * kWarpsPerBlock;
     const uint32_t total = (uint32_t)a.n * (uint32_t)a.n_slabs;
     for (uint32_t item = blockIdx.x * kWarpsPerBlock + (threadIdx.x >> 5); item < total; item += n_warps) {
@@ -337,6 +340,7 @@ __global__ void __launch_bounds__(kThreads) decompress_cw_reg_kernel(const Codec
 {
     const int lane = threadIdx.x & 31;
     const CwGeo geo(head_dim, lane);
+    // fixed split: with drawn slabs this kernel, which keeps no load ahead of its stores, ran 5% slower (0.580 -> 0.611 ms)
     const uint32_t n_warps = gridDim.x * kWarpsPerBlock;
     const uint32_t total = (uint32_t)a.n * (uint32_t)a.n_slabs;
     for (uint32_t item = blockIdx.x * kWarpsPerBlock + (threadIdx.x >> 5); item < total; item += n_warps) {
