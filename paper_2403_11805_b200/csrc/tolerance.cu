@@ -730,10 +730,12 @@ static int seg_len(int chunk_len)
     return s;
 }
 
-// slices of rows in the column kernel: enough blocks to fill the GPU, and no slice longer than the kernel's arrays
-static int row_slices(int rows)
+// slices of rows in the column kernel: enough blocks to fill the GPU - with many rows about 512 blocks over the n_x
+// groups of 32 segments (measured: 64 slices at 8 groups, 16 at 32 groups; 8 or 128 slices cost 3-10% of the stage) -
+// and no slice longer than the kernel's arrays
+static int row_slices(int rows, int n_x)
 {
-    const int y = rows >= 4096 ? 64 : (rows >= 512 ? 16 : (rows >= 64 ? 4 : 1));
+    const int y = rows >= 4096 ? std::min(64, std::max(16, 512 / std::max(1, n_x))) : (rows >= 512 ? 16 : (rows >= 64 ? 4 : 1));
     return std::max(y, (rows + kMaxSliceRows - 1) / kMaxSliceRows);
 }
 
@@ -750,12 +752,12 @@ static TolLayout tol_layout(const llms_kv_desc &d, int W)
     t.n_seg = (d.n_tokens + t.SEG - 1) / t.SEG;
     t.seg_tail0 = std::min(t.n_seg, (d.n_tokens - W + 1) / t.SEG);
     t.rows = d.n_layers * d.n_q_heads * W;
-    t.Y = row_slices(t.rows);
+    t.n_x = (t.n_seg + 31) / 32;
+    t.Y = row_slices(t.rows, t.n_x);
     t.off_pl = 0;
     t.off_pw = round_up((uint64_t)t.rows * t.n_seg * 4, 256);
     t.off_rlse = t.off_pw + round_up((uint64_t)t.rows * (t.n_seg - t.seg_tail0) * 4, 256);
     t.off_part = t.off_rlse + round_up((uint64_t)t.rows * 4, 256);
-    t.n_x = (t.n_seg + 31) / 32;
     t.off_rpart = t.off_part + round_up((uint64_t)t.Y * t.n_seg * 4, 256);
     t.off_colsum = t.off_rpart + round_up((uint64_t)t.rows * kMaxRowSlots * sizeof(float2), 256);
     t.off_tickets = t.off_colsum + round_up((uint64_t)t.n_seg * 4, 256);
