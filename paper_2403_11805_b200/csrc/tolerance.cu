@@ -443,7 +443,7 @@ __global__ void __launch_bounds__(kTileWarps * 32, 2) logits_mma_kernel(const To
     if (blockIdx.x == 0 && blockIdx.y == 0)
         for (int i = threadIdx.x; i <= a.n_x; i += blockDim.x) a.tickets[i] = 0;
     // Every row's (max, sum of exp) over this CTA's tiles: the warps' running pairs, combined in warp order.  The
-    // column kernel combines a row's n_slots such pairs into the row's softmax normaliser.
+    // column kernel combines a row's n_slots such pairs into the row's softmax denominator.
     __syncthreads();
     if (a.n_slots > 0) {
         constexpr float kLog2e = 1.4426950408889634f;
@@ -570,7 +570,7 @@ __device__ __forceinline__ bool arrives_last(uint32_t *counter, uint32_t expecte
     return last;
 }
 
-constexpr int kMaxSliceRows = 1024;   // rows of one slice of the column kernel (their normalisers sit in shared memory)
+constexpr int kMaxSliceRows = 1024;   // rows of one slice of the column kernel (their denominators sit in shared memory)
 
 // Column sums, then chunk means, in one launch.  Block (32 row lanes x 8 segment lanes) over 32 segments; blockIdx.y
 // picks a slice of rows.
@@ -957,7 +957,7 @@ int llms::chunk_tolerance_impl(const llms_kv_desc *desc, const void *kv, const v
         splits = std::max(1, std::min({splits, (n_tiles + cta_warps - 1) / cta_warps, kMaxRowSlots}));
         // With up to 16 rows per KV head and segments of 16 or 32 tokens every CTA leaves its rows' (max, sum of exp)
         // for the column kernel (7B shape: 2 us more in this kernel, 6 us of row_stats_kernel and a launch less).
-        // Elsewhere the normalisers come from a pass of row_stats_kernel over all statistics: with 32 rows per KV
+        // Elsewhere the denominators come from a pass of row_stats_kernel over all statistics: with 32 rows per KV
         // head the running sums made this kernel 24 us slower (32K grouped-query shape), more than that pass costs.
         a.n_slots = t.SEG >= 16 && a.NR <= 16 ? splits : 0;
         const dim3 grid(splits, pairs);

@@ -21,9 +21,13 @@
 //
 // Measured (B200, whole launches, K bytes / time): 32K-token grouped-query shape (32 rows per KV head) 352.8 us against
 // 356.9 us for the warp-level kernel; 7B shape (8 rows) 177.6 against 165.3 us - so it is used from 32 rows per KV head
-// on.  Taking the MMAs or the statistics out of it showed the feeding side alone at the plain read stream's pace
-// (6.9 TB/s); MMAs and statistics each add their time instead of hiding behind the copies, whatever the number of
-// stages (2 to 5 made no difference), and asking tiles into L2 ahead of the ring made it slower.
+// on.  Taking the MMAs or the statistics out of it showed the feeding side alone at the pace of a resident-CTA read
+// stream (6.9 TB/s); MMAs and statistics each add their time instead of hiding behind the copies, whatever the number
+// of stages (2 to 5 made no difference), and asking tiles into L2 ahead of the ring made it slower.  Cycle counters
+// around the waits (32K shape, per tile of 1332 cycles): the issuing thread is held 890 cycles by a tile's eight MMAs
+// and waits 440, the feeding thread waits 970 for a free stage, a statistics warp works 750 cycles on a tile of its
+// own and waits 4400.  With the query rows in tensor memory instead of shared memory (three accumulators, tcgen05.st)
+// the tile took 1282 cycles and the same time: the kernel runs under the power cap.
 #pragma once
 
 #include <cuda.h>
@@ -147,7 +151,8 @@ __device__ __forceinline__ void tc_load(uint32_t taddr, float (&v)[N])
 }
 
 // Softmax statistics of this thread's window row over its N consecutive tokens (tok0 ..), per SEG-token segment, stored
-// like the MMA kernel's (see row_statistics): segment max, sum of exp and, in the last W columns, the weighted sum.
+// like the MMA kernel's (see row_statistics): log2 of the segment's sum of exp and, in the last W columns, of the
+// weighted sum.
 // N >= SEG: whole segments inside the thread.  N < SEG: the SEG/N threads that hold a segment's pieces are N lanes
 // apart (copies of the row); they combine by shuffles and the one with the first piece stores.
 // run_m, run_z: the thread's running (max, sum) pair over the segment values it has stored for its row (see
