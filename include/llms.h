@@ -291,6 +291,17 @@ int llms_swap_in(const void *pinned_src, uint64_t host_bytes, const uint64_t *ho
 /* Poll a cudaEvent_t until it has completed or timeout_ms has passed (LLMS_ERR_TIMEOUT). */
 int llms_wait(void *event, uint32_t timeout_ms);
 
+/* ------------------------------------------------------------------ checked build */
+
+/* Not a step of the method (the paper has no counterpart).  The library can be built a second time with a bounds check
+ * in front of every access the group-wise codec kernels make to the KV tensor and the swap buffer (a file of its
+ * own, for tests; see the package's build module).  In that build this call waits for the device and reports how many
+ * accesses fell outside the two buffers of their call since the library was loaded (they were skipped) and the address
+ * of the first one; in the ordinary build it sets *compiled_in = 0 and the other two to 0.  The checked build keeps
+ * one pair of ranges per device: its codec calls must not overlap on different streams.  All three pointers are host
+ * pointers and must not be NULL (LLMS_ERR_INVALID_ARG). */
+int llms_debug_bounds(uint32_t *compiled_in, uint32_t *violations, uint64_t *first_address);
+
 /* ------------------------------------------------------------------ measurement aid */
 
 /* Not a step of the method (the paper has no counterpart): a plain streaming kernel with the codec kernels' access

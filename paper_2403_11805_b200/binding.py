@@ -9,7 +9,8 @@ import os
 import numpy as np
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
-LIB_PATH = os.path.join(_HERE, "libllms.so")
+# LLMS_LIBRARY names another build of the library to load instead of the in-tree one (the checked build's test uses it)
+LIB_PATH = os.environ.get("LLMS_LIBRARY") or os.path.join(_HERE, "libllms.so")
 _lib = None
 
 OK = 0
@@ -74,6 +75,7 @@ _SIGNATURES = {
                                C.c_void_p, C.c_void_p, C.c_void_p]),
     "llms_wait": (C.c_int, [C.c_void_p, C.c_uint32]),
     "llms_stream_probe": (C.c_int, [C.c_void_p, C.c_uint64, C.c_void_p, C.c_uint64, C.c_uint64, C.c_int, C.c_int, C.c_void_p]),
+    "llms_debug_bounds": (C.c_int, [C.c_void_p, C.c_void_p, C.c_void_p]),
     "llms_stream_probe_split": (C.c_int, [C.c_void_p, C.c_uint64, C.c_void_p, C.c_uint64, C.c_uint64, C.c_int, C.c_int, C.c_int,
                                           C.c_void_p]),
 }
@@ -376,6 +378,15 @@ def swap_in(pinned_src, meta, dev_buf, host_offsets=None, side_stream=None, afte
 
 def wait(event, timeout_ms=10000):
     _check(lib().llms_wait(_event(event), int(timeout_ms)), "llms_wait")
+
+
+# ----------------------------------------------------------------------------- checked build
+
+def debug_bounds():
+    """llms_debug_bounds: (compiled_in, violations, first_address) of the loaded library."""
+    c, v, a = C.c_uint32(0), C.c_uint32(0), C.c_uint64(0)
+    _check(lib().llms_debug_bounds(C.byref(c), C.byref(v), C.byref(a)), "llms_debug_bounds")
+    return int(c.value), int(v.value), int(a.value)
 
 
 # ----------------------------------------------------------------------------- measurement aid

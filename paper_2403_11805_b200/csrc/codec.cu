@@ -172,10 +172,41 @@ __device__ __forceinline__ float fma_f32_f16(unsigned short x, unsigned short y,
     return d;
 }
 
+// ---------------------------------------------------------------------------------------------- checked build
+// Compiled with LLMS_DEBUG_BOUNDS (python -m paper_2403_11805_b200.build --debug-bounds: a library of its own, never the
+// one the binding loads by default) every access the group-wise kernels make to the KV tensor and to the swap buffer
+// is first compared with the two address ranges the host set for the call; an access outside them is counted, its
+// address kept if it is the first, and skipped (loads give zeros).  Nothing of this exists in the ordinary build.
+#ifdef LLMS_DEBUG_BOUNDS
+struct DebugRanges {
+    unsigned long long lo[2], hi[2];
+};
+__device__ DebugRanges g_debug_ranges;
+__device__ unsigned int g_debug_violations;
+__device__ unsigned long long g_debug_first_address;
+
+__device__ __forceinline__ bool access_ok(const void *p, unsigned int bytes)
+{
+    const unsigned long long a = reinterpret_cast<unsigned long long>(p);
+#pragma unroll
+    for (int r = 0; r < 2; ++r)
+        if (a >= g_debug_ranges.lo[r] && a + bytes <= g_debug_ranges.hi[r]) return true;
+    if (atomicAdd(&g_debug_violations, 1u) == 0) g_debug_first_address = a;
+    return false;
+}
+#else
+__device__ __forceinline__ bool access_ok(const void *, unsigned int) { return true; }
+#endif
+
 // Global accesses of data that is touched once: no L1 allocation.  WIDE: one 256-bit access (32-byte aligned).
 template <bool WIDE>
 __device__ __forceinline__ void load32(const void *p, uint32_t (&w)[8])
 {
+    if (!access_ok(p, 32)) {
+#pragma unroll
+        for (int k = 0; k < 8; ++k) w[k] = 0;
+        return;
+    }
     if constexpr (WIDE) {
         asm volatile("ld.global.nc.L1::no_allocate.v8.b32 {%0,%1,%2,%3,%4,%5,%6,%7}, [%8];"
                      : "=r"(w[0]), "=r"(w[1]), "=r"(w[2]), "=r"(w[3]), "=r"(w[4]), "=r"(w[5]), "=r"(w[6]), "=r"(w[7])
@@ -191,46 +222,82 @@ __device__ __forceinline__ void load32(const void *p, uint32_t (&w)[8])
 __device__ __forceinline__ void st256(void *p, uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t a4,
                                       uint32_t a5, uint32_t a6, uint32_t a7)
 {
+    if (!access_ok(p, 32)) return;
     asm volatile("st.global.L1::no_allocate.v8.b32 [%8], {%0,%1,%2,%3,%4,%5,%6,%7};"
                  :: "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(a4), "r"(a5), "r"(a6), "r"(a7), "l"(p) : "memory");
 }
 __device__ __forceinline__ void st128(void *p, uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3)
 {
+    if (!access_ok(p, 16)) return;
     asm volatile("st.global.L1::no_allocate.v4.b32 [%4], {%0,%1,%2,%3};" :: "r"(a0), "r"(a1), "r"(a2), "r"(a3), "l"(p) : "memory");
 }
 __device__ __forceinline__ void st64(void *p, uint32_t a0, uint32_t a1)
 {
+    if (!access_ok(p, 8)) return;
     asm volatile("st.global.L1::no_allocate.v2.b32 [%2], {%0,%1};" :: "r"(a0), "r"(a1), "l"(p) : "memory");
 }
 __device__ __forceinline__ void st32(void *p, uint32_t a0)
 {
+    if (!access_ok(p, 4)) return;
     asm volatile("st.global.L1::no_allocate.b32 [%1], %0;" :: "r"(a0), "l"(p) : "memory");
 }
 __device__ __forceinline__ void st16(void *p, uint32_t a0)
 {
+    if (!access_ok(p, 2)) return;
     asm volatile("st.global.L1::no_allocate.b16 [%1], %0;" :: "h"((unsigned short)a0), "l"(p) : "memory");
 }
 __device__ __forceinline__ void ld16(const void *p, uint32_t *w)
 {
+    if (!access_ok(p, 2)) {
+        w[0] = 0;
+        return;
+    }
     unsigned short v;
     asm volatile("ld.global.nc.L1::no_allocate.b16 %0, [%1];" : "=h"(v) : "l"(p));
     w[0] = v;
 }
 __device__ __forceinline__ void ld256(const void *p, uint32_t *w)
 {
+    if (!access_ok(p, 32)) {
+        w[0] = 0;
+        w[1] = 0;
+        w[2] = 0;
+        w[3] = 0;
+        w[4] = 0;
+        w[5] = 0;
+        w[6] = 0;
+        w[7] = 0;
+        return;
+    }
     asm volatile("ld.global.nc.L1::no_allocate.v8.b32 {%0,%1,%2,%3,%4,%5,%6,%7}, [%8];"
                  : "=r"(w[0]), "=r"(w[1]), "=r"(w[2]), "=r"(w[3]), "=r"(w[4]), "=r"(w[5]), "=r"(w[6]), "=r"(w[7]) : "l"(p));
 }
 __device__ __forceinline__ void ld128(const void *p, uint32_t *w)
 {
+    if (!access_ok(p, 16)) {
+        w[0] = 0;
+        w[1] = 0;
+        w[2] = 0;
+        w[3] = 0;
+        return;
+    }
     asm volatile("ld.global.nc.L1::no_allocate.v4.b32 {%0,%1,%2,%3}, [%4];" : "=r"(w[0]), "=r"(w[1]), "=r"(w[2]), "=r"(w[3]) : "l"(p));
 }
 __device__ __forceinline__ void ld64(const void *p, uint32_t *w)
 {
+    if (!access_ok(p, 8)) {
+        w[0] = 0;
+        w[1] = 0;
+        return;
+    }
     asm volatile("ld.global.nc.L1::no_allocate.v2.b32 {%0,%1}, [%2];" : "=r"(w[0]), "=r"(w[1]) : "l"(p));
 }
 __device__ __forceinline__ void ld32(const void *p, uint32_t *w)
 {
+    if (!access_ok(p, 4)) {
+        w[0] = 0;
+        return;
+    }
     asm volatile("ld.global.nc.L1::no_allocate.b32 %0, [%1];" : "=r"(w[0]) : "l"(p));
 }
 
@@ -496,10 +563,12 @@ __device__ __forceinline__ uint32_t compress_unit_bits(const CodecArgs &a, const
 // Zero the two padding runs of a record (after the parameter block, after the code stream).
 __device__ __forceinline__ void zero_padding(const CodecArgs &a, uint8_t *rec, uint32_t bits, int lane)
 {
-    for (uint32_t k = a.params_bytes + lane; k < a.codes_off; k += 32) rec[k] = 0;
+    for (uint32_t k = a.params_bytes + lane; k < a.codes_off; k += 32)
+        if (access_ok(rec + k, 1)) rec[k] = 0;
     const uint64_t codes_end = a.codes_off + (uint64_t)a.n_slabs * a.slab_elems * bits / 8;
     const uint64_t nbytes = (codes_end + 255) / 256 * 256;
-    for (uint64_t k = codes_end + lane; k < nbytes; k += 32) rec[k] = 0;
+    for (uint64_t k = codes_end + lane; k < nbytes; k += 32)
+        if (access_ok(rec + k, 1)) rec[k] = 0;
 }
 
 // The unit is fetched so that every load instruction of the warp reads 1 KiB of consecutive bytes (piece j of
@@ -787,7 +856,7 @@ __device__ __forceinline__ void load_unit_codes(const DecodePos &u, uint32_t (&c
             else if constexpr (BITS == 4) ld64(src, c[j]);
             else if constexpr (BITS == 2) ld32(src, c[j]);
             else ld16(src, c[j]);
-            p[j] = __ldg(u.params + j * (kPieceStride / G));
+            p[j] = access_ok(u.params + j * (kPieceStride / G), 4) ? __ldg(u.params + j * (kPieceStride / G)) : 0u;
         } else {
 #pragma unroll
             for (int k = 0; k < piece_words(BITS); ++k) c[j][k] = 0;
@@ -1203,13 +1272,40 @@ static int check_common(const llms_kv_desc *desc, int n, const void *workspace, 
     return LLMS_OK;
 }
 
+#ifdef LLMS_DEBUG_BOUNDS
+// For the test of the check itself: the swap buffer's range is declared this much shorter than it is, so that accesses to
+// its (perfectly valid) last bytes are counted and skipped.
+static uint64_t g_debug_shrink_bytes = 0;
+extern "C" void llms_debug_shrink_swap_range(uint64_t bytes) { g_debug_shrink_bytes = bytes; }
+#endif
+
+// The checked build's two address ranges for the kernels of a call: the KV tensor as the strides span it, and the swap
+// buffer.  The ordinary build does nothing here.
+static int set_debug_ranges(const llms_kv_desc &d, const void *kv, const void *buf, uint64_t buf_bytes, cudaStream_t st)
+{
+#ifdef LLMS_DEBUG_BOUNDS
+    const uint64_t span = (uint64_t)(d.n_layers - 1) * d.stride_l + (uint64_t)d.stride_s + (uint64_t)(d.n_kv_heads - 1) * d.stride_h +
+                          (uint64_t)d.n_tokens * d.head_dim;   // elements up to the end of the last slab
+    DebugRanges r;
+    r.lo[0] = reinterpret_cast<unsigned long long>(kv);
+    r.hi[0] = r.lo[0] + span * 2;
+    r.lo[1] = reinterpret_cast<unsigned long long>(buf);
+    r.hi[1] = r.lo[1] + buf_bytes - std::min<uint64_t>(buf_bytes, g_debug_shrink_bytes);
+    LLMS_CUDA_TRY(cudaMemcpyToSymbolAsync(g_debug_ranges, &r, sizeof(r), 0, cudaMemcpyHostToDevice, st));
+#else
+    (void)d; (void)kv; (void)buf; (void)buf_bytes; (void)st;
+#endif
+    return LLMS_OK;
+}
+
 // Launch the encoder over the chunk tables that sit in the workspace (entries, unit table, order grouped by bit-width;
 // first[k] / count[k]: where the chunks of width 8, 4, 2, 1 start in the grouped order and how many there are), and see
 // to it that the checksums reach `meta` (host) in stream order.
-static int launch_compress(const llms_kv_desc &desc, const void *kv, void *out_buf, void *workspace, int n,
+static int launch_compress(const llms_kv_desc &desc, const void *kv, void *out_buf, uint64_t out_bytes, void *workspace, int n,
                            const int (&first)[kNumWidths], const int (&count)[kNumWidths], llms_chunk_meta *meta, cudaStream_t st,
                            bool after_kernel = false)
 {
+    if (int rc = set_debug_ranges(desc, kv, out_buf, out_bytes, st)) return rc;
     CodecArgs a{};
     const bool wide = wide_ok(desc, kv);
     fill_args(desc, a, n, workspace, wide);
@@ -1324,12 +1420,12 @@ extern "C" int llms_compress_chunks(const llms_kv_desc *desc, const void *kv, co
     const BitGroups groups = group_by_bits(n, staged.data(), [&](int i) { return (uint32_t)bits[i]; });
     rc = upload_tables(workspace, staged.data(), groups, n, false, st);
     if (rc) return rc;
-    return launch_compress(*desc, kv, out_buf, workspace, n, groups.first, groups.count, meta, st);
+    return launch_compress(*desc, kv, out_buf, out_bytes, workspace, n, groups.first, groups.count, meta, st);
 }
 
 // The encoder over chunk tables that a kernel has already put into the workspace (llms_compress_context's stream-ordered
 // path): chunks 0 .. n-1 in index order, count[k] of them at width 8, 4, 2, 1.
-int llms::compress_planned(const llms_kv_desc *desc, const void *kv, int n, const int count[4], void *out_buf,
+int llms::compress_planned(const llms_kv_desc *desc, const void *kv, int n, const int count[4], void *out_buf, uint64_t out_bytes,
                            llms_chunk_meta *meta, void *workspace, void *stream)
 {
     int first[kNumWidths], cnt[kNumWidths], at = 0;
@@ -1339,7 +1435,7 @@ int llms::compress_planned(const llms_kv_desc *desc, const void *kv, int n, cons
         at += count[k];
     }
     if (at != n) return LLMS_ERR_INVALID_ARG;
-    return launch_compress(*desc, kv, out_buf, workspace, n, first, cnt, meta, static_cast<cudaStream_t>(stream), true);
+    return launch_compress(*desc, kv, out_buf, out_bytes, workspace, n, first, cnt, meta, static_cast<cudaStream_t>(stream), true);
 }
 
 int llms::check_compress_args(const llms_kv_desc *desc, int n, const void *kv, const void *out_buf, const void *workspace,
@@ -1388,6 +1484,8 @@ static int decompress_chunks(const llms_kv_desc *desc, const void *buf, uint64_t
         seen[dst] = 1;
         staged[i].chunk_id = dst;
     }
+    rc = set_debug_ranges(*desc, kv_out, buf, buf_bytes, static_cast<cudaStream_t>(stream));
+    if (rc) return rc;
     CodecArgs a{};
     const bool wide = wide_ok(*desc, kv_out);
     fill_args(*desc, a, n, workspace, wide);
@@ -1465,6 +1563,25 @@ extern "C" int llms_codec_corrupt_count(const void *workspace, uint32_t *n_corru
     LLMS_CUDA_TRY(cudaStreamSynchronize(st));
     if (n_corrupt) *n_corrupt = status;
     return status ? LLMS_ERR_CORRUPT : LLMS_OK;
+}
+
+extern "C" int llms_debug_bounds(uint32_t *compiled_in, uint32_t *violations, uint64_t *first_address)
+{
+    if (!compiled_in || !violations || !first_address) return LLMS_ERR_INVALID_ARG;
+    *compiled_in = 0;
+    *violations = 0;
+    *first_address = 0;
+#ifdef LLMS_DEBUG_BOUNDS
+    unsigned int count = 0;
+    unsigned long long first = 0;
+    LLMS_CUDA_TRY(cudaDeviceSynchronize());
+    LLMS_CUDA_TRY(cudaMemcpyFromSymbol(&count, g_debug_violations, sizeof(count)));
+    LLMS_CUDA_TRY(cudaMemcpyFromSymbol(&first, g_debug_first_address, sizeof(first)));
+    *compiled_in = 1;
+    *violations = count;
+    *first_address = first;
+#endif
+    return LLMS_OK;
 }
 
 // ---------------------------------------------------------------------------------------------- no-allocation variant

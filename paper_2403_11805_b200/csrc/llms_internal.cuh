@@ -76,7 +76,7 @@ int chunk_tolerance_impl(const llms_kv_desc *desc, const void *kv, const void *q
 
 // The encoder over chunk tables already present in the workspace (see codec.cu), and the argument checks of the
 // compress call that do not depend on the chunk list.
-int compress_planned(const llms_kv_desc *desc, const void *kv, int n, const int count[4], void *out_buf,
+int compress_planned(const llms_kv_desc *desc, const void *kv, int n, const int count[4], void *out_buf, uint64_t out_bytes,
                      llms_chunk_meta *meta, void *workspace, void *stream);
 int check_compress_args(const llms_kv_desc *desc, int n, const void *kv, const void *out_buf, const void *workspace,
                         uint64_t workspace_bytes);

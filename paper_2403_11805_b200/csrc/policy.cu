@@ -352,7 +352,7 @@ extern "C" int llms_compress_context(const llms_kv_desc *desc, const void *kv, c
         p.bits_out = bits_live;
         LLMS_CUDA_TRY(launch_dependent(plan_context_kernel, dim3(1), dim3(kPlanThreads), 0, st, p));
         if (after_scores) LLMS_CUDA_TRY(cudaEventRecord(static_cast<cudaEvent_t>(after_scores), st));
-        return compress_planned(desc, kv, n, count, out_buf, meta, codec_workspace, stream);
+        return compress_planned(desc, kv, n, count, out_buf, out_bytes, meta, codec_workspace, stream);
     }
 
     // ---- the ranking as a host step: one synchronisation, when the scores have reached the host
