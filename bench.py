@@ -64,11 +64,11 @@ def measured_peaks():
 CODEC_SOURCES = ("paper_2403_11805_b200/csrc/codec.cu", "paper_2403_11805_b200/csrc/codec_cw.cuh",
                  "paper_2403_11805_b200/csrc/llms_internal.cuh")
 NCU_DRAM_TRAFFIC = {
-    "codec_sha256_16": "b1334cf685818d9e",      # hash of CODEC_SOURCES at the capture
-    "source": "ncu dram__bytes_read.sum + dram__bytes_write.sum of one full-size launch, commit bea5d12 "
+    "codec_sha256_16": "01417c4ecd867fea",      # hash of CODEC_SOURCES at the capture
+    "source": "ncu dram__bytes_read.sum + dram__bytes_write.sum of one full-size launch, commit 97f4083 "
               "(profiles/codec_and_score_kernels_llama7b.md)",
-    ("llama7b", 32, "compress_kernel"): 2148803328 + 646520832,
-    ("llama7b", 32, "decompress_kernel"): 659694336 + 2088079104,
+    ("llama7b", 32, "compress_kernel"): 2149007616 + 646748160,
+    ("llama7b", 32, "decompress_kernel"): 659704064 + 2085752576,
 }
 
 
