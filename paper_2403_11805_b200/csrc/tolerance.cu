@@ -950,10 +950,15 @@ int llms::chunk_tolerance_impl(const llms_kv_desc *desc, const void *kv, const v
     const int cta_warps = 2 * (mma_q_bytes + kTileWarps * tile_bytes + 1024) <= 227 * 1024 ? kTileWarps : kTileWarpsSmall;
     const size_t mma_smem = mma_q_bytes + (size_t)cta_warps * tile_bytes;
     if ((a.d == 64 || a.d == 128 || a.d == 256) && mma_smem <= 200 * 1024) {
-        // enough blocks per (layer, KV head) to fill the GPU a few times over
+        // enough blocks per (layer, KV head) to fill the GPU a few times over - many times over where a block then still
+        // has two tiles per warp: the blocks are handed out as earlier ones leave, and the shorter they are the less the
+        // last ones leave idle (7B shape, 1024 pairs of 128 tiles: 1 / 2 / 3 / 4 / 6 blocks per pair 193.6 / 193.4 /
+        // 191.5 / 191.5 / 195.6 us for the stage; 1024 pairs of 32 tiles: 1 / 3 blocks 72.7 / 75.2 us)
         const int n_tiles = (a.T + kTileTokens - 1) / kTileTokens;
         const int pairs = a.L * a.Hkv;
         int splits = (sm_count() * 6 + pairs - 1) / pairs;
+        const int more = (sm_count() * 18 + pairs - 1) / pairs;
+        if (n_tiles / more >= 2 * cta_warps) splits = more;
         splits = std::max(1, std::min({splits, (n_tiles + cta_warps - 1) / cta_warps, kMaxRowSlots}));
         // With up to 16 rows per KV head and segments of 16 or 32 tokens every CTA leaves its rows' (max, sum of exp)
         // for the column kernel (7B shape: 2 us more in this kernel, 6 us of row_stats_kernel and a launch less).
