@@ -548,7 +548,7 @@ __global__ void __launch_bounds__(256) row_combine_kernel(const TolArgs a)
     grid_launch_dependents();
     const int row = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5), lane = threadIdx.x & 31;
     if (row >= a.rows) return;
-    const int tiles_per_pair = (a.T + 127) / 128;
+    const int tiles_per_pair = ((a.T + 127) / 128 + 1) / 2;      // the tcgen05 kernel's double tiles
     const int64_t total = (int64_t)a.L * a.Hkv * tiles_per_pair;
     const int64_t first = (int64_t)(row / a.NR) * tiles_per_pair;
     const int n = (tc_cta_of_tile(first + tiles_per_pair - 1, total, a.tc_grid) - tc_cta_of_tile(first, total, a.tc_grid) + 1) * a.tc_spr;
@@ -801,9 +801,9 @@ static bool tc_path_ok(const TolArgs &a, int SEG)
 template <int SEG, int D, int R>
 static int launch_logits_tc_inst(const TolArgs &a, const CUtensorMap &map_k, const CUtensorMap &map_q, cudaStream_t st)
 {
-    const size_t operand = (size_t)(D / 64) * kTcBlockBytes;
-    const int n_stages = (int)std::min<size_t>(8, (227 * 1024 - 2 * operand - sizeof(TcBarriers) - 1024) / operand);
-    const size_t smem = 1024 + (2 + (size_t)n_stages) * operand + sizeof(TcBarriers);
+    const size_t operand = (size_t)(D / 64) * kTcBlockBytes, stage = (size_t)(D / 64) * kTcWideBlockBytes;
+    const int n_stages = (int)std::min<size_t>(8, (227 * 1024 - 2 * operand - sizeof(TcBarriers) - 1024) / stage);
+    const size_t smem = 1024 + 2 * operand + (size_t)n_stages * stage + sizeof(TcBarriers);
     LLMS_CUDA_TRY(cudaFuncSetAttribute(logits_tc_kernel<SEG, D, R>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
     logits_tc_kernel<SEG, D, R><<<a.tc_grid, kTcThreads, smem, st>>>(a, map_k, map_q, n_stages);
     return LLMS_OK;
@@ -833,7 +833,7 @@ static int launch_logits_tc(const TolArgs &a, int SEG, cudaStream_t st)
     {
         const cuuint64_t dims[4] = {(cuuint64_t)a.d, (cuuint64_t)a.T, (cuuint64_t)a.Hkv, (cuuint64_t)a.L};
         const cuuint64_t strides[3] = {(cuuint64_t)a.d * 2, (cuuint64_t)a.stride_h * 2, (cuuint64_t)a.stride_l * 2};
-        const cuuint32_t box[4] = {64, (cuuint32_t)kTcTile, 1, 1}, elem[4] = {1, 1, 1, 1};
+        const cuuint32_t box[4] = {64, (cuuint32_t)kTcWide, 1, 1}, elem[4] = {1, 1, 1, 1};
         if (encode(&map_k, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 4, const_cast<__half *>(a.kv), dims, strides, box, elem,
                    CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                    CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
@@ -926,7 +926,7 @@ int llms::chunk_tolerance_impl(const llms_kv_desc *desc, const void *kv, const v
         // one CTA per SM, each with an equal run of the sequence of all 128-token tiles.  Every statistics thread
         // keeps the partial sums of its row while it runs, if a row's slots - threads per row x the most CTAs that
         // share a (layer, KV head) pair - fit; else a pass over the statistics follows.
-        const int tiles_per_pair = (a.T + kTcTile - 1) / kTcTile;
+        const int tiles_per_pair = ((a.T + kTcTile - 1) / kTcTile + 1) / 2;      // double tiles: what an MMA takes
         const int64_t total = (int64_t)a.L * a.Hkv * tiles_per_pair;
         a.tc_grid = (int)std::min<int64_t>(total, sm_count());
         a.tc_spr = kTcAcc * (kTcTile / tc_rows(a));

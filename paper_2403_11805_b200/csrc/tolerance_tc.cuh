@@ -4,10 +4,12 @@
 // Why: the warp-level MMA kernel is bound by the latency of each warp's own instruction chain (fragment loads,
 // MMAs, shuffles, one tile at a time), not by memory - with 32 rows per KV head it stays near 6.0 TB/s of K while a
 // plain read stream reaches 6.9.  Here the product leaves the warps altogether:
-//   * one thread feeds tiles of 128 tokens (and, per (layer, KV head) pair, the query rows) into shared memory with
-//     TMA tensor copies, 128-byte swizzled, a ring of stages ahead of the arithmetic;
-//   * one thread issues the MMAs: S[128 rows x 128 tokens] = q[128 x d] K_tile[128 x d]^T, operands read from shared
-//     memory by the tensor core, the accumulator in tensor memory (four accumulators of 128 columns take turns);
+//   * one thread feeds pairs of 128-token tiles (and, per (layer, KV head) pair, the query rows) into shared memory
+//     with TMA tensor copies, 128-byte swizzled, a ring of stages ahead of the arithmetic;
+//   * one thread issues the MMAs: S[128 rows x 256 tokens] = q[128 x d] K_tiles[256 x d]^T, two neighbouring tiles of
+//     a pair at a time (an MMA of 256 columns holds the issuing thread hardly longer than one of 128: with one tile per
+//     MMA that thread was the pacemaker of the kernel), operands read from shared memory by the tensor core, the
+//     accumulator in tensor memory (two accumulators of 256 columns take turns);
 //   * the other warps only do the softmax statistics: a thread reads ITS window row's consecutive tokens from tensor
 //     memory, so maxima and sums over a segment of tokens stay inside the thread (one or two shuffle steps where a
 //     thread holds fewer tokens than a segment has).
@@ -19,29 +21,32 @@
 // long raises a flag that turns the scores of the call into NaN, and still leaves through the common exit, where
 // tensor memory is given back.
 //
-// Measured (B200, whole launches, K bytes / time): 32K-token grouped-query shape (32 rows per KV head) 352.8 us against
-// 356.9 us for the warp-level kernel; 7B shape (8 rows) 177.6 against 165.3 us - so it is used from 32 rows per KV head
-// on.  Taking the MMAs or the statistics out of it showed the feeding side alone at the pace of a resident-CTA read
-// stream (6.9 TB/s); MMAs and statistics each add their time instead of hiding behind the copies, whatever the number
-// of stages (2 to 5 made no difference), and asking tiles into L2 ahead of the ring made it slower.  Cycle counters
-// around the waits (32K shape, per tile of 1332 cycles): the issuing thread is held 890 cycles by a tile's eight MMAs
-// and waits 440, the feeding thread waits 970 for a free stage, a statistics warp works 750 cycles on a tile of its
-// own and waits 4400.  With the query rows in tensor memory instead of shared memory (three accumulators, tcgen05.st)
-// the tile took 1282 cycles and the same time: the kernel runs under the power cap.
+// Measured (B200, whole launches, K bytes / time): 32K-token grouped-query shape (32 rows per KV head), one tile per MMA:
+// 352.8 us against 356.9 us for the warp-level kernel; 7B shape (8 rows) 177.6 against 165.3 us - so it is used from 32
+// rows per KV head on.  Taking the MMAs or the statistics out of that kernel showed the feeding side alone at the pace of
+// a resident-CTA read stream (6.9 TB/s); MMAs and statistics each added their time instead of hiding behind the copies,
+// whatever the number of stages (2 to 5 made no difference), and asking tiles into L2 ahead of the ring made it slower.
+// Cycle counters around the waits (32K shape, per tile of 1332 cycles) then showed the issuing thread held 890 cycles by
+// a tile's eight MMAs (111 each, where the tensor pipe alone needs 68) and waiting 440, the feeding thread waiting 970
+// for a free stage, a statistics warp working 750 cycles on a tile of its own and waiting 4400.  With the query rows in
+// tensor memory instead of shared memory (three accumulators, tcgen05.st) a tile took 1282 cycles and the same time
+// (not kept); with two tiles per MMA (this kernel) the score stage of the 32K shape went from 384 to 357 us.
 #pragma once
 
 #include <cuda.h>
 
 namespace llms {
 
-constexpr int kTcTile = 128;                         // tokens per tile = N of the MMA = columns of an accumulator
-constexpr int kTcAcc = 4;                            // accumulators in tensor memory (4 x 128 = all 512 columns)
+constexpr int kTcTile = 128;                         // tokens per tile: what a statistics warp group takes at a time
+constexpr int kTcWide = 2 * kTcTile;                 // tokens per MMA (N = 256): two neighbouring tiles of a pair
+constexpr int kTcAcc = 4;                            // tile-wide halves of the two 256-column accumulators (all 512 columns)
 constexpr int kTcEpiWarps = 4 * kTcAcc;              // per accumulator one warp for each quarter of the 128 lanes
 constexpr int kTcProducerWarp = kTcEpiWarps, kTcMmaWarp = kTcEpiWarps + 1;
 constexpr int kTcThreads = (kTcEpiWarps + 2) * 32;
 constexpr uint32_t kTcSpinLimit = 1u << 22;          // polls (with a pause in between) before a wait is given up
 constexpr uint32_t kTcGaveUp = 0x7E57DEADu;          // value of the status word after a wait was given up
-constexpr int kTcBlockBytes = kTcTile * 128;         // one 64-channel block of a 128-row operand: 128 rows x 128 bytes
+constexpr int kTcBlockBytes = kTcTile * 128;         // one 64-channel block of the 128-row A operand: 128 rows x 128 bytes
+constexpr int kTcWideBlockBytes = kTcWide * 128;     // one 64-channel block of the 256-row B operand (two tiles of K)
 
 struct TcBarriers {
     unsigned long long full[8], empty[8];            // tile stages (as many as fit, at most 8)
@@ -104,7 +109,7 @@ __device__ __forceinline__ uint64_t tc_operand_desc(uint32_t smem_addr)
 
 // Instruction descriptor: fp32 accumulator (bits 4-5 = 1), fp16 A and B (bits 7-9, 10-12 = 0), both with the
 // contraction dimension contiguous (bits 15, 16 = 0), N / 8 in bits 17-22, M / 16 in bits 24-28.
-constexpr uint32_t kTcInstrDesc = (1u << 4) | ((uint32_t)(kTcTile >> 3) << 17) | ((128u >> 4) << 24);
+constexpr uint32_t kTcInstrDesc = (1u << 4) | ((uint32_t)(kTcWide >> 3) << 17) | ((128u >> 4) << 24);
 
 __device__ __forceinline__ void tc_mma(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t accumulate)
 {
@@ -234,13 +239,14 @@ __global__ void __launch_bounds__(kTcThreads, 1) logits_tc_kernel(const TolArgs 
                                                                   const __grid_constant__ CUtensorMap map_q, int n_stages)
 {
     constexpr int kBlocks = D / 64;                              // 64-channel blocks of an operand
-    constexpr int kOperandBytes = kBlocks * kTcBlockBytes;       // one tile of K, or one buffer of query rows
+    constexpr int kOperandBytes = kBlocks * kTcBlockBytes;       // one buffer of query rows
+    constexpr int kStageBytes = kBlocks * kTcWideBlockBytes;     // two neighbouring tiles of K
     extern __shared__ __align__(1024) unsigned char tc_smem_raw[];
     // operands need 1 KiB alignment for the swizzle; the barriers sit behind them
     unsigned char *base = reinterpret_cast<unsigned char *>((reinterpret_cast<uintptr_t>(tc_smem_raw) + 1023) & ~(uintptr_t)1023);
     unsigned char *q_buf = base;                                 // [2][kOperandBytes]
-    unsigned char *k_buf = base + 2 * kOperandBytes;             // [n_stages][kOperandBytes]
-    TcBarriers *bar = reinterpret_cast<TcBarriers *>(k_buf + (size_t)n_stages * kOperandBytes);
+    unsigned char *k_buf = base + 2 * kOperandBytes;             // [n_stages][kStageBytes]
+    TcBarriers *bar = reinterpret_cast<TcBarriers *>(k_buf + (size_t)n_stages * kStageBytes);
     volatile uint32_t *gave_up = &bar->gave_up;
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -254,9 +260,9 @@ __global__ void __launch_bounds__(kTcThreads, 1) logits_tc_kernel(const TolArgs 
             mbar_init(&bar->q_full[b], 1);
             mbar_init(&bar->q_empty[b], 1);
         }
-        for (int g = 0; g < kTcAcc; ++g) {
+        for (int g = 0; g < 2; ++g) {                            // the two accumulators of 256 columns
             mbar_init(&bar->acc_full[g], 1);
-            mbar_init(&bar->acc_empty[g], n_quarters);
+            mbar_init(&bar->acc_empty[g], 2 * n_quarters);       // both halves' four statistics warps
         }
         bar->gave_up = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -273,8 +279,9 @@ __global__ void __launch_bounds__(kTcThreads, 1) logits_tc_kernel(const TolArgs 
     tc_fence_after();
     const uint32_t tmem_base = bar->tmem_base;
 
-    // this CTA's run of the sequence of all tiles (pair-major)
-    const int tiles_per_pair = (a.T + kTcTile - 1) / kTcTile;
+    // this CTA's run of the sequence of all double tiles (pair-major); a pair's last one may have only its first half
+    const int n_tiles = (a.T + kTcTile - 1) / kTcTile;
+    const int tiles_per_pair = (n_tiles + 1) / 2;                // double tiles of a pair
     const int64_t total = (int64_t)a.L * a.Hkv * tiles_per_pair;
     const int64_t run_begin = total * blockIdx.x / gridDim.x, run_end = total * (blockIdx.x + 1) / gridDim.x;
     const int n_items = (int)(run_end - run_begin);
@@ -303,10 +310,10 @@ __global__ void __launch_bounds__(kTcThreads, 1) logits_tc_kernel(const TolArgs 
                     ++stage_round;
                 }
                 if (!mbar_wait(&bar->empty[s], parity ^ 1, gave_up)) break;
-                mbar_expect_tx(&bar->full[s], kOperandBytes);
+                mbar_expect_tx(&bar->full[s], kStageBytes);
 #pragma unroll
                 for (int b = 0; b < kBlocks; ++b)
-                    tma_load_4d(smem_u32(k_buf + (size_t)s * kOperandBytes + b * kTcBlockBytes), &map_k, b * 64, at.tile * kTcTile, at.kvh,
+                    tma_load_4d(smem_u32(k_buf + (size_t)s * kStageBytes + b * kTcWideBlockBytes), &map_k, b * 64, at.tile * kTcWide, at.kvh,
                                 at.l, &bar->full[s]);
             }
         }
@@ -326,16 +333,16 @@ __global__ void __launch_bounds__(kTcThreads, 1) logits_tc_kernel(const TolArgs 
                     stage = 0;
                     ++stage_round;
                 }
-                const int g = it & (kTcAcc - 1), ka = it / kTcAcc;
+                const int g = it & 1, ka = it >> 1;              // accumulator, its turn
                 if (!mbar_wait(&bar->acc_empty[g], (ka & 1) ^ 1, gave_up)) break;
                 tc_fence_after();
-                const uint32_t q_addr = smem_u32(q_buf + qb * kOperandBytes), k_addr = smem_u32(k_buf + (size_t)s * kOperandBytes);
+                const uint32_t q_addr = smem_u32(q_buf + qb * kOperandBytes), k_addr = smem_u32(k_buf + (size_t)s * kStageBytes);
 #pragma unroll
                 for (int b = 0; b < kBlocks; ++b)
 #pragma unroll
                     for (int kk = 0; kk < 4; ++kk)               // 16 channels (32 bytes) per MMA
-                        tc_mma(tmem_base + g * kTcTile, tc_operand_desc(q_addr + b * kTcBlockBytes + kk * 32),
-                               tc_operand_desc(k_addr + b * kTcBlockBytes + kk * 32), (b | kk) != 0);
+                        tc_mma(tmem_base + g * kTcWide, tc_operand_desc(q_addr + b * kTcBlockBytes + kk * 32),
+                               tc_operand_desc(k_addr + b * kTcWideBlockBytes + kk * 32), (b | kk) != 0);
                 tc_commit(&bar->empty[s]);                       // the stage is free once these MMAs have read it
                 tc_commit(&bar->acc_full[g]);
                 const bool pair_ends = tile == tiles_per_pair - 1;
@@ -344,7 +351,8 @@ __global__ void __launch_bounds__(kTcThreads, 1) logits_tc_kernel(const TolArgs 
             }
         }
     } else {
-        const int g = warp >> 2, quarter = warp & 3;             // accumulator, lanes 32*quarter .. +31 of it
+        const int g = warp >> 2, quarter = warp & 3;             // half accumulator, lanes 32*quarter .. +31 of it
+        const int acc = g >> 1, half = g & 1;                    // accumulator of 256 columns, which tile of its two
         constexpr int kPiece = R < 32 ? R : 32;                  // tokens a thread takes from one load of 32 columns
         const int m_index = quarter * 32 + lane;                 // this thread's row of the product
         const int j = m_index % R;                               // ... is copy m_index / R of row j of the pair,
@@ -356,8 +364,8 @@ __global__ void __launch_bounds__(kTcThreads, 1) logits_tc_kernel(const TolArgs 
         const int copy_index = g * (kTcTile / R) + m_index / R;
         const bool keep = a.n_slots > 0;
         TcCursor at;
-        at.start(run_begin + g, tiles_per_pair, a.Hkv);
-        int it = g;                                              // this thread's next tile, counted from the run's first
+        at.start(run_begin + acc, tiles_per_pair, a.Hkv);
+        int it = acc;                                            // this thread's next double tile, counted from the run's first
         bool alive = true;
         // pair by pair: every thread leaves a (max, sum) pair for every (layer, KV head) pair the run touches, also
         // where none of the pair's tiles fell to its accumulator
@@ -365,13 +373,13 @@ __global__ void __launch_bounds__(kTcThreads, 1) logits_tc_kernel(const TolArgs 
             const int64_t next_pair = (pair + 1) * tiles_per_pair;
             const int pair_end = (int)((run_end < next_pair ? run_end : next_pair) - run_begin);
             float run_m = -INFINITY, run_z = 0.0f;
-            for (; it < pair_end; it += kTcAcc) {
-                const int tile = at.tile;
+            for (; it < pair_end; it += 2) {
+                const int tile = 2 * at.tile + half;
                 const int64_t out = pair * a.NR + j;             // this thread's row among all rows
                 const int last_col = valid ? a.T - a.W + row_in_window : -1;
 #pragma unroll
-                for (int k = 0; k < kTcAcc; ++k) at.next(tiles_per_pair, a.Hkv);   // where the next trip is
-                if (!mbar_wait(&bar->acc_full[g], (it / kTcAcc) & 1, gave_up)) {
+                for (int k = 0; k < 2; ++k) at.next(tiles_per_pair, a.Hkv);        // where the next trip is
+                if (!mbar_wait(&bar->acc_full[acc], (it >> 1) & 1, gave_up)) {
                     alive = false;
                     break;
                 }
@@ -381,7 +389,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) logits_tc_kernel(const TolArgs 
                 // columns and every thread keeps the piece of its copy
                 const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + g * kTcTile + (R < 32 ? quarter * 32 : col0);
 #pragma unroll
-                for (int c = 0; c < (R < 32 ? 1 : R / 32); ++c) {
+                for (int c = 0; c < (R < 32 ? 1 : R / 32) && tile < n_tiles; ++c) {   // a pair's odd last tile has no second half
                     float got[32], dot[kPiece];
                     tc_load<32>(taddr + c * 32, got);
 #pragma unroll
@@ -398,7 +406,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) logits_tc_kernel(const TolArgs 
                 }
                 tc_fence_before();
                 __syncwarp();
-                if (lane == 0) mbar_arrive(&bar->acc_empty[g]);
+                if (lane == 0) mbar_arrive(&bar->acc_empty[acc]);
             }
             if (alive && keep && valid) {
                 const int first_cta = tc_cta_of_tile(pair * tiles_per_pair, total, (int)gridDim.x);
