@@ -593,20 +593,24 @@ __device__ __forceinline__ void load_unit(const CodecArgs &a, const UnitPos &u, 
 }
 
 // ... and brought to the layout the arithmetic wants (lane L holds elements [L*64, +64) of the pass) through the
-// warp's patch of shared memory.  Rows of 128 bytes are padded to 144: both the 32-byte-per-lane writes and the
+// warp's patch of shared memory: stored from the registers the loads landed in, read back into others.  Rows of 128 bytes are padded to 144: both the 32-byte-per-lane writes and the
 // 128-byte-per-lane reads are then free of bank conflicts.
 constexpr int kTransposeRowBytes = 128 + 16;
 constexpr int kTransposeBytes = 32 * kTransposeRowBytes;
 
-__device__ __forceinline__ void to_lane_contiguous(uint32_t (&w)[kPieces][8], unsigned char *patch, int lane)
+__device__ __forceinline__ void patch_store(const uint32_t (&raw)[kPieces][8], unsigned char *patch, int lane)
 {
 #pragma unroll
     for (int j = 0; j < kPieces; ++j) {
         // piece j of this lane = 16-byte chunks 64j + 2L and 64j + 2L + 1 of the unit; chunk n -> row n/8, column n%8
         unsigned char *dst = patch + (8 * j + (lane >> 2)) * kTransposeRowBytes + (lane & 3) * 32;
-        *reinterpret_cast<uint4 *>(dst) = make_uint4(w[j][0], w[j][1], w[j][2], w[j][3]);
-        *reinterpret_cast<uint4 *>(dst + 16) = make_uint4(w[j][4], w[j][5], w[j][6], w[j][7]);
+        *reinterpret_cast<uint4 *>(dst) = make_uint4(raw[j][0], raw[j][1], raw[j][2], raw[j][3]);
+        *reinterpret_cast<uint4 *>(dst + 16) = make_uint4(raw[j][4], raw[j][5], raw[j][6], raw[j][7]);
     }
+}
+
+__device__ __forceinline__ void patch_load(unsigned char *patch, int lane, uint32_t (&w)[kPieces][8])
+{
     __syncwarp();
     const unsigned char *row = patch + lane * kTransposeRowBytes;
 #pragma unroll
@@ -703,23 +707,26 @@ __device__ __forceinline__ void compress_phase(const CodecArgs &a, uint32_t *cou
     if (unit < a.total_units) {
         unsigned char *patch = patches[threadIdx.x >> 5];
         // A unit is decoded once, two turns ahead of its own: then its bytes are asked into L2, one trip later its
-        // loads are issued (pn -> pb), another trip later it is computed (pb -> pa).  One unit per trip, the next
-        // unit's registers copied over at the end: unrolled by two, so that the buffers swap roles without the 32
-        // copies, the loop no longer fits the instruction cache well and the kernel is 1.5% slower (measured).
+        // loads are issued (pn -> pb), another trip later it is computed (pb -> pa).  The loads land in `raw`; a trip
+        // first puts the current unit's raw registers into the warp's patch of shared memory, then issues the next
+        // unit's loads into the same registers, then reads the current unit back in the layout the arithmetic wants
+        // (`cur`).  One unit per trip: unrolled by two the loop no longer fits the instruction cache well and the
+        // kernel is 1.5% slower (measured).
         static_assert(kPrefetchAhead == 2, "the loop below looks exactly two units ahead");
         UnitPos pa, pb, pn;
-        uint32_t wa[kPieces][8], wb[kPieces][8];
+        uint32_t raw[kPieces][8], cur[kPieces][8];
         decode_unit<PACKED>(a, unit, lane, pa);
-        load_unit<WIDE, PACKED>(a, pa, lane, wa);
+        load_unit<WIDE, PACKED>(a, pa, lane, raw);
         uint32_t ahead = feed.pop(lane);
         bool has_next = ahead < a.total_units;
         if (has_next) decode_unit<PACKED>(a, ahead, lane, pn);
 #pragma unroll 1
         for (;;) {
+            patch_store(raw, patch, lane);
             const bool more = has_next;
             if (more) {
                 pb = pn;
-                load_unit<WIDE, PACKED>(a, pb, lane, wb);
+                load_unit<WIDE, PACKED>(a, pb, lane, raw);
             }
             ahead = feed.pop(lane);
             has_next = ahead < a.total_units;
@@ -727,14 +734,10 @@ __device__ __forceinline__ void compress_phase(const CodecArgs &a, uint32_t *cou
                 decode_unit<PACKED>(a, ahead, lane, pn);
                 prefetch_unit_l2<PACKED>(a, pn, lane);
             }
-            to_lane_contiguous(wa, patch, lane);
-            compress_unit<BITS, G, WIDE>(a, pa, wa, lane, sum_slots);
+            patch_load(patch, lane, cur);
+            compress_unit<BITS, G, WIDE>(a, pa, cur, lane, sum_slots);
             if (!more) break;
             pa = pb;
-#pragma unroll
-            for (int j = 0; j < kPieces; ++j)
-#pragma unroll
-                for (int k = 0; k < 8; ++k) wa[j][k] = wb[j][k];
         }
     }
     __syncthreads();
