@@ -100,7 +100,7 @@ struct CodecArgs {
 // meaning for every record offset, with e0 running past the end of slab s_idx; only the KV addresses have to be
 // looked up slab by slab.
 struct UnitPos {
-    uint32_t i, k, s_idx, chunk_id, bits;  // i: entry index (caller's order), k: position in this launch's list
+    uint32_t i, k, s_idx, chunk_id;  // i: entry index (caller's order), k: position in this launch's list
     uint64_t rec_off;
     int e0;                // first element of this lane, counted from the start of slab s_idx
     int limit;             // elements of this unit that exist, counted from the unit's first element
@@ -123,11 +123,10 @@ __device__ __forceinline__ void decode_unit(const CodecArgs &a, uint32_t unit, i
     uint32_t row;
     a.div_n.divmod(item, row, k);
     u.k = k;
-    u.i = a.order[k];
-    const uint4 head = *reinterpret_cast<const uint4 *>(a.entries + u.i);  // chunk_id, bits, offset
-    u.chunk_id = head.x;
-    u.bits = head.y;
-    u.rec_off = (uint64_t)head.z | ((uint64_t)head.w << 32);
+    const uint4 ent = *reinterpret_cast<const uint4 *>(a.table + k);       // chunk, entry, record offset: one load
+    u.chunk_id = ent.x;
+    u.i = ent.y;
+    u.rec_off = (uint64_t)ent.z | ((uint64_t)ent.w << 32);
     if constexpr (PACKED) {
         u.s_idx = row * (uint32_t)a.slabs_per_unit;
         u.e0 = lane * kLaneElems;
@@ -136,7 +135,7 @@ __device__ __forceinline__ void decode_unit(const CodecArgs &a, uint32_t unit, i
         u.s_idx = row;
         u.e0 = (int)pass * kPassElems + lane * kLaneElems;
         u.limit = min(kPassElems, a.slab_elems - (int)pass * kPassElems);
-        u.kv_off = slab_offset(a, row, head.x) + (int)pass * kPassElems;
+        u.kv_off = slab_offset(a, row, ent.x) + (int)pass * kPassElems;
     }
 }
 
