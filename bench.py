@@ -64,11 +64,11 @@ def measured_peaks():
 CODEC_SOURCES = ("paper_2403_11805_b200/csrc/codec.cu", "paper_2403_11805_b200/csrc/codec_cw.cuh",
                  "paper_2403_11805_b200/csrc/llms_internal.cuh")
 NCU_DRAM_TRAFFIC = {
-    "codec_sha256_16": "01417c4ecd867fea",      # hash of CODEC_SOURCES at the capture
-    "source": "ncu dram__bytes_read.sum + dram__bytes_write.sum of one full-size launch, commit 97f4083 "
+    "codec_sha256_16": "78c2b6ab0867d80c",      # hash of CODEC_SOURCES at the capture
+    "source": "ncu dram__bytes_read.sum + dram__bytes_write.sum of one full-size launch, commit 396a81d "
               "(profiles/codec_and_score_kernels_llama7b.md)",
-    ("llama7b", 32, "compress_kernel"): 2149007616 + 646748160,
-    ("llama7b", 32, "decompress_kernel"): 659704064 + 2085752576,
+    ("llama7b", 32, "compress_kernel"): 2149846528 + 646908672,
+    ("llama7b", 32, "decompress_kernel"): 659665408 + 2085249792,
 }
 
 
