@@ -139,7 +139,7 @@ int llms_compress_chunks(const llms_kv_desc *desc, const void *kv, const uint32_
  * would stall inference because cudaMalloc synchronises the device), or code running where the CUDA
  * allocator must not be entered at all.  The paper has no counterpart to this call; it is a
  * convenience of this library.  The chunk table lives in a fixed array inside the library image
- * (about 57 KB, present on every GPU that loads the library until the process exits), which limits
+ * (about 64 KiB, present on every GPU that loads the library until the process exits), which limits
  * one call to LLMS_STATIC_MAX_CHUNKS chunks: a larger n returns LLMS_ERR_BUF_TOO_SMALL and nothing
  * is launched.  No device memory is allocated or freed.  All other arguments, results and errors
  * are those of llms_compress_chunks.
